@@ -1,0 +1,21 @@
+"""CPU oracle for routed structured-sparse causal prefill attention (RouteSparse).
+
+TEST INFRASTRUCTURE ONLY.  This package is the slow, plain restatement of what the CUDA
+path computes, written from the paper's definitions in float64 numpy.  It is imported only
+by the tests, by the smoke check and by the benchmark's CPU-baseline leg; the product
+path never calls it, and it imports nothing from the CUDA package.
+
+Parts and what pins them (tests/test_oracle_*.py):
+  attention.dense_attention      Eq. 1, plain definition.        Pinned: row 0, K=0 mean, torch SDPA.
+  attention.masked_attention     Section 2.1 masked variant.      Pinned: causal mask == dense, LSE merge, explicit bitset.
+  probe.probe                    Eq. 3 in the last-64-query form. Pinned: row sums, brute force vs the full matrix A.
+  patterns.*                     Section 3.1 pattern library.     Pinned: brute-force pair counts, coverage vs plain
+                                                                  definition, nesting, k >= n.  The concrete tie-break
+                                                                  and the block expansion of slashes are this build's
+                                                                  reading: beyond those invariants "parity unpinned".
+  routing.route                  Eq. 4, Eq. 6-8, fallback.        Pinned: constraints, trivial budgets, exhaustive optimum
+                                                                  as a lower bound.  The exact substitution order is this
+                                                                  build's reading: "parity unpinned".
+  certificate.certificate        Eq. 5.                           Pinned: equality case, L1 identity, bound on every row.
+"""
+from . import attention, certificate, patterns, probe, routing  # noqa: F401

@@ -1,0 +1,157 @@
+"""Oracle: risk score (Eq. 4), latency-constrained routing (Eq. 6-8) and the fallback rule (Section 3.4).
+
+Test infrastructure only; never imported by the product path.
+
+Items are (segment, head) pairs; every item picks exactly one candidate of the library (Eq. 7) and the
+summed cost plus the probe cost must not exceed the layer budget T (Eq. 8).  The paper solves this with
+a greedy heuristic: start from the zero-risk dense choice everywhere and repeatedly apply the
+substitution with the best risk increase per unit of cost saved until the budget is met.  Then items
+whose lower-confidence mass is too small first take a larger budget of the same family and finally
+dense.  The paper names no tie-break and no order of the fallback walk; the order used here is this
+build's reading (parity unpinned beyond the invariants the tests check).
+
+Arithmetic: coverage arrives as exact fixed-point integers, costs are integers (FLOPs or nanoseconds),
+so totals are exact; risks are IEEE doubles computed as (1 - m_hat) + alpha * u with each operation
+rounded separately; ratios are compared by cross-multiplication.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from itertools import product
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+from .patterns import DENSE, Candidate, m_hat_from_fx
+
+CERT_ABS, CERT_REL = 0, 1
+
+
+@dataclass
+class RouteParams:
+    budget: int                      # T_l, same integer unit as cost
+    t_probe: int = 0
+    alpha: float = 1.0               # weight of the probe-subset disagreement u (beta = 0: training-free router)
+    delta_q: float = 0.0             # one-sided residual quantile: m_low = max(0, m_hat - delta_q)
+    cert_max: Optional[float] = None  # fallback fires while certificate > cert_max (None: no fallback)
+    cert_mode: int = CERT_REL        # REL: 2(1 - m_low);  ABS: 2(1 - m_low) * vmax
+    expand_first: bool = True        # try the next larger budget of the family before dense
+    forced_dense: Sequence[int] = field(default_factory=list)   # items forced to dense last
+    fixed_choice: Optional[Sequence[int]] = None                 # bypasses the solve and the fallback
+
+
+@dataclass
+class RouteReport:
+    total_cost: int
+    total_risk: float
+    n_fallback: int
+    feasible: int
+
+
+def risks(lib: List[Candidate], cov_fx: np.ndarray, alpha: float):
+    """R[item][c] = (1 - m_hat) + alpha * u (Eq. 4 with beta = 0); dense has m_hat = 1, u = 0, R = 0."""
+    n_items, n_cand = cov_fx.shape[0], len(lib)
+    R = np.zeros((n_items, n_cand), dtype=np.float64)
+    M = np.ones((n_items, n_cand), dtype=np.float64)
+    for it in range(n_items):
+        for c, cand in enumerate(lib):
+            if cand.pattern == DENSE:
+                continue
+            m_hat, u = m_hat_from_fx(cov_fx[it, c])
+            M[it, c] = m_hat
+            R[it, c] = (1.0 - m_hat) + alpha * u
+    return R, M
+
+
+def _dense_index(lib: List[Candidate]) -> int:
+    for c, cand in enumerate(lib):
+        if cand.pattern == DENSE:
+            return c
+    raise ValueError("the library must contain the dense candidate")
+
+
+def greedy_solve(R: np.ndarray, cost: np.ndarray, dense_c: int, budget: int, t_probe: int):
+    """Greedy substitution for Eq. 6-8. Returns (choice, total, feasible)."""
+    n_items, n_cand = R.shape
+    choice = [dense_c] * n_items
+    total = int(t_probe) + sum(int(cost[it, dense_c]) for it in range(n_items))
+    feasible = 1
+    while total > budget:
+        best = None                                   # (dR, dT, item, cand)
+        for it in range(n_items):
+            cur = choice[it]
+            for k in range(n_cand):
+                dT = int(cost[it, cur]) - int(cost[it, k])
+                if dT <= 0:
+                    continue
+                dR = float(R[it, k]) - float(R[it, cur])
+                if best is None:
+                    best = (dR, dT, it, k)
+                    continue
+                lhs = dR * float(best[1])             # dR / dT < best_dR / best_dT  <=>  dR * best_dT < best_dR * dT
+                rhs = best[0] * float(dT)
+                if lhs < rhs or (lhs == rhs and dT > best[1]):
+                    best = (dR, dT, it, k)
+        if best is None:
+            feasible = 0
+            break
+        _, dT, it, k = best
+        choice[it] = k
+        total -= dT
+    return choice, total, feasible
+
+
+def _next_larger(lib: List[Candidate], c: int) -> Optional[int]:
+    """Index of the next entry of the same family after c (library lists a family by increasing budget)."""
+    for k in range(c + 1, len(lib)):
+        if lib[k].pattern == lib[c].pattern:
+            return k
+    return None
+
+
+def route(lib: List[Candidate], cov_fx: np.ndarray, cost: np.ndarray, vmax: np.ndarray, p: RouteParams):
+    """Full routing of one layer. cov_fx[items, n_cand, 4] uint64, cost[items, n_cand] int64, vmax[items] fp32."""
+    n_items = cov_fx.shape[0]
+    dense_c = _dense_index(lib)
+    R, M = risks(lib, cov_fx, p.alpha)
+    n_fallback = 0
+    if p.fixed_choice is not None:
+        choice = [int(c) for c in p.fixed_choice]
+        feasible = 1
+    else:
+        choice, _, feasible = greedy_solve(R, cost, dense_c, int(p.budget), int(p.t_probe))
+        if p.cert_max is not None:
+            for it in range(n_items):
+                fired = False
+                while lib[choice[it]].pattern != DENSE:
+                    m_low = max(0.0, float(M[it, choice[it]]) - p.delta_q)
+                    cert = 2.0 * (1.0 - m_low)
+                    if p.cert_mode == CERT_ABS:
+                        cert = cert * float(np.float32(vmax[it]))
+                    if not cert > p.cert_max:
+                        break
+                    fired = True
+                    nxt = _next_larger(lib, choice[it]) if p.expand_first else None
+                    choice[it] = nxt if nxt is not None else dense_c
+                n_fallback += int(fired)
+    for it in p.forced_dense:
+        choice[int(it)] = dense_c
+    total = int(p.t_probe) + sum(int(cost[it, choice[it]]) for it in range(n_items))
+    risk = 0.0
+    for it in range(n_items):
+        risk += float(R[it, choice[it]])
+    return np.asarray(choice, dtype=np.int32), RouteReport(total, risk, n_fallback, feasible)
+
+
+def exhaustive_optimum(R: np.ndarray, cost: np.ndarray, budget: int, t_probe: int):
+    """Exact multiple-choice knapsack by enumeration (tiny instances only). Returns (risk, choice) or None."""
+    n_items, n_cand = R.shape
+    best = None
+    for combo in product(range(n_cand), repeat=n_items):
+        tot = int(t_probe) + sum(int(cost[i, c]) for i, c in enumerate(combo))
+        if tot > budget:
+            continue
+        r = sum(float(R[i, c]) for i, c in enumerate(combo))
+        if best is None or r < best[0]:
+            best = (r, combo)
+    return best

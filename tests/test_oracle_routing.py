@@ -1,0 +1,114 @@
+"""Pins for the oracle's risk (Eq. 4), routing (Eq. 6-8) and fallback (Section 3.4). CPU only."""
+import numpy as np
+import pytest
+
+from oracle import patterns as PT
+from oracle import routing as RT
+
+C = PT.Candidate
+LIB = [C(PT.A_SHAPE, 8, 64), C(PT.A_SHAPE, 8, 128), C(PT.VERTICAL_SLASH, 8, 8), C(PT.BLOCK_SPARSE, 2), C(PT.DENSE)]
+DENSE_C = 4
+
+
+def _instance(rng, n_items=4):
+    cov = np.zeros((n_items, len(LIB), 4), dtype=np.uint64)
+    cost = np.zeros((n_items, len(LIB)), dtype=np.int64)
+    for it in range(n_items):
+        for c in range(len(LIB) - 1):
+            base = rng.uniform(0.2, 1.0)
+            cov[it, c] = (np.clip(base + rng.uniform(-0.1, 0.1, 4), 0, 1) * 16 * 2 ** 32).astype(np.uint64)
+            cost[it, c] = rng.integers(10, 90)
+        cov[it, 1] = np.maximum(cov[it, 1], cov[it, 0])      # larger budget of a family covers at least as much
+        cost[it, 1] = max(cost[it, 1], cost[it, 0] + 1)
+        cost[it, DENSE_C] = 100
+    return cov, cost
+
+
+def test_risk_formula():
+    cov = np.zeros((1, len(LIB), 4), dtype=np.uint64)
+    cov[0, 0] = np.array([0.5, 0.75, 1.0, 0.25]) * 16 * 2 ** 32
+    R, M = RT.risks(LIB, cov, alpha=2.0)
+    assert M[0, 0] == 0.625 and R[0, 0] == (1 - 0.625) + 2.0 * 0.75
+    assert R[0, DENSE_C] == 0.0 and M[0, DENSE_C] == 1.0
+
+
+def test_constraints_and_bound_against_exhaustive_optimum():
+    rng = np.random.default_rng(0)
+    n_opt = 0
+    for trial in range(60):
+        cov, cost = _instance(rng)
+        budget = int(rng.integers(30, 420))
+        choice, rep = RT.route(LIB, cov, cost, np.ones(4, np.float32), RT.RouteParams(budget=budget, t_probe=5))
+        assert choice.shape == (4,) and np.all((choice >= 0) & (choice < len(LIB)))      # Eq. 7
+        R, _ = RT.risks(LIB, cov, 1.0)
+        best = RT.exhaustive_optimum(R, cost, budget, 5)
+        if best is None:
+            assert rep.feasible == 0
+            assert all(cost[i, choice[i]] == cost[i].min() for i in range(4))
+        else:
+            assert rep.feasible == 1 and rep.total_cost <= budget                          # Eq. 8
+            assert rep.total_risk >= best[0] - 1e-12
+            n_opt += abs(rep.total_risk - best[0]) < 1e-12
+        assert rep.total_cost == 5 + sum(cost[i, choice[i]] for i in range(4))
+    assert n_opt > 5          # the heuristic does find the optimum on a fair share of instances
+
+
+def test_trivial_budgets():
+    rng = np.random.default_rng(1)
+    cov, cost = _instance(rng)
+    choice, rep = RT.route(LIB, cov, cost, np.ones(4, np.float32), RT.RouteParams(budget=405, t_probe=5))
+    assert np.all(choice == DENSE_C) and rep.total_risk == 0.0 and rep.feasible == 1
+    choice, rep = RT.route(LIB, cov, cost, np.ones(4, np.float32), RT.RouteParams(budget=1, t_probe=5))
+    assert rep.feasible == 0
+
+
+def test_greedy_takes_best_ratio_first():
+    lib = [C(PT.A_SHAPE, 8, 64), C(PT.DENSE)]
+    cov = np.zeros((2, 2, 4), dtype=np.uint64)
+    cov[0, 0] = np.uint64(int(0.9 * 16 * 2 ** 32))      # item 0 loses 0.1 mass for 50 units
+    cov[1, 0] = np.uint64(int(0.5 * 16 * 2 ** 32))      # item 1 loses 0.5 mass for 50 units
+    cost = np.array([[50, 100], [50, 100]], dtype=np.int64)
+    choice, rep = RT.route(lib, cov, cost, np.ones(2, np.float32), RT.RouteParams(budget=150))
+    assert choice.tolist() == [0, 1]
+    # equal ratios: the larger saving wins, then the lower item
+    cov[1, 0] = cov[0, 0]
+    choice, _ = RT.route(lib, cov, cost, np.ones(2, np.float32), RT.RouteParams(budget=150))
+    assert choice.tolist() == [0, 1]
+
+
+def test_fallback_expands_then_goes_dense_and_never_lowers_coverage():
+    rng = np.random.default_rng(2)
+    for trial in range(30):
+        cov, cost = _instance(rng)
+        base, _ = RT.route(LIB, cov, cost, np.ones(4, np.float32), RT.RouteParams(budget=200))
+        fb, rep = RT.route(LIB, cov, cost, np.ones(4, np.float32),
+                           RT.RouteParams(budget=200, cert_max=0.3, cert_mode=RT.CERT_REL))
+        _, M = RT.risks(LIB, cov, 1.0)
+        for it in range(4):
+            assert M[it, fb[it]] >= M[it, base[it]]
+            assert LIB[fb[it]].pattern == PT.DENSE or 2 * (1 - M[it, fb[it]]) <= 0.3
+            if fb[it] != base[it]:
+                assert LIB[fb[it]].pattern in (PT.DENSE, LIB[base[it]].pattern)
+        assert rep.n_fallback == int((fb != base).sum())
+        direct, _ = RT.route(LIB, cov, cost, np.ones(4, np.float32),
+                             RT.RouteParams(budget=200, cert_max=0.3, expand_first=False))
+        assert all(direct[it] in (base[it], DENSE_C) for it in range(4))
+
+
+def test_abs_mode_scales_with_vmax_and_delta_q_shifts():
+    cov = np.zeros((1, len(LIB), 4), dtype=np.uint64)
+    cov[0, :4] = np.uint64(int(0.99 * 16 * 2 ** 32))
+    cost = np.array([[10, 20, 30, 40, 100]], dtype=np.int64)
+    p = dict(budget=50, cert_max=0.05)
+    assert RT.route(LIB, cov, cost, np.float32([1.0]), RT.RouteParams(cert_mode=RT.CERT_ABS, **p))[0][0] != DENSE_C
+    assert RT.route(LIB, cov, cost, np.float32([13.5]), RT.RouteParams(cert_mode=RT.CERT_ABS, **p))[0][0] == DENSE_C
+    assert RT.route(LIB, cov, cost, np.float32([1.0]), RT.RouteParams(delta_q=0.02, **p))[0][0] == DENSE_C
+
+
+def test_forced_dense_and_fixed_choice():
+    rng = np.random.default_rng(3)
+    cov, cost = _instance(rng)
+    choice, _ = RT.route(LIB, cov, cost, np.ones(4, np.float32), RT.RouteParams(budget=150, forced_dense=[1, 3]))
+    assert choice[1] == DENSE_C and choice[3] == DENSE_C
+    choice, rep = RT.route(LIB, cov, cost, np.ones(4, np.float32), RT.RouteParams(budget=1, fixed_choice=[0, 1, 2, 3]))
+    assert choice.tolist() == [0, 1, 2, 3] and rep.n_fallback == 0
