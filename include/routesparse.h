@@ -1,0 +1,183 @@
+/*
+ * routesparse.h -- C ABI of the routed structured-sparse causal prefill attention path (RouteSparse).
+ *
+ * One attention layer at a time, on one GPU (sm_100a).  The calls follow the paper's per-layer procedure
+ * (Section 3.4, the six-step table): probe -> candidate indices, coverage, uncertainty -> routing under the
+ * layer budget with fallback -> one sparse attention launch for all heads -> certificate.
+ *
+ * Conventions (all entry points)
+ *   - Return value: RS_OK or a negative rs_status.  Nothing is thrown; nothing is printed.
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller unless the comment says "host".
+ *     The library allocates no device memory: scratch comes from the caller's workspace
+ *     (rs_workspace_bytes), which must be 256-byte aligned.
+ *   - Every call only enqueues work on `stream` (a cudaStream_t passed as void*); it neither synchronises nor
+ *     copies to the host.  Conditions only knowable on the device (a bounded wait that expired, an
+ *     infeasible budget) are written to `status` (device int32[RS_STATUS_WORDS], may be NULL).
+ *   - Layouts are contiguous, row-major: Q[n_q_heads][n_keys][d], K and V [n_kv_heads][n_keys][d], bf16,
+ *     d = 128.  Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ *   - A segment s is the query range [seg_bounds[s], seg_bounds[s+1]) attending keys [0, seg_bounds[s+1]).
+ *     Bounds are multiples of 64; seg_bounds[0] = 0; seg_bounds[n_segments] = n_keys.  Items are
+ *     (segment, head) pairs, item = s * n_q_heads + h.
+ *   - Probe rows: the last 64 query rows of a segment, in four groups of 16 consecutive rows.
+ */
+#ifndef ROUTESPARSE_H_
+#define ROUTESPARSE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RS_BLOCK 64          /* block edge of block-sparse blocks and of block diagonals */
+#define RS_PROBE_ROWS 64
+#define RS_PROBE_GROUPS 4
+#define RS_HEAD_DIM 128
+#define RS_STATUS_WORDS 8    /* [0] first error code, [1] where, [2..] kernel specific */
+#define RS_MAX_KEYS 262144
+#define RS_MAX_CANDIDATES 32
+
+typedef enum {
+  RS_OK = 0,
+  RS_ERR_INVALID_ARG = -1,
+  RS_ERR_UNSUPPORTED_SHAPE = -2,
+  RS_ERR_WORKSPACE_TOO_SMALL = -3,
+  RS_ERR_CUDA = -4,
+  RS_ERR_UNSUPPORTED_DEVICE = -5,
+  RS_ERR_TIMEOUT = -6
+} rs_status;
+
+/* Pattern library of Section 3.1. */
+typedef enum { RS_DENSE = 0, RS_A_SHAPE = 1, RS_VERTICAL_SLASH = 2, RS_BLOCK_SPARSE = 3 } rs_pattern;
+
+/* One (pattern, budget) pair.  Budgets "in units that match the kernel" (Section 3.1):
+ *   A-shape: b0 = sink tokens, b1 = local window width (tokens, diagonal included)
+ *   vertical-slash: b0 = k_v columns, b1 = k_s slash offsets (offset 0 is always kept and counted)
+ *   block-sparse: b0 = k_b key blocks per query block (the diagonal block is always kept and counted)
+ *   dense: none.
+ * Within a family the library lists candidates by increasing budget ("expand" = next of the family). */
+typedef struct { int32_t pattern, b0, b1, flags; } rs_candidate;
+
+typedef struct {
+  int32_t n_q_heads, n_kv_heads, head_dim, n_keys;
+  int32_t n_segments;
+  const int32_t* seg_bounds;   /* HOST array, n_segments + 1 entries */
+} rs_problem;
+
+/* Index storage (device arrays owned by the caller).  Two uses:
+ *   evaluation  (choice == NULL): VS slot = item * n_cand + c;  bs_blk holds, per slot, only the list of the
+ *                segment's last query block: bs_rows = n_items * n_cand.
+ *   materialised (choice != NULL): VS slot = item;  bs_blk is indexed by (head, global query block):
+ *                bs_rows = n_q_heads * n_keys / 64.
+ * Lists are ascending.  Unused tail entries are unspecified. */
+typedef struct {
+  int32_t n_vs_slots, kv_cap, ks_cap, nd_cap;   /* capacities per slot (>= largest budget / n_keys/64) */
+  int32_t bs_rows, kb_cap;
+  int32_t* vs_cols;    /* [n_vs_slots][kv_cap]  vertical key indices */
+  int32_t* vs_offs;    /* [n_vs_slots][ks_cap]  slash offsets */
+  int32_t* vs_diag;    /* [n_vs_slots][nd_cap]  block-diagonal deltas D */
+  int32_t* vs_count;   /* [n_vs_slots][4]       n_cols, n_offs, n_diag, 0 */
+  int32_t* bs_blk;     /* [bs_rows][kb_cap]     selected key blocks */
+  int32_t* bs_count;   /* [bs_rows] */
+} rs_index_set;
+
+/* Per (item, candidate): fixed-point covered probe mass per probe group (unit 2^-32; m_hat_g = cov_fx[g] /
+ * (16 * 2^32)) and the exact number of selected causal query-key pairs. Dense: cov_fx unused. */
+typedef struct { uint64_t cov_fx[RS_PROBE_GROUPS]; uint64_t pairs; } rs_cand_stats;
+
+typedef enum { RS_CERT_ABS = 0, RS_CERT_REL = 1 } rs_cert_mode;
+
+typedef struct {
+  int64_t budget;          /* T_l of Eq. 8, same integer unit as cost */
+  int64_t t_probe;         /* t_probe of Eq. 8 */
+  double alpha;            /* weight of u in Eq. 4 (beta = 0: training-free router) */
+  double delta_q;          /* m_low = max(0, m_hat - delta_q) */
+  double cert_max;         /* fallback fires while certificate > cert_max */
+  int32_t use_cert;        /* 0: no fallback step */
+  int32_t cert_mode;       /* rs_cert_mode: REL 2(1-m_low), ABS 2(1-m_low) * V_max */
+  int32_t expand_first;    /* 1: next larger budget of the family before dense */
+  int32_t reserved;
+  const int32_t* forced_dense;  /* device int32[n_items], non-zero = force dense last; may be NULL */
+  const int32_t* fixed_choice;  /* device int32[n_items]; when set, bypasses solve and fallback; may be NULL */
+} rs_route_params;
+
+typedef struct { int64_t total_cost; double total_risk; int32_t n_fallback; int32_t feasible; } rs_route_report;
+
+const char* rs_error_string(int code);
+int rs_version(void);
+
+/* Bytes of scratch that any hot-path call below needs for this problem and library (host computation). */
+int rs_workspace_bytes(const rs_problem* p, const rs_candidate* lib, int n_cand, size_t* bytes);
+
+/* Shared attention probe, Eq. 3 (Section 3.2) in the last-64-query form, for every (segment, head):
+ * exact softmax rows of the last 64 queries over all causal keys, reduced to
+ *   vert  [n_seg][n_q_heads][4][n_keys]  column mass per probe group          (fp32, 0 beyond the segment end)
+ *   slash [n_seg][n_q_heads][4][n_keys]  diagonal mass per offset i - j        (fp32)
+ *   lse_probe [n_seg][n_q_heads][64]     log-sum-exp of each probe row         (fp32)
+ * plus the pooled signals of the coarse block candidates and the value norms of Eq. 5:
+ *   qpool [n_q_heads][n_keys/64][d], kpool [n_kv_heads][n_keys/64][d]  64-row means (fp32)
+ *   vmax  [n_seg][n_kv_heads]   max_j ||v_j||_2 over j < segment end             (fp32)
+ * vert and slash are fully overwritten.  descr (may be NULL) is reserved for the entropy /
+ * local-concentration descriptors. */
+int rs_probe(const rs_problem* p, const void* Q, const void* K, const void* V,
+             float* vert, float* slash, float* lse_probe, float* qpool, float* kpool, float* vmax,
+             float* descr, void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* Candidate index construction and coverage (Section 3.1, 3.2; step 2 of the procedure table).
+ * Ranking keys are the integers sum_g floor(mass_g * 2^32); order is key descending, index ascending.
+ * vertical-slash: V = top-k_v columns, S = {0} + top-(k_s-1) offsets, D = {floor(o/64), ceil(o/64)}.
+ * block-sparse: per query block the diagonal block plus the top-(k_b-1) pooled scores
+ *   (qpool . kpool / sqrt(d); `bscore` [n_items][n_keys/64][n_keys/64], indexed by global query block,
+ *   replaces the fused product when not NULL).
+ * choice == NULL: evaluate every candidate of every item (lists + stats, see rs_index_set).
+ * choice != NULL (device int32[n_items]): materialise only the chosen candidate of each item. */
+int rs_build_indices(const rs_problem* p, const rs_candidate* lib, int n_cand,
+                     const float* vert, const float* slash, const float* qpool, const float* kpool,
+                     const float* bscore, const int32_t* choice,
+                     const rs_index_set* out, rs_cand_stats* stats,
+                     void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* Risk (Eq. 4), greedy substitution for the budgeted routing problem (Eq. 6-8), fallback walk and forced
+ * dense (Section 3.4), solved by one thread block on the device.
+ * cost: device int64[n_items][n_cand] or NULL (then 4 * d * pairs, i.e. FLOPs of the selected pairs).
+ * vmax: [n_seg][n_kv_heads].  choice: device int32[n_items] out.  report: device, may be NULL. */
+int rs_route(const rs_problem* p, const rs_candidate* lib, int n_cand,
+             const rs_cand_stats* stats, const int64_t* cost, const float* vmax,
+             const rs_route_params* params, int32_t* choice, rs_route_report* report,
+             int32_t* status, void* stream);
+
+/* Masked attention O~ = softmax(Q K^T / sqrt(d) + C + mask(M)) V (Section 2.1) for every head under its
+ * routed pattern, one launch for all heads (Section 3.4, step 6).
+ * idx: materialised index set; choice: device int32[n_items].
+ * O: [n_q_heads][n_keys][d], bf16 (o_dtype 0) or fp32 (o_dtype 1).
+ * lse_sel [n_q_heads][n_keys]: log-sum-exp over the selected keys;  onorm (may be NULL): ||O~_i||_2.
+ * counters (may be NULL): device uint64[2], incremented by the 64-key chunks issued and by the work items. */
+int rs_sparse_prefill_attn(const rs_problem* p, const void* Q, const void* K, const void* V,
+                           const rs_candidate* lib, int n_cand, const rs_index_set* idx, const int32_t* choice,
+                           void* O, int o_dtype, float* lse_sel, float* onorm, uint64_t* counters,
+                           void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* Dense causal attention, Eq. 1, with the same engine (the denominator of "speed-up over own dense").
+ * lse [n_q_heads][n_keys] is the full-row log-sum-exp (the audit input of rs_certificate). */
+int rs_dense_prefill_attn(const rs_problem* p, const void* Q, const void* K, const void* V,
+                          void* O, int o_dtype, float* lse, float* onorm, uint64_t* counters,
+                          void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* Error certificate, Eq. 5: for audited rows with both log-sum-exps known,
+ *   m_i = min(1, exp(lse_sel_i - lse_full_i)),  cert_i = 2 (1 - m_i) V_max,
+ *   tight_i = (1 - m_i) (V_max + onorm_i) (written when onorm and cert_tight are given),
+ * and per head: m_head = mean_i m_i, cert_head[h][0] = 2 (1 - max(0, m_head - delta_q)) V_max,
+ * cert_head[h][1] = max_i cert_i.
+ * lse_sel, onorm: [n_q_heads][n_keys].  rows: device int32[n_rows] query row ids (same for every head);
+ * lse_full: [n_q_heads][n_rows].  vmax_head: [n_q_heads] (V_max of the head's KV head).
+ * Outputs m_row, cert_row, cert_tight: [n_q_heads][n_rows]; m_head [n_q_heads]; cert_head [n_q_heads][2]. */
+int rs_certificate(int n_q_heads, int n_keys, const float* lse_sel, const float* lse_full,
+                   const int32_t* rows, int n_rows, const float* vmax_head, const float* onorm, float delta_q,
+                   float* m_row, float* cert_row, float* cert_tight, float* m_head, float* cert_head,
+                   int32_t* status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROUTESPARSE_H_ */

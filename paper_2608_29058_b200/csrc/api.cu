@@ -1,0 +1,113 @@
+// Host-side glue of the C ABI: argument checks, error strings, tensor-map encoding, workspace sizing.
+#include <mutex>
+
+#include "common.cuh"
+
+size_t rs_attn_workspace_bytes(const rs_problem* p, int max_kv);
+size_t rs_probe_workspace_bytes(const rs_problem* p);
+size_t rs_indices_workspace_bytes(const rs_problem* p, const rs_candidate* lib, int n_cand);
+
+extern "C" const char* rs_error_string(int code) {
+  switch (code) {
+    case RS_OK: return "ok";
+    case RS_ERR_INVALID_ARG: return "invalid argument";
+    case RS_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (d must be 128; n_keys and segment bounds multiples of 64)";
+    case RS_ERR_WORKSPACE_TOO_SMALL: return "workspace too small (see rs_workspace_bytes)";
+    case RS_ERR_CUDA: return "CUDA runtime or driver error";
+    case RS_ERR_UNSUPPORTED_DEVICE: return "device is not sm_100";
+    case RS_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown error";
+  }
+}
+
+extern "C" int rs_version(void) { return 100; }
+
+int rs_check_problem(const rs_problem* p) {
+  if (p == nullptr || p->seg_bounds == nullptr) return RS_ERR_INVALID_ARG;
+  if (p->n_q_heads <= 0 || p->n_kv_heads <= 0 || p->n_q_heads % p->n_kv_heads != 0) return RS_ERR_INVALID_ARG;
+  if (p->head_dim != RS_HEAD_DIM) return RS_ERR_UNSUPPORTED_SHAPE;
+  if (p->n_keys <= 0 || p->n_keys % RS_BLOCK != 0 || p->n_keys > RS_MAX_KEYS) return RS_ERR_UNSUPPORTED_SHAPE;
+  if (p->n_segments <= 0 || p->n_segments > RS_MAX_SEGMENTS) return RS_ERR_UNSUPPORTED_SHAPE;
+  if (p->seg_bounds[0] != 0 || p->seg_bounds[p->n_segments] != p->n_keys) return RS_ERR_INVALID_ARG;
+  for (int s = 0; s < p->n_segments; ++s) {
+    const int a = p->seg_bounds[s], b = p->seg_bounds[s + 1];
+    if (b <= a) return RS_ERR_INVALID_ARG;
+    if (b % RS_BLOCK != 0) return RS_ERR_UNSUPPORTED_SHAPE;
+  }
+  if ((long long)p->n_q_heads * p->n_keys >= (1ll << 31)) return RS_ERR_UNSUPPORTED_SHAPE;
+  return RS_OK;
+}
+
+int rs_check_device() {
+  static int cached[64];
+  static bool init = false;
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return RS_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!init) { for (int i = 0; i < 64; ++i) cached[i] = 1; init = true; }
+  if (dev < 0 || dev >= 64) return RS_ERR_UNSUPPORTED_DEVICE;
+  if (cached[dev] == 1) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return RS_ERR_CUDA;
+    cached[dev] = (major == 10) ? RS_OK : RS_ERR_UNSUPPORTED_DEVICE;
+  }
+  return cached[dev];
+}
+
+typedef CUresult (*encode_fn_t)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static encode_fn_t get_encode() {
+  static encode_fn_t fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<encode_fn_t>(ptr);
+  });
+  return fn;
+}
+
+static int make_tmap_2d(CUtensorMap* out, CUtensorMapDataType dt, size_t esize, const void* base, uint64_t rows,
+                        uint64_t cols, uint32_t box_rows, uint32_t box_cols) {
+  encode_fn_t enc = get_encode();
+  if (enc == nullptr) return RS_ERR_CUDA;
+  if (((uintptr_t)base & 15) != 0) return RS_ERR_INVALID_ARG;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * esize};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(out, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? RS_OK : RS_ERR_CUDA;
+}
+
+int rs_make_tmap_bf16_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                         uint32_t box_cols) {
+  return make_tmap_2d(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, rows, cols, box_rows, box_cols);
+}
+int rs_make_tmap_f32_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                        uint32_t box_cols) {
+  return make_tmap_2d(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, rows, cols, box_rows, box_cols);
+}
+
+extern "C" int rs_workspace_bytes(const rs_problem* p, const rs_candidate* lib, int n_cand, size_t* bytes) {
+  int rc = rs_check_problem(p);
+  if (rc != RS_OK) return rc;
+  if (bytes == nullptr || n_cand < 0 || n_cand > RS_MAX_CANDIDATES || (n_cand > 0 && lib == nullptr))
+    return RS_ERR_INVALID_ARG;
+  int max_kv = 0;
+  for (int c = 0; c < n_cand; ++c)
+    if (lib[c].pattern == RS_VERTICAL_SLASH && lib[c].b0 > max_kv) max_kv = lib[c].b0;
+  size_t need = rs_attn_workspace_bytes(p, max_kv);
+  size_t b = rs_probe_workspace_bytes(p);
+  if (b > need) need = b;
+  b = rs_indices_workspace_bytes(p, lib, n_cand);
+  if (b > need) need = b;
+  *bytes = rs_align_up(need, 256);
+  return RS_OK;
+}

@@ -1,0 +1,667 @@
+// Routed sparse prefill attention (Section 2.1 masked attention, Section 3.4 step 6) and the dense causal
+// kernel of Eq. 1, on tcgen05 tensor cores with TMEM accumulators and TMA-fed shared memory.
+//
+// One CTA owns one 128-row query tile of one head.  The keys a tile visits are a list of 64-key chunks:
+// key blocks of K/V selected by the head's pattern (dense, A-shape, the block diagonals of vertical-slash,
+// block-sparse) followed by chunks of gathered vertical columns.  Two chunks form one 128-key MMA tile:
+//   S = Q K^T        tcgen05.mma, A and B from shared memory (K-major, 128-byte swizzle), S in TMEM
+//   P = exp2(S - m)  softmax warps: tcgen05.ld, mask, online max / sum, bf16 P written back over S in TMEM
+//   O += P V         tcgen05.mma, A = P from TMEM, B = V from shared memory (MN-major)
+// Roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warps 2-5 = softmax / correction / epilogue.
+// Two CTAs share an SM (256 TMEM columns each) so that one tile's softmax overlaps the other's MMAs.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kTileM = 128;
+constexpr int kChunk = 64;
+constexpr int kTmemCols = 256;
+constexpr uint32_t kColS = 0;     // S (fp32, 128 columns); P (bf16 pairs, 64 columns) overwrites its start
+constexpr uint32_t kColO = 128;   // O (fp32, 128 columns)
+
+constexpr uint32_t F_LO = 1u << 12, F_HI = 1u << 13, F_CAUSAL = 1u << 14, F_EDGE = 1u << 15;
+
+struct AttnParams {
+  int n, Hq, Hkv, group, n_seg, n_cand;
+  int seg_bounds[RS_MAX_SEGMENTS + 1];
+  int tile_base[RS_MAX_SEGMENTS + 1];   // first tile id of each segment within one head
+  int tiles_per_head;
+  rs_candidate lib[RS_MAX_CANDIDATES];
+  const int32_t* choice;      // [n_items] or nullptr (all dense)
+  rs_index_set idx;
+  int kv_pad;                 // rows per slot of the packed vertical K/V
+  const int2* order;          // [n_work] (item, tile in segment), heavy first
+  void* O;
+  int o_f32;
+  float* lse;
+  float* onorm;
+  unsigned long long* counters;
+  int32_t* status;
+  float scale_log2e;
+};
+
+struct SmemLayout {   // offsets from the 1024-aligned base
+  static constexpr uint32_t q = 0, k = 32768, v = 65536, end_tiles = 98304;
+};
+
+__device__ __forceinline__ uint32_t range_mask(int lo, int hi, int w) {
+  int a = max(lo, 32 * w), b = min(hi, 32 * w + 31);
+  if (a > b) return 0u;
+  uint32_t len = (uint32_t)(b - a + 1);
+  uint32_t m = (len == 32u) ? 0xffffffffu : ((1u << len) - 1u);
+  return m << (a - 32 * w);
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+               const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmKp,
+               const __grid_constant__ CUtensorMap tmVp, const __grid_constant__ AttnParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // ---- work item
+  const int2 w = P.order[blockIdx.x];
+  const int item = w.x, tile = w.y;
+  const int s = item / P.Hq, h = item - s * P.Hq, g = h / P.group;
+  const int q0 = P.seg_bounds[s], q1 = P.seg_bounds[s + 1];
+  const int i0 = q0 + tile * kTileM;
+  const int rows_valid = min(kTileM, q1 - i0);
+  const int qb0 = i0 >> 6;
+  const bool has_hi = rows_valid > kChunk;
+  const int qb_last = has_hi ? qb0 + 1 : qb0;
+  const rs_candidate cand = (P.choice != nullptr) ? P.lib[P.choice[item]] : rs_candidate{RS_DENSE, 0, 0, 0};
+  const int pattern = cand.pattern;
+  const int nb_words = (qb_last >> 5) + 1;
+
+  // ---- shared memory carve-up
+  const int list_cap = (P.n >> 6) + 64;
+  uint16_t* list = reinterpret_cast<uint16_t*>(sm + SmemLayout::end_tiles);
+  uint32_t* lo_bits = reinterpret_cast<uint32_t*>(sm + SmemLayout::end_tiles + ((list_cap * 2 + 15) & ~15));
+  uint32_t* hi_bits = lo_bits + 128;
+  uint32_t* d_bits = hi_bits + 128;
+  int* wprefix = reinterpret_cast<int*>(d_bits + 128);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(wprefix + 132);
+  volatile int* misc = reinterpret_cast<volatile int*>(bars + 8);   // [0] tmem base, [1] abort, [2] n_block, [3] n_vert
+  const uint32_t bar_q = smem_u32(&bars[0]), bar_kf = smem_u32(&bars[1]), bar_ke = smem_u32(&bars[2]),
+                 bar_vf = smem_u32(&bars[3]), bar_ve = smem_u32(&bars[4]), bar_s = smem_u32(&bars[5]),
+                 bar_p = smem_u32(&bars[6]), bar_o = smem_u32(&bars[7]);
+  volatile int* abort_flag = misc + 1;
+
+  if (tid == 0) {
+    mbar_init(bar_q, 1); mbar_init(bar_kf, 1); mbar_init(bar_ke, 1); mbar_init(bar_vf, 1);
+    mbar_init(bar_ve, 1); mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+    misc[1] = 0; misc[2] = 0; misc[3] = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32((const void*)&misc[0]), kTmemCols);
+    tmem_relinquish();
+  }
+  for (int i = tid; i < 128; i += kThreads) { lo_bits[i] = 0; hi_bits[i] = 0; d_bits[i] = 0; }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = (uint32_t)misc[0];
+
+  // Q tile load goes out before the chunk list is built.
+  if (tid == 0) {
+    mbar_arrive_expect_tx(bar_q, 32768);
+    tma_load_2d(base + SmemLayout::q, &tmQ, bar_q, 0, h * P.n + i0);
+    tma_load_2d(base + SmemLayout::q + 16384, &tmQ, bar_q, 64, h * P.n + i0);
+  }
+
+  // ---- chunk list: bitmaps of key blocks wanted by the low / high 64 query rows, then ordered compaction
+  int vs_slot = 0, n_vcols = 0;
+  if (pattern == RS_VERTICAL_SLASH) {
+    vs_slot = item;
+    const int* cnt = P.idx.vs_count + 4 * vs_slot;
+    n_vcols = cnt[0];
+    const int n_diag = cnt[2];
+    const int* dl = P.idx.vs_diag + (size_t)vs_slot * P.idx.nd_cap;
+    for (int i = tid; i < n_diag; i += kThreads) {
+      int dlt = dl[i];
+      if (dlt >= 0 && dlt < 4096) atomicOr(&d_bits[dlt >> 5], 1u << (dlt & 31));
+    }
+  } else if (pattern == RS_BLOCK_SPARSE) {
+    for (int half = 0; half < (has_hi ? 2 : 1); ++half) {
+      const size_t row = (size_t)h * (P.n >> 6) + qb0 + half;
+      const int cnt = P.idx.bs_count[row];
+      const int* bl = P.idx.bs_blk + row * P.idx.kb_cap;
+      uint32_t* dst = half ? hi_bits : lo_bits;
+      for (int i = tid; i < cnt; i += kThreads) {
+        int kb = bl[i];
+        if (kb >= 0 && kb <= qb0 + half) atomicOr(&dst[kb >> 5], 1u << (kb & 31));
+      }
+    }
+  }
+  __syncthreads();
+  if (pattern != RS_BLOCK_SPARSE) {
+    for (int wd = tid; wd < nb_words; wd += kThreads) {
+      uint32_t lo = 0, hi = 0;
+      if (pattern == RS_DENSE) {
+        lo = range_mask(0, qb0, wd);
+        hi = range_mask(0, qb0 + 1, wd);
+      } else if (pattern == RS_A_SHAPE) {
+        const int n_sink = cand.b0, win = cand.b1;
+        const uint32_t sink0 = (n_sink > 0) ? range_mask(0, min(qb0, (n_sink - 1) >> 6), wd) : 0u;
+        const uint32_t sink1 = (n_sink > 0) ? range_mask(0, min(qb0 + 1, (n_sink - 1) >> 6), wd) : 0u;
+        lo = sink0 | range_mask(max(0, i0 - win + 1) >> 6, qb0, wd);
+        hi = sink1 | range_mask(max(0, i0 + 64 - win + 1) >> 6, qb0 + 1, wd);
+      } else {   // vertical-slash: block kb is wanted by query block qb when (qb - kb) is in D
+        for (int b = 0; b < 32; ++b) {
+          const int kb = 32 * wd + b;
+          const int d0 = qb0 - kb, d1 = qb0 + 1 - kb;
+          if (d0 >= 0 && ((d_bits[d0 >> 5] >> (d0 & 31)) & 1u)) lo |= 1u << b;
+          if (d1 >= 0 && ((d_bits[d1 >> 5] >> (d1 & 31)) & 1u)) hi |= 1u << b;
+        }
+      }
+      lo_bits[wd] = lo;
+      hi_bits[wd] = has_hi ? hi : 0u;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int acc = 0;
+    for (int wd = 0; wd < nb_words; ++wd) { wprefix[wd] = acc; acc += __popc(lo_bits[wd] | hi_bits[wd]); }
+    misc[2] = acc;
+    int nv = 0;
+    if (pattern == RS_VERTICAL_SLASH && n_vcols > 0) {   // verticals with j <= last valid row are a prefix
+      const int* vc = P.idx.vs_cols + (size_t)vs_slot * P.idx.kv_cap;
+      const int i_last = i0 + rows_valid - 1;
+      int lo = 0, hi = n_vcols;
+      while (lo < hi) { int mid = (lo + hi) >> 1; if (vc[mid] <= i_last) lo = mid + 1; else hi = mid; }
+      nv = (lo + kChunk - 1) / kChunk;
+    }
+    misc[3] = nv;
+  }
+  __syncthreads();
+  for (int wd = tid; wd < nb_words; wd += kThreads) {
+    uint32_t lo = lo_bits[wd], hi = hi_bits[wd], any = lo | hi;
+    int at = wprefix[wd];
+    while (any) {
+      const int b = __ffs(any) - 1;
+      any &= any - 1;
+      const int kb = 32 * wd + b;
+      uint32_t e = (uint32_t)kb;
+      if ((lo >> b) & 1u) e |= F_LO;
+      if ((hi >> b) & 1u) e |= F_HI;
+      if (kb >= qb0) e |= F_CAUSAL;
+      if (pattern == RS_A_SHAPE) {
+        const bool in_window = kb * 64 >= i0 + kTileM - cand.b1;
+        const bool in_sink = (kb + 1) * 64 <= cand.b0;
+        if (!in_window && !in_sink) e |= F_EDGE;
+      }
+      list[at++] = (uint16_t)e;
+    }
+  }
+  __syncthreads();
+  const int n_block = misc[2], n_vert = misc[3];
+  const int n_chunks = n_block + n_vert;
+  const int n_pairs = (n_chunks + 1) >> 1;
+
+  // =========================================================================================== roles
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------------------------------------------ TMA producer
+      bool ok = true;
+      for (int t = 0; t < n_pairs && ok; ++t) {
+        const int nch = min(2, n_chunks - 2 * t);
+        const uint32_t ph = (uint32_t)(t & 1);
+        ok = mbar_wait(bar_ke, ph ^ 1u, abort_flag);
+        if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, 1); break; }
+        mbar_arrive_expect_tx(bar_kf, (uint32_t)nch * 16384u);
+        for (int c = 0; c < nch; ++c) {
+          const int ch = 2 * t + c;
+          const uint32_t dst = base + SmemLayout::k + (uint32_t)c * 8192u;
+          if (ch < n_block) {
+            const int row = g * P.n + (int)(list[ch] & 0xfffu) * kChunk;
+            tma_load_2d(dst, &tmK, bar_kf, 0, row);
+            tma_load_2d(dst + 16384, &tmK, bar_kf, 64, row);
+          } else {
+            const int row = vs_slot * P.kv_pad + (ch - n_block) * kChunk;
+            tma_load_2d(dst, &tmKp, bar_kf, 0, row);
+            tma_load_2d(dst + 16384, &tmKp, bar_kf, 64, row);
+          }
+        }
+        ok = mbar_wait(bar_ve, ph ^ 1u, abort_flag);
+        if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, 2); break; }
+        mbar_arrive_expect_tx(bar_vf, (uint32_t)nch * 16384u);
+        for (int c = 0; c < nch; ++c) {
+          const int ch = 2 * t + c;
+          const uint32_t dst = base + SmemLayout::v + (uint32_t)c * 8192u;
+          if (ch < n_block) {
+            const int row = g * P.n + (int)(list[ch] & 0xfffu) * kChunk;
+            tma_load_2d(dst, &tmV, bar_vf, 0, row);
+            tma_load_2d(dst + 16384, &tmV, bar_vf, 64, row);
+          } else {
+            const int row = vs_slot * P.kv_pad + (ch - n_block) * kChunk;
+            tma_load_2d(dst, &tmVp, bar_vf, 0, row);
+            tma_load_2d(dst + 16384, &tmVp, bar_vf, 64, row);
+          }
+        }
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ------------------------------------------------------------------ MMA issuer
+      const uint32_t d_s = tmem + kColS, d_o = tmem + kColO;
+      const uint64_t qdesc = umma_smem_desc(base + SmemLayout::q, 16, 1024);
+      const uint64_t kdesc = umma_smem_desc(base + SmemLayout::k, 16, 1024);
+      const uint64_t vdesc = umma_smem_desc(base + SmemLayout::v, 16384, 1024);
+      auto issue_qk = [&](int nch) {
+        const uint32_t idesc = umma_idesc_bf16(128, 64 * nch, 0, 0);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t off = (uint64_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+          umma_ss(d_s, qdesc + off, kdesc + off, idesc, kk > 0 ? 1u : 0u);
+        }
+      };
+      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      int site = 3;
+      for (int t = 0; t < n_pairs && ok; ++t) {
+        const int nch = min(2, n_chunks - 2 * t);
+        const uint32_t ph = (uint32_t)(t & 1);
+        if (t == 0) {
+          ok = mbar_wait(bar_kf, 0, abort_flag); site = 4;
+          if (!ok) break;
+          tc_fence_after();
+          issue_qk(nch);
+          umma_commit(bar_s);
+          umma_commit(bar_ke);
+        }
+        ok = mbar_wait(bar_p, ph, abort_flag); site = 5;
+        if (!ok) break;
+        ok = mbar_wait(bar_vf, ph, abort_flag); site = 6;
+        if (!ok) break;
+        tc_fence_after();
+        {
+          const uint32_t idesc = umma_idesc_bf16(128, 128, 0, 1);
+          for (int kk = 0; kk < 4 * nch; ++kk) {   // 16 keys per step: P columns advance by 8, V rows by 16
+            umma_ts(d_o, d_s + 8u * (uint32_t)kk, vdesc + (uint64_t)((kk * 2048) >> 4), idesc,
+                    (t > 0 || kk > 0) ? 1u : 0u);
+          }
+        }
+        umma_commit(bar_ve);
+        if (t + 1 < n_pairs) {
+          const int nch2 = min(2, n_chunks - 2 * (t + 1));
+          ok = mbar_wait(bar_kf, ph ^ 1u, abort_flag); site = 7;
+          if (!ok) break;
+          tc_fence_after();
+          issue_qk(nch2);
+          umma_commit(bar_s);
+          umma_commit(bar_ke);
+        } else {
+          umma_commit(bar_o);
+        }
+      }
+      if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, site); *abort_flag = 1; }
+    }
+  } else {
+    // -------------------------------------------------------------------- softmax / correction / epilogue
+    const int quad = warp & 3;
+    const int r = quad * 32 + lane;            // row of the tile = TMEM lane
+    const int i = i0 + r;                      // global query row
+    const int half = r >> 6;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t t_s = tmem + lane_addr + kColS, t_o = tmem + lane_addr + kColO;
+    const float sl2 = P.scale_log2e;
+    const float NEG_INF = -INFINITY;
+    float m_run = NEG_INF, l_run = 0.f;
+    const int* vcols = P.idx.vs_cols + (size_t)vs_slot * P.idx.kv_cap;
+    bool ok = true;
+    uint32_t v[32];
+
+    for (int t = 0; t < n_pairs; ++t) {
+      const int nch = min(2, n_chunks - 2 * t);
+      ok = mbar_wait(bar_s, (uint32_t)(t & 1), abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      // pass 1: masks (written back to TMEM) and the tile's row maximum
+      float m_tile = NEG_INF;
+      for (int c4 = 0; c4 < 2 * nch; ++c4) {
+        const int ch = 2 * t + (c4 >> 1);
+        const int cb = (c4 & 1) * 32;
+        tmem_ld32(t_s + (uint32_t)c4 * 32u, v);
+        tc_wait_ld();
+        bool masked = false;
+        if (ch < n_block) {
+          const uint32_t e = list[ch];
+          const bool half_ok = (e & (half ? F_HI : F_LO)) != 0;
+          if (!half_ok) {
+            masked = true;
+#pragma unroll
+            for (int x = 0; x < 32; ++x) v[x] = __float_as_uint(NEG_INF);
+          } else if (e & (F_CAUSAL | F_EDGE)) {
+            masked = true;
+            const int j0 = (int)(e & 0xfffu) * kChunk + cb;
+            const bool edge = (e & F_EDGE) != 0;
+#pragma unroll
+            for (int x = 0; x < 32; ++x) {
+              const int j = j0 + x;
+              bool keep = j <= i;
+              if (edge) keep = keep && (j < cand.b0 || i - j < cand.b1);
+              if (!keep) v[x] = __float_as_uint(NEG_INF);
+            }
+          }
+        } else {
+          masked = true;
+          const int vbase = (ch - n_block) * kChunk + cb;
+          const int qb_i = i >> 6;
+#pragma unroll
+          for (int x = 0; x < 32; ++x) {
+            const int vi = vbase + x;
+            bool keep = false;
+            if (vi < n_vcols) {
+              const int j = __ldg(vcols + vi);
+              if (j <= i) {
+                const int dlt = qb_i - (j >> 6);
+                keep = !((d_bits[dlt >> 5] >> (dlt & 31)) & 1u);   // not already covered by a block diagonal
+              }
+            }
+            if (!keep) v[x] = __float_as_uint(NEG_INF);
+          }
+        }
+        if (masked) {
+          tmem_st32(t_s + (uint32_t)c4 * 32u, v);
+        }
+#pragma unroll
+        for (int x = 0; x < 32; ++x) m_tile = fmaxf(m_tile, __uint_as_float(v[x]));
+      }
+      tc_wait_st();
+      m_tile *= sl2;
+      const float m_new = fmaxf(m_run, m_tile);
+      // lazy rescale: only when some row of the warp moved its maximum by more than 2^8
+      const bool need = m_new > m_run + 8.0f;
+      if (__any_sync(0xffffffffu, need)) {
+        const float alpha = (m_new == NEG_INF) ? 1.0f : fast_exp2(m_run - m_new);
+        l_run *= alpha;
+        m_run = m_new;
+        if (t > 0) {
+#pragma unroll 1
+          for (int c4 = 0; c4 < 4; ++c4) {
+            tmem_ld32(t_o + (uint32_t)c4 * 32u, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int x = 0; x < 32; ++x) v[x] = __float_as_uint(__uint_as_float(v[x]) * alpha);
+            tmem_st32(t_o + (uint32_t)c4 * 32u, v);
+          }
+          tc_wait_st();
+        }
+      }
+      const float m_use = (m_run == NEG_INF) ? 0.f : m_run;
+      // pass 2: P = exp2(S * scale*log2e - m), row sum, bf16 pairs written over the start of S
+      for (int c4 = 0; c4 < 2 * nch; ++c4) {
+        tmem_ld32(t_s + (uint32_t)c4 * 32u, v);
+        tc_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int x = 0; x < 16; ++x) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * x]), sl2, -m_use));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * x + 1]), sl2, -m_use));
+          l_run += p0 + p1;
+          pk[x] = pack_bf16x2(p0, p1);
+        }
+        tmem_st16(t_s + (uint32_t)c4 * 16u, pk);
+      }
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_p);
+    }
+
+    if (ok) ok = mbar_wait(bar_o, 0, abort_flag);
+    if (ok) {
+      tc_fence_after();
+      const float inv = (l_run > 0.f) ? 1.0f / l_run : 0.f;
+      const bool valid = r < rows_valid;
+      float ss = 0.f;
+      const size_t orow = ((size_t)h * P.n + (size_t)i) * RS_HEAD_DIM;
+#pragma unroll 1
+      for (int c4 = 0; c4 < 4; ++c4) {
+        tmem_ld32(t_o + (uint32_t)c4 * 32u, v);
+        tc_wait_ld();
+        float f[32];
+#pragma unroll
+        for (int x = 0; x < 32; ++x) { f[x] = __uint_as_float(v[x]) * inv; ss = fmaf(f[x], f[x], ss); }
+        if (valid) {
+          if (P.o_f32) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(P.O) + orow + c4 * 32);
+#pragma unroll
+            for (int x = 0; x < 8; ++x) dst[x] = make_float4(f[4 * x], f[4 * x + 1], f[4 * x + 2], f[4 * x + 3]);
+          } else {
+            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(P.O) + orow + c4 * 32);
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+              dst[x] = make_uint4(pack_bf16x2(f[8 * x], f[8 * x + 1]), pack_bf16x2(f[8 * x + 2], f[8 * x + 3]),
+                                  pack_bf16x2(f[8 * x + 4], f[8 * x + 5]), pack_bf16x2(f[8 * x + 6], f[8 * x + 7]));
+          }
+        }
+      }
+      if (valid) {
+        const size_t ridx = (size_t)h * P.n + (size_t)i;
+        P.lse[ridx] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+        if (P.onorm != nullptr) P.onorm[ridx] = sqrtf(ss);
+      }
+    } else if (lane == 0 && quad == 0) {
+      rs_report(P.status, RS_ERR_TIMEOUT, 8);
+      *abort_flag = 1;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && P.counters != nullptr) {
+    atomicAdd(&P.counters[0], (unsigned long long)n_chunks);
+    atomicAdd(&P.counters[1], 1ull);
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kTmemCols);
+  }
+}
+
+// -------------------------------------------------------------------------------------------- work list
+// One thread per (item, tile): estimated number of 64-key chunks, used only to order the launch (heavy first).
+__global__ void rs_attn_cost_kernel(AttnParams P, int n_work, int* cost, int2* items) {
+  const int wid = blockIdx.x * blockDim.x + threadIdx.x;
+  if (wid >= n_work) return;
+  const int h = wid / P.tiles_per_head;
+  const int tt = wid - h * P.tiles_per_head;
+  int s = 0;
+  while (s + 1 < P.n_seg && tt >= P.tile_base[s + 1]) ++s;
+  const int tile = tt - P.tile_base[s];
+  const int item = s * P.Hq + h;
+  const int q0 = P.seg_bounds[s], q1 = P.seg_bounds[s + 1];
+  const int i0 = q0 + tile * kTileM;
+  const int rows_valid = min(kTileM, q1 - i0);
+  const int qb0 = i0 >> 6;
+  const int qb_last = rows_valid > kChunk ? qb0 + 1 : qb0;
+  const rs_candidate cand = (P.choice != nullptr) ? P.lib[P.choice[item]] : rs_candidate{RS_DENSE, 0, 0, 0};
+  int c = qb_last + 1;
+  if (cand.pattern == RS_A_SHAPE) {
+    c = min(qb_last + 1, (cand.b0 + 63) / 64 + (cand.b1 + 63) / 64 + 2);
+  } else if (cand.pattern == RS_VERTICAL_SLASH) {
+    const int* cnt = P.idx.vs_count + 4 * item;
+    const int* dl = P.idx.vs_diag + (size_t)item * P.idx.nd_cap;
+    int lo = 0, hi = cnt[2];
+    while (lo < hi) { int mid = (lo + hi) >> 1; if (dl[mid] <= qb_last) lo = mid + 1; else hi = mid; }
+    c = min(qb_last + 1, lo + 1) + (cnt[0] + 63) / 64;
+  } else if (cand.pattern == RS_BLOCK_SPARSE) {
+    const size_t row = (size_t)h * (P.n >> 6) + qb0;
+    c = P.idx.bs_count[row] + (qb_last > qb0 ? P.idx.bs_count[row + 1] : 0);
+  }
+  cost[wid] = c;
+  items[wid] = make_int2(item, tile);
+}
+
+// Counting sort by cost, descending (single block).
+__global__ void rs_attn_order_kernel(int n_work, int n_bins, const int* cost, const int2* items, int2* order) {
+  extern __shared__ int hist[];
+  for (int i = threadIdx.x; i <= n_bins; i += blockDim.x) hist[i] = 0;
+  __syncthreads();
+  for (int i = threadIdx.x; i < n_work; i += blockDim.x) atomicAdd(&hist[min(cost[i], n_bins - 1)], 1);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int acc = 0;
+    for (int b = n_bins - 1; b >= 0; --b) { int c = hist[b]; hist[b] = acc; acc += c; }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < n_work; i += blockDim.x) {
+    const int pos = atomicAdd(&hist[min(cost[i], n_bins - 1)], 1);
+    order[pos] = items[i];
+  }
+}
+
+// Gathers the vertical key / value rows of every vertical-slash item into a contiguous, zero-padded buffer.
+__global__ void rs_pack_vertical_kernel(AttnParams P, const __nv_bfloat16* K, const __nv_bfloat16* V,
+                                        __nv_bfloat16* Kp, __nv_bfloat16* Vp) {
+  const int item = blockIdx.y;
+  if (P.choice == nullptr || P.lib[P.choice[item]].pattern != RS_VERTICAL_SLASH) return;
+  const int h = item % P.Hq, g = h / P.group;
+  const int n_cols = P.idx.vs_count[4 * item];
+  const int row = blockIdx.x * (blockDim.x >> 4) + (threadIdx.x >> 4);   // 16 threads move one 256-byte row
+  if (row >= P.kv_pad) return;
+  const int l16 = threadIdx.x & 15;
+  uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
+  if (row < n_cols) {
+    const int j = P.idx.vs_cols[(size_t)item * P.idx.kv_cap + row];
+    const size_t src = ((size_t)g * P.n + (size_t)j) * RS_HEAD_DIM;
+    kv = reinterpret_cast<const uint4*>(K + src)[l16];
+    vv = reinterpret_cast<const uint4*>(V + src)[l16];
+  }
+  const size_t dst = ((size_t)item * P.kv_pad + row) * RS_HEAD_DIM;
+  reinterpret_cast<uint4*>(Kp + dst)[l16] = kv;
+  reinterpret_cast<uint4*>(Vp + dst)[l16] = vv;
+}
+
+size_t attn_smem_bytes(int n) {
+  const int list_cap = (n >> 6) + 64;
+  return 1024 + SmemLayout::end_tiles + ((list_cap * 2 + 15) & ~15) + 3 * 128 * 4 + 132 * 4 + 8 * 8 + 64;
+}
+
+struct WsPlan { size_t cost, items, order, kpack, vpack, total; int n_work, kv_pad, n_items; };
+
+WsPlan plan_ws(const rs_problem* p, int max_kv) {
+  WsPlan w{};
+  int tiles = 0;
+  for (int s = 0; s < p->n_segments; ++s) tiles += (p->seg_bounds[s + 1] - p->seg_bounds[s] + kTileM - 1) / kTileM;
+  w.n_work = tiles * p->n_q_heads;
+  w.n_items = p->n_segments * p->n_q_heads;
+  w.kv_pad = (int)rs_align_up((size_t)(max_kv > 0 ? max_kv : 0), 64);
+  size_t off = 0;
+  w.cost = off;  off += rs_align_up((size_t)w.n_work * 4, 256);
+  w.items = off; off += rs_align_up((size_t)w.n_work * 8, 256);
+  w.order = off; off += rs_align_up((size_t)w.n_work * 8, 256);
+  const size_t pack = rs_align_up((size_t)w.n_items * (size_t)(w.kv_pad > 0 ? w.kv_pad : 64) * RS_HEAD_DIM * 2, 256);
+  w.kpack = off; off += pack;
+  w.vpack = off; off += pack;
+  w.total = off;
+  return w;
+}
+
+int launch_attn(const rs_problem* p, const void* Q, const void* K, const void* V, const rs_candidate* lib,
+                int n_cand, const rs_index_set* idx, const int32_t* choice, void* O, int o_dtype, float* lse,
+                float* onorm, uint64_t* counters, void* ws, size_t ws_bytes, int32_t* status, void* stream_) {
+  int rc = rs_check_problem(p);
+  if (rc != RS_OK) return rc;
+  if (!Q || !K || !V || !O || !lse || !ws) return RS_ERR_INVALID_ARG;
+  if (n_cand < 0 || n_cand > RS_MAX_CANDIDATES) return RS_ERR_INVALID_ARG;
+  if (choice != nullptr && (lib == nullptr || idx == nullptr || n_cand == 0)) return RS_ERR_INVALID_ARG;
+  rc = rs_check_device();
+  if (rc != RS_OK) return rc;
+  cudaStream_t stream = (cudaStream_t)stream_;
+
+  int max_kv = 0;
+  bool any_vs = false;
+  for (int c = 0; c < n_cand; ++c) {
+    if (lib[c].pattern == RS_VERTICAL_SLASH) { any_vs = true; if (lib[c].b0 > max_kv) max_kv = lib[c].b0; }
+    if (lib[c].pattern == RS_A_SHAPE && (lib[c].b1 < 1 || lib[c].b0 < 0)) return RS_ERR_INVALID_ARG;
+    if (lib[c].pattern < 0 || lib[c].pattern > 3) return RS_ERR_INVALID_ARG;
+  }
+  if (choice != nullptr && any_vs) {
+    if (idx->kv_cap < max_kv || idx->n_vs_slots < p->n_segments * p->n_q_heads) return RS_ERR_INVALID_ARG;
+  }
+  const WsPlan w = plan_ws(p, max_kv);
+  if (ws_bytes < w.total) return RS_ERR_WORKSPACE_TOO_SMALL;
+  if (((uintptr_t)ws & 255) != 0) return RS_ERR_INVALID_ARG;
+
+  AttnParams P{};
+  P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = p->n_q_heads / p->n_kv_heads;
+  P.n_seg = p->n_segments; P.n_cand = n_cand;
+  int tiles = 0;
+  for (int s = 0; s <= p->n_segments; ++s) {
+    P.seg_bounds[s] = p->seg_bounds[s];
+    P.tile_base[s] = tiles;
+    if (s < p->n_segments) tiles += (p->seg_bounds[s + 1] - p->seg_bounds[s] + kTileM - 1) / kTileM;
+  }
+  P.tiles_per_head = tiles;
+  for (int c = 0; c < n_cand; ++c) P.lib[c] = lib[c];
+  P.choice = choice;
+  if (idx) P.idx = *idx;
+  P.kv_pad = w.kv_pad > 0 ? w.kv_pad : 64;
+  uint8_t* wsb = reinterpret_cast<uint8_t*>(ws);
+  P.order = reinterpret_cast<const int2*>(wsb + w.order);
+  P.O = O; P.o_f32 = o_dtype; P.lse = lse; P.onorm = onorm;
+  P.counters = reinterpret_cast<unsigned long long*>(counters);
+  P.status = status;
+  P.scale_log2e = (float)(1.4426950408889634 / sqrt((double)RS_HEAD_DIM));
+
+  __nv_bfloat16* Kp = reinterpret_cast<__nv_bfloat16*>(wsb + w.kpack);
+  __nv_bfloat16* Vp = reinterpret_cast<__nv_bfloat16*>(wsb + w.vpack);
+  CUtensorMap tmQ, tmK, tmV, tmKp, tmVp;
+  const uint64_t pack_rows = (uint64_t)w.n_items * (uint64_t)P.kv_pad;
+  if (rs_make_tmap_bf16_2d(&tmQ, Q, (uint64_t)P.Hq * P.n, RS_HEAD_DIM, kTileM, 64) ||
+      rs_make_tmap_bf16_2d(&tmK, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kChunk, 64) ||
+      rs_make_tmap_bf16_2d(&tmV, V, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kChunk, 64) ||
+      rs_make_tmap_bf16_2d(&tmKp, Kp, pack_rows, RS_HEAD_DIM, kChunk, 64) ||
+      rs_make_tmap_bf16_2d(&tmVp, Vp, pack_rows, RS_HEAD_DIM, kChunk, 64))
+    return RS_ERR_CUDA;
+
+  const int n_work = w.n_work;
+  int* cost = reinterpret_cast<int*>(wsb + w.cost);
+  int2* items = reinterpret_cast<int2*>(wsb + w.items);
+  int2* order = reinterpret_cast<int2*>(wsb + w.order);
+  rs_attn_cost_kernel<<<(n_work + 255) / 256, 256, 0, stream>>>(P, n_work, cost, items);
+  const int n_bins = (P.n >> 6) + 66;
+  rs_attn_order_kernel<<<1, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work, n_bins, cost, items, order);
+  if (choice != nullptr && any_vs) {
+    dim3 grid((P.kv_pad + 15) / 16, w.n_items);
+    rs_pack_vertical_kernel<<<grid, 256, 0, stream>>>(P, reinterpret_cast<const __nv_bfloat16*>(K),
+                                                      reinterpret_cast<const __nv_bfloat16*>(V), Kp, Vp);
+  }
+  const size_t smem = attn_smem_bytes(P.n);
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(rs_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024) != cudaSuccess)
+      return RS_ERR_CUDA;
+    attr_set = true;
+  }
+  rs_attn_kernel<<<n_work, kThreads, smem, stream>>>(tmQ, tmK, tmV, tmKp, tmVp, P);
+  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+}
+
+}  // namespace
+
+size_t rs_attn_workspace_bytes(const rs_problem* p, int max_kv) { return plan_ws(p, max_kv).total; }
+
+extern "C" int rs_sparse_prefill_attn(const rs_problem* p, const void* Q, const void* K, const void* V,
+                                      const rs_candidate* lib, int n_cand, const rs_index_set* idx,
+                                      const int32_t* choice, void* O, int o_dtype, float* lse_sel, float* onorm,
+                                      uint64_t* counters, void* ws, size_t ws_bytes, int32_t* status, void* stream) {
+  if (!lib || !idx || !choice || n_cand <= 0) return RS_ERR_INVALID_ARG;
+  return launch_attn(p, Q, K, V, lib, n_cand, idx, choice, O, o_dtype, lse_sel, onorm, counters, ws, ws_bytes, status,
+                     stream);
+}
+
+extern "C" int rs_dense_prefill_attn(const rs_problem* p, const void* Q, const void* K, const void* V, void* O,
+                                     int o_dtype, float* lse, float* onorm, uint64_t* counters, void* ws,
+                                     size_t ws_bytes, int32_t* status, void* stream) {
+  return launch_attn(p, Q, K, V, nullptr, 0, nullptr, nullptr, O, o_dtype, lse, onorm, counters, ws, ws_bytes, status,
+                     stream);
+}
