@@ -122,11 +122,11 @@ def mask_rows(ix: IndexSet, rows: np.ndarray, n_keys: int) -> np.ndarray:
         col = np.zeros(n_keys, dtype=bool)
         col[ix.V[ix.V < n_keys]] = True
         if c.strict:
-            off = np.zeros(max(n_keys, int(rows.max()) + 1) + 1, dtype=bool)
+            off = np.zeros(max(n_keys, int(rows.max()) + 1, int(ix.S.max()) + 1) + 1, dtype=bool)
             off[ix.S] = True
             diff = i - j
             return col[None, :] | ((diff >= 0) & off[np.clip(diff, 0, len(off) - 1)])
-        nb = max(n_keys, int(rows.max()) + 1) // B + 2
+        nb = max(max(n_keys, int(rows.max()) + 1) // B, int(ix.D.max())) + 2
         dl = np.zeros(nb, dtype=bool)
         dl[ix.D] = True
         delta = i // B - j // B
