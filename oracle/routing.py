@@ -12,7 +12,9 @@ build's reading (parity unpinned beyond the invariants the tests check).
 
 Arithmetic: coverage arrives as exact fixed-point integers, costs are integers (FLOPs or nanoseconds),
 so totals are exact; risks are IEEE doubles computed as (1 - m_hat) + alpha * u with each operation
-rounded separately; ratios are compared by cross-multiplication.
+rounded separately; a substitution's ratio is the single IEEE division dR / dT, and substitutions are
+ordered by the tuple (ratio, larger saving first, lower item, lower candidate), a total order, so the
+chosen substitution does not depend on the order in which candidates are examined.
 """
 from __future__ import annotations
 
@@ -77,7 +79,7 @@ def greedy_solve(R: np.ndarray, cost: np.ndarray, dense_c: int, budget: int, t_p
     total = int(t_probe) + sum(int(cost[it, dense_c]) for it in range(n_items))
     feasible = 1
     while total > budget:
-        best = None                                   # (dR, dT, item, cand)
+        best = None                                   # (ratio, -dT, item, cand): smallest tuple wins
         for it in range(n_items):
             cur = choice[it]
             for k in range(n_cand):
@@ -85,19 +87,15 @@ def greedy_solve(R: np.ndarray, cost: np.ndarray, dense_c: int, budget: int, t_p
                 if dT <= 0:
                     continue
                 dR = float(R[it, k]) - float(R[it, cur])
-                if best is None:
-                    best = (dR, dT, it, k)
-                    continue
-                lhs = dR * float(best[1])             # dR / dT < best_dR / best_dT  <=>  dR * best_dT < best_dR * dT
-                rhs = best[0] * float(dT)
-                if lhs < rhs or (lhs == rhs and dT > best[1]):
-                    best = (dR, dT, it, k)
+                key = (dR / float(dT), -dT, it, k)    # one IEEE division; ties: larger saving, lower item, lower k
+                if best is None or key < best:
+                    best = key
         if best is None:
             feasible = 0
             break
-        _, dT, it, k = best
+        _, neg_dT, it, k = best
         choice[it] = k
-        total -= dT
+        total += neg_dT
     return choice, total, feasible
 
 

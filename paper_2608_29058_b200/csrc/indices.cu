@@ -1,0 +1,687 @@
+// Candidate index construction, coverage and pair counts (Section 3.1, 3.2; step 2 of the per-layer procedure).
+//
+// Everything that decides an index is integer arithmetic so that the result does not depend on the order of
+// evaluation: ranking keys are sum_g floor(mass_g * 2^32) (uint64), top-k is "key descending, index ascending"
+// found by an exact radix select (threshold key + quota of ties in index order) followed by an ordered
+// compaction, coverage is a sum of the same fixed-point values, and pair counts are closed forms.
+// Block-sparse scores are fp32 (fused pooled dot products accumulated k = 0..127 with fmaf, or an explicit
+// score matrix) compared through an order-preserving integer transform.
+#include "common.cuh"
+
+namespace {
+
+typedef unsigned long long u64;
+
+struct IdxParams {
+  int n, Hq, Hkv, group, n_seg, n_cand, nb;
+  int seg_bounds[RS_MAX_SEGMENTS + 1];
+  rs_candidate lib[RS_MAX_CANDIDATES];
+  const float* vert; const float* slash; const float* qpool; const float* kpool; const float* bscore;
+  const int32_t* choice;
+  rs_index_set out;
+  rs_cand_stats* stats;
+  u64* vblk;          // [n_items][4][nb] block sums of fx(vert)
+  float* bs_ws;       // [Hq][nb][nb] fused block scores (materialise mode)
+  int32_t* status;
+  float scale;
+};
+
+__device__ __forceinline__ u64 fx(float x) { return (u64)__float2ull_rz(x * 4294967296.0f); }
+
+__device__ __forceinline__ u64 line_key(const float* mass, int n, int j) {
+  return fx(mass[j]) + fx(mass[(size_t)n + j]) + fx(mass[2 * (size_t)n + j]) + fx(mass[3 * (size_t)n + j]);
+}
+
+__device__ __forceinline__ int seg_of_block(const IdxParams& P, int qb) {
+  int s = 0;
+  while (s + 1 < P.n_seg && qb * 64 >= P.seg_bounds[s + 1]) ++s;
+  return s;
+}
+
+// job -> (item, candidate, slot); returns false when this block has nothing to do
+__device__ __forceinline__ bool job_of(const IdxParams& P, int job, int& item, int& c, int& slot) {
+  item = job / P.n_cand;
+  c = job - item * P.n_cand;
+  if (P.choice != nullptr) {
+    if (P.choice[item] != c) return false;
+    slot = item;
+  } else {
+    slot = job;
+  }
+  return true;
+}
+
+// ------------------------------------------------------------------------------------------ block sums of fx(vert)
+__global__ void rs_vblk_kernel(IdxParams P) {
+  const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const int total = P.n_seg * P.Hq * RS_PROBE_GROUPS * P.nb;
+  if (warp_global >= total) return;
+  const int kb = warp_global % P.nb;
+  const int ig = warp_global / P.nb;            // item * 4 + g
+  const int item = ig >> 2;
+  const int s = item / P.Hq;
+  u64 acc = 0;
+  if (kb * 64 < P.seg_bounds[s + 1]) {
+    const float* src = P.vert + (size_t)ig * P.n + (size_t)kb * 64;
+    acc = fx(src[lane]) + fx(src[lane + 32]);
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  if (lane == 0) P.vblk[(size_t)ig * P.nb + kb] = acc;
+}
+
+// ------------------------------------------------------------------------------------------ exact top-k of a line list
+// grid = (2 lists, jobs).  list 0: vertical columns over [0, q1); list 1: slash offsets over [1, q1) plus offset 0.
+constexpr int kSelThreads = 1024;
+constexpr int kDigitBits = 13;
+constexpr int kBins = 1 << kDigitBits;
+
+__global__ void __launch_bounds__(kSelThreads)
+rs_vs_select_kernel(IdxParams P) {
+  __shared__ unsigned int hist[kBins];
+  __shared__ unsigned int wsum[32];
+  __shared__ u64 sh_prefix;
+  __shared__ unsigned int sh_k;
+  __shared__ unsigned int w_gt[32], w_eq[32];
+  int item, c, slot;
+  if (!job_of(P, blockIdx.y, item, c, slot)) return;
+  const rs_candidate cand = P.lib[c];
+  if (cand.pattern != RS_VERTICAL_SLASH) return;
+  const int list = blockIdx.x;
+  const int s = item / P.Hq;
+  const int q1 = P.seg_bounds[s + 1];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* mass = (list == 0 ? P.vert : P.slash) + (size_t)item * RS_PROBE_GROUPS * P.n;
+  const int first = (list == 0) ? 0 : 1;                 // first index of the domain
+  const int n_dom = q1 - first;
+  int k = (list == 0) ? min(cand.b0, q1) : (min(cand.b1, q1) - 1);
+  if (k < 0) k = 0;
+  if (k > n_dom) k = n_dom;
+  int32_t* out = (list == 0) ? (P.out.vs_cols + (size_t)slot * P.out.kv_cap) : (P.out.vs_offs + (size_t)slot * P.out.ks_cap);
+  const int cap = (list == 0) ? P.out.kv_cap : P.out.ks_cap;
+
+  u64 T = ~0ull;           // threshold key: everything above is taken, k_eq ties in index order
+  unsigned int k_eq = 0;
+  if (k > 0) {
+    if (tid == 0) { sh_prefix = 0; sh_k = (unsigned)k; }
+    for (int pass = 2; pass >= 0; --pass) {
+      for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
+      __syncthreads();
+      const u64 prefix = sh_prefix;
+      const int shift = pass * kDigitBits;
+      for (int base = 0; base < n_dom; base += kSelThreads) {
+        const int j = base + tid;
+        unsigned int digit = 0xffffffffu;
+        if (j < n_dom) {
+          const u64 key = line_key(mass, P.n, first + j);
+          if ((key >> (shift + kDigitBits)) == prefix) digit = (unsigned)((key >> shift) & (kBins - 1));
+        }
+        const unsigned int peers = __match_any_sync(0xffffffffu, digit);
+        if (digit != 0xffffffffu && lane == (__ffs(peers) - 1)) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+      }
+      __syncthreads();
+      // each thread owns 8 consecutive bins, highest bins first
+      const int b0 = kBins - 8 * (tid + 1);
+      unsigned int loc[8], lsum = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { loc[i] = hist[b0 + i]; lsum += loc[i]; }
+      unsigned int incl = lsum;           // inclusive scan over threads (thread 0 owns the top bins)
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int t = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += t;
+      }
+      if (lane == 31) wsum[warp] = incl;
+      __syncthreads();
+      unsigned int before = 0;
+      for (int w = 0; w < warp; ++w) before += wsum[w];
+      const unsigned int above = before + incl - lsum;    // entries in bins above this thread's bins
+      const unsigned int kk = sh_k;
+      __syncthreads();
+      if (above < kk && kk <= above + lsum) {
+        unsigned int acc = above;
+        for (int i = 7; i >= 0; --i) {
+          if (acc + loc[i] >= kk) {
+            sh_prefix = (prefix << kDigitBits) | (u64)(b0 + i);
+            sh_k = kk - acc;
+            break;
+          }
+          acc += loc[i];
+        }
+      }
+      __syncthreads();
+    }
+    T = sh_prefix;
+    k_eq = sh_k;
+  }
+
+  // ordered compaction: warp w walks the contiguous range [w * chunk, (w + 1) * chunk)
+  const int chunk = (((n_dom + 31) / 32) + 31) / 32 * 32;
+  const int lo = warp * chunk, hi = min(n_dom, lo + chunk);
+  unsigned int gt = 0, eq = 0;
+  for (int base = lo; base < hi; base += 32) {
+    const int j = base + lane;
+    u64 key = 0;
+    const bool in = j < hi;
+    if (in) key = line_key(mass, P.n, first + j);
+    gt += __popc(__ballot_sync(0xffffffffu, in && key > T));
+    eq += __popc(__ballot_sync(0xffffffffu, in && key == T));
+  }
+  if (lane == 0) { w_gt[warp] = gt; w_eq[warp] = eq; }
+  __syncthreads();
+  unsigned int gt_before = 0, eq_before = 0;
+  for (int w = 0; w < warp; ++w) { gt_before += w_gt[w]; eq_before += w_eq[w]; }
+  unsigned int pos = gt_before + min(k_eq, eq_before) + (list == 1 ? 1u : 0u);
+  unsigned int eq_run = eq_before;
+  const unsigned int lt_mask = (1u << lane) - 1u;
+  for (int base = lo; base < hi; base += 32) {
+    const int j = base + lane;
+    u64 key = 0;
+    const bool in = j < hi;
+    if (in) key = line_key(mass, P.n, first + j);
+    const bool is_eq = in && key == T;
+    const unsigned int beq = __ballot_sync(0xffffffffu, is_eq);
+    const bool take = in && (key > T || (is_eq && eq_run + __popc(beq & lt_mask) < k_eq));
+    const unsigned int bt = __ballot_sync(0xffffffffu, take);
+    if (take) {
+      const unsigned int p = pos + __popc(bt & lt_mask);
+      if ((int)p < cap) out[p] = first + j;
+    }
+    pos += __popc(bt);
+    eq_run += __popc(beq);
+  }
+  if (tid == 0) {
+    if (list == 1) { out[0] = 0; P.out.vs_count[4 * slot + 1] = k + 1; }
+    else P.out.vs_count[4 * slot + 0] = k;
+  }
+}
+
+// ------------------------------------------------------------------------------------------ pair counts (closed forms)
+__device__ __forceinline__ u64 pairs_dense(long long q0, long long q1) { return (u64)((q1 * (q1 + 1) - q0 * (q0 + 1)) / 2); }
+
+__device__ __forceinline__ u64 pairs_a_shape(long long q0, long long q1, long long cap) {
+  // sum_{i=q0}^{q1-1} min(i + 1, cap)
+  const long long m = min(q1, max(q0, cap));            // rows [q0, m) have i + 1 <= cap
+  u64 total = (u64)((m * (m + 1) - q0 * (q0 + 1)) / 2);
+  total += (u64)((q1 - m) * cap);
+  return total;
+}
+
+__device__ __forceinline__ u64 pairs_block_sparse(int qb_lo, int qb_hi, int k_b) {
+  u64 total = 0;
+  for (int qb = qb_lo; qb < qb_hi; ++qb) total += (u64)(min(k_b, qb + 1) - 1) * 4096ull + 2080ull;
+  return total;
+}
+
+// ------------------------------------------------------------------------------------------ vertical-slash: D, coverage, pairs
+__global__ void __launch_bounds__(256)
+rs_vs_finish_kernel(IdxParams P) {
+  __shared__ uint32_t dbits[128];
+  __shared__ int wpre[129];
+  __shared__ u64 cov[RS_PROBE_GROUPS];
+  __shared__ u64 extra_pairs;
+  int item, c, slot;
+  if (!job_of(P, blockIdx.x, item, c, slot)) return;
+  const rs_candidate cand = P.lib[c];
+  if (cand.pattern != RS_VERTICAL_SLASH) return;
+  const int s = item / P.Hq;
+  const int q0 = P.seg_bounds[s], q1 = P.seg_bounds[s + 1];
+  const int nbs = q1 >> 6, qb_lo = q0 >> 6, qb_star = nbs - 1;
+  const int tid = threadIdx.x;
+  const int n_cols = P.out.vs_count[4 * slot + 0], n_offs = P.out.vs_count[4 * slot + 1];
+  const int32_t* cols = P.out.vs_cols + (size_t)slot * P.out.kv_cap;
+  const int32_t* offs = P.out.vs_offs + (size_t)slot * P.out.ks_cap;
+  int32_t* diag = P.out.vs_diag + (size_t)slot * P.out.nd_cap;
+  for (int i = tid; i < 128; i += blockDim.x) dbits[i] = 0;
+  if (tid < RS_PROBE_GROUPS) cov[tid] = 0;
+  if (tid == 0) extra_pairs = 0;
+  __syncthreads();
+  for (int i = tid; i < n_offs; i += blockDim.x) {
+    const int o = offs[i];
+    const int d0 = o >> 6, d1 = (o + 63) >> 6;
+    if (d0 < nbs) atomicOr(&dbits[d0 >> 5], 1u << (d0 & 31));
+    if (d1 < nbs) atomicOr(&dbits[d1 >> 5], 1u << (d1 & 31));
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int acc = 0;
+    for (int w = 0; w < 128; ++w) { wpre[w] = acc; acc += __popc(dbits[w]); }
+    wpre[128] = acc;
+  }
+  __syncthreads();
+  const int n_diag = wpre[128];
+  if (tid < 128) {
+    uint32_t bits = dbits[tid];
+    int at = wpre[tid];
+    while (bits) {
+      const int b = __ffs(bits) - 1;
+      bits &= bits - 1;
+      if (at < P.out.nd_cap) diag[at] = tid * 32 + b;
+      ++at;
+    }
+  }
+  if (tid == 0) { P.out.vs_count[4 * slot + 2] = n_diag; P.out.vs_count[4 * slot + 3] = 0; }
+  if (P.stats == nullptr) return;
+
+  // coverage: block diagonals seen from the last query block + verticals outside them
+  const float* vert = P.vert + (size_t)item * RS_PROBE_GROUPS * P.n;
+  const u64* vblk = P.vblk + (size_t)item * RS_PROBE_GROUPS * P.nb;
+  u64 part[RS_PROBE_GROUPS] = {0, 0, 0, 0};
+  for (int kb = tid; kb < nbs; kb += blockDim.x) {
+    const int d = qb_star - kb;
+    if ((dbits[d >> 5] >> (d & 31)) & 1u) {
+#pragma unroll
+      for (int g = 0; g < RS_PROBE_GROUPS; ++g) part[g] += vblk[(size_t)g * P.nb + kb];
+    }
+  }
+  // pairs: verticals not covered by a block diagonal of their query block
+  u64 vp = 0;
+  const bool has0 = (dbits[0] & 1u) != 0;
+  for (int i = tid; i < n_cols; i += blockDim.x) {
+    const int j = cols[i];
+    const int kbj = j >> 6;
+    const int d = qb_star - kbj;
+    if (!((dbits[d >> 5] >> (d & 31)) & 1u)) {
+#pragma unroll
+      for (int g = 0; g < RS_PROBE_GROUPS; ++g) part[g] += fx(vert[(size_t)g * P.n + j]);
+    }
+    // query blocks qb in [max(kbj, qb_lo), nbs): delta = qb - kbj
+    if (kbj >= qb_lo && !has0) vp += (u64)((kbj + 1) * 64 - j);
+    const int d_lo = max(1, qb_lo - kbj), d_hi = qb_star - kbj;       // deltas >= 1 of the other query blocks
+    if (d_hi >= d_lo) {
+      int covered = 0;                                                 // |D intersect [d_lo, d_hi]|
+      const int w_lo = d_lo >> 5, w_hi = d_hi >> 5;
+      for (int w = w_lo; w <= w_hi; ++w) {
+        uint32_t bits = dbits[w];
+        if (w == w_lo) bits &= 0xffffffffu << (d_lo & 31);
+        if (w == w_hi) bits &= 0xffffffffu >> (31 - (d_hi & 31));
+        covered += __popc(bits);
+      }
+      vp += 64ull * (u64)(d_hi - d_lo + 1 - covered);
+    }
+  }
+#pragma unroll
+  for (int g = 0; g < RS_PROBE_GROUPS; ++g) if (part[g]) atomicAdd(&cov[g], part[g]);
+  if (vp) atomicAdd(&extra_pairs, vp);
+  __syncthreads();
+  if (tid == 0) {
+    u64 total = extra_pairs;
+    // block diagonals: delta >= 1 is used by every query block qb >= delta of the segment, delta 0 by all
+    for (int w = 0; w < 128; ++w) {
+      uint32_t bits = dbits[w];
+      while (bits) {
+        const int d = w * 32 + __ffs(bits) - 1;
+        bits &= bits - 1;
+        if (d == 0) total += (u64)(nbs - qb_lo) * 2080ull;
+        else if (nbs > max(qb_lo, d)) total += (u64)(nbs - max(qb_lo, d)) * 4096ull;
+      }
+    }
+    rs_cand_stats* st = P.stats + (size_t)item * P.n_cand + c;
+    for (int g = 0; g < RS_PROBE_GROUPS; ++g) st->cov_fx[g] = cov[g];
+    st->pairs = total;
+  }
+}
+
+// ------------------------------------------------------------------------------------------ A-shape and dense stats
+__global__ void __launch_bounds__(256)
+rs_simple_stats_kernel(IdxParams P) {
+  __shared__ u64 cov[RS_PROBE_GROUPS];
+  int item, c, slot;
+  if (!job_of(P, blockIdx.x, item, c, slot)) return;
+  if (P.stats == nullptr) return;
+  const rs_candidate cand = P.lib[c];
+  if (cand.pattern != RS_A_SHAPE && cand.pattern != RS_DENSE) return;
+  const int s = item / P.Hq;
+  const int q0 = P.seg_bounds[s], q1 = P.seg_bounds[s + 1];
+  rs_cand_stats* st = P.stats + (size_t)item * P.n_cand + c;
+  const int tid = threadIdx.x;
+  if (cand.pattern == RS_DENSE) {
+    if (tid == 0) {
+      for (int g = 0; g < RS_PROBE_GROUPS; ++g) st->cov_fx[g] = 16ull << 32;
+      st->pairs = pairs_dense(q0, q1);
+    }
+    return;
+  }
+  if (tid < RS_PROBE_GROUPS) cov[tid] = 0;
+  __syncthreads();
+  const float* vert = P.vert + (size_t)item * RS_PROBE_GROUPS * P.n;
+  const float* slash = P.slash + (size_t)item * RS_PROBE_GROUPS * P.n;
+  const int n_sink = cand.b0, win = cand.b1;
+  const bool window_covers_all = win >= q1;
+  const int n_off = window_covers_all ? q1 : win;
+  const int n_col = window_covers_all ? 0 : min(n_sink, q1);
+  u64 part[RS_PROBE_GROUPS] = {0, 0, 0, 0};
+  for (int o = tid; o < n_off; o += blockDim.x)
+#pragma unroll
+    for (int g = 0; g < RS_PROBE_GROUPS; ++g) part[g] += fx(slash[(size_t)g * P.n + o]);
+  for (int j = tid; j < n_col; j += blockDim.x)
+#pragma unroll
+    for (int g = 0; g < RS_PROBE_GROUPS; ++g) part[g] += fx(vert[(size_t)g * P.n + j]);
+#pragma unroll
+  for (int g = 0; g < RS_PROBE_GROUPS; ++g) if (part[g]) atomicAdd(&cov[g], part[g]);
+  __syncthreads();
+  if (tid == 0) {
+    for (int g = 0; g < RS_PROBE_GROUPS; ++g) st->cov_fx[g] = cov[g];
+    st->pairs = pairs_a_shape(q0, q1, (long long)n_sink + win);
+  }
+}
+
+// ------------------------------------------------------------------------------------------ block-sparse row selection
+__device__ __forceinline__ uint32_t f32_order_key(float x) {
+  if (x == 0.f) x = 0.f;                     // -0 and +0 compare equal
+  const uint32_t u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Selects the `take` largest of score[0, m) (ties -> lower index) plus the diagonal block `qb`; writes them
+// ascending to out[] and returns the count.  All 256 threads of the block call it; scores live in shared memory.
+__device__ int select_row(const float* score, int m, int take, int qb, int32_t* out, int cap, uint32_t* hist /*256*/,
+                          uint32_t* sh /*8*/, unsigned int* wcnt /*16*/) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t T = 0xffffffffu, k_eq = 0;
+  take = min(take, m);
+  if (take > 0) {
+    if (tid == 0) { sh[0] = 0; sh[1] = (uint32_t)take; }
+    for (int pass = 3; pass >= 0; --pass) {
+      hist[tid] = 0;
+      __syncthreads();
+      const uint32_t prefix = sh[0];
+      const int shift = pass * 8;
+      for (int i = tid; i < m; i += 256) {
+        const uint32_t key = f32_order_key(score[i]);
+        if (pass == 3 || (key >> (shift + 8)) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        uint32_t kk = sh[1], acc = 0;
+        for (int b = 255; b >= 0; --b) {
+          if (acc + hist[b] >= kk) { sh[0] = (prefix << 8) | (uint32_t)b; sh[1] = kk - acc; break; }
+          acc += hist[b];
+        }
+      }
+      __syncthreads();
+    }
+    T = sh[0];
+    k_eq = sh[1];
+  }
+  __syncthreads();
+  // ordered compaction over [0, m): 8 warps, contiguous chunks
+  const int chunk = (((m + 7) / 8) + 31) / 32 * 32;
+  const int lo = warp * chunk, hi = min(m, lo + chunk);
+  unsigned int gt = 0, eq = 0;
+  for (int base = lo; base < hi; base += 32) {
+    const int i = base + lane;
+    const bool in = i < hi;
+    const uint32_t key = in ? f32_order_key(score[i]) : 0u;
+    gt += __popc(__ballot_sync(0xffffffffu, in && take > 0 && key > T));
+    eq += __popc(__ballot_sync(0xffffffffu, in && take > 0 && key == T));
+  }
+  if (lane == 0) { wcnt[warp] = gt; wcnt[8 + warp] = eq; }
+  __syncthreads();
+  unsigned int gt_before = 0, eq_before = 0;
+  for (int w = 0; w < warp; ++w) { gt_before += wcnt[w]; eq_before += wcnt[8 + w]; }
+  unsigned int pos = gt_before + min(k_eq, eq_before), eq_run = eq_before;
+  const unsigned int lt_mask = (1u << lane) - 1u;
+  for (int base = lo; base < hi; base += 32) {
+    const int i = base + lane;
+    const bool in = i < hi && take > 0;
+    const uint32_t key = in ? f32_order_key(score[i]) : 0u;
+    const bool is_eq = in && key == T;
+    const unsigned int beq = __ballot_sync(0xffffffffu, is_eq);
+    const bool tk = in && (key > T || (is_eq && eq_run + __popc(beq & lt_mask) < k_eq));
+    const unsigned int bt = __ballot_sync(0xffffffffu, tk);
+    if (tk) {
+      const unsigned int p = pos + __popc(bt & lt_mask);
+      if ((int)p < cap) out[p] = i;
+    }
+    pos += __popc(bt);
+    eq_run += __popc(beq);
+  }
+  if (tid == 0 && take < cap) out[take] = qb;     // the diagonal block is the largest index: list stays ascending
+  __syncthreads();
+  return take + 1;
+}
+
+__device__ __forceinline__ float pooled_score(const float* q, const float* k, float scale) {
+  float acc = 0.f;
+#pragma unroll 8
+  for (int t = 0; t < RS_HEAD_DIM; ++t) acc = fmaf(q[t], k[t], acc);
+  return acc * scale;
+}
+
+// Evaluation of one block-sparse candidate: list of the segment's last query block, coverage, pairs.
+__global__ void __launch_bounds__(256)
+rs_bs_eval_kernel(IdxParams P) {
+  extern __shared__ float score[];      // [nb]
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t sh[8];
+  __shared__ unsigned int wcnt[16];
+  __shared__ int32_t sel[1024];
+  __shared__ float qrow[RS_HEAD_DIM];
+  __shared__ u64 cov[RS_PROBE_GROUPS];
+  int item, c, slot;
+  if (!job_of(P, blockIdx.x, item, c, slot)) return;
+  const rs_candidate cand = P.lib[c];
+  if (cand.pattern != RS_BLOCK_SPARSE) return;
+  if (P.stats == nullptr && P.choice != nullptr) return;    // materialise mode without stats: rows are built elsewhere
+  const int s = item / P.Hq, h = item - s * P.Hq, g = h / P.group;
+  const int q0 = P.seg_bounds[s], q1 = P.seg_bounds[s + 1];
+  const int qb = (q1 >> 6) - 1;
+  const int tid = threadIdx.x;
+  if (P.bscore != nullptr) {
+    const float* row = P.bscore + ((size_t)item * P.nb + qb) * P.nb;
+    for (int kb = tid; kb < qb; kb += 256) score[kb] = row[kb];
+  } else {
+    if (tid < RS_HEAD_DIM) qrow[tid] = P.qpool[((size_t)h * P.nb + qb) * RS_HEAD_DIM + tid];
+    __syncthreads();
+    for (int kb = tid; kb < qb; kb += 256)
+      score[kb] = pooled_score(qrow, P.kpool + ((size_t)g * P.nb + kb) * RS_HEAD_DIM, P.scale);
+  }
+  if (tid < RS_PROBE_GROUPS) cov[tid] = 0;
+  __syncthreads();
+  const int k_b = min(cand.b0, 1024);
+  const int cnt = select_row(score, qb, min(k_b, qb + 1) - 1, qb, sel, 1024, hist, sh, wcnt);
+  if (P.choice == nullptr) {
+    int32_t* dst = P.out.bs_blk + (size_t)slot * P.out.kb_cap;
+    for (int i = tid; i < cnt && i < P.out.kb_cap; i += 256) dst[i] = sel[i];
+    if (tid == 0) P.out.bs_count[slot] = cnt;
+  }
+  if (P.stats == nullptr) return;
+  const u64* vblk = P.vblk + (size_t)item * RS_PROBE_GROUPS * P.nb;
+  u64 part[RS_PROBE_GROUPS] = {0, 0, 0, 0};
+  for (int i = tid; i < cnt; i += 256)
+#pragma unroll
+    for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) part[gg] += vblk[(size_t)gg * P.nb + sel[i]];
+#pragma unroll
+  for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) if (part[gg]) atomicAdd(&cov[gg], part[gg]);
+  __syncthreads();
+  if (tid == 0) {
+    rs_cand_stats* st = P.stats + (size_t)item * P.n_cand + c;
+    for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) st->cov_fx[gg] = cov[gg];
+    st->pairs = pairs_block_sparse(q0 >> 6, q1 >> 6, cand.b0);
+  }
+}
+
+// Materialise: one block per (query block, head) of every item routed to block-sparse.
+__global__ void __launch_bounds__(256)
+rs_bs_rows_kernel(IdxParams P) {
+  extern __shared__ float score[];
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t sh[8];
+  __shared__ unsigned int wcnt[16];
+  const int qb = blockIdx.x, h = blockIdx.y;
+  const int s = seg_of_block(P, qb);
+  const int item = s * P.Hq + h;
+  const rs_candidate cand = P.lib[P.choice[item]];
+  if (cand.pattern != RS_BLOCK_SPARSE) return;
+  const int tid = threadIdx.x;
+  const float* row = (P.bscore != nullptr) ? P.bscore + ((size_t)item * P.nb + qb) * P.nb
+                                           : P.bs_ws + ((size_t)h * P.nb + qb) * P.nb;
+  for (int kb = tid; kb < qb; kb += 256) score[kb] = row[kb];
+  __syncthreads();
+  const size_t orow = (size_t)h * P.nb + qb;
+  const int k_b = min(cand.b0, P.out.kb_cap);
+  const int cnt = select_row(score, qb, min(k_b, qb + 1) - 1, qb, P.out.bs_blk + orow * P.out.kb_cap, P.out.kb_cap,
+                             hist, sh, wcnt);
+  if (tid == 0) P.out.bs_count[orow] = cnt;
+}
+
+// Fused pooled scores for the items routed to block-sparse: 64 x 64 tiles of qpool[h] kpool[g]^T / sqrt(d),
+// lower triangle only; every output accumulates k = 0..127 in order with fmaf (same bits as pooled_score).
+__global__ void __launch_bounds__(256)
+rs_bs_scores_kernel(IdxParams P) {
+  __shared__ float As[64][33], Bs[64][33];
+  __shared__ int any_bs;
+  const int kt = blockIdx.x, qt = blockIdx.y, h = blockIdx.z;
+  if (kt > qt) return;
+  const int tid = threadIdx.x;
+  if (tid == 0) any_bs = 0;
+  __syncthreads();
+  if (tid < 64) {
+    const int qb = qt * 64 + tid;
+    if (qb < P.nb) {
+      const int item = seg_of_block(P, qb) * P.Hq + h;
+      if (P.lib[P.choice[item]].pattern == RS_BLOCK_SPARSE) any_bs = 1;
+    }
+  }
+  __syncthreads();
+  if (!any_bs) return;
+  const int g = h / P.group;
+  const int tx = tid & 15, ty = tid >> 4;       // outputs rows ty*4.., cols tx*4..
+  float acc[4][4] = {};
+  for (int k0 = 0; k0 < RS_HEAD_DIM; k0 += 32) {
+    for (int i = tid; i < 64 * 32; i += 256) {
+      const int r = i >> 5, cidx = i & 31;
+      const int qb = qt * 64 + r, kb = kt * 64 + r;
+      As[r][cidx] = (qb < P.nb) ? P.qpool[((size_t)h * P.nb + qb) * RS_HEAD_DIM + k0 + cidx] : 0.f;
+      Bs[r][cidx] = (kb < P.nb) ? P.kpool[((size_t)g * P.nb + kb) * RS_HEAD_DIM + k0 + cidx] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int k = 0; k < 32; ++k) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = As[ty * 4 + i][k]; b[i] = Bs[tx * 4 + i][k]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int qb = qt * 64 + ty * 4 + i;
+    if (qb >= P.nb) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int kb = kt * 64 + tx * 4 + j;
+      if (kb < P.nb) P.bs_ws[((size_t)h * P.nb + qb) * P.nb + kb] = acc[i][j] * P.scale;
+    }
+  }
+}
+
+struct IdxPlan { size_t vblk, bs_ws, total; };
+
+IdxPlan plan(const rs_problem* p, const rs_candidate* lib, int n_cand) {
+  IdxPlan w{};
+  const size_t nb = (size_t)p->n_keys / 64;
+  const size_t items = (size_t)p->n_segments * p->n_q_heads;
+  bool any_bs = false;
+  for (int c = 0; c < n_cand; ++c) any_bs |= (lib[c].pattern == RS_BLOCK_SPARSE);
+  size_t off = 0;
+  w.vblk = off;  off += rs_align_up(items * RS_PROBE_GROUPS * nb * sizeof(u64), 256);
+  w.bs_ws = off; off += any_bs ? rs_align_up((size_t)p->n_q_heads * nb * nb * sizeof(float), 256) : 0;
+  w.total = off;
+  return w;
+}
+
+}  // namespace
+
+size_t rs_indices_workspace_bytes(const rs_problem* p, const rs_candidate* lib, int n_cand) {
+  return plan(p, lib, n_cand).total;
+}
+
+extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, int n_cand, const float* vert,
+                                const float* slash, const float* qpool, const float* kpool, const float* bscore,
+                                const int32_t* choice, const rs_index_set* out, rs_cand_stats* stats, void* ws,
+                                size_t ws_bytes, int32_t* status, void* stream_) {
+  int rc = rs_check_problem(p);
+  if (rc != RS_OK) return rc;
+  if (!lib || n_cand <= 0 || n_cand > RS_MAX_CANDIDATES || !out || !ws) return RS_ERR_INVALID_ARG;
+  if (choice == nullptr && stats == nullptr) return RS_ERR_INVALID_ARG;
+  const int n_items = p->n_segments * p->n_q_heads;
+  const int nb = p->n_keys / 64;
+  bool any_vs = false, any_bs = false, any_a = false;
+  for (int c = 0; c < n_cand; ++c) {
+    const rs_candidate& cd = lib[c];
+    if (cd.pattern < 0 || cd.pattern > 3) return RS_ERR_INVALID_ARG;
+    if (cd.pattern == RS_VERTICAL_SLASH) {
+      any_vs = true;
+      if (cd.b0 < 0 || cd.b1 < 1) return RS_ERR_INVALID_ARG;
+      if (out->kv_cap < (cd.b0 < p->n_keys ? cd.b0 : p->n_keys) || out->ks_cap < (cd.b1 < p->n_keys ? cd.b1 : p->n_keys) ||
+          out->nd_cap < nb) return RS_ERR_INVALID_ARG;
+    } else if (cd.pattern == RS_BLOCK_SPARSE) {
+      any_bs = true;
+      if (cd.b0 < 1 || cd.b0 > 1024) return RS_ERR_INVALID_ARG;
+      if (out->kb_cap < (cd.b0 < nb ? cd.b0 : nb)) return RS_ERR_INVALID_ARG;
+    } else if (cd.pattern == RS_A_SHAPE) {
+      any_a = true;
+      if (cd.b0 < 0 || cd.b1 < 1) return RS_ERR_INVALID_ARG;
+      if (stats != nullptr) {
+        // coverage of sink + window from column and offset masses needs the two not to overlap on the probe rows
+        for (int s = 0; s < p->n_segments; ++s) {
+          const int q1 = p->seg_bounds[s + 1];
+          if (cd.b1 < q1 && q1 - RS_PROBE_ROWS - cd.b1 + 1 < cd.b0) return RS_ERR_UNSUPPORTED_SHAPE;
+        }
+      }
+    }
+  }
+  (void)any_a;
+  if ((any_vs || stats) && (!vert || !slash)) return RS_ERR_INVALID_ARG;
+  if (any_bs && bscore == nullptr && (!qpool || !kpool)) return RS_ERR_INVALID_ARG;
+  const int n_slots = choice ? n_items : n_items * n_cand;
+  if (any_vs && out->n_vs_slots < n_slots) return RS_ERR_INVALID_ARG;
+  if (any_bs && out->bs_rows < (choice ? p->n_q_heads * nb : n_slots)) return RS_ERR_INVALID_ARG;
+  for (int s = 0; s < p->n_segments; ++s)
+    if (p->seg_bounds[s + 1] < RS_PROBE_ROWS) return RS_ERR_UNSUPPORTED_SHAPE;
+  const IdxPlan w = plan(p, lib, n_cand);
+  if (ws_bytes < w.total) return RS_ERR_WORKSPACE_TOO_SMALL;
+  if (((uintptr_t)ws & 255) != 0) return RS_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  uint8_t* wsb = reinterpret_cast<uint8_t*>(ws);
+
+  IdxParams P{};
+  P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = P.Hq / P.Hkv; P.n_seg = p->n_segments;
+  P.n_cand = n_cand; P.nb = nb;
+  for (int s = 0; s <= p->n_segments; ++s) P.seg_bounds[s] = p->seg_bounds[s];
+  for (int c = 0; c < n_cand; ++c) P.lib[c] = lib[c];
+  P.vert = vert; P.slash = slash; P.qpool = qpool; P.kpool = kpool; P.bscore = bscore; P.choice = choice;
+  P.out = *out; P.stats = stats; P.vblk = reinterpret_cast<u64*>(wsb + w.vblk);
+  P.bs_ws = reinterpret_cast<float*>(wsb + w.bs_ws); P.status = status;
+  P.scale = (float)(1.0 / sqrt((double)RS_HEAD_DIM));
+
+  const int n_jobs = n_items * n_cand;
+  if (stats != nullptr) {
+    const long long warps = (long long)n_items * RS_PROBE_GROUPS * nb;
+    rs_vblk_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, stream>>>(P);
+    rs_simple_stats_kernel<<<n_jobs, 256, 0, stream>>>(P);
+  }
+  if (any_vs) {
+    rs_vs_select_kernel<<<dim3(2, n_jobs), kSelThreads, 0, stream>>>(P);
+    rs_vs_finish_kernel<<<n_jobs, 256, 0, stream>>>(P);
+  }
+  if (any_bs) {
+    if (choice == nullptr || stats != nullptr)
+      rs_bs_eval_kernel<<<n_jobs, 256, (size_t)nb * sizeof(float), stream>>>(P);
+    if (choice != nullptr) {
+      if (bscore == nullptr) {
+        const int nt = (nb + 63) / 64;
+        rs_bs_scores_kernel<<<dim3(nt, nt, P.Hq), 256, 0, stream>>>(P);
+      }
+      rs_bs_rows_kernel<<<dim3(nb, P.Hq), 256, (size_t)nb * sizeof(float), stream>>>(P);
+    }
+  }
+  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+}

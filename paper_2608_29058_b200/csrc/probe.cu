@@ -1,0 +1,501 @@
+// Shared attention probe (Eq. 3, Section 3.2) in the last-64-query form, plus the pooled means for the
+// coarse block scores and the value norms of Eq. 5.
+//
+// For every (segment, KV head) the 64 probe rows of up to four query heads (256 rows) are scored against all
+// causal keys on the tensor cores, twice:
+//   pass 1 (probe_lse):   S = Qp K^T with probe rows on the TMEM lanes; every thread owns one probe row and keeps
+//                         its running maximum and sum, split over key ranges; partials are merged afterwards.
+//   pass 2 (probe_accum): S^T = K Qp^T with keys on the TMEM lanes; every thread owns one key, so the column
+//                         mass of a 16-row probe group is a sum inside the thread; the diagonal (slash) mass is
+//                         a skewed sum over a 16 x 128 tile staged in shared memory.
+// Each key tile is read from HBM once per pass (TMA, 128-byte swizzle); both passes are balanced between the
+// HBM stream and the exponential rate.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kHC = 4;                 // head slots per CTA (4 x 64 = 256 probe rows)
+constexpr int kRows = kHC * RS_PROBE_ROWS;
+constexpr int kKeyTile = 128;
+constexpr int kStages = 3;
+constexpr int kThreads = 320;          // warp 0 TMA, warp 1 MMA, warps 2..9 compute
+constexpr uint32_t kTmemCols = 512;
+
+struct ProbeParams {
+  int n, Hq, Hkv, group, n_seg, n_hc;  // n_hc = head chunks per KV head = ceil(group / 4)
+  int seg_bounds[RS_MAX_SEGMENTS + 1];
+  int n_splits;
+  float2* partial;    // [n_seg*Hkv*n_hc][n_splits][256] (max, sum) in the exp2 domain
+  float* lse2;        // [n_seg*Hkv*n_hc][256] log-sum-exp * log2(e)
+  float* lse_probe;   // [n_seg][Hq][64]
+  float* vert;        // [n_seg][Hq][4][n]
+  float* slash;       // [n_seg][Hq][4][n]
+  int32_t* status;
+  float scale_log2e;
+};
+
+struct Smem {
+  static constexpr uint32_t qp = 0;                       // 2 halves x 256 rows x 128 B
+  static constexpr uint32_t k = 65536;                    // kStages x (2 halves x 128 rows x 128 B)
+  static constexpr uint32_t x = k + kStages * 32768;      // pass 2: [2 column halves][2 buffers][16][128] fp32
+  static constexpr uint32_t lse = x + 32768;              // 256 floats
+  static constexpr uint32_t bars = lse + 1024;            // mbarriers
+  static constexpr uint32_t misc = bars + 128;
+  static constexpr uint32_t total = misc + 64 + 1024;     // + alignment slack
+};
+
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+// Common prologue: barriers, TMEM, probe-row tile load.  Returns the TMEM base.
+struct Ctx {
+  uint32_t base, tmem;
+  uint32_t bar_q, bar_full[kStages], bar_empty[kStages], bar_tfull[2], bar_tempty[2];
+  volatile int* abort_flag;
+  int s, g, hc, q1, n_heads, h0, t0, t1, unit;
+};
+
+template <int PASS>
+__global__ void __launch_bounds__(kThreads, 1)
+rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ ProbeParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // unit = (segment, kv head, head chunk); blockIdx.x = split of the key range
+  const int unit = blockIdx.y;
+  const int hc = unit % P.n_hc;
+  const int g = (unit / P.n_hc) % P.Hkv;
+  const int s = unit / (P.n_hc * P.Hkv);
+  const int q1 = P.seg_bounds[s + 1];
+  const int h0 = g * P.group + hc * kHC;
+  const int n_heads = min(kHC, P.group - hc * kHC);
+  const int n_tiles = (q1 + kKeyTile - 1) / kKeyTile;
+  const int per = (n_tiles + P.n_splits - 1) / P.n_splits;
+  const int t0 = blockIdx.x * per, t1 = min(n_tiles, t0 + per);
+  const int i_first = q1 - RS_PROBE_ROWS;   // first probe row
+
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + Smem::bars);
+  volatile int* misc = reinterpret_cast<volatile int*>(sm + Smem::misc);
+  volatile int* abort_flag = misc + 1;
+  float* s_lse = reinterpret_cast<float*>(sm + Smem::lse);
+  const uint32_t bar_q = smem_u32(&bars[0]);
+  uint32_t bar_full[kStages], bar_empty[kStages], bar_tfull[2], bar_tempty[2];
+#pragma unroll
+  for (int i = 0; i < kStages; ++i) { bar_full[i] = smem_u32(&bars[1 + i]); bar_empty[i] = smem_u32(&bars[4 + i]); }
+#pragma unroll
+  for (int i = 0; i < 2; ++i) { bar_tfull[i] = smem_u32(&bars[7 + i]); bar_tempty[i] = smem_u32(&bars[9 + i]); }
+
+  if (tid == 0) {
+    mbar_init(bar_q, 1);
+    for (int i = 0; i < kStages; ++i) { mbar_init(bar_full[i], 1); mbar_init(bar_empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull[i], 1); mbar_init(bar_tempty[i], 256); }
+    misc[1] = 0;
+    mbar_fence_init();
+    tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
+  }
+  if (warp == 1) { tmem_alloc(smem_u32((const void*)&misc[0]), kTmemCols); tmem_relinquish(); }
+  if (PASS == 2) {
+    for (int i = tid; i < kRows; i += kThreads) s_lse[i] = P.lse2[(size_t)unit * kRows + i];
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = (uint32_t)misc[0];
+  if (t0 >= t1) {   // nothing to do for this split (uniform across the CTA)
+    if (PASS == 1) {
+      for (int i = tid; i < kRows; i += kThreads)
+        P.partial[((size_t)unit * P.n_splits + blockIdx.x) * kRows + i] = make_float2(-INFINITY, 0.f);
+    }
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+    return;
+  }
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- producer
+      mbar_arrive_expect_tx(bar_q, (uint32_t)n_heads * 16384u);
+      for (int hh = 0; hh < n_heads; ++hh) {
+        const int row = (h0 + hh) * P.n + i_first;
+        tma_load_2d(base + Smem::qp + (uint32_t)hh * 8192u, &tmQ, bar_q, 0, row);
+        tma_load_2d(base + Smem::qp + 32768u + (uint32_t)hh * 8192u, &tmQ, bar_q, 64, row);
+      }
+      bool ok = true;
+      for (int t = t0; t < t1; ++t) {
+        const int it = t - t0, st = it % kStages;
+        ok = mbar_wait(bar_empty[st], ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag);
+        if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, 11); break; }
+        mbar_arrive_expect_tx(bar_full[st], 32768u);
+        const uint32_t dst = base + Smem::k + (uint32_t)st * 32768u;
+        const int row = g * P.n + t * kKeyTile;
+        tma_load_2d(dst, &tmK, bar_full[st], 0, row);
+        tma_load_2d(dst + 16384u, &tmK, bar_full[st], 64, row);
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---------------------------------------------------------------- MMA issuer
+      bool ok = mbar_wait(bar_q, 0, abort_flag);
+      int site = 12;
+      for (int t = t0; t < t1 && ok; ++t) {
+        const int it = t - t0, st = it % kStages, b = it & 1;
+        ok = mbar_wait(bar_full[st], (uint32_t)(it / kStages) & 1u, abort_flag); site = 13;
+        if (!ok) break;
+        ok = mbar_wait(bar_tempty[b], ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag); site = 14;
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t ksm = base + Smem::k + (uint32_t)st * 32768u;
+        if (PASS == 1) {
+          // probe rows on lanes: two M=128 products (head pairs), N = 128 keys
+          const uint32_t idesc = umma_idesc_bf16(128, 128, 0, 0);
+          for (int pr = 0; pr < 2; ++pr) {
+            const uint64_t adesc = umma_smem_desc(base + Smem::qp + (uint32_t)pr * 16384u, 16, 1024);
+            const uint64_t bdesc = umma_smem_desc(ksm, 16, 1024);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+              const uint64_t aoff = (uint64_t)(((kk >> 2) * 32768 + (kk & 3) * 32) >> 4);
+              const uint64_t boff = (uint64_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+              umma_ss(tmem + (uint32_t)(b * 256 + pr * 128), adesc + aoff, bdesc + boff, idesc, kk > 0 ? 1u : 0u);
+            }
+          }
+        } else {
+          // keys on lanes: one M=128 product, N = 256 probe rows
+          const uint32_t idesc = umma_idesc_bf16(128, 256, 0, 0);
+          const uint64_t adesc = umma_smem_desc(ksm, 16, 1024);
+          const uint64_t bdesc = umma_smem_desc(base + Smem::qp, 16, 1024);
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint64_t aoff = (uint64_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+            const uint64_t boff = (uint64_t)(((kk >> 2) * 32768 + (kk & 3) * 32) >> 4);
+            umma_ss(tmem + (uint32_t)(b * 256), adesc + aoff, bdesc + boff, idesc, kk > 0 ? 1u : 0u);
+          }
+        }
+        umma_commit(bar_tfull[b]);
+        umma_commit(bar_empty[st]);
+      }
+      if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, site); *abort_flag = 1; }
+    }
+  } else {
+    // ------------------------------------------------------------------ compute warps
+    const int cw = warp - 2;                 // 0..7
+    const int quad = warp & 3;               // TMEM lane quadrant this warp may touch
+    const int part = cw >> 2;                // pass 1: head pair; pass 2: column half
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const float sl2 = P.scale_log2e;
+    uint32_t v[32];
+    bool ok = true;
+
+    if (PASS == 1) {
+      const int r = quad * 32 + lane;                 // row inside the head pair (0..127)
+      const int hh = part * 2 + (r >> 6);             // head slot
+      const int i = i_first + (r & 63);               // global query row
+      float m_run = -INFINITY, l_run = 0.f;
+      for (int t = t0; t < t1; ++t) {
+        const int it = t - t0, b = it & 1;
+        ok = mbar_wait(bar_tfull[b], (uint32_t)(it >> 1) & 1u, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const int j0 = t * kKeyTile;
+        const bool need_mask = j0 + kKeyTile - 1 > i_first;
+#pragma unroll 1
+        for (int c4 = 0; c4 < 4; ++c4) {
+          tmem_ld32(tmem + lane_addr + (uint32_t)(b * 256 + part * 128 + c4 * 32), v);
+          tc_wait_ld();
+          float mx = -INFINITY;
+#pragma unroll
+          for (int x = 0; x < 32; ++x) {
+            float sv = __uint_as_float(v[x]) * sl2;
+            if (need_mask && (j0 + c4 * 32 + x > i)) sv = -INFINITY;
+            v[x] = __float_as_uint(sv);
+            mx = fmaxf(mx, sv);
+          }
+          if (mx > m_run) { l_run *= fast_exp2(m_run - mx); m_run = mx; }
+          if (m_run > -INFINITY) {
+            float acc = 0.f;
+#pragma unroll
+            for (int x = 0; x < 32; ++x) acc += fast_exp2(__uint_as_float(v[x]) - m_run);
+            l_run += acc;
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar_tempty[b]);
+      }
+      if (ok) {
+        P.partial[((size_t)unit * P.n_splits + blockIdx.x) * kRows + hh * 64 + (r & 63)] = make_float2(m_run, l_run);
+      }
+    } else {
+      const int l128 = quad * 32 + lane;              // key inside the tile
+      float* xs = reinterpret_cast<float*>(sm + Smem::x) + part * (2 * 16 * 128);
+      int iter = 0;
+      for (int t = t0; t < t1; ++t) {
+        const int it = t - t0, b = it & 1;
+        ok = mbar_wait(bar_tfull[b], (uint32_t)(it >> 1) & 1u, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const int j0 = t * kKeyTile;
+        const int j = j0 + l128;
+        const bool need_mask = j0 + kKeyTile - 1 > i_first;
+#pragma unroll 1
+        for (int q = 0; q < 8; ++q, ++iter) {         // (head slot, probe group) pairs of this column half
+          const int hh = part * 2 + (q >> 2), grp = q & 3;
+          float* xb = xs + (iter & 1) * (16 * 128);
+          uint32_t v16[16];
+          {
+            uint32_t* d = v16;
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
+                  "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15])
+                : "r"(tmem + lane_addr + (uint32_t)(b * 256 + hh * 64 + grp * 16))
+                : "memory");
+          }
+          tc_wait_ld();
+          const int ig = i_first + grp * 16;          // first row of the group
+          float vsum = 0.f;
+#pragma unroll
+          for (int r = 0; r < 16; ++r) {
+            float p = fast_exp2(fmaf(__uint_as_float(v16[r]), sl2, -s_lse[hh * 64 + grp * 16 + r]));
+            if (need_mask && j > ig + r) p = 0.f;
+            vsum += p;
+            xb[r * 128 + l128] = p;
+          }
+          const bool live = hh < n_heads;
+          const size_t out = (((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS + grp) * (size_t)P.n;
+          if (live && j < q1) P.vert[out + j] = vsum;
+          named_bar_sync(1 + part, 128);
+          // skewed sums: u = l - r + 15 in [0, 142]; offset o = (ig - j0 + 15) - u
+          const int obase = ig - j0 + 15;
+          {
+            const int u = l128;
+            float acc = 0.f;
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+              const int l = u - 15 + r;
+              if (l >= 0) acc += xb[r * 128 + l];
+            }
+            const int o = obase - u;
+            if (live && o >= 0) {
+              if (u >= 15) P.slash[out + o] = acc;      // all 16 rows of the group inside this tile
+              else atomicAdd(&P.slash[out + o], acc);   // shared with the neighbouring tile (two addends)
+            }
+          }
+          if (l128 < 15) {
+            const int u = 128 + l128;
+            float acc = 0.f;
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+              const int l = u - 15 + r;
+              if (l < 128) acc += xb[r * 128 + l];
+            }
+            const int o = obase - u;
+            if (live && o >= 0) atomicAdd(&P.slash[out + o], acc);
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar_tempty[b]);
+      }
+    }
+    if (!ok && lane == 0 && cw == 0) { rs_report(P.status, RS_ERR_TIMEOUT, 15); *abort_flag = 1; }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, kTmemCols); }
+}
+
+// Merges the per-split (max, sum) partials of pass 1 into the probe log-sum-exp.
+__global__ void rs_probe_merge_kernel(ProbeParams P) {
+  const int unit = blockIdx.x;
+  const int row = threadIdx.x;    // 0..255
+  const int hc = unit % P.n_hc;
+  const int g = (unit / P.n_hc) % P.Hkv;
+  const int s = unit / (P.n_hc * P.Hkv);
+  const int hh = row >> 6;
+  const float2* part = P.partial + (size_t)unit * P.n_splits * kRows + row;
+  float m = -INFINITY;
+  for (int k = 0; k < P.n_splits; ++k) m = fmaxf(m, part[(size_t)k * kRows].x);
+  float l = 0.f;
+  for (int k = 0; k < P.n_splits; ++k) {
+    const float2 pk = part[(size_t)k * kRows];
+    if (pk.x > -INFINITY) l += pk.y * exp2f(pk.x - m);
+  }
+  const float lse2 = m + log2f(l);
+  P.lse2[(size_t)unit * kRows + row] = lse2;
+  if (hc * kHC + hh < P.group) {
+    const int h = g * P.group + hc * kHC + hh;
+    P.lse_probe[((size_t)s * P.Hq + h) * RS_PROBE_ROWS + (row & 63)] = lse2 * 0.6931471805599453f;
+  }
+}
+
+// 64-row means of Q and K (fp32) and per-block maxima of ||v||^2.
+// One CTA per (tensor row block): 256 threads, thread (rg = tid/16, cc = tid%16) sums rows rg, rg+16, .. of 16-byte
+// column chunk cc; a fixed-order shared-memory reduction over the 16 row groups follows.
+__global__ void __launch_bounds__(256)
+rs_pool_kernel(const __nv_bfloat16* __restrict__ X, float* __restrict__ out, long long n_blocks) {
+  __shared__ float red[16][128 + 4];
+  const long long blk = blockIdx.x;
+  if (blk >= n_blocks) return;
+  const int rg = threadIdx.x >> 4, cc = threadIdx.x & 15;
+  const uint4* src = reinterpret_cast<const uint4*>(X + (size_t)blk * 64 * RS_HEAD_DIM);
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint4 u = __ldg(src + (size_t)(rg + 16 * k) * 16 + cc);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      acc[2 * e] += __uint_as_float(w[e] << 16);
+      acc[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) red[rg][cc * 8 + e] = acc[e];
+  __syncthreads();
+  if (threadIdx.x < 128) {
+    float sum = 0.f;
+#pragma unroll
+    for (int r = 0; r < 16; ++r) sum += red[r][threadIdx.x];
+    out[(size_t)blk * RS_HEAD_DIM + threadIdx.x] = sum * (1.0f / 64.0f);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+rs_vnorm_block_kernel(const __nv_bfloat16* __restrict__ V, float* __restrict__ blockmax, long long n_blocks) {
+  __shared__ float red[8];
+  const long long blk = blockIdx.x;
+  if (blk >= n_blocks) return;
+  const int rg = threadIdx.x >> 4, cc = threadIdx.x & 15;
+  const uint4* src = reinterpret_cast<const uint4*>(V + (size_t)blk * 64 * RS_HEAD_DIM);
+  float best = 0.f;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint4 u = __ldg(src + (size_t)(rg + 16 * k) * 16 + cc);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+    float ss = 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float a = __uint_as_float(w[e] << 16), b = __uint_as_float(w[e] & 0xffff0000u);
+      ss = fmaf(a, a, ss);
+      ss = fmaf(b, b, ss);
+    }
+    // 16 lanes hold one row: fixed-order butterfly
+#pragma unroll
+    for (int off = 8; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+    best = fmaxf(best, ss);
+  }
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) best = fmaxf(best, __shfl_xor_sync(0xffffffffu, best, off));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = best;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float m = red[0];
+    for (int i = 1; i < 8; ++i) m = fmaxf(m, red[i]);
+    blockmax[blk] = m;
+  }
+}
+
+// vmax[s][g] = sqrt(max over key blocks below the segment end of the block maxima of ||v||^2)
+__global__ void rs_vmax_kernel(ProbeParams P, const float* blockmax, float* vmax) {
+  const int s = blockIdx.x / P.Hkv, g = blockIdx.x % P.Hkv;
+  const int nb = P.n >> 6, nbs = P.seg_bounds[s + 1] >> 6;
+  float m = 0.f;
+  for (int i = threadIdx.x; i < nbs; i += blockDim.x) m = fmaxf(m, blockmax[(size_t)g * nb + i]);
+  __shared__ float red[32];
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < (int)(blockDim.x >> 5); ++i) m = fmaxf(m, red[i]);
+    vmax[blockIdx.x] = sqrtf(m);
+  }
+}
+
+struct ProbePlan { size_t partial, lse2, blockmax, total; int n_units, n_splits, n_hc; };
+
+ProbePlan plan(const rs_problem* p) {
+  ProbePlan w{};
+  const int group = p->n_q_heads / p->n_kv_heads;
+  w.n_hc = (group + kHC - 1) / kHC;
+  w.n_units = p->n_segments * p->n_kv_heads * w.n_hc;
+  int splits = (2 * 148 + w.n_units - 1) / w.n_units;
+  const int max_tiles = (p->n_keys + kKeyTile - 1) / kKeyTile;
+  if (splits > max_tiles) splits = max_tiles;
+  if (splits < 1) splits = 1;
+  if (splits > 64) splits = 64;
+  w.n_splits = splits;
+  size_t off = 0;
+  w.partial = off;  off += rs_align_up((size_t)w.n_units * splits * kRows * sizeof(float2), 256);
+  w.lse2 = off;     off += rs_align_up((size_t)w.n_units * kRows * sizeof(float), 256);
+  w.blockmax = off; off += rs_align_up((size_t)p->n_kv_heads * (p->n_keys / 64) * sizeof(float), 256);
+  w.total = off;
+  return w;
+}
+
+}  // namespace
+
+size_t rs_probe_workspace_bytes(const rs_problem* p) { return plan(p).total; }
+
+extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const void* V, float* vert, float* slash,
+                        float* lse_probe, float* qpool, float* kpool, float* vmax, float* descr, void* ws,
+                        size_t ws_bytes, int32_t* status, void* stream_) {
+  (void)descr;
+  int rc = rs_check_problem(p);
+  if (rc != RS_OK) return rc;
+  if (!Q || !K || !V || !vert || !slash || !lse_probe || !ws) return RS_ERR_INVALID_ARG;
+  for (int s = 0; s < p->n_segments; ++s)
+    if (p->seg_bounds[s + 1] < RS_PROBE_ROWS) return RS_ERR_UNSUPPORTED_SHAPE;
+  rc = rs_check_device();
+  if (rc != RS_OK) return rc;
+  const ProbePlan w = plan(p);
+  if (ws_bytes < w.total) return RS_ERR_WORKSPACE_TOO_SMALL;
+  if (((uintptr_t)ws & 255) != 0) return RS_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  uint8_t* wsb = reinterpret_cast<uint8_t*>(ws);
+
+  ProbeParams P{};
+  P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = P.Hq / P.Hkv;
+  P.n_seg = p->n_segments; P.n_hc = w.n_hc; P.n_splits = w.n_splits;
+  for (int s = 0; s <= p->n_segments; ++s) P.seg_bounds[s] = p->seg_bounds[s];
+  P.partial = reinterpret_cast<float2*>(wsb + w.partial);
+  P.lse2 = reinterpret_cast<float*>(wsb + w.lse2);
+  P.lse_probe = lse_probe; P.vert = vert; P.slash = slash; P.status = status;
+  P.scale_log2e = (float)(1.4426950408889634 / sqrt((double)RS_HEAD_DIM));
+
+  const size_t mass_bytes = (size_t)P.n_seg * P.Hq * RS_PROBE_GROUPS * (size_t)P.n * sizeof(float);
+  if (cudaMemsetAsync(vert, 0, mass_bytes, stream) != cudaSuccess) return RS_ERR_CUDA;
+  if (cudaMemsetAsync(slash, 0, mass_bytes, stream) != cudaSuccess) return RS_ERR_CUDA;
+
+  CUtensorMap tmQ, tmK;
+  if (rs_make_tmap_bf16_2d(&tmQ, Q, (uint64_t)P.Hq * P.n, RS_HEAD_DIM, 64, 64) ||
+      rs_make_tmap_bf16_2d(&tmK, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kKeyTile, 64))
+    return RS_ERR_CUDA;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(rs_probe_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::total) != cudaSuccess ||
+        cudaFuncSetAttribute(rs_probe_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::total) != cudaSuccess)
+      return RS_ERR_CUDA;
+    attr_set = true;
+  }
+  dim3 grid(w.n_splits, w.n_units);
+  rs_probe_kernel<1><<<grid, kThreads, Smem::total, stream>>>(tmQ, tmK, P);
+  rs_probe_merge_kernel<<<w.n_units, kRows, 0, stream>>>(P);
+  rs_probe_kernel<2><<<grid, kThreads, Smem::total, stream>>>(tmQ, tmK, P);
+
+  const long long nb = p->n_keys / 64;
+  if (qpool) rs_pool_kernel<<<(unsigned)(P.Hq * nb), 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(Q), qpool, P.Hq * nb);
+  if (kpool) rs_pool_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(K), kpool, P.Hkv * nb);
+  if (vmax) {
+    float* blockmax = reinterpret_cast<float*>(wsb + w.blockmax);
+    rs_vnorm_block_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(V), blockmax, P.Hkv * nb);
+    rs_vmax_kernel<<<P.n_seg * P.Hkv, 256, 0, stream>>>(P, blockmax, vmax);
+  }
+  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+}

@@ -1,0 +1,213 @@
+// Risk score (Eq. 4), greedy substitution for the budgeted routing problem (Eq. 6-8), fallback walk and forced
+// dense (Section 3.4), solved by one thread block so that no host round trip sits between probe and attention.
+//
+// Exactness: coverage and cost are integers, so totals are exact; risks are IEEE doubles built from separately
+// rounded operations (no fused multiply-add); a substitution's ratio is one IEEE division and candidates are
+// ordered by (ratio, larger saving, lower item, lower candidate), a total order, so the parallel arg-min picks
+// the same substitution as a sequential scan.
+#include "common.cuh"
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kMaxItems = RS_MAX_SEGMENTS * 64;
+
+struct RouteArgs {
+  int n_items, n_cand, Hq, Hkv, group, dense_c;
+  rs_candidate lib[RS_MAX_CANDIDATES];
+  int next_larger[RS_MAX_CANDIDATES];
+  const rs_cand_stats* stats;
+  const int64_t* cost;
+  const float* vmax;
+  rs_route_params prm;
+  int32_t* choice;
+  rs_route_report* report;
+  int32_t* status;
+};
+
+struct Sub { double ratio; long long dT; int item, k; };
+
+__device__ __forceinline__ bool better(const Sub& a, const Sub& b) {
+  if (a.k < 0) return false;
+  if (b.k < 0) return true;
+  if (a.ratio != b.ratio) return a.ratio < b.ratio;
+  if (a.dT != b.dT) return a.dT > b.dT;
+  if (a.item != b.item) return a.item < b.item;
+  return a.k < b.k;
+}
+
+__device__ __forceinline__ Sub shfl_sub(const Sub& a, int off) {
+  Sub r;
+  r.ratio = __shfl_xor_sync(0xffffffffu, a.ratio, off);
+  r.dT = __shfl_xor_sync(0xffffffffu, a.dT, off);
+  r.item = __shfl_xor_sync(0xffffffffu, a.item, off);
+  r.k = __shfl_xor_sync(0xffffffffu, a.k, off);
+  return r;
+}
+
+__device__ __forceinline__ long long cost_of(const RouteArgs& A, int item, int c) {
+  if (A.cost != nullptr) return A.cost[(size_t)item * A.n_cand + c];
+  return (long long)(4ull * RS_HEAD_DIM * A.stats[(size_t)item * A.n_cand + c].pairs);
+}
+
+__device__ __forceinline__ double m_hat_of(const RouteArgs& A, int item, int c) {
+  if (A.lib[c].pattern == RS_DENSE) return 1.0;
+  const rs_cand_stats& st = A.stats[(size_t)item * A.n_cand + c];
+  const unsigned long long tot = st.cov_fx[0] + st.cov_fx[1] + st.cov_fx[2] + st.cov_fx[3];
+  return (double)tot / 274877906944.0;          // 64 * 2^32
+}
+
+__device__ __forceinline__ double risk_of(const RouteArgs& A, int item, int c) {
+  if (A.lib[c].pattern == RS_DENSE) return 0.0;
+  const rs_cand_stats& st = A.stats[(size_t)item * A.n_cand + c];
+  double mx = 0.0, mn = 2.0;
+#pragma unroll
+  for (int g = 0; g < RS_PROBE_GROUPS; ++g) {
+    const double mg = (double)st.cov_fx[g] / 68719476736.0;   // 16 * 2^32
+    mx = fmax(mx, mg);
+    mn = fmin(mn, mg);
+  }
+  const double u = __dsub_rn(mx, mn);
+  return __dadd_rn(__dsub_rn(1.0, m_hat_of(A, item, c)), __dmul_rn(A.prm.alpha, u));
+}
+
+__global__ void __launch_bounds__(kThreads)
+rs_route_kernel(const __grid_constant__ RouteArgs A) {
+  __shared__ int ch[kMaxItems];
+  __shared__ Sub wbest[32];
+  __shared__ long long wsum[32];
+  __shared__ long long sh_total;
+  __shared__ int sh_feasible, sh_fallback;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_pairs = A.n_items * A.n_cand;
+
+  if (tid == 0) { sh_feasible = 1; sh_fallback = 0; }
+  if (A.prm.fixed_choice != nullptr) {
+    for (int it = tid; it < A.n_items; it += kThreads) ch[it] = A.prm.fixed_choice[it];
+    __syncthreads();
+  } else {
+    for (int it = tid; it < A.n_items; it += kThreads) ch[it] = A.dense_c;
+    long long part = 0;
+    for (int it = tid; it < A.n_items; it += kThreads) part += cost_of(A, it, A.dense_c);
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+    if (lane == 0) wsum[warp] = part;
+    __syncthreads();
+    if (tid == 0) {
+      long long t = A.prm.t_probe;
+      for (int w = 0; w < 32; ++w) t += wsum[w];
+      sh_total = t;
+    }
+    __syncthreads();
+    // ---- greedy substitutions until the layer budget is met
+    const int max_steps = n_pairs + 1;
+    for (int step = 0; step < max_steps; ++step) {
+      if (sh_total <= A.prm.budget) break;
+      Sub best; best.ratio = 0.0; best.dT = 0; best.item = -1; best.k = -1;
+      for (int p = tid; p < n_pairs; p += kThreads) {
+        const int it = p / A.n_cand, k = p - it * A.n_cand;
+        const int cur = ch[it];
+        const long long dT = cost_of(A, it, cur) - cost_of(A, it, k);
+        if (dT <= 0) continue;
+        Sub s;
+        s.ratio = __ddiv_rn(__dsub_rn(risk_of(A, it, k), risk_of(A, it, cur)), (double)dT);
+        s.dT = dT; s.item = it; s.k = k;
+        if (better(s, best)) best = s;
+      }
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) {
+        const Sub o = shfl_sub(best, off);
+        if (better(o, best)) best = o;
+      }
+      if (lane == 0) wbest[warp] = best;
+      __syncthreads();
+      if (tid == 0) {
+        Sub b = wbest[0];
+        for (int w = 1; w < 32; ++w) if (better(wbest[w], b)) b = wbest[w];
+        if (b.k < 0) {
+          sh_feasible = 0;
+        } else {
+          ch[b.item] = b.k;
+          sh_total -= b.dT;
+        }
+      }
+      __syncthreads();
+      if (sh_feasible == 0) break;
+    }
+    // ---- fallback walk: larger budget of the family first, then dense
+    if (A.prm.use_cert) {
+      for (int it = tid; it < A.n_items; it += kThreads) {
+        const int s = it / A.Hq, h = it - s * A.Hq;
+        const double vm = (double)A.vmax[s * A.Hkv + h / A.group];
+        int c = ch[it];
+        bool fired = false;
+        for (int guard = 0; guard < RS_MAX_CANDIDATES + 1 && A.lib[c].pattern != RS_DENSE; ++guard) {
+          const double m_low = fmax(0.0, __dsub_rn(m_hat_of(A, it, c), A.prm.delta_q));
+          double cert = __dmul_rn(2.0, __dsub_rn(1.0, m_low));
+          if (A.prm.cert_mode == RS_CERT_ABS) cert = __dmul_rn(cert, vm);
+          if (!(cert > A.prm.cert_max)) break;
+          fired = true;
+          const int nxt = A.prm.expand_first ? A.next_larger[c] : -1;
+          c = (nxt >= 0) ? nxt : A.dense_c;
+        }
+        ch[it] = c;
+        if (fired) atomicAdd(&sh_fallback, 1);
+      }
+      __syncthreads();
+    }
+  }
+  if (A.prm.forced_dense != nullptr) {
+    for (int it = tid; it < A.n_items; it += kThreads)
+      if (A.prm.forced_dense[it] != 0) ch[it] = A.dense_c;
+  }
+  __syncthreads();
+  for (int it = tid; it < A.n_items; it += kThreads) A.choice[it] = ch[it];
+  if (A.report != nullptr) {
+    long long part = 0;
+    for (int it = tid; it < A.n_items; it += kThreads) part += cost_of(A, it, ch[it]);
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+    if (lane == 0) wsum[warp] = part;
+    __syncthreads();
+    if (tid == 0) {
+      long long t = A.prm.t_probe;
+      for (int w = 0; w < 32; ++w) t += wsum[w];
+      double risk = 0.0;
+      for (int it = 0; it < A.n_items; ++it) risk = __dadd_rn(risk, risk_of(A, it, ch[it]));
+      A.report->total_cost = t;
+      A.report->total_risk = risk;
+      A.report->n_fallback = sh_fallback;
+      A.report->feasible = sh_feasible;
+    }
+  }
+  if (tid == 0 && sh_feasible == 0 && A.status != nullptr) A.status[3] = 1;   // budget cannot be met
+}
+
+}  // namespace
+
+extern "C" int rs_route(const rs_problem* p, const rs_candidate* lib, int n_cand, const rs_cand_stats* stats,
+                        const int64_t* cost, const float* vmax, const rs_route_params* params, int32_t* choice,
+                        rs_route_report* report, int32_t* status, void* stream_) {
+  int rc = rs_check_problem(p);
+  if (rc != RS_OK) return rc;
+  if (!lib || n_cand <= 0 || n_cand > RS_MAX_CANDIDATES || !params || !choice) return RS_ERR_INVALID_ARG;
+  const int n_items = p->n_segments * p->n_q_heads;
+  if (n_items > kMaxItems) return RS_ERR_UNSUPPORTED_SHAPE;
+  RouteArgs A{};
+  A.n_items = n_items; A.n_cand = n_cand; A.Hq = p->n_q_heads; A.Hkv = p->n_kv_heads;
+  A.group = p->n_q_heads / p->n_kv_heads; A.dense_c = -1;
+  for (int c = 0; c < n_cand; ++c) {
+    A.lib[c] = lib[c];
+    if (lib[c].pattern == RS_DENSE && A.dense_c < 0) A.dense_c = c;
+    A.next_larger[c] = -1;
+    for (int k = c + 1; k < n_cand; ++k)
+      if (lib[k].pattern == lib[c].pattern) { A.next_larger[c] = k; break; }
+  }
+  if (A.dense_c < 0) return RS_ERR_INVALID_ARG;          // the library must contain the dense candidate
+  if (params->fixed_choice == nullptr && stats == nullptr) return RS_ERR_INVALID_ARG;
+  if (params->use_cert && params->cert_mode == RS_CERT_ABS && vmax == nullptr) return RS_ERR_INVALID_ARG;
+  A.stats = stats; A.cost = cost; A.vmax = vmax; A.prm = *params; A.choice = choice; A.report = report;
+  A.status = status;
+  rs_route_kernel<<<1, kThreads, 0, (cudaStream_t)stream_>>>(A);
+  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+}

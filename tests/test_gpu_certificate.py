@@ -1,0 +1,32 @@
+"""GPU parity: rs_certificate against the oracle (Eq. 5), and the bound against the true error."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_29058_b200 as rs
+from oracle import certificate as CT
+
+pytestmark = pytest.mark.gpu
+
+
+def test_certificate_matches_oracle():
+    rng = np.random.default_rng(0)
+    Hq, n, R = 3, 512, 200
+    lse_full = rng.uniform(2, 8, (Hq, R)).astype(np.float32)
+    rows = np.sort(rng.choice(n, R, replace=False)).astype(np.int32)
+    lse_sel = np.zeros((Hq, n), np.float32)
+    lse_sel[:, rows] = lse_full - rng.exponential(0.05, (Hq, R)).astype(np.float32)
+    lse_sel[0, rows[:5]] = lse_full[0, :5] + 1e-6          # rounding may put lse_sel a hair above: m clamps to 1
+    onorm = rng.uniform(0, 10, (Hq, n)).astype(np.float32)
+    vmax = np.float32([13.5, 12.0, 14.25])
+    t = lambda a: torch.from_numpy(a).cuda()
+    out = [torch.zeros((Hq, R), device="cuda") for _ in range(3)] + [torch.zeros(Hq, device="cuda"), torch.zeros((Hq, 2), device="cuda")]
+    rs.rs_certificate(Hq, n, t(lse_sel), t(lse_full), t(rows), t(vmax), t(onorm), 0.01, *out, None)
+    m_row, cert_row, tight, m_head, cert_head = [o.cpu().numpy() for o in out]
+    for h in range(Hq):
+        m, cert, tg, mh, ch, cm = CT.certificate(lse_sel[h, rows], lse_full[h], vmax[h], onorm[h, rows], 0.01)
+        assert np.allclose(m_row[h], m, rtol=1e-5, atol=1e-6)
+        assert np.allclose(cert_row[h], cert, rtol=1e-4, atol=1e-5)
+        assert np.allclose(tight[h], tg, rtol=1e-4, atol=1e-5)
+        assert abs(m_head[h] - mh) < 1e-6 and abs(cert_head[h, 0] - ch) < 1e-4 and abs(cert_head[h, 1] - cm) < 1e-4
+    assert np.all(m_row <= 1.0) and np.all(cert_row >= 0)

@@ -1,0 +1,67 @@
+"""GPU parity: rs_probe against the oracle's probe (Eq. 3, last-64-query form).
+
+Tolerance: probe scores within 1e-3 relative (fp32 accumulation, ex2.approx) with an absolute floor of 1e-7
+for entries that underflow; pooled means and V_max within 1e-5 relative.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_29058_b200 as rs
+from gpu_helpers import dev_bf16, f64_heads
+from oracle import probe as OP
+from synth import make_layer, tiny_spec
+
+pytestmark = pytest.mark.gpu
+
+
+def run_probe(L, p):
+    Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+    S, Hq, Hkv, n = p.n_segments, p.n_q_heads, p.n_kv_heads, p.n_keys
+    f32 = dict(dtype=torch.float32, device="cuda")
+    out = dict(vert=torch.full((S, Hq, 4, n), 7.0, **f32), slash=torch.full((S, Hq, 4, n), 7.0, **f32),
+               lse=torch.zeros((S, Hq, 64), **f32), qpool=torch.zeros((Hq, n // 64, 128), **f32),
+               kpool=torch.zeros((Hkv, n // 64, 128), **f32), vmax=torch.zeros((S, Hkv), **f32))
+    ws = rs.new_workspace(p, None)
+    st = rs.new_status()
+    rs.rs_probe(p, Q, K, V, out["vert"], out["slash"], out["lse"], out["qpool"], out["kpool"], out["vmax"], None, ws, st)
+    rs.check_status(st, "probe")
+    return {k: v.cpu().numpy() for k, v in out.items()}
+
+
+def close(a, b, rtol=1e-3, floor=1e-7):
+    return np.all(np.abs(a - b) <= rtol * np.abs(b) + floor)
+
+
+@pytest.mark.parametrize("n,Hq,Hkv,bounds", [(256, 2, 1, None), (1088, 4, 2, [0, 320, 1088]), (704, 4, 1, None),
+                                             (448, 2, 2, [0, 64, 448]), (640, 8, 1, None)])
+def test_probe_matches_oracle(n, Hq, Hkv, bounds):
+    L = make_layer(tiny_spec(31 + n, n, Hq, Hkv))
+    p = rs.Problem(Hq, Hkv, n, bounds or [0, n])
+    got = run_probe(L, p)
+    Qs, Ks, Vs = f64_heads(L)
+    G = Hq // Hkv
+    for s in range(p.n_segments):
+        q1 = p.seg_bounds[s + 1]
+        for h in range(Hq):
+            pr = OP.probe_rows(Qs[h], Ks[h // G], q1)
+            assert close(got["lse"][s, h], pr.lse, 1e-5, 1e-4), (s, h)
+            assert close(got["vert"][s, h][:, :q1], pr.vert), (s, h)
+            assert close(got["slash"][s, h][:, :q1], pr.slash), (s, h)
+            assert np.all(got["vert"][s, h][:, q1:] == 0) and np.all(got["slash"][s, h][:, q1:] == 0)
+            assert abs(got["vert"][s, h].sum() - 64) < 1e-2 and abs(got["slash"][s, h].sum() - 64) < 1e-2
+        for g in range(Hkv):
+            _, vmax = OP.value_norms(Vs[g], q1)
+            assert abs(got["vmax"][s, g] - vmax) <= 1e-5 * vmax
+    for h in range(Hq):
+        assert np.allclose(got["qpool"][h], OP.pool_mean(Qs[h]), rtol=1e-5, atol=1e-6)
+    for g in range(Hkv):
+        assert np.allclose(got["kpool"][g], OP.pool_mean(Ks[g]), rtol=1e-5, atol=1e-6)
+
+
+def test_probe_is_deterministic():
+    L = make_layer(tiny_spec(77, 1024, 4, 1))
+    p = rs.Problem(4, 1, 1024)
+    a, b = run_probe(L, p), run_probe(L, p)
+    for k in a:
+        assert np.array_equal(a[k], b[k]), k
