@@ -114,7 +114,8 @@ int rs_workspace_bytes(const rs_problem* p, const rs_candidate* lib, int n_cand,
  * exact softmax rows of the last 64 queries over all causal keys, reduced to
  *   vert  [n_seg][n_q_heads][4][n_keys]  column mass per probe group          (fp32, 0 beyond the segment end)
  *   slash [n_seg][n_q_heads][4][n_keys]  diagonal mass per offset i - j        (fp32)
- *   lse_probe [n_seg][n_q_heads][64]     log-sum-exp of each probe row         (fp32)
+ *   lse_probe [n_q_heads][n_seg][64]     log-sum-exp of each probe row         (fp32; the layout rs_certificate
+ *                                        takes as lse_full for rows = the segments' last 64 rows)
  * plus the pooled signals of the coarse block candidates and the value norms of Eq. 5:
  *   qpool [n_q_heads][n_keys/64][d], kpool [n_kv_heads][n_keys/64][d]  64-row means (fp32)
  *   vmax  [n_seg][n_kv_heads]   max_j ||v_j||_2 over j < segment end             (fp32)
@@ -170,10 +171,12 @@ int rs_dense_prefill_attn(const rs_problem* p, const void* Q, const void* K, con
  * and per head: m_head = mean_i m_i, cert_head[h][0] = 2 (1 - max(0, m_head - delta_q)) V_max,
  * cert_head[h][1] = max_i cert_i.
  * lse_sel, onorm: [n_q_heads][n_keys].  rows: device int32[n_rows] query row ids (same for every head);
- * lse_full: [n_q_heads][n_rows].  vmax_head: [n_q_heads] (V_max of the head's KV head).
- * Outputs m_row, cert_row, cert_tight: [n_q_heads][n_rows]; m_head [n_q_heads]; cert_head [n_q_heads][2]. */
-int rs_certificate(int n_q_heads, int n_keys, const float* lse_sel, const float* lse_full,
-                   const int32_t* rows, int n_rows, const float* vmax_head, const float* onorm, float delta_q,
+ * lse_full: [n_q_heads][n_rows].  vmax: [n_kv_heads], any upper bound of the value norms of that KV head
+ * (rs_probe's vmax row of the last segment qualifies).
+ * Outputs (each may be NULL) m_row, cert_row, cert_tight: [n_q_heads][n_rows]; m_head [n_q_heads];
+ * cert_head [n_q_heads][2]. */
+int rs_certificate(int n_q_heads, int n_kv_heads, int n_keys, const float* lse_sel, const float* lse_full,
+                   const int32_t* rows, int n_rows, const float* vmax, const float* onorm, float delta_q,
                    float* m_row, float* cert_row, float* cert_tight, float* m_head, float* cert_head,
                    int32_t* status, void* stream);
 

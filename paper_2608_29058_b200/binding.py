@@ -205,12 +205,12 @@ def rs_dense_prefill_attn(p: Problem, Q, K, V, O, lse, onorm, counters, ws, stat
                                         _stream()), "rs_dense_prefill_attn")
 
 
-def rs_certificate(n_q_heads: int, n_keys: int, lse_sel, lse_full, rows, vmax_head, onorm, delta_q: float,
-                   m_row, cert_row, cert_tight, m_head, cert_head, status):
-    _check(load().rs_certificate(n_q_heads, n_keys, _ptr(lse_sel), _ptr(lse_full), _ptr(rows), int(rows.numel()),
-                                 _ptr(vmax_head), _ptr(onorm), C.c_float(delta_q), _ptr(m_row), _ptr(cert_row),
-                                 _ptr(cert_tight), _ptr(m_head), _ptr(cert_head), _ptr(status), _stream()),
-           "rs_certificate")
+def rs_certificate(n_q_heads: int, n_kv_heads: int, n_keys: int, lse_sel, lse_full, rows, vmax, onorm,
+                   delta_q: float, m_row, cert_row, cert_tight, m_head, cert_head, status):
+    _check(load().rs_certificate(n_q_heads, n_kv_heads, n_keys, _ptr(lse_sel), _ptr(lse_full), _ptr(rows),
+                                 int(rows.numel()), _ptr(vmax), _ptr(onorm), C.c_float(delta_q), _ptr(m_row),
+                                 _ptr(cert_row), _ptr(cert_tight), _ptr(m_head), _ptr(cert_head), _ptr(status),
+                                 _stream()), "rs_certificate")
 
 
 def check_status(status: torch.Tensor, what: str = "kernel"):

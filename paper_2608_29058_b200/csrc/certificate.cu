@@ -5,13 +5,13 @@
 namespace {
 
 __global__ void __launch_bounds__(256)
-rs_certificate_kernel(int n_keys, const float* lse_sel, const float* lse_full, const int32_t* rows, int n_rows,
+rs_certificate_kernel(int n_keys, int group, const float* lse_sel, const float* lse_full, const int32_t* rows, int n_rows,
                       const float* vmax_head, const float* onorm, float delta_q, float* m_row, float* cert_row,
                       float* cert_tight, float* m_head, float* cert_head) {
   __shared__ double s_sum[8];
   __shared__ float s_max[8];
   const int h = blockIdx.x;
-  const float vmax = vmax_head[h];
+  const float vmax = vmax_head[h / group];
   double sum = 0.0;
   float cmax = 0.f;
   for (int r = threadIdx.x; r < n_rows; r += blockDim.x) {
@@ -45,14 +45,14 @@ rs_certificate_kernel(int n_keys, const float* lse_sel, const float* lse_full, c
 
 }  // namespace
 
-extern "C" int rs_certificate(int n_q_heads, int n_keys, const float* lse_sel, const float* lse_full,
+extern "C" int rs_certificate(int n_q_heads, int n_kv_heads, int n_keys, const float* lse_sel, const float* lse_full,
                               const int32_t* rows, int n_rows, const float* vmax_head, const float* onorm,
                               float delta_q, float* m_row, float* cert_row, float* cert_tight, float* m_head,
                               float* cert_head, int32_t* status, void* stream_) {
   (void)status;
-  if (n_q_heads <= 0 || n_keys <= 0 || n_rows <= 0 || !lse_sel || !lse_full || !rows || !vmax_head)
+  if (n_q_heads <= 0 || n_kv_heads <= 0 || n_q_heads % n_kv_heads != 0 || n_keys <= 0 || n_rows <= 0 || !lse_sel || !lse_full || !rows || !vmax_head)
     return RS_ERR_INVALID_ARG;
-  rs_certificate_kernel<<<n_q_heads, 256, 0, (cudaStream_t)stream_>>>(n_keys, lse_sel, lse_full, rows, n_rows, vmax_head,
+  rs_certificate_kernel<<<n_q_heads, 256, 0, (cudaStream_t)stream_>>>(n_keys, n_q_heads / n_kv_heads, lse_sel, lse_full, rows, n_rows, vmax_head,
                                                                      onorm, delta_q, m_row, cert_row, cert_tight, m_head,
                                                                      cert_head);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;

@@ -27,7 +27,7 @@ struct ProbeParams {
   int n_splits;
   float2* partial;    // [n_seg*Hkv*n_hc][n_splits][256] (max, sum) in the exp2 domain
   float* lse2;        // [n_seg*Hkv*n_hc][256] log-sum-exp * log2(e)
-  float* lse_probe;   // [n_seg][Hq][64]
+  float* lse_probe;   // [Hq][n_seg][64]
   float* vert;        // [n_seg][Hq][4][n]
   float* slash;       // [n_seg][Hq][4][n]
   int32_t* status;
@@ -47,14 +47,6 @@ struct Smem {
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
-
-// Common prologue: barriers, TMEM, probe-row tile load.  Returns the TMEM base.
-struct Ctx {
-  uint32_t base, tmem;
-  uint32_t bar_q, bar_full[kStages], bar_empty[kStages], bar_tfull[2], bar_tempty[2];
-  volatile int* abort_flag;
-  int s, g, hc, q1, n_heads, h0, t0, t1, unit;
-};
 
 template <int PASS>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -330,7 +322,7 @@ __global__ void rs_probe_merge_kernel(ProbeParams P) {
   P.lse2[(size_t)unit * kRows + row] = lse2;
   if (hc * kHC + hh < P.group) {
     const int h = g * P.group + hc * kHC + hh;
-    P.lse_probe[((size_t)s * P.Hq + h) * RS_PROBE_ROWS + (row & 63)] = lse2 * 0.6931471805599453f;
+    P.lse_probe[((size_t)h * P.n_seg + s) * RS_PROBE_ROWS + (row & 63)] = lse2 * 0.6931471805599453f;
   }
 }
 

@@ -47,6 +47,7 @@ __device__ __forceinline__ Sub shfl_sub(const Sub& a, int off) {
 
 __device__ __forceinline__ long long cost_of(const RouteArgs& A, int item, int c) {
   if (A.cost != nullptr) return A.cost[(size_t)item * A.n_cand + c];
+  if (A.stats == nullptr) return 0;
   return (long long)(4ull * RS_HEAD_DIM * A.stats[(size_t)item * A.n_cand + c].pairs);
 }
 
@@ -58,7 +59,7 @@ __device__ __forceinline__ double m_hat_of(const RouteArgs& A, int item, int c) 
 }
 
 __device__ __forceinline__ double risk_of(const RouteArgs& A, int item, int c) {
-  if (A.lib[c].pattern == RS_DENSE) return 0.0;
+  if (A.lib[c].pattern == RS_DENSE || A.stats == nullptr) return 0.0;
   const rs_cand_stats& st = A.stats[(size_t)item * A.n_cand + c];
   double mx = 0.0, mn = 2.0;
 #pragma unroll

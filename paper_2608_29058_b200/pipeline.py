@@ -1,0 +1,177 @@
+"""Call sequence of one routed prefill attention layer (the six-step procedure of Section 3.4).
+
+This is the public, user-level entry of the package: it owns the device buffers of one layer and enqueues the
+C-ABI calls in order on the current CUDA stream.  It contains no arithmetic of the method -- every step runs
+in the library's kernels.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence
+
+import torch
+
+from . import binding as rs
+
+
+def default_library() -> List[tuple]:
+    """13-candidate online library: four budgets per sparse family by increasing budget, then dense."""
+    lib = [(rs.RS_A_SHAPE, 128, w) for w in (1024, 2048, 4096, 8192)]
+    lib += [(rs.RS_VERTICAL_SLASH, kv, ks) for kv, ks in ((500, 3048), (1000, 6096), (2000, 12192), (4000, 24384))]
+    lib += [(rs.RS_BLOCK_SPARSE, kb, 0) for kb in (50, 100, 200, 400)]
+    lib += [(rs.RS_DENSE, 0, 0)]
+    return lib
+
+
+def dense_flops(seg_bounds: Sequence[int], n_q_heads: int, d: int = 128) -> int:
+    n = seg_bounds[-1]
+    return 4 * d * n_q_heads * (n * (n + 1) // 2)
+
+
+def probe_flops(seg_bounds: Sequence[int], n_q_heads: int, d: int = 128) -> int:
+    tot = 0
+    for q0, q1 in zip(seg_bounds[:-1], seg_bounds[1:]):
+        tot += 2 * 64 * q1 * d * n_q_heads + 2 * d * n_q_heads * ((q1 // 64) * (q1 // 64 + 1) // 2 - (q0 // 64) * (q0 // 64 + 1) // 2)
+    return tot
+
+
+@dataclass
+class RouteConfig:
+    budget_frac: float = 0.15          # layer budget T as a fraction of the dense FLOPs of the layer
+    alpha: float = 1.0
+    delta_q: float = 0.0
+    cert_max: Optional[float] = 0.05   # None disables the fallback step
+    cert_mode: int = rs.RS_CERT_REL
+    expand_first: bool = True
+
+
+class RoutedPrefillLayer:
+    """Device buffers and call order for one layer; reuse one instance for every layer of the same shape."""
+
+    def __init__(self, problem: rs.Problem, library: Optional[Sequence[Sequence[int]]] = None,
+                 route: Optional[RouteConfig] = None, out_dtype=torch.bfloat16, device="cuda"):
+        self.p = problem
+        self.cands = list(library) if library is not None else default_library()
+        self.lib = rs.make_library(self.cands)
+        self.cfg = route or RouteConfig()
+        p, S, Hq, Hkv, n = problem, problem.n_segments, problem.n_q_heads, problem.n_kv_heads, problem.n_keys
+        f32 = dict(dtype=torch.float32, device=device)
+        self.vert = torch.empty((S, Hq, 4, n), **f32)
+        self.slash = torch.empty((S, Hq, 4, n), **f32)
+        self.lse_probe = torch.empty((Hq, S, 64), **f32)
+        self.qpool = torch.empty((Hq, n // 64, 128), **f32)
+        self.kpool = torch.empty((Hkv, n // 64, 128), **f32)
+        self.vmax = torch.empty((S, Hkv), **f32)
+        self.stats = torch.zeros((p.n_items, len(self.cands), 5), dtype=torch.int64, device=device)
+        self.idx_eval = rs.IndexSet.for_library(p, self.lib, materialised=False, device=device)
+        self.idx = rs.IndexSet.for_library(p, self.lib, materialised=True, device=device)
+        self.choice = torch.zeros(p.n_items, dtype=torch.int32, device=device)
+        self.report = torch.zeros(24, dtype=torch.uint8, device=device)
+        self.O = torch.empty((Hq, n, 128), dtype=out_dtype, device=device)
+        self.lse_sel = torch.empty((Hq, n), **f32)
+        self.onorm = torch.empty((Hq, n), **f32)
+        self.counters = torch.zeros(2, dtype=torch.int64, device=device)
+        self.status = rs.new_status(device)
+        self.ws = rs.new_workspace(p, self.lib, device)
+        rows = []
+        for s in range(S):
+            rows += list(range(p.seg_bounds[s + 1] - 64, p.seg_bounds[s + 1]))
+        self.probe_rows = torch.tensor(rows, dtype=torch.int32, device=device)
+        R = len(rows)
+        self.m_row = torch.empty((Hq, R), **f32)
+        self.cert_row = torch.empty((Hq, R), **f32)
+        self.m_head = torch.empty((Hq,), **f32)
+        self.cert_head = torch.empty((Hq, 2), **f32)
+        self.prm = rs.rs_route_params()
+        self._forced = None
+        self.events = None
+
+    # ------------------------------------------------------------------ steps (each only enqueues kernels)
+    def probe(self, Q, K, V):
+        rs.rs_probe(self.p, Q, K, V, self.vert, self.slash, self.lse_probe, self.qpool, self.kpool, self.vmax, None,
+                    self.ws, self.status)
+
+    def evaluate_candidates(self):
+        rs.rs_build_indices(self.p, self.lib, self.vert, self.slash, self.qpool, self.kpool, None, None,
+                            self.idx_eval, self.stats, self.ws, self.status)
+
+    def route(self, forced_dense: Optional[torch.Tensor] = None):
+        c, prm = self.cfg, self.prm
+        prm.budget = int(c.budget_frac * dense_flops(self.p.seg_bounds, self.p.n_q_heads))
+        prm.t_probe = probe_flops(self.p.seg_bounds, self.p.n_q_heads)
+        prm.alpha, prm.delta_q = c.alpha, c.delta_q
+        prm.use_cert = 0 if c.cert_max is None else 1
+        prm.cert_max = 0.0 if c.cert_max is None else c.cert_max
+        prm.cert_mode, prm.expand_first = c.cert_mode, int(c.expand_first)
+        self._forced = forced_dense
+        prm.forced_dense = None if forced_dense is None else forced_dense.data_ptr()
+        prm.fixed_choice = None
+        rs.rs_route(self.p, self.lib, self.stats, None, self.vmax, prm, self.choice, self.report, self.status)
+
+    def materialise(self):
+        rs.rs_build_indices(self.p, self.lib, self.vert, self.slash, self.qpool, self.kpool, None, self.choice,
+                            self.idx, None, self.ws, self.status)
+
+    def attention(self, Q, K, V):
+        rs.rs_sparse_prefill_attn(self.p, Q, K, V, self.lib, self.idx, self.choice, self.O, self.lse_sel, self.onorm,
+                                  self.counters, self.ws, self.status)
+
+    def certificate(self):
+        p = self.p
+        rs.rs_certificate(p.n_q_heads, p.n_kv_heads, p.n_keys, self.lse_sel, self.lse_probe, self.probe_rows,
+                          self.vmax[p.n_segments - 1], self.onorm, self.cfg.delta_q, self.m_row, self.cert_row, None,
+                          self.m_head, self.cert_head, self.status)
+
+    # ------------------------------------------------------------------ whole layer
+    def forward(self, Q, K, V, fixed_choice: Optional[torch.Tensor] = None,
+                forced_dense: Optional[torch.Tensor] = None, record_events: bool = False) -> torch.Tensor:
+        """Routed sparse prefill attention of one layer; returns O (device). Nothing synchronises."""
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(7)] if record_events else None
+        mark = (lambda i: ev[i].record()) if record_events else (lambda i: None)
+        mark(0)
+        self.probe(Q, K, V)
+        mark(1)
+        if fixed_choice is None:
+            self.evaluate_candidates()
+            mark(2)
+            self.route(forced_dense)
+        else:
+            self.choice.copy_(fixed_choice)
+            mark(2)
+        mark(3)
+        self.materialise()
+        mark(4)
+        self.attention(Q, K, V)
+        mark(5)
+        self.certificate()
+        mark(6)
+        self.events = ev
+        return self.O
+
+    def stage_ms(self):
+        """Milliseconds per stage of the last forward(record_events=True): probe, evaluate, route, materialise,
+        attention, certificate (synchronises)."""
+        torch.cuda.synchronize()
+        e = self.events
+        names = ["probe", "evaluate", "route", "materialise", "attention", "certificate"]
+        return {names[i]: e[i].elapsed_time(e[i + 1]) for i in range(6)}
+
+    def route_report(self):
+        import numpy as np
+        r = self.report.cpu().numpy()
+        return dict(total_cost=int(r[:8].view(np.int64)[0]), total_risk=float(r[8:16].view(np.float64)[0]),
+                    n_fallback=int(r[16:20].view(np.int32)[0]), feasible=int(r[20:24].view(np.int32)[0]))
+
+
+def prefill_from_host(layer: RoutedPrefillLayer, Q_host: torch.Tensor, K_host: torch.Tensor, V_host: torch.Tensor,
+                      O_host: torch.Tensor, dev_bufs=None) -> torch.Tensor:
+    """End-to-end call with pinned HOST buffers: copies Q, K, V to the device, runs the layer, copies O back."""
+    if dev_bufs is None:
+        dev_bufs = tuple(torch.empty_like(t, device=layer.O.device) for t in (Q_host, K_host, V_host))
+    Qd, Kd, Vd = dev_bufs
+    Qd.copy_(Q_host, non_blocking=True)
+    Kd.copy_(K_host, non_blocking=True)
+    Vd.copy_(V_host, non_blocking=True)
+    O = layer.forward(Qd, Kd, Vd)
+    O_host.copy_(O, non_blocking=True)
+    return O_host

@@ -21,7 +21,7 @@ def test_certificate_matches_oracle():
     vmax = np.float32([13.5, 12.0, 14.25])
     t = lambda a: torch.from_numpy(a).cuda()
     out = [torch.zeros((Hq, R), device="cuda") for _ in range(3)] + [torch.zeros(Hq, device="cuda"), torch.zeros((Hq, 2), device="cuda")]
-    rs.rs_certificate(Hq, n, t(lse_sel), t(lse_full), t(rows), t(vmax), t(onorm), 0.01, *out, None)
+    rs.rs_certificate(Hq, Hq, n, t(lse_sel), t(lse_full), t(rows), t(vmax), t(onorm), 0.01, *out, None)
     m_row, cert_row, tight, m_head, cert_head = [o.cpu().numpy() for o in out]
     for h in range(Hq):
         m, cert, tg, mh, ch, cm = CT.certificate(lse_sel[h, rows], lse_full[h], vmax[h], onorm[h, rows], 0.01)

@@ -1,0 +1,130 @@
+"""GPU end-to-end: probe -> candidate evaluation -> routing -> materialisation -> attention -> certificate,
+checked stage by stage against the oracle (each stage is fed what the previous GPU stage produced, so that a
+1e-3 difference in probe scores cannot flip a later integer decision inside the comparison)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_29058_b200 as rs
+from gpu_helpers import assert_attention_close, dev_bf16, f64_heads
+from oracle import attention as A
+from oracle import certificate as CT
+from oracle import patterns as PT
+from oracle import probe as OP
+from oracle import routing as RT
+from synth import config1_spec, make_layer, tiny_spec
+
+pytestmark = pytest.mark.gpu
+C = PT.Candidate
+
+
+def download_sets(layer, cands, choice):
+    p = layer.p
+    nb = p.n_keys // 64
+    cnt = layer.idx.vs_count.cpu().numpy()
+    cols, offs, diag = (t.cpu().numpy() for t in (layer.idx.vs_cols, layer.idx.vs_offs, layer.idx.vs_diag))
+    blk, bcnt = layer.idx.bs_blk.cpu().numpy(), layer.idx.bs_count.cpu().numpy()
+    sets = []
+    for item in range(p.n_items):
+        s, h = divmod(item, p.n_q_heads)
+        q0, q1 = p.seg_bounds[s], p.seg_bounds[s + 1]
+        cand = cands[choice[item]]
+        ix = PT.IndexSet(cand=cand, q0=q0, q1=q1)
+        if cand.pattern == PT.VERTICAL_SLASH:
+            ix.V, ix.S, ix.D = cols[item, :cnt[item, 0]], offs[item, :cnt[item, 1]], diag[item, :cnt[item, 2]]
+        elif cand.pattern == PT.BLOCK_SPARSE:
+            ix.blk = [blk[h * nb + qb, :bcnt[h * nb + qb]] for qb in range(q0 // 64, q1 // 64)]
+        sets.append(ix)
+    return sets
+
+
+def run_and_check(spec, bounds, cands, cfg, seed_name):
+    L = make_layer(spec)
+    Hq, Hkv, n = spec.n_q_heads, spec.n_kv_heads, spec.n
+    p = rs.Problem(Hq, Hkv, n, bounds)
+    layer = rs.RoutedPrefillLayer(p, [(c.pattern, c.b0, c.b1) for c in cands], cfg, out_dtype=torch.float32)
+    Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+    O = layer.forward(Q, K, V).cpu().numpy()
+    rs.check_status(layer.status, seed_name)
+    Qs, Ks, Vs = f64_heads(L)
+    G = Hq // Hkv
+    vert, slash = layer.vert.cpu().numpy(), layer.slash.cpu().numpy()
+    stats = layer.stats.cpu().numpy()
+    choice = layer.choice.cpu().numpy()
+    # stage 2: candidate stats from the GPU's own probe scores (A-shape, vertical-slash, dense: bit-exact)
+    cov = stats[:, :, :4].astype(np.uint64)
+    pairs = stats[:, :, 4]
+    for item in range(p.n_items):
+        s, h = divmod(item, Hq)
+        q0, q1 = p.seg_bounds[s], p.seg_bounds[s + 1]
+        for c, cand in enumerate(cands):
+            if cand.pattern == PT.BLOCK_SPARSE:
+                assert pairs[item, c] == sum((min(cand.b0, qb + 1) - 1) * 4096 + 2080 for qb in range(q0 // 64, q1 // 64))
+                continue
+            ix = PT.build_indices(cand, q0, q1, vert[s, h][:, :q1], slash[s, h][:, :q1], None)
+            assert pairs[item, c] == PT.pairs(ix), (item, cand)
+            if cand.pattern != PT.DENSE:
+                assert cov[item, c].tolist() == PT.coverage_fx(ix, vert[s, h][:, :q1], slash[s, h][:, :q1]).tolist()
+    # stage 3: routing from the GPU's stats
+    vmax = layer.vmax.cpu().numpy()
+    vmax_item = np.array([vmax[it // Hq, (it % Hq) // G] for it in range(p.n_items)], np.float32)
+    want, wrep = RT.route(cands, cov, 512 * pairs, vmax_item, RT.RouteParams(
+        budget=int(cfg.budget_frac * rs.dense_flops(p.seg_bounds, Hq)), t_probe=rs.probe_flops(p.seg_bounds, Hq),
+        alpha=cfg.alpha, delta_q=cfg.delta_q, cert_max=cfg.cert_max, cert_mode=cfg.cert_mode,
+        expand_first=cfg.expand_first))
+    assert np.array_equal(choice, want)
+    rep = layer.route_report()
+    assert rep["total_cost"] == wrep.total_cost and rep["feasible"] == wrep.feasible and rep["n_fallback"] == wrep.n_fallback
+    # stage 4: attention under the materialised index sets; stage 5: certificate against the true error
+    sets = download_sets(layer, cands, choice)
+    lse_sel, onorm = layer.lse_sel.cpu().numpy(), layer.onorm.cpu().numpy()
+    m_head, cert_head = layer.m_head.cpu().numpy(), layer.cert_head.cpu().numpy()
+    m_rows = layer.m_row.cpu().numpy()
+    for item, ix in enumerate(sets):
+        s, h = divmod(item, Hq)
+        g = h // G
+        rows = np.arange(ix.q0, ix.q1)
+        if ix.cand.pattern == PT.VERTICAL_SLASH:      # lists equal the oracle's selection on the same scores
+            ref = PT.build_indices(ix.cand, ix.q0, ix.q1, vert[s, h][:, :ix.q1], slash[s, h][:, :ix.q1], None)
+            assert np.array_equal(ix.V, ref.V) and np.array_equal(ix.S, ref.S) and np.array_equal(ix.D, ref.D)
+        Om, lo, no = A.masked_attention(Qs[h], Ks[g], Vs[g], lambda r, nk: PT.mask_rows(ix, r, nk), rows)
+        assert_attention_close(O[h, rows], Om, f"item {item} {ix.cand}")
+        assert np.abs(lse_sel[h, rows] - lo).max() < 2e-3
+        Od, ld = A.dense_attention(Qs[h], Ks[g], Vs[g], rows)
+        _, vm = OP.value_norms(Vs[g], n)
+        m, cert, tight, _, _, _ = CT.certificate(lse_sel[h, rows], ld, vm, onorm[h, rows])
+        # Eq. 5 on every row: the certificate built from the kernel's log-sum-exp bounds the exact error of the mask
+        # (1e-2 absorbs the fp32 rounding of lse_sel, which enters as 2 * V_max * |d lse|)
+        err = np.linalg.norm(Od.astype(np.float64) - Om.astype(np.float64), axis=1)
+        assert np.all(cert + 1e-2 >= err), (item, ix.cand)
+        # online certificate on the probe rows: kernel-side mass equals builder-side coverage
+        if ix.cand.pattern != PT.DENSE:
+            m_hat, _ = PT.m_hat_from_fx(cov[item, choice[item]])
+            assert abs(m_rows[h, 64 * s:64 * s + 64].mean() - m_hat) < 2e-3, (item, ix.cand)
+    for h in range(Hq):
+        assert abs(m_head[h] - m_rows[h].mean()) < 1e-5
+        assert cert_head[h, 1] >= 0
+    return layer, choice
+
+
+def test_pipeline_small_layer_with_segments():
+    cands = [C(PT.A_SHAPE, 8, 128), C(PT.A_SHAPE, 8, 256), C(PT.VERTICAL_SLASH, 32, 48), C(PT.VERTICAL_SLASH, 64, 96),
+             C(PT.BLOCK_SPARSE, 3), C(PT.BLOCK_SPARSE, 6), C(PT.DENSE)]
+    cfg = rs.RouteConfig(budget_frac=0.45, cert_max=0.6)
+    layer, choice = run_and_check(tiny_spec(61, 1536, 4, 2), [0, 768, 1536], cands, cfg, "small")
+    assert len(set(choice.tolist())) > 1          # the router really mixes patterns on this input
+
+
+def test_pipeline_tight_budget_and_abs_certificate():
+    cands = [C(PT.A_SHAPE, 8, 128), C(PT.VERTICAL_SLASH, 32, 48), C(PT.BLOCK_SPARSE, 3), C(PT.DENSE)]
+    cfg = rs.RouteConfig(budget_frac=0.2, cert_max=0.05, cert_mode=rs.RS_CERT_ABS, expand_first=False)
+    run_and_check(tiny_spec(63, 1024, 4, 4), [0, 1024], cands, cfg, "abs")
+
+
+def test_config1_single_head_vertical_slash():
+    """n = 4096, one head, vertical-slash (256 verticals, 512 slashes) forced through a two-entry library."""
+    spec = config1_spec(toeplitz=True)
+    cands = [C(PT.VERTICAL_SLASH, 256, 512), C(PT.DENSE)]
+    cfg = rs.RouteConfig(budget_frac=0.6, cert_max=None)
+    layer, choice = run_and_check(spec, [0, 4096], cands, cfg, "config1")
+    assert choice.tolist() == [0]

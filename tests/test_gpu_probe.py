@@ -20,7 +20,7 @@ def run_probe(L, p):
     S, Hq, Hkv, n = p.n_segments, p.n_q_heads, p.n_kv_heads, p.n_keys
     f32 = dict(dtype=torch.float32, device="cuda")
     out = dict(vert=torch.full((S, Hq, 4, n), 7.0, **f32), slash=torch.full((S, Hq, 4, n), 7.0, **f32),
-               lse=torch.zeros((S, Hq, 64), **f32), qpool=torch.zeros((Hq, n // 64, 128), **f32),
+               lse=torch.zeros((Hq, S, 64), **f32), qpool=torch.zeros((Hq, n // 64, 128), **f32),
                kpool=torch.zeros((Hkv, n // 64, 128), **f32), vmax=torch.zeros((S, Hkv), **f32))
     ws = rs.new_workspace(p, None)
     st = rs.new_status()
@@ -45,7 +45,7 @@ def test_probe_matches_oracle(n, Hq, Hkv, bounds):
         q1 = p.seg_bounds[s + 1]
         for h in range(Hq):
             pr = OP.probe_rows(Qs[h], Ks[h // G], q1)
-            assert close(got["lse"][s, h], pr.lse, 1e-5, 1e-4), (s, h)
+            assert close(got["lse"][h, s], pr.lse, 1e-5, 1e-4), (s, h)
             assert close(got["vert"][s, h][:, :q1], pr.vert), (s, h)
             assert close(got["slash"][s, h][:, :q1], pr.slash), (s, h)
             assert np.all(got["vert"][s, h][:, q1:] == 0) and np.all(got["slash"][s, h][:, q1:] == 0)
