@@ -1,0 +1,438 @@
+#!/usr/bin/env python
+"""Benchmark of the routed sparse prefill attention layer (one JSON line on stdout).
+
+A step is one pass of the whole hot path over one layer: probe -> candidate evaluation -> routing ->
+materialisation -> one sparse attention launch -> certificate.  Default workload: the Llama-3.1-8B-shaped
+layer (32 query heads, 8 KV heads, d = 128) at n = 131072 with routing decided online (budget 15 % of the
+dense FLOPs, relative certificate threshold 0.05), synthetic seeded inputs.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config3|config2|config1] [--n N]
+  python bench.py --impl reference ...        # times the CPU oracle on the host cores instead
+
+Multi-GPU: the path has no exchange step, so N ranks run N independent replicas of the layer (weak scaling);
+the only cross-rank traffic is the barrier and the max-over-ranks of the measured time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["source"] = "fallback"
+    return d
+
+
+# ----------------------------------------------------------------------------------------- workloads
+def workload_spec(name: str, n_override: int | None):
+    from synth import config1_spec, config2_spec
+    if name == "config1":
+        spec = config1_spec(toeplitz=True, n=n_override or 4096)
+        lib = [(2, 256, 512), (0, 0, 0)]
+        route = dict(budget_frac=0.6, cert_max=None)
+        fixed = None
+    elif name == "config2":
+        spec = config2_spec(n=n_override or 32768)
+        lib = [(1, 128, 1024), (2, 1000, 6096), (3, 100, 0), (0, 0, 0)]
+        route = dict(budget_frac=1.0, cert_max=None)
+        fixed = "seeded 30/30/30/10"
+    else:
+        spec = config2_spec(n=n_override or 131072, seed_offset=3)
+        lib = None     # 13-candidate default library
+        route = dict(budget_frac=0.15, cert_max=0.05)
+        fixed = None
+    return spec, lib, route, fixed
+
+
+def fixed_choice_for(lib, n_q_heads):
+    from synth import fixed_routes_config2
+    pat = fixed_routes_config2(n_q_heads)
+    index_of = {c[0]: i for i, c in enumerate(lib)}
+    return np.array([index_of[int(x)] for x in pat], dtype=np.int32)
+
+
+# ----------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7 or not (t0 - 0.05 <= ts <= t1 + 0.15):
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------- rank plumbing
+def init_ranks(n_gpus: int, backend: str = "nccl"):
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1 and not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, world
+
+
+def aggregate_over_ranks(ms_local: float, units_local: float, device=None):
+    """Max of the time and sum of the processed units over all ranks (replicas: no data-path collective)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return ms_local, units_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ----------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float = 20.0):
+    """Times the oracle's masked attention on sampled query blocks under the routed masks.
+
+    Returns (effective TFLOP/s, description, cores, max abs difference to gpu_O on the sampled rows).
+    """
+    from oracle import attention as OA
+    from oracle import patterns as PT
+    from synth import bf16_bits_to_f64
+    G = spec.n_q_heads // spec.n_kv_heads
+    nb = spec.n // 64
+    heads = sorted(set(int(h) for h in np.linspace(0, spec.n_q_heads - 1, 4)))
+    blocks = sorted(set([nb // 4, nb // 2, nb - 1]))
+    t_used, pairs_done, rows_done, worst = 0.0, 0, 0, 0.0
+    kv_cache = {}
+    for h in heads:
+        g = h // G
+        if g not in kv_cache:
+            kv_cache = {g: (bf16_bits_to_f64(L["K"][g]), bf16_bits_to_f64(L["V"][g]))}
+        Kf, Vf = kv_cache[g]
+        Qf = bf16_bits_to_f64(L["Q"][h])
+        ix = sets_fn(h)
+        for qb in blocks:
+            if t_used > budget_s:
+                break
+            rows = np.arange(qb * 64, qb * 64 + 64)
+            t0 = time.perf_counter()
+            Om, _, _ = OA.masked_attention(Qf, Kf, Vf, lambda r, nk: PT.mask_rows(ix, r, nk), rows, chunk=64)
+            t_used += time.perf_counter() - t0
+            M = PT.mask_rows(ix, rows, int(rows.max()) + 1) & (np.arange(int(rows.max()) + 1)[None, :] <= rows[:, None])
+            pairs_done += int(M.sum())
+            rows_done += 64
+            if gpu_O is not None:
+                worst = max(worst, float(np.abs(gpu_O[h, rows].astype(np.float64) - Om).max()))
+    tflops = 512.0 * pairs_done / max(t_used, 1e-9) / 1e12
+    desc = (f"oracle masked attention on {rows_done} sampled query rows (heads {heads}, query blocks {blocks}) of the "
+            f"same routed layer, {t_used:.1f} s; effective = 512 FLOP x selected pairs / time")
+    return tflops, desc, os.cpu_count(), worst
+
+
+def download_sets(layer, cands, choice):
+    """Device index lists of the routed candidates -> the oracle's IndexSet objects (CPU-baseline leg only)."""
+    from oracle import patterns as PT
+    p = layer.p
+    nb = p.n_keys // 64
+    cnt = layer.idx.vs_count.cpu().numpy()
+    cols, offs, diag = (t.cpu().numpy() for t in (layer.idx.vs_cols, layer.idx.vs_offs, layer.idx.vs_diag))
+    blk, bcnt = layer.idx.bs_blk.cpu().numpy(), layer.idx.bs_count.cpu().numpy()
+    sets = []
+    for item in range(p.n_items):
+        s, h = divmod(item, p.n_q_heads)
+        q0, q1 = p.seg_bounds[s], p.seg_bounds[s + 1]
+        cand = cands[choice[item]]
+        ix = PT.IndexSet(cand=cand, q0=q0, q1=q1)
+        if cand.pattern == PT.VERTICAL_SLASH:
+            ix.V, ix.S, ix.D = cols[item, :cnt[item, 0]], offs[item, :cnt[item, 1]], diag[item, :cnt[item, 2]]
+        elif cand.pattern == PT.BLOCK_SPARSE:
+            ix.blk = [blk[h * nb + qb, :bcnt[h * nb + qb]] for qb in range(q0 // 64, q1 // 64)]
+        sets.append(ix)
+    return sets
+
+
+# ----------------------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config3", choices=["config1", "config2", "config3"])
+    ap.add_argument("--n", type=int, default=None, help="override the sequence length (smaller profiling case)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-dense", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from synth import make_layer
+    spec, lib, route_kw, fixed = workload_spec(args.workload, args.n)
+    metric = "effective TFLOP/s of routed sparse prefill attention (FLOPs of selected query-key pairs / layer time)"
+    config = {"workload": f"{args.workload}: Hq={spec.n_q_heads} Hkv={spec.n_kv_heads} d=128 n={spec.n}, "
+                          + ("routes fixed from seed" if fixed else
+                             f"online routing, budget {route_kw['budget_frac']:.2f} of dense FLOPs, cert_max {route_kw['cert_max']}"),
+              "l2": "inputs (Q,K,V,O > 126 MB) exceed L2; no explicit flush" if spec.n >= 32768 else "small case, L2 resident",
+              "replicas": args.gpus}
+
+    if args.impl == "reference":
+        rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+        if rank != 0:
+            return 0
+        return reference_arm(args, spec, lib, route_kw, fixed, metric, config)
+
+    import torch
+    import paper_2608_29058_b200 as rs
+    rank, world = init_ranks(args.gpus)
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    peaks = measured_peaks()
+
+    L = make_layer(spec)
+    to_dev = lambda bits: torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    Q, K, V = to_dev(L["Q"]), to_dev(L["K"]), to_dev(L["V"])
+    p = rs.Problem(spec.n_q_heads, spec.n_kv_heads, spec.n, [int(x) for x in L["seg_bounds"]])
+    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(**route_kw), device=dev)
+    fixed_t = None
+    if fixed:
+        fixed_t = torch.from_numpy(fixed_choice_for(layer.cands, spec.n_q_heads)).to(dev)
+
+    def step(record=False):
+        return layer.forward(Q, K, V, fixed_choice=fixed_t, record_events=record)
+
+    def sync_all():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    rs.check_status(layer.status, "warm-up")
+
+    # ---- timed region: K steps, CUDA events on the launching stream, per-stage events inside every step
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stage_events = []
+    layer.counters.zero_()
+    t_wall0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        step(record=True)
+        stage_events.append(layer.events)
+    e1.record()
+    sync_all()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    ms_local = e0.elapsed_time(e1) / args.steps
+    rs.check_status(layer.status, "timed region")
+
+    names = ["probe", "evaluate", "route", "materialise", "attention", "certificate"]
+    stages = {nm: float(np.mean([ev[i].elapsed_time(ev[i + 1]) for ev in stage_events])) for i, nm in enumerate(names)}
+    counters = layer.counters.cpu().numpy()
+    chunks_per_step = int(counters[0]) // args.steps
+    choice = layer.choice.cpu().numpy()
+    stats = layer.stats.cpu().numpy()
+    if fixed:
+        layer.evaluate_candidates()      # pair counts of the fixed routes (outside the timed region)
+        torch.cuda.synchronize()
+        stats = layer.stats.cpu().numpy()
+    pairs_sel = int(sum(int(stats[it, choice[it], 4]) for it in range(p.n_items)))
+    f_mask = 512.0 * pairs_sel
+    f_tile = chunks_per_step * (128 * 64 * 512.0)
+    f_dense = float(rs.dense_flops(p.seg_bounds, p.n_q_heads))
+
+    ms, units = aggregate_over_ranks(ms_local, f_mask, dev)
+    value = units / (ms * 1e-3) / 1e12
+
+    # ---- own dense kernel (denominator of the speed-up), same inputs
+    dense_ms = None
+    if not args.no_dense:
+        ws = layer.ws
+        lse_d = torch.empty((p.n_q_heads, p.n_keys), dtype=torch.float32, device=dev)
+        O_d = torch.empty_like(layer.O)
+        reps = 2 if spec.n > 65536 else 3
+        rs.rs_dense_prefill_attn(p, Q, K, V, O_d, lse_d, None, None, ws, layer.status)
+        torch.cuda.synchronize()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record()
+        for _ in range(reps):
+            rs.rs_dense_prefill_attn(p, Q, K, V, O_d, lse_d, None, None, ws, layer.status)
+        d1.record()
+        torch.cuda.synchronize()
+        dense_ms = d0.elapsed_time(d1) / reps
+        del O_d, lse_d
+
+    # ---- end to end through the public call with pinned host buffers
+    e2e = None
+    if not args.no_e2e:
+        Qh, Kh, Vh = (torch.from_numpy(L[k].view(np.int16)).view(torch.bfloat16).pin_memory() for k in ("Q", "K", "V"))
+        Oh = torch.empty(tuple(layer.O.shape), dtype=layer.O.dtype).pin_memory()
+        bufs = (Q, K, V)
+        # fixed routes need the route tensor inside forward: bind it through a small closure
+        def e2e_step():
+            Q.copy_(Qh, non_blocking=True); K.copy_(Kh, non_blocking=True); V.copy_(Vh, non_blocking=True)
+            layer.forward(Q, K, V, fixed_choice=fixed_t)
+            Oh.copy_(layer.O, non_blocking=True)
+        e2e_step()
+        sync_all()
+        k_e2e = max(2, min(args.steps, 3))
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(k_e2e):
+            e2e_step()
+        g1.record()
+        sync_all()
+        ms_e2e, units_e2e = aggregate_over_ranks(g0.elapsed_time(g1) / k_e2e, f_mask, dev)
+        h2d = sum(int(t.numel() * t.element_size()) for t in (Qh, Kh, Vh))
+        d2h = int(Oh.numel() * Oh.element_size())
+        e2e = {"value": units_e2e / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        del Qh, Kh, Vh
+
+    if rank != 0:
+        return 0
+
+    # ---- CPU oracle on a bounded sample of the same workload (also a full-size parity spot check)
+    cpu = None
+    if not args.no_cpu_baseline:
+        from oracle import patterns as PT
+        cands = [PT.Candidate(c[0], c[1], c[2]) for c in layer.cands]
+        sets = download_sets(layer, cands, choice)
+        O_host = layer.O.float().cpu().numpy()
+        tf, desc, cores, worst = oracle_sample(L, spec, cands, choice, lambda h: sets[(p.n_segments - 1) * p.n_q_heads + h],
+                                               O_host)
+        cpu = {"value": tf, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc,
+               "max_abs_diff_vs_gpu_on_sample": worst}
+
+    peak = peaks["bf16_tflops_sustained"]
+    attn_ms = stages["attention"]
+    achieved = f_tile / (attn_ms * 1e-3) / 1e12
+    overhead_ms = stages["probe"] + stages["evaluate"] + stages["route"] + stages["materialise"] + stages["certificate"]
+    hist = {}
+    for it in range(p.n_items):
+        c = layer.cands[choice[it]]
+        key = {0: "dense", 1: "a_shape", 2: "vertical_slash", 3: "block_sparse"}[c[0]] + (f"({c[1]},{c[2]})" if c[0] else "")
+        hist[key] = hist.get(key, 0) + 1
+    any_vs = any(c[0] == 2 for c in layer.cands)
+    any_bs = any(c[0] == 3 for c in layer.cands)
+    launches_per_step = (7 + (0 if fixed else 2 + 2 * any_vs + any_bs + 1) + 2 * any_vs + 2 * any_bs
+                         + 3 + any_vs + 1)      # probe, evaluate + route, materialise, attention, certificate
+    out = {
+        "metric": metric, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "config": config,
+        "ms_per_layer": ms, "dense_ms_per_layer": dense_ms,
+        "speedup_vs_own_dense": (dense_ms / ms) if dense_ms else None,
+        "dense_tflops": (f_dense / (dense_ms * 1e-3) / 1e12) if dense_ms else None,
+        "stage_ms": stages, "overhead_over_attention": overhead_ms / attn_ms,
+        "flops": {"selected_pairs": f_mask, "issued_tiles": f_tile, "dense": f_dense,
+                  "selected_fraction_of_dense": f_mask / f_dense},
+        "routes": hist, "route_report": layer.route_report() if not fixed else None,
+        "roofline": {"kernel": "rs_attn_kernel (one launch, all heads)", "bound": "tensor", "achieved": achieved,
+                     "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "peak_source": f"bf16_tflops_sustained, {peaks['source']}",
+                     "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "traffic": None,
+                     "note": "achieved = 512 FLOP x 128 x 64 pairs per issued chunk / attention-call time (CUDA events)"},
+        "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
+    }
+    print(json.dumps(out))
+    return 0
+
+
+def reference_arm(args, spec, lib, route_kw, fixed, metric, config):
+    """The oracle as it stands, timed on the host cores on a bounded sample of the same workload per step."""
+    from synth import make_layer
+    from oracle import patterns as PT
+    from oracle import probe as OP
+    from synth import bf16_bits_to_f64
+    import paper_2608_29058_b200.pipeline as pl     # library list only (host data, no GPU work)
+    cands_raw = lib if lib is not None else pl.default_library()
+    cands = [PT.Candidate(c[0], c[1], c[2]) for c in cands_raw]
+    heads = sorted(set(int(h) for h in np.linspace(0, spec.n_q_heads - 1, 4)))
+    L = make_layer(spec, heads=heads)
+    Lq = {"Q": {h: L["Q"][i] for i, h in enumerate(heads)}, "K": L["K"], "V": L["V"]}
+    G = spec.n_q_heads // spec.n_kv_heads
+    # routes of the sampled heads: a sparse candidate per head in turn (the oracle's own probe builds the indices)
+    sparse = [c for c in cands if c.pattern != PT.DENSE]
+    sets = {}
+    for t, h in enumerate(heads):
+        Qf, Kf = bf16_bits_to_f64(Lq["Q"][h]), bf16_bits_to_f64(L["K"][h // G])
+        pr = OP.probe_rows(Qf, Kf, spec.n)
+        cand = sparse[(t * 5 + 1) % len(sparse)]
+        bs = OP.block_scores(Qf, Kf, 0, spec.n) if cand.pattern == PT.BLOCK_SPARSE else None
+        sets[h] = PT.build_indices(cand, 0, spec.n, pr.vert, pr.slash, bs)
+    Lfull = {"Q": [Lq["Q"].get(h) for h in range(spec.n_q_heads)], "K": L["K"], "V": L["V"]}
+    vals, times = [], []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        tf, desc, cores, _ = oracle_sample(Lfull, spec, cands, None, lambda h: sets[h], None,
+                                           budget_s=max(2.0, 60.0 / max(1, args.steps + args.warmup)))
+        if it >= args.warmup:
+            vals.append(tf); times.append((time.perf_counter() - t0) * 1e3)
+    v = float(np.mean(vals))
+    out = {"impl": "reference", "metric": metric, "value": v, "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": float(np.mean(times)), "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config,
+           "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc},
+           "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
