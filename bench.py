@@ -44,7 +44,7 @@ def measured_peaks():
 
 # ----------------------------------------------------------------------------------------- workloads
 def workload_spec(name: str, n_override: int | None):
-    from synth import config1_spec, config2_spec
+    from synth import config1_spec, config2_spec, config3_spec
     if name == "config1":
         spec = config1_spec(toeplitz=True, n=n_override or 4096)
         lib = [(2, 256, 512), (0, 0, 0)]
@@ -56,7 +56,7 @@ def workload_spec(name: str, n_override: int | None):
         route = dict(budget_frac=1.0, cert_max=None)
         fixed = "seeded 30/30/30/10"
     else:
-        spec = config2_spec(n=n_override or 131072, seed_offset=3)
+        spec = config3_spec(n=n_override or 131072)
         lib = None     # 13-candidate default library
         route = dict(budget_frac=0.15, cert_max=0.05)
         fixed = None
@@ -150,7 +150,7 @@ def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float =
     G = spec.n_q_heads // spec.n_kv_heads
     nb = spec.n // 64
     heads = sorted(set(int(h) for h in np.linspace(0, spec.n_q_heads - 1, 4)))
-    blocks = sorted(set([nb // 4, nb // 2, nb - 1]))
+    blocks = sorted(set([nb // 8, nb // 4, nb // 2, (5 * nb) // 8, (7 * nb) // 8, nb - 1]))
     t_used, pairs_done, rows_done, worst = 0.0, 0, 0, 0.0
     kv_cache = {}
     for h in heads:

@@ -11,6 +11,7 @@ from .generator import (  # noqa: F401
     bf16_bits_to_f64,
     config1_spec,
     config2_spec,
+    config3_spec,
     config4_layer_spec,
     f32_to_bf16_bits,
     fixed_routes_config2,

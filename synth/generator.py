@@ -31,7 +31,7 @@ import numpy as np
 GAMMA0 = 4.0          # strength of the key-side boost direction
 N_SINK_KEYS = 4       # keys 0..3 act as attention sinks
 TOEPLITZ_F = 8        # number of rotary-like frequency pairs
-_T_Q, _T_K, _T_V, _T_U, _T_MISC = 0, 1, 2, 3, 4
+_T_Q, _T_K, _T_V, _T_U, _T_MISC, _T_V2, _T_TOPIC = 0, 1, 2, 3, 4, 5, 6
 
 
 # ----------------------------------------------------------------------------- dtype helpers
@@ -84,7 +84,17 @@ class LayerSpec:
     a_vert: Optional[Sequence[float]] = None     # per KV head
     n_vert: int = 8
     toeplitz: bool = True
-    toeplitz_boost: float = 6.0                  # logit boost on the diagonal from T
+    toeplitz_boost: object = 6.0                 # logit boost on the diagonal from T (float, or one per query head)
+    toeplitz_periods: Optional[Sequence[float]] = None   # (shortest, longest) period; default (512, 8 n)
+    toeplitz_f: int = TOEPLITZ_F                 # number of frequency pairs (first 2 F dimensions)
+    disjoint_dims: bool = False                  # keep the planted directions out of the rotary dimensions
+    q_noise: Optional[Sequence[float]] = None    # per query head, scale of the unstructured part Qr (1 = literal)
+    nu: Optional[Sequence[float]] = None         # per query head, response to planted verticals along a second
+                                                 # direction v_g (None: verticals share the sink direction u_g)
+    topic_q: Optional[Sequence[float]] = None    # per query head, strength of the chunk-topic component
+    topic_k: Optional[Sequence[float]] = None    # per KV head, strength of the chunk-topic component
+    n_topics: int = 24
+    topic_chunk: int = 256
     segments: List[SegmentSpec] = field(default_factory=list)
 
     @property
@@ -127,6 +137,55 @@ def config2_spec(n: int = 32768, seed_offset: int = 2, n_q_heads: int = 32, n_kv
                      n_vert=8, toeplitz=True)
 
 
+def config3_spec(n: int = 131072, seed_offset: int = 3, n_q_heads: int = 32, n_kv_heads: int = 8) -> LayerSpec:
+    """Llama-3.1-8B-shaped layer whose heads follow four archetypes, with boosts that grow with log(n) so that the
+    mass split between structure and the diffuse background stays what it is at n = 4096:
+      local/sink heads (window + initial tokens), vertical heads (planted columns), topic heads (separated key
+      blocks of the same topic as the query's chunk) and diffuse heads (little structure: dense fallback).
+    Archetypes are dealt to the heads of every KV group by a seeded permutation."""
+    seed = 260829058 + seed_offset
+    r = _rng(seed, 0, _T_MISC, 1004)
+    sd, comp = np.sqrt(128.0), np.log(max(n, 4096) / 4096.0)
+    G = n_q_heads // n_kv_heads
+    kinds = []
+    for g in range(n_kv_heads):
+        base = ["local", "vertical", "topic", "local" if g % 2 == 0 else "vertical"][:G] if G <= 4 else ["local", "vertical", "topic"] * G
+        base = list(base[:G])
+        if g % 3 == 2 and G >= 2:
+            base[-1] = "diffuse"
+        kinds += [base[i] for i in r.permutation(G)]
+    # Log-weights (natural log of a component's total unnormalised softmax weight) relative to a top level w_top;
+    # the diffuse background has log-weight ~ ln(n) + 0.5.  Sinks: 4 keys, verticals: 8 keys, topic: ~ n / (2 T) keys.
+    gamma0_k = 4.0                                   # query-side response that realises the key-side base logit
+    w_top = 14.5
+    B_s = [w_top - np.log(4.0) + r.uniform(-0.3, 0.3) + comp for _ in range(n_kv_heads)]     # key-side base logits
+    B_v = [w_top - np.log(8.0) + r.uniform(-0.3, 0.3) + comp for _ in range(n_kv_heads)]
+    B_t = [w_top - 4.4 + r.uniform(-0.3, 0.3) for _ in range(n_kv_heads)]                    # key count grows with n
+    a_sink = [b * sd / (GAMMA0 * gamma0_k) for b in B_s]
+    a_vert = [b * sd / (GAMMA0 * gamma0_k) for b in B_v]
+    topic_k = [float(np.sqrt(b * sd)) for b in B_t]
+    # per archetype: offsets below the top level for (sink, vertical, local, topic)
+    drop = {"local": (0.5, 6.0, 0.0, None), "vertical": (0.5, 0.0, 0.5, None), "topic": (2.0, 6.0, 1.0, 0.0),
+            "diffuse": (7.0, 8.0, 7.0, None)}
+    gamma, nu, lam, qn, tq, tb = [], [], [], [], [], []
+    for h, kind in enumerate(kinds):
+        g = h // G
+        ds, dv, dl, dt = drop[kind]
+        jit = lambda: r.uniform(-0.25, 0.25)
+        lam_h = 0.5 if kind == "diffuse" else r.uniform(0.1, 0.3)
+        gamma.append(gamma0_k * (B_s[g] - ds + jit()) / B_s[g])
+        nu.append(gamma0_k * (B_v[g] - dv + jit()) / B_v[g])
+        tb.append(w_top - dl - lam_h * sd - 0.7 + comp + jit())
+        tq.append(0.0 if dt is None else topic_k[g] * (B_t[g] - dt + jit()) / B_t[g])
+        lam.append(lam_h)
+        qn.append(1.0 if kind == "diffuse" else 0.25)
+    spec = LayerSpec(seed=seed, n=n, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, gamma=gamma, lam=lam,
+                     a_sink=a_sink, a_vert=a_vert, n_vert=8, toeplitz=True, toeplitz_boost=tb,
+                     toeplitz_periods=(37.0, 5300.0), toeplitz_f=28, disjoint_dims=True, q_noise=qn, nu=nu, topic_q=tq, topic_k=topic_k)
+    spec.kinds = kinds
+    return spec
+
+
 def config4_layer_spec(layer: int, n: int = 131072, seg_len: int = 32768,
                        n_q_heads: int = 32, n_kv_heads: int = 8) -> LayerSpec:
     """One layer of the segmented stack: structure switches every seg_len tokens, order seeded per layer."""
@@ -164,11 +223,11 @@ def fixed_routes_config2(n_q_heads: int = 32, seed: int = 260829058 + 2) -> np.n
 
 
 # ----------------------------------------------------------------------------- generation
-def _toeplitz_table(n: int, d: int, boost: float) -> np.ndarray:
+def _toeplitz_table(n: int, d: int, boost: float, period_range=None, F: int = TOEPLITZ_F) -> np.ndarray:
     """[n, 2F] float32 rows c * (cos, sin)(2 pi p / P_f); c^2 * F / sqrt(d) = boost."""
-    F = TOEPLITZ_F
     c = np.sqrt(boost * np.sqrt(d) / F)
-    periods = np.geomspace(512.0, 8.0 * n, F)
+    lo, hi = period_range if period_range is not None else (512.0, 8.0 * n)
+    periods = np.geomspace(float(lo), float(hi), F)
     pos = np.arange(n, dtype=np.float64)[:, None]
     ang = 2.0 * np.pi * pos / periods[None, :]
     t = np.empty((n, 2 * F), dtype=np.float32)
@@ -194,6 +253,8 @@ def make_layer(spec: LayerSpec, heads: Optional[Sequence[int]] = None) -> Dict[s
     kv_needed = sorted({h // G for h in q_heads})
 
     segs = spec.segments or [SegmentSpec(0, n, "planted")]
+    tb_heads = np.broadcast_to(np.asarray(spec.toeplitz_boost, dtype=np.float64), (Hq,))
+    tb_mean = float(tb_heads.mean())     # the key side carries the mean boost, each query head rescales its side
     # per-position modifiers shared by all heads
     lam_scale = np.ones(n, dtype=np.float32)      # multiplies lambda_h
     lam_abs = np.full(n, -1.0, dtype=np.float32)  # >= 0 overrides lambda_h
@@ -203,12 +264,13 @@ def make_layer(spec: LayerSpec, heads: Optional[Sequence[int]] = None) -> Dict[s
         sl = slice(s.start, s.end)
         if s.kind == "local":
             lam_abs[sl] = 1.0
-            tz_amp[sl] = np.sqrt(8.0 / spec.toeplitz_boost) if spec.toeplitz else 0.0
+            tz_amp[sl] = np.sqrt(8.0 / tb_mean) if spec.toeplitz else 0.0
         elif s.kind == "diffuse":
             lam_scale[sl] = 0.0
             gam_scale[sl] = 0.0
             tz_amp[sl] = 0.0
-    ttab = _toeplitz_table(n, d, spec.toeplitz_boost) if tz_amp.any() else None
+    ttab = _toeplitz_table(n, d, tb_mean, spec.toeplitz_periods, spec.toeplitz_f) if tz_amp.any() else None
+    TF2 = 2 * spec.toeplitz_f
 
     Q = np.zeros((len(q_heads), n, d), dtype=np.uint16)
     K = np.zeros((Hkv, n, d), dtype=np.uint16)
@@ -217,9 +279,13 @@ def make_layer(spec: LayerSpec, heads: Optional[Sequence[int]] = None) -> Dict[s
     kr_cache: Dict[int, np.ndarray] = {}
     u_cache: Dict[int, np.ndarray] = {}
     needle_cache: Dict[int, Dict[str, np.ndarray]] = {}
+    v_cache: Dict[int, np.ndarray] = {}
+    topic_cache: Dict[int, np.ndarray] = {}
 
     for g in kv_needed:
         u = _normals(spec.seed, spec.layer, _T_U, g, (d,)).astype(np.float64)
+        if spec.disjoint_dims:
+            u[:TF2] = 0.0
         u = (u / np.linalg.norm(u)).astype(np.float32)
         u_cache[g] = u
         Kr = _normals(spec.seed, spec.layer, _T_K, g, (n, d))
@@ -253,9 +319,31 @@ def make_layer(spec: LayerSpec, heads: Optional[Sequence[int]] = None) -> Dict[s
         needle_cache[g] = needles
         vert_pos[g] = np.asarray(sorted(planted), dtype=np.int64)
         kr_cache[g] = Kr
-        Kf = Kr + (kboost * GAMMA0)[:, None] * u[None, :]
+        if spec.nu is not None:          # verticals along a second direction, sinks along u
+            v2 = _normals(spec.seed, spec.layer, _T_V2, g, (d,)).astype(np.float64)
+            if spec.disjoint_dims:
+                v2[:TF2] = 0.0
+            v2 = v2 - (v2 @ u.astype(np.float64)) * u.astype(np.float64)
+            v2 = (v2 / np.linalg.norm(v2)).astype(np.float32)
+            v_cache[g] = v2
+            sink_part = np.zeros(n, dtype=np.float32)
+            sink_part[:min(N_SINK_KEYS, n)] = kboost[:min(N_SINK_KEYS, n)]
+            vert_part = kboost - sink_part
+            Kf = Kr + (sink_part * GAMMA0)[:, None] * u[None, :] + (vert_part * GAMMA0)[:, None] * v2[None, :]
+        else:
+            Kf = Kr + (kboost * GAMMA0)[:, None] * u[None, :]
+        if spec.topic_k is not None:
+            rt = _rng(spec.seed, spec.layer, _T_TOPIC, g)
+            E = rt.standard_normal((spec.n_topics, d), dtype=np.float32)
+            if spec.disjoint_dims:
+                E[:, :TF2] = 0.0
+            E /= np.linalg.norm(E, axis=1, keepdims=True)
+            n_chunks = (n + spec.topic_chunk - 1) // spec.topic_chunk
+            topic_of_pos = np.repeat(rt.integers(0, spec.n_topics, n_chunks), spec.topic_chunk)[:n]
+            topic_cache[g] = E[topic_of_pos]
+            Kf += np.float32(spec.topic_k[g]) * topic_cache[g]
         if ttab is not None:
-            Kf[:, :2 * TOEPLITZ_F] += tz_amp[:, None] * ttab
+            Kf[:, :TF2] += tz_amp[:, None] * ttab
         K[g] = f32_to_bf16_bits(Kf)
         V[g] = f32_to_bf16_bits(_normals(spec.seed, spec.layer, _T_V, g, (n, d)))
 
@@ -263,9 +351,15 @@ def make_layer(spec: LayerSpec, heads: Optional[Sequence[int]] = None) -> Dict[s
         g = h // G
         Qr = _normals(spec.seed, spec.layer, _T_Q, h, (n, d))
         lam_pos = np.where(lam_abs >= 0, lam_abs, lam[h] * lam_scale).astype(np.float32)
+        if spec.q_noise is not None:
+            Qr = Qr * np.float32(spec.q_noise[h])
         Qf = Qr + (gamma[h] * gam_scale)[:, None] * u_cache[g][None, :] + lam_pos[:, None] * kr_cache[g]
+        if spec.nu is not None:
+            Qf += (np.float32(spec.nu[h]) * gam_scale)[:, None] * v_cache[g][None, :]
+        if spec.topic_q is not None and spec.topic_k is not None:
+            Qf += np.float32(spec.topic_q[h]) * topic_cache[g]
         if ttab is not None:
-            Qf[:, :2 * TOEPLITZ_F] += tz_amp[:, None] * ttab
+            Qf[:, :TF2] += (np.float32(tb_heads[h] / tb_mean) * tz_amp)[:, None] * ttab
         for si, s in enumerate(segs):
             if s.kind == "needle" and str(si) in needle_cache[g]:
                 nv = needle_cache[g][str(si)]
