@@ -371,8 +371,17 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if (masked) {
           tmem_st32(t_s + (uint32_t)c4 * 32u, v);
         }
+        {
+          float mx0 = m_tile, mx1 = NEG_INF, mx2 = NEG_INF, mx3 = NEG_INF;   // four independent chains
 #pragma unroll
-        for (int x = 0; x < 32; ++x) m_tile = fmaxf(m_tile, __uint_as_float(v[x]));
+          for (int x = 0; x < 32; x += 4) {
+            mx0 = fmaxf(mx0, __uint_as_float(v[x]));
+            mx1 = fmaxf(mx1, __uint_as_float(v[x + 1]));
+            mx2 = fmaxf(mx2, __uint_as_float(v[x + 2]));
+            mx3 = fmaxf(mx3, __uint_as_float(v[x + 3]));
+          }
+          m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        }
       }
       tc_wait_st();
       m_tile *= sl2;
@@ -401,13 +410,16 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         tmem_ld32(t_s + (uint32_t)c4 * 32u, v);
         tc_wait_ld();
         uint32_t pk[16];
+        float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
         for (int x = 0; x < 16; ++x) {
           const float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * x]), sl2, -m_use));
           const float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * x + 1]), sl2, -m_use));
-          l_run += p0 + p1;
+          acc0 += p0;
+          acc1 += p1;
           pk[x] = pack_bf16x2(p0, p1);
         }
+        l_run += acc0 + acc1;
         tmem_st16(t_s + (uint32_t)c4 * 16u, pk);
       }
       tc_wait_st();
