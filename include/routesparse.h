@@ -45,7 +45,8 @@ typedef enum {
   RS_ERR_WORKSPACE_TOO_SMALL = -3,
   RS_ERR_CUDA = -4,
   RS_ERR_UNSUPPORTED_DEVICE = -5,
-  RS_ERR_TIMEOUT = -6
+  RS_ERR_TIMEOUT = -6,
+  RS_ERR_NOALLOC_TOO_LARGE = -7
 } rs_status;
 
 /* Pattern library of Section 3.1. */
@@ -164,6 +165,24 @@ int rs_sparse_prefill_attn(const rs_problem* p, const void* Q, const void* K, co
 int rs_dense_prefill_attn(const rs_problem* p, const void* Q, const void* K, const void* V,
                           void* O, int o_dtype, float* lse, float* onorm, uint64_t* counters,
                           void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* Dense causal attention for callers that cannot pass a workspace (the paper has no counterpart: this is a
+ * convenience of this library, not a step of the method).  Same computation and outputs as rs_dense_prefill_attn,
+ * but the launch's work list lives in a fixed array inside the library image instead of caller scratch, so the call
+ * needs no device allocation of any kind.  Meant for callers that cannot allocate where they call from: a plugin
+ * that only receives its input and output tensors, code running inside an allocator or memory-pool callback, a
+ * serving loop in which cudaMalloc (a device-wide synchronisation) is not allowed.
+ *   limit   n_q_heads x (number of 128-row query tiles) <= 16384 (e.g. 32 heads at n = 65536); larger problems
+ *           return RS_ERR_NOALLOC_TOO_LARGE and nothing is launched.  The array is 320 KB and every GPU that loads
+ *           the library keeps it until the process ends.
+ *   set-up  the first call on each device looks up the array's device address (with that device current); make that
+ *           first call outside any stream capture.  Later calls on the device do no set-up.
+ *   sharing all calls on a device use the same array and it keeps the previous call's contents; each call rewrites
+ *           every entry it reads, so nothing needs clearing, but two calls whose kernels overlap on the GPU (different
+ *           streams without ordering) race on it.  Calls on one stream are safe.
+ * No counters output; status as for the other calls (may be NULL). */
+int rs_dense_prefill_attn_noalloc(const rs_problem* p, const void* Q, const void* K, const void* V,
+                                  void* O, int o_dtype, float* lse, float* onorm, int32_t* status, void* stream);
 
 /* Error certificate, Eq. 5: for audited rows with both log-sum-exps known,
  *   m_i = min(1, exp(lse_sel_i - lse_full_i)),  cert_i = 2 (1 - m_i) V_max,

@@ -46,7 +46,7 @@ class rs_route_params(C.Structure):
 
 
 EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "rs_build_indices", "rs_route",
-           "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_certificate"]
+           "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate"]
 
 
 def lib_path() -> str:
@@ -203,6 +203,13 @@ def rs_dense_prefill_attn(p: Problem, Q, K, V, O, lse, onorm, counters, ws, stat
     _check(load().rs_dense_prefill_attn(C.byref(p.c), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), o_dtype, _ptr(lse),
                                         _ptr(onorm), _ptr(counters), _ptr(ws), C.c_size_t(ws.numel()), _ptr(status),
                                         _stream()), "rs_dense_prefill_attn")
+
+
+def rs_dense_prefill_attn_noalloc(p: Problem, Q, K, V, O, lse, onorm, status):
+    """Dense causal attention with the library's built-in scratch: no workspace argument, no allocation."""
+    o_dtype = 1 if O.dtype == torch.float32 else 0
+    _check(load().rs_dense_prefill_attn_noalloc(C.byref(p.c), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), o_dtype, _ptr(lse),
+                                                _ptr(onorm), _ptr(status), _stream()), "rs_dense_prefill_attn_noalloc")
 
 
 def rs_certificate(n_q_heads: int, n_kv_heads: int, n_keys: int, lse_sel, lse_full, rows, vmax, onorm,

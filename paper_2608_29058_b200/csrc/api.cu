@@ -16,6 +16,8 @@ extern "C" const char* rs_error_string(int code) {
     case RS_ERR_CUDA: return "CUDA runtime or driver error";
     case RS_ERR_UNSUPPORTED_DEVICE: return "device is not sm_100";
     case RS_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case RS_ERR_NOALLOC_TOO_LARGE:
+      return "problem exceeds the built-in scratch of the no-allocation entry point (heads x 128-row tiles > 16384)";
     default: return "unknown error";
   }
 }

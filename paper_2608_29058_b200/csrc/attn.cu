@@ -9,6 +9,8 @@
 //   O += P V         tcgen05.mma, A = P from TMEM, B = V from shared memory (MN-major)
 // Roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warps 2-5 = softmax / correction / epilogue.
 // Two CTAs share an SM (256 TMEM columns each) so that one tile's softmax overlaps the other's MMAs.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace {
@@ -676,4 +678,91 @@ extern "C" int rs_dense_prefill_attn(const rs_problem* p, const void* Q, const v
                                      size_t ws_bytes, int32_t* status, void* stream) {
   return launch_attn(p, Q, K, V, nullptr, 0, nullptr, nullptr, O, o_dtype, lse, onorm, counters, ws, ws_bytes, status,
                      stream);
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Dense causal attention without a caller workspace.
+//
+// Some callers cannot hand the library a scratch buffer because they cannot allocate device memory at the point of
+// the call: code running inside a framework's memory-pool callback, a plugin that is given only its input and
+// output tensors, or a latency-critical serving loop in which any cudaMalloc (which synchronises the device) is
+// forbidden.  For them the work list of the attention launch lives in a fixed array inside this library image.
+// The array is part of the module, so every GPU that loads the library holds these bytes until the process exits.
+namespace {
+
+constexpr int kNoAllocMaxTiles = 16384;                         // (query heads) x (128-row query tiles) per call
+constexpr size_t kNoAllocBytes = (size_t)kNoAllocMaxTiles * 20; // cost (4 B) + items (8 B) + order (8 B) per tile
+static __device__ __align__(256) unsigned char rs_noalloc_scratch[kNoAllocBytes];
+
+// In host code the array's name is only a handle for the runtime; the device address must be asked for, once per
+// device and with that device current.
+int noalloc_scratch_ptr(void** out) {
+  static void* cached[64] = {nullptr};
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return RS_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return RS_ERR_UNSUPPORTED_DEVICE;
+  std::lock_guard<std::mutex> lock(mu);
+  if (cached[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, rs_noalloc_scratch) != cudaSuccess || ptr == nullptr) return RS_ERR_CUDA;
+    cached[dev] = ptr;
+  }
+  *out = cached[dev];
+  return RS_OK;
+}
+
+}  // namespace
+
+extern "C" int rs_dense_prefill_attn_noalloc(const rs_problem* p, const void* Q, const void* K, const void* V, void* O,
+                                             int o_dtype, float* lse, float* onorm, int32_t* status, void* stream_) {
+  int rc = rs_check_problem(p);
+  if (rc != RS_OK) return rc;
+  if (!Q || !K || !V || !O || !lse) return RS_ERR_INVALID_ARG;
+  int tiles = 0;
+  for (int s = 0; s < p->n_segments; ++s) tiles += (p->seg_bounds[s + 1] - p->seg_bounds[s] + kTileM - 1) / kTileM;
+  const long long n_work_ll = (long long)tiles * p->n_q_heads;
+  if (n_work_ll > kNoAllocMaxTiles) return RS_ERR_NOALLOC_TOO_LARGE;
+  rc = rs_check_device();
+  if (rc != RS_OK) return rc;
+  void* scratch = nullptr;
+  rc = noalloc_scratch_ptr(&scratch);
+  if (rc != RS_OK) return rc;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  const int n_work = (int)n_work_ll;
+
+  AttnParams P{};
+  P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = p->n_q_heads / p->n_kv_heads;
+  P.n_seg = p->n_segments; P.n_cand = 0;
+  int acc = 0;
+  for (int s = 0; s <= p->n_segments; ++s) {
+    P.seg_bounds[s] = p->seg_bounds[s];
+    P.tile_base[s] = acc;
+    if (s < p->n_segments) acc += (p->seg_bounds[s + 1] - p->seg_bounds[s] + kTileM - 1) / kTileM;
+  }
+  P.tiles_per_head = acc;
+  P.choice = nullptr;
+  P.kv_pad = 64;
+  unsigned char* sb = reinterpret_cast<unsigned char*>(scratch);
+  int* cost = reinterpret_cast<int*>(sb);
+  int2* items = reinterpret_cast<int2*>(sb + (size_t)kNoAllocMaxTiles * 4);
+  int2* order = reinterpret_cast<int2*>(sb + (size_t)kNoAllocMaxTiles * 12);
+  P.order = order;
+  P.O = O; P.o_f32 = o_dtype; P.lse = lse; P.onorm = onorm; P.counters = nullptr; P.status = status;
+  P.scale_log2e = (float)(1.4426950408889634 / sqrt((double)RS_HEAD_DIM));
+
+  CUtensorMap tmQ, tmK, tmV;
+  if (rs_make_tmap_bf16_2d(&tmQ, Q, (uint64_t)P.Hq * P.n, RS_HEAD_DIM, kTileM, 64) ||
+      rs_make_tmap_bf16_2d(&tmK, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kChunk, 64) ||
+      rs_make_tmap_bf16_2d(&tmV, V, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kChunk, 64))
+    return RS_ERR_CUDA;
+  // every entry of cost / items / order is rewritten by the two kernels below, so nothing has to be cleared
+  rs_attn_cost_kernel<<<(n_work + 255) / 256, 256, 0, stream>>>(P, n_work, cost, items);
+  const int n_bins = (P.n >> 6) + 66;
+  rs_attn_order_kernel<<<1, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work, n_bins, cost, items, order);
+  if (cudaFuncSetAttribute(rs_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024) != cudaSuccess)
+    return RS_ERR_CUDA;
+  // the gathered-column maps are never read by dense tiles; they alias K and V
+  rs_attn_kernel<<<n_work, kThreads, attn_smem_bytes(P.n), stream>>>(tmQ, tmK, tmV, tmK, tmV, P);
+  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }
