@@ -5,7 +5,8 @@
 // key blocks of K/V selected by the head's pattern (dense, A-shape, the block diagonals of vertical-slash,
 // block-sparse) followed by chunks of gathered vertical columns.  Two chunks form one 128-key MMA tile:
 //   S = Q K^T        tcgen05.mma, A and B from shared memory (K-major, 128-byte swizzle), S in TMEM
-//   P = exp2(S - m)  softmax warps: tcgen05.ld, mask, online max / sum, bf16 P written back over S in TMEM
+//   P = exp2(S - m)  softmax warps: tcgen05.ld, online max / sum in one pass per 64-key chunk (rare chunks are
+//                    masked in place first), bf16 P written back over S in TMEM
 //   O += P V         tcgen05.mma, A = P from TMEM, B = V from shared memory (MN-major)
 // Roles: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM), warps 2-5 = softmax / correction / epilogue.
 // Two CTAs share an SM (256 TMEM columns each) so that one tile's softmax overlaps the other's MMAs.
@@ -53,6 +54,52 @@ __device__ __forceinline__ uint32_t range_mask(int lo, int hi, int w) {
   uint32_t len = (uint32_t)(b - a + 1);
   uint32_t m = (len == 32u) ? 0xffffffffu : ((1u << len) - 1u);
   return m << (a - 32 * w);
+}
+
+// Masks one 64-key chunk of a score row in place in TMEM (rare chunks only: the causal diagonal, A-shape edges,
+// chunks another quarter wants, gathered vertical columns).  Kept out of line so that the common, unmasked chunk
+// pays one uniform branch and nothing else.
+//   mode 0: every column to -inf;  mode 1: keep j <= i (and, with `edge`, j < n_sink or i - j < window);
+//   mode 2: gathered columns: keep vcols[vbase + x] <= i unless a block diagonal of D already covers that key.
+__device__ __noinline__ void rs_mask_chunk(uint32_t taddr, int mode, int i, int j0, int edge, int n_sink, int window,
+                                           const int* vcols, int vbase, int n_vcols, const uint32_t* d_bits) {
+  const uint32_t NEG = 0xff800000u;
+  uint32_t x[32];
+#pragma unroll 1
+  for (int part = 0; part < 2; ++part) {
+    tmem_ld32(taddr + 32u * part, x);
+    tc_wait_ld();
+    const int cb = 32 * part;
+    if (mode == 0) {
+#pragma unroll
+      for (int q = 0; q < 32; ++q) x[q] = NEG;
+    } else if (mode == 1) {
+#pragma unroll
+      for (int q = 0; q < 32; ++q) {
+        const int j = j0 + cb + q;
+        bool keep = j <= i;
+        if (edge) keep = keep && (j < n_sink || i - j < window);
+        if (!keep) x[q] = NEG;
+      }
+    } else {
+      const int qb_i = i >> 6;
+#pragma unroll
+      for (int q = 0; q < 32; ++q) {
+        const int vi = vbase + cb + q;
+        bool keep = false;
+        if (vi < n_vcols) {
+          const int j = __ldg(vcols + vi);
+          if (j <= i) {
+            const int dlt = qb_i - (j >> 6);
+            keep = !((d_bits[dlt >> 5] >> (dlt & 31)) & 1u);
+          }
+        }
+        if (!keep) x[q] = NEG;
+      }
+    }
+    tmem_st32(taddr + 32u * part, x);
+  }
+  tc_wait_st();
 }
 
 __global__ void __launch_bounds__(kThreads, 2)
@@ -254,15 +301,31 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     if (lane == 0) {
       // ------------------------------------------------------------------ MMA issuer
       const uint32_t d_s = tmem + kColS, d_o = tmem + kColO;
-      const uint64_t qdesc = umma_smem_desc(base + SmemLayout::q, 16, 1024);
-      const uint64_t kdesc = umma_smem_desc(base + SmemLayout::k, 16, 1024);
-      const uint64_t vdesc = umma_smem_desc(base + SmemLayout::v, 16384, 1024);
+      // Descriptor words are formed once; an instruction then costs the issuing thread two adds and the MMA itself.
+      const uint64_t q_desc = umma_smem_desc(base + SmemLayout::q, 16, 1024);
+      const uint64_t k_desc = umma_smem_desc(base + SmemLayout::k, 16, 1024);
+      const uint64_t v_desc = umma_smem_desc(base + SmemLayout::v, 16384, 1024);
+      const uint32_t q_lo = (uint32_t)q_desc, q_hi = (uint32_t)(q_desc >> 32);
+      const uint32_t k_lo = (uint32_t)k_desc, k_hi = (uint32_t)(k_desc >> 32);
+      const uint32_t v_lo = (uint32_t)v_desc, v_hi = (uint32_t)(v_desc >> 32);
+      constexpr uint32_t kIdescQK128 = umma_idesc_bf16(128, 128, 0, 0), kIdescQK64 = umma_idesc_bf16(128, 64, 0, 0);
+      constexpr uint32_t kIdescPV = umma_idesc_bf16(128, 128, 0, 1);
       auto issue_qk = [&](int nch) {
-        const uint32_t idesc = umma_idesc_bf16(128, 64 * nch, 0, 0);
+        const uint32_t idesc = (nch == 2) ? kIdescQK128 : kIdescQK64;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-          const uint64_t off = (uint64_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
-          umma_ss(d_s, qdesc + off, kdesc + off, idesc, kk > 0 ? 1u : 0u);
+          const uint32_t off = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
+          umma_ss2(d_s, q_lo + off, q_hi, k_lo + off, k_hi, idesc, kk > 0 ? 1u : 0u);
+        }
+      };
+      auto issue_pv = [&](int nch, bool accumulate) {
+        // 16 keys per step: P columns advance by 8, V rows by 16 (2048 bytes)
+        umma_ts2(d_o, d_s, v_lo, v_hi, kIdescPV, accumulate ? 1u : 0u);
+#pragma unroll
+        for (int kk = 1; kk < 4; ++kk) umma_ts2(d_o, d_s + 8u * kk, v_lo + 128u * kk, v_hi, kIdescPV, 1u);
+        if (nch == 2) {
+#pragma unroll
+          for (int kk = 4; kk < 8; ++kk) umma_ts2(d_o, d_s + 8u * kk, v_lo + 128u * kk, v_hi, kIdescPV, 1u);
         }
       };
       bool ok = mbar_wait(bar_q, 0, abort_flag);
@@ -283,13 +346,7 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         ok = mbar_wait(bar_vf, ph, abort_flag); site = 6;
         if (!ok) break;
         tc_fence_after();
-        {
-          const uint32_t idesc = umma_idesc_bf16(128, 128, 0, 1);
-          for (int kk = 0; kk < 4 * nch; ++kk) {   // 16 keys per step: P columns advance by 8, V rows by 16
-            umma_ts(d_o, d_s + 8u * (uint32_t)kk, vdesc + (uint64_t)((kk * 2048) >> 4), idesc,
-                    (t > 0 || kk > 0) ? 1u : 0u);
-          }
-        }
+        issue_pv(nch, t > 0);
         umma_commit(bar_ve);
         if (t + 1 < n_pairs) {
           const int nch2 = min(2, n_chunks - 2 * (t + 1));
@@ -318,111 +375,98 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     float m_run = NEG_INF, l_run = 0.f;
     const int* vcols = P.idx.vs_cols + (size_t)vs_slot * P.idx.kv_cap;
     bool ok = true;
-    uint32_t v[32];
+    uint32_t v[32], v2[32];
+    auto max32 = [&](const uint32_t (&x)[32]) -> float {
+      float mx0 = NEG_INF, mx1 = NEG_INF, mx2 = NEG_INF, mx3 = NEG_INF;   // four independent chains
+#pragma unroll
+      for (int q = 0; q < 32; q += 4) {
+        mx0 = fmaxf(mx0, __uint_as_float(x[q]));
+        mx1 = fmaxf(mx1, __uint_as_float(x[q + 1]));
+        mx2 = fmaxf(mx2, __uint_as_float(x[q + 2]));
+        mx3 = fmaxf(mx3, __uint_as_float(x[q + 3]));
+      }
+      return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+    };
+    auto exp_chunk = [&](const uint32_t (&x)[32], uint32_t dst, float m_use) {
+      uint32_t pk[16];
+      float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+      for (int q = 0; q < 16; ++q) {
+        const float p0 = fast_exp2(fmaf(__uint_as_float(x[2 * q]), sl2, -m_use));
+        const float p1 = fast_exp2(fmaf(__uint_as_float(x[2 * q + 1]), sl2, -m_use));
+        acc0 += p0;
+        acc1 += p1;
+        pk[q] = pack_bf16x2(p0, p1);
+      }
+      l_run += acc0 + acc1;
+      tmem_st16(dst, pk);
+    };
 
     for (int t = 0; t < n_pairs; ++t) {
       const int nch = min(2, n_chunks - 2 * t);
       ok = mbar_wait(bar_s, (uint32_t)(t & 1), abort_flag);
       if (!ok) break;
       tc_fence_after();
-      // pass 1: masks (written back to TMEM) and the tile's row maximum
-      float m_tile = NEG_INF;
-      for (int c4 = 0; c4 < 2 * nch; ++c4) {
-        const int ch = 2 * t + (c4 >> 1);
-        const int cb = (c4 & 1) * 32;
-        tmem_ld32(t_s + (uint32_t)c4 * 32u, v);
-        tc_wait_ld();
-        bool masked = false;
-        if (ch < n_block) {
-          const uint32_t e = list[ch];
-          const bool half_ok = (e & (half ? F_HI : F_LO)) != 0;
-          if (!half_ok) {
-            masked = true;
-#pragma unroll
-            for (int x = 0; x < 32; ++x) v[x] = __float_as_uint(NEG_INF);
-          } else if (e & (F_CAUSAL | F_EDGE)) {
-            masked = true;
-            const int j0 = (int)(e & 0xfffu) * kChunk + cb;
-            const bool edge = (e & F_EDGE) != 0;
-#pragma unroll
-            for (int x = 0; x < 32; ++x) {
-              const int j = j0 + x;
-              bool keep = j <= i;
-              if (edge) keep = keep && (j < cand.b0 || i - j < cand.b1);
-              if (!keep) v[x] = __float_as_uint(NEG_INF);
-            }
-          }
-        } else {
-          masked = true;
-          const int vbase = (ch - n_block) * kChunk + cb;
-          const int qb_i = i >> 6;
-#pragma unroll
-          for (int x = 0; x < 32; ++x) {
-            const int vi = vbase + x;
-            bool keep = false;
-            if (vi < n_vcols) {
-              const int j = __ldg(vcols + vi);
-              if (j <= i) {
-                const int dlt = qb_i - (j >> 6);
-                keep = !((d_bits[dlt >> 5] >> (dlt & 31)) & 1u);   // not already covered by a block diagonal
-              }
-            }
-            if (!keep) v[x] = __float_as_uint(NEG_INF);
-          }
-        }
-        if (masked) {
-          tmem_st32(t_s + (uint32_t)c4 * 32u, v);
-        }
+      // One pass per 64-key chunk: rare chunks are masked in place first, then the scores go to registers (two
+      // 32-column loads per wait), chunk maximum, P = exp2(S * scale*log2e - m) against the running maximum.  The
+      // maximum only moves when some row of the warp exceeds it by more than 2^8; then l, O and the part of P already
+      // written for this tile are rescaled.
+      for (int c = 0; c < nch; ++c) {
+        const int ch = 2 * t + c;
         {
-          float mx0 = m_tile, mx1 = NEG_INF, mx2 = NEG_INF, mx3 = NEG_INF;   // four independent chains
-#pragma unroll
-          for (int x = 0; x < 32; x += 4) {
-            mx0 = fmaxf(mx0, __uint_as_float(v[x]));
-            mx1 = fmaxf(mx1, __uint_as_float(v[x + 1]));
-            mx2 = fmaxf(mx2, __uint_as_float(v[x + 2]));
-            mx3 = fmaxf(mx3, __uint_as_float(v[x + 3]));
+          int mode = -1, j0 = 0, edge = 0, vbase = 0;
+          if (ch < n_block) {
+            const uint32_t e = list[ch];
+            if (!(e & (half ? F_HI : F_LO))) {
+              mode = 0;
+            } else if (e & (F_CAUSAL | F_EDGE)) {
+              mode = 1;
+              j0 = (int)(e & 0xfffu) * kChunk;
+              edge = (e & F_EDGE) ? 1 : 0;
+            }
+          } else {
+            mode = 2;
+            vbase = (ch - n_block) * kChunk;
           }
-          m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+          if (mode >= 0)
+            rs_mask_chunk(t_s + (uint32_t)c * 64u, mode, i, j0, edge, cand.b0, cand.b1, vcols, vbase, n_vcols, d_bits);
         }
-      }
-      tc_wait_st();
-      m_tile *= sl2;
-      const float m_new = fmaxf(m_run, m_tile);
-      // lazy rescale: only when some row of the warp moved its maximum by more than 2^8
-      const bool need = m_new > m_run + 8.0f;
-      if (__any_sync(0xffffffffu, need)) {
-        const float alpha = (m_new == NEG_INF) ? 1.0f : fast_exp2(m_run - m_new);
-        l_run *= alpha;
-        m_run = m_new;
-        if (t > 0) {
+        tmem_ld32(t_s + (uint32_t)c * 64u, v);
+        tmem_ld32(t_s + (uint32_t)c * 64u + 32u, v2);
+        tc_wait_ld();
+        const float m_chunk = fmaxf(max32(v), max32(v2)) * sl2;
+        const float m_new = fmaxf(m_run, m_chunk);
+        const bool need = m_new > m_run + 8.0f;
+        if (__any_sync(0xffffffffu, need)) {
+          const float alpha = (m_new == NEG_INF) ? 1.0f : fast_exp2(m_run - m_new);
+          l_run *= alpha;
+          m_run = m_new;
+          uint32_t w32[32];
+          if (t > 0) {
 #pragma unroll 1
-          for (int c4 = 0; c4 < 4; ++c4) {
-            tmem_ld32(t_o + (uint32_t)c4 * 32u, v);
+            for (int c4 = 0; c4 < 4; ++c4) {
+              tmem_ld32(t_o + (uint32_t)c4 * 32u, w32);
+              tc_wait_ld();
+#pragma unroll
+              for (int q = 0; q < 32; ++q) w32[q] = __float_as_uint(__uint_as_float(w32[q]) * alpha);
+              tmem_st32(t_o + (uint32_t)c4 * 32u, w32);
+            }
+          }
+          if (c == 1) {        // P of the tile's first chunk was written against the old maximum
+            tmem_ld32(t_s, w32);
             tc_wait_ld();
 #pragma unroll
-            for (int x = 0; x < 32; ++x) v[x] = __float_as_uint(__uint_as_float(v[x]) * alpha);
-            tmem_st32(t_o + (uint32_t)c4 * 32u, v);
+            for (int q = 0; q < 32; ++q) {
+              const float lo = __uint_as_float(w32[q] << 16) * alpha, hi = __uint_as_float(w32[q] & 0xffff0000u) * alpha;
+              w32[q] = pack_bf16x2(lo, hi);
+            }
+            tmem_st32(t_s, w32);
           }
           tc_wait_st();
         }
-      }
-      const float m_use = (m_run == NEG_INF) ? 0.f : m_run;
-      // pass 2: P = exp2(S * scale*log2e - m), row sum, bf16 pairs written over the start of S
-      for (int c4 = 0; c4 < 2 * nch; ++c4) {
-        tmem_ld32(t_s + (uint32_t)c4 * 32u, v);
-        tc_wait_ld();
-        uint32_t pk[16];
-        float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll
-        for (int x = 0; x < 16; ++x) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(v[2 * x]), sl2, -m_use));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(v[2 * x + 1]), sl2, -m_use));
-          acc0 += p0;
-          acc1 += p1;
-          pk[x] = pack_bf16x2(p0, p1);
-        }
-        l_run += acc0 + acc1;
-        tmem_st16(t_s + (uint32_t)c4 * 16u, pk);
+        const float m_use = (m_run == NEG_INF) ? 0.f : m_run;
+        exp_chunk(v, t_s + (uint32_t)c * 32u, m_use);
+        exp_chunk(v2, t_s + (uint32_t)c * 32u + 16u, m_use);
       }
       tc_wait_st();
       tc_fence_before();
