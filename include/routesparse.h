@@ -71,7 +71,11 @@ typedef struct {
  *                segment's last query block: bs_rows = n_items * n_cand.
  *   materialised (choice != NULL): VS slot = item;  bs_blk is indexed by (head, global query block):
  *                bs_rows = n_q_heads * n_keys / 64.
- * Lists are ascending.  Unused tail entries are unspecified. */
+ * Lists are ascending.  Unused tail entries are unspecified.
+ * rs_sparse_prefill_attn accepts the vertical-slash arrays in either layout (it tells them apart by n_vs_slots ==
+ * n_items * n_cand), so a caller that has evaluated every candidate need not build the chosen lists again: it passes
+ * n_vs_slots = 0 to the materialising rs_build_indices call (block-sparse rows only) and hands the attention call the
+ * evaluation's vertical-slash arrays together with the materialised block-sparse arrays. */
 typedef struct {
   int32_t n_vs_slots, kv_cap, ks_cap, nd_cap;   /* capacities per slot (>= largest budget / n_keys/64) */
   int32_t bs_rows, kb_cap;

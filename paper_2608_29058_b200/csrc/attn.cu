@@ -34,6 +34,7 @@ struct AttnParams {
   const int32_t* choice;      // [n_items] or nullptr (all dense)
   rs_index_set idx;
   int kv_pad;                 // rows per slot of the packed vertical K/V
+  int vs_eval_layout;         // 1: vertical-slash lists sit in the evaluation layout, slot = item * n_cand + candidate
   const int2* order;          // [n_work] (item, tile in segment), heavy first
   void* O;
   int o_f32;
@@ -168,7 +169,7 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   // ---- chunk list: bitmaps of key blocks wanted by the low / high 64 query rows, then ordered compaction
   int vs_slot = 0, n_vcols = 0;
   if (pattern == RS_VERTICAL_SLASH) {
-    vs_slot = item;
+    vs_slot = P.vs_eval_layout ? item * P.n_cand + P.choice[item] : item;
     const int* cnt = P.idx.vs_count + 4 * vs_slot;
     n_vcols = cnt[0];
     const int n_diag = cnt[2];
@@ -273,7 +274,7 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             tma_load_2d(dst, &tmK, bar_kf, 0, row);
             tma_load_2d(dst + 16384, &tmK, bar_kf, 64, row);
           } else {
-            const int row = vs_slot * P.kv_pad + (ch - n_block) * kChunk;
+            const int row = item * P.kv_pad + (ch - n_block) * kChunk;
             tma_load_2d(dst, &tmKp, bar_kf, 0, row);
             tma_load_2d(dst + 16384, &tmKp, bar_kf, 64, row);
           }
@@ -289,7 +290,7 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             tma_load_2d(dst, &tmV, bar_vf, 0, row);
             tma_load_2d(dst + 16384, &tmV, bar_vf, 64, row);
           } else {
-            const int row = vs_slot * P.kv_pad + (ch - n_block) * kChunk;
+            const int row = item * P.kv_pad + (ch - n_block) * kChunk;
             tma_load_2d(dst, &tmVp, bar_vf, 0, row);
             tma_load_2d(dst + 16384, &tmVp, bar_vf, 64, row);
           }
@@ -545,8 +546,9 @@ __global__ void rs_attn_cost_kernel(AttnParams P, int n_work, int* cost, int2* i
   if (cand.pattern == RS_A_SHAPE) {
     c = min(qb_last + 1, (cand.b0 + 63) / 64 + (cand.b1 + 63) / 64 + 2);
   } else if (cand.pattern == RS_VERTICAL_SLASH) {
-    const int* cnt = P.idx.vs_count + 4 * item;
-    const int* dl = P.idx.vs_diag + (size_t)item * P.idx.nd_cap;
+    const int slot = P.vs_eval_layout ? item * P.n_cand + P.choice[item] : item;
+    const int* cnt = P.idx.vs_count + 4 * slot;
+    const int* dl = P.idx.vs_diag + (size_t)slot * P.idx.nd_cap;
     int lo = 0, hi = cnt[2];
     while (lo < hi) { int mid = (lo + hi) >> 1; if (dl[mid] <= qb_last) lo = mid + 1; else hi = mid; }
     c = min(qb_last + 1, lo + 1) + (cnt[0] + 63) / 64;
@@ -582,13 +584,14 @@ __global__ void rs_pack_vertical_kernel(AttnParams P, const __nv_bfloat16* K, co
   const int item = blockIdx.y;
   if (P.choice == nullptr || P.lib[P.choice[item]].pattern != RS_VERTICAL_SLASH) return;
   const int h = item % P.Hq, g = h / P.group;
-  const int n_cols = P.idx.vs_count[4 * item];
+  const int slot = P.vs_eval_layout ? item * P.n_cand + P.choice[item] : item;
+  const int n_cols = P.idx.vs_count[4 * slot];
   const int row = blockIdx.x * (blockDim.x >> 4) + (threadIdx.x >> 4);   // 16 threads move one 256-byte row
   if (row >= P.kv_pad) return;
   const int l16 = threadIdx.x & 15;
   uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
   if (row < n_cols) {
-    const int j = P.idx.vs_cols[(size_t)item * P.idx.kv_cap + row];
+    const int j = P.idx.vs_cols[(size_t)slot * P.idx.kv_cap + row];
     const size_t src = ((size_t)g * P.n + (size_t)j) * RS_HEAD_DIM;
     kv = reinterpret_cast<const uint4*>(K + src)[l16];
     vv = reinterpret_cast<const uint4*>(V + src)[l16];
@@ -642,8 +645,11 @@ int launch_attn(const rs_problem* p, const void* Q, const void* K, const void* V
     if (lib[c].pattern == RS_A_SHAPE && (lib[c].b1 < 1 || lib[c].b0 < 0)) return RS_ERR_INVALID_ARG;
     if (lib[c].pattern < 0 || lib[c].pattern > 3) return RS_ERR_INVALID_ARG;
   }
+  bool vs_eval_layout = false;
   if (choice != nullptr && any_vs) {
-    if (idx->kv_cap < max_kv || idx->n_vs_slots < p->n_segments * p->n_q_heads) return RS_ERR_INVALID_ARG;
+    const int n_items_ = p->n_segments * p->n_q_heads;
+    if (idx->kv_cap < max_kv || idx->n_vs_slots < n_items_) return RS_ERR_INVALID_ARG;
+    vs_eval_layout = n_cand > 1 && idx->n_vs_slots == n_items_ * n_cand;
   }
   const WsPlan w = plan_ws(p, max_kv);
   if (ws_bytes < w.total) return RS_ERR_WORKSPACE_TOO_SMALL;
@@ -662,6 +668,7 @@ int launch_attn(const rs_problem* p, const void* Q, const void* K, const void* V
   for (int c = 0; c < n_cand; ++c) P.lib[c] = lib[c];
   P.choice = choice;
   if (idx) P.idx = *idx;
+  P.vs_eval_layout = vs_eval_layout ? 1 : 0;
   P.kv_pad = w.kv_pad > 0 ? w.kv_pad : 64;
   uint8_t* wsb = reinterpret_cast<uint8_t*>(ws);
   P.order = reinterpret_cast<const int2*>(wsb + w.order);

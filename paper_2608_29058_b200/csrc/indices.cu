@@ -450,7 +450,8 @@ __device__ __forceinline__ float pooled_score(const float* q, const float* k, fl
   return acc * scale;
 }
 
-// Evaluation of one block-sparse candidate: list of the segment's last query block, coverage, pairs.
+// Evaluation of the block-sparse candidates of one item: the pooled scores of the segment's last query block are
+// computed once, then every block-sparse candidate selects from them (list, coverage, pairs).
 __global__ void __launch_bounds__(256)
 rs_bs_eval_kernel(IdxParams P) {
   extern __shared__ float score[];      // [nb]
@@ -460,11 +461,12 @@ rs_bs_eval_kernel(IdxParams P) {
   __shared__ int32_t sel[1024];
   __shared__ float qrow[RS_HEAD_DIM];
   __shared__ u64 cov[RS_PROBE_GROUPS];
-  int item, c, slot;
-  if (!job_of(P, blockIdx.x, item, c, slot)) return;
-  const rs_candidate cand = P.lib[c];
-  if (cand.pattern != RS_BLOCK_SPARSE) return;
+  const int item = blockIdx.x;
   if (P.stats == nullptr && P.choice != nullptr) return;    // materialise mode without stats: rows are built elsewhere
+  bool any = false;
+  for (int c = 0; c < P.n_cand; ++c)
+    any |= P.lib[c].pattern == RS_BLOCK_SPARSE && (P.choice == nullptr || P.choice[item] == c);
+  if (!any) return;
   const int s = item / P.Hq, h = item - s * P.Hq, g = h / P.group;
   const int q0 = P.seg_bounds[s], q1 = P.seg_bounds[s + 1];
   const int qb = (q1 >> 6) - 1;
@@ -478,28 +480,37 @@ rs_bs_eval_kernel(IdxParams P) {
     for (int kb = tid; kb < qb; kb += 256)
       score[kb] = pooled_score(qrow, P.kpool + ((size_t)g * P.nb + kb) * RS_HEAD_DIM, P.scale);
   }
-  if (tid < RS_PROBE_GROUPS) cov[tid] = 0;
   __syncthreads();
-  const int k_b = min(cand.b0, 1024);
-  const int cnt = select_row(score, qb, min(k_b, qb + 1) - 1, qb, sel, 1024, hist, sh, wcnt);
-  if (P.choice == nullptr) {
-    int32_t* dst = P.out.bs_blk + (size_t)slot * P.out.kb_cap;
-    for (int i = tid; i < cnt && i < P.out.kb_cap; i += 256) dst[i] = sel[i];
-    if (tid == 0) P.out.bs_count[slot] = cnt;
-  }
-  if (P.stats == nullptr) return;
-  const u64* vblk = P.vblk + (size_t)item * RS_PROBE_GROUPS * P.nb;
-  u64 part[RS_PROBE_GROUPS] = {0, 0, 0, 0};
-  for (int i = tid; i < cnt; i += 256)
+  for (int c = 0; c < P.n_cand; ++c) {
+    const rs_candidate cand = P.lib[c];
+    if (cand.pattern != RS_BLOCK_SPARSE) continue;
+    if (P.choice != nullptr && P.choice[item] != c) continue;
+    const int slot = (P.choice != nullptr) ? item : item * P.n_cand + c;
+    if (tid < RS_PROBE_GROUPS) cov[tid] = 0;
+    __syncthreads();
+    const int k_b = min(cand.b0, 1024);
+    const int cnt = select_row(score, qb, min(k_b, qb + 1) - 1, qb, sel, 1024, hist, sh, wcnt);
+    if (P.choice == nullptr) {
+      int32_t* dst = P.out.bs_blk + (size_t)slot * P.out.kb_cap;
+      for (int i = tid; i < cnt && i < P.out.kb_cap; i += 256) dst[i] = sel[i];
+      if (tid == 0) P.out.bs_count[slot] = cnt;
+    }
+    if (P.stats != nullptr) {
+      const u64* vblk = P.vblk + (size_t)item * RS_PROBE_GROUPS * P.nb;
+      u64 part[RS_PROBE_GROUPS] = {0, 0, 0, 0};
+      for (int i = tid; i < cnt; i += 256)
 #pragma unroll
-    for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) part[gg] += vblk[(size_t)gg * P.nb + sel[i]];
+        for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) part[gg] += vblk[(size_t)gg * P.nb + sel[i]];
 #pragma unroll
-  for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) if (part[gg]) atomicAdd(&cov[gg], part[gg]);
-  __syncthreads();
-  if (tid == 0) {
-    rs_cand_stats* st = P.stats + (size_t)item * P.n_cand + c;
-    for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) st->cov_fx[gg] = cov[gg];
-    st->pairs = pairs_block_sparse(q0 >> 6, q1 >> 6, cand.b0);
+      for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) if (part[gg]) atomicAdd(&cov[gg], part[gg]);
+      __syncthreads();
+      if (tid == 0) {
+        rs_cand_stats* st = P.stats + (size_t)item * P.n_cand + c;
+        for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) st->cov_fx[gg] = cov[gg];
+        st->pairs = pairs_block_sparse(q0 >> 6, q1 >> 6, cand.b0);
+      }
+    }
+    __syncthreads();
   }
 }
 
@@ -642,7 +653,9 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   if ((any_vs || stats) && (!vert || !slash)) return RS_ERR_INVALID_ARG;
   if (any_bs && bscore == nullptr && (!qpool || !kpool)) return RS_ERR_INVALID_ARG;
   const int n_slots = choice ? n_items : n_items * n_cand;
-  if (any_vs && out->n_vs_slots < n_slots) return RS_ERR_INVALID_ARG;
+  // materialise mode with n_vs_slots == 0: the caller keeps using the lists of an earlier evaluation call
+  const bool skip_vs = choice != nullptr && out->n_vs_slots == 0 && stats == nullptr;
+  if (any_vs && !skip_vs && out->n_vs_slots < n_slots) return RS_ERR_INVALID_ARG;
   if (any_bs && out->bs_rows < (choice ? p->n_q_heads * nb : n_slots)) return RS_ERR_INVALID_ARG;
   for (int s = 0; s < p->n_segments; ++s)
     if (p->seg_bounds[s + 1] < RS_PROBE_ROWS) return RS_ERR_UNSUPPORTED_SHAPE;
@@ -668,13 +681,13 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
     rs_vblk_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, stream>>>(P);
     rs_simple_stats_kernel<<<n_jobs, 256, 0, stream>>>(P);
   }
-  if (any_vs) {
+  if (any_vs && !skip_vs) {
     rs_vs_select_kernel<<<dim3(2, n_jobs), kSelThreads, 0, stream>>>(P);
     rs_vs_finish_kernel<<<n_jobs, 256, 0, stream>>>(P);
   }
   if (any_bs) {
     if (choice == nullptr || stats != nullptr)
-      rs_bs_eval_kernel<<<n_jobs, 256, (size_t)nb * sizeof(float), stream>>>(P);
+      rs_bs_eval_kernel<<<n_items, 256, (size_t)nb * sizeof(float), stream>>>(P);
     if (choice != nullptr) {
       if (bscore == nullptr) {
         const int nt = (nb + 63) / 64;

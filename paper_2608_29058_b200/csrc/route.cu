@@ -10,7 +10,8 @@
 namespace {
 
 constexpr int kThreads = 1024;
-constexpr int kMaxItems = RS_MAX_SEGMENTS * 64;
+constexpr int kMaxItems = 2048;
+constexpr int kCachePairs = 1792;     // (item, candidate) pairs whose risk / cost are kept in shared memory
 
 struct RouteArgs {
   int n_items, n_cand, Hq, Hkv, group, dense_c;
@@ -75,21 +76,34 @@ __device__ __forceinline__ double risk_of(const RouteArgs& A, int item, int c) {
 __global__ void __launch_bounds__(kThreads)
 rs_route_kernel(const __grid_constant__ RouteArgs A) {
   __shared__ int ch[kMaxItems];
+  __shared__ double c_risk[kCachePairs];
+  __shared__ long long c_cost[kCachePairs];
   __shared__ Sub wbest[32];
   __shared__ long long wsum[32];
   __shared__ long long sh_total;
   __shared__ int sh_feasible, sh_fallback;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_pairs = A.n_items * A.n_cand;
+  const bool cached = n_pairs <= kCachePairs;
+  if (cached) {
+    for (int p = tid; p < n_pairs; p += kThreads) {
+      const int it = p / A.n_cand, k = p - it * A.n_cand;
+      c_risk[p] = risk_of(A, it, k);
+      c_cost[p] = cost_of(A, it, k);
+    }
+  }
+  auto riskf = [&](int it, int k) -> double { return cached ? c_risk[it * A.n_cand + k] : risk_of(A, it, k); };
+  auto costf = [&](int it, int k) -> long long { return cached ? c_cost[it * A.n_cand + k] : cost_of(A, it, k); };
 
   if (tid == 0) { sh_feasible = 1; sh_fallback = 0; }
+  __syncthreads();
   if (A.prm.fixed_choice != nullptr) {
     for (int it = tid; it < A.n_items; it += kThreads) ch[it] = A.prm.fixed_choice[it];
     __syncthreads();
   } else {
     for (int it = tid; it < A.n_items; it += kThreads) ch[it] = A.dense_c;
     long long part = 0;
-    for (int it = tid; it < A.n_items; it += kThreads) part += cost_of(A, it, A.dense_c);
+    for (int it = tid; it < A.n_items; it += kThreads) part += costf(it, A.dense_c);
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
     if (lane == 0) wsum[warp] = part;
@@ -108,10 +122,10 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
       for (int p = tid; p < n_pairs; p += kThreads) {
         const int it = p / A.n_cand, k = p - it * A.n_cand;
         const int cur = ch[it];
-        const long long dT = cost_of(A, it, cur) - cost_of(A, it, k);
+        const long long dT = costf(it, cur) - costf(it, k);
         if (dT <= 0) continue;
         Sub s;
-        s.ratio = __ddiv_rn(__dsub_rn(risk_of(A, it, k), risk_of(A, it, cur)), (double)dT);
+        s.ratio = __ddiv_rn(__dsub_rn(riskf(it, k), riskf(it, cur)), (double)dT);
         s.dT = dT; s.item = it; s.k = k;
         if (better(s, best)) best = s;
       }

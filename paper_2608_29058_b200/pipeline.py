@@ -45,6 +45,13 @@ class RouteConfig:
     expand_first: bool = True
 
 
+class _IdxView:
+    """An rs_index_set struct that points into arrays owned by IndexSet objects."""
+
+    def __init__(self, c_struct):
+        self.c = c_struct
+
+
 class RoutedPrefillLayer:
     """Device buffers and call order for one layer; reuse one instance for every layer of the same shape."""
 
@@ -65,6 +72,14 @@ class RoutedPrefillLayer:
         self.stats = torch.zeros((p.n_items, len(self.cands), 5), dtype=torch.int64, device=device)
         self.idx_eval = rs.IndexSet.for_library(p, self.lib, materialised=False, device=device)
         self.idx = rs.IndexSet.for_library(p, self.lib, materialised=True, device=device)
+        # online routing reuses the evaluation's vertical-slash lists: materialise only block-sparse rows, and hand the
+        # attention call the evaluation's vertical-slash arrays next to the materialised block-sparse arrays
+        e, m = self.idx_eval.c, self.idx.c
+        self._idx_bs_only = rs.rs_index_set(0, m.kv_cap, m.ks_cap, m.nd_cap, m.bs_rows, m.kb_cap, m.vs_cols, m.vs_offs,
+                                            m.vs_diag, m.vs_count, m.bs_blk, m.bs_count)
+        self._idx_hybrid = rs.rs_index_set(e.n_vs_slots, e.kv_cap, e.ks_cap, e.nd_cap, m.bs_rows, m.kb_cap, e.vs_cols,
+                                           e.vs_offs, e.vs_diag, e.vs_count, m.bs_blk, m.bs_count)
+        self._reuse_eval = False
         self.choice = torch.zeros(p.n_items, dtype=torch.int32, device=device)
         self.report = torch.zeros(24, dtype=torch.uint8, device=device)
         self.O = torch.empty((Hq, n, 128), dtype=out_dtype, device=device)
@@ -108,12 +123,15 @@ class RoutedPrefillLayer:
         prm.fixed_choice = None
         rs.rs_route(self.p, self.lib, self.stats, None, self.vmax, prm, self.choice, self.report, self.status)
 
-    def materialise(self):
+    def materialise(self, reuse_evaluation: bool = False):
+        self._reuse_eval = reuse_evaluation and len(self.cands) > 1
+        out = _IdxView(self._idx_bs_only) if self._reuse_eval else self.idx
         rs.rs_build_indices(self.p, self.lib, self.vert, self.slash, self.qpool, self.kpool, None, self.choice,
-                            self.idx, None, self.ws, self.status)
+                            out, None, self.ws, self.status)
 
     def attention(self, Q, K, V):
-        rs.rs_sparse_prefill_attn(self.p, Q, K, V, self.lib, self.idx, self.choice, self.O, self.lse_sel, self.onorm,
+        idx = _IdxView(self._idx_hybrid) if self._reuse_eval else self.idx
+        rs.rs_sparse_prefill_attn(self.p, Q, K, V, self.lib, idx, self.choice, self.O, self.lse_sel, self.onorm,
                                   self.counters, self.ws, self.status)
 
     def certificate(self):
@@ -139,7 +157,7 @@ class RoutedPrefillLayer:
             self.choice.copy_(fixed_choice)
             mark(2)
         mark(3)
-        self.materialise()
+        self.materialise(reuse_evaluation=fixed_choice is None)
         mark(4)
         self.attention(Q, K, V)
         mark(5)

@@ -21,8 +21,10 @@ C = PT.Candidate
 def download_sets(layer, cands, choice):
     p = layer.p
     nb = p.n_keys // 64
-    cnt = layer.idx.vs_count.cpu().numpy()
-    cols, offs, diag = (t.cpu().numpy() for t in (layer.idx.vs_cols, layer.idx.vs_offs, layer.idx.vs_diag))
+    reuse = getattr(layer, "_reuse_eval", False)       # vertical-slash lists may still sit in the evaluation layout
+    vs = layer.idx_eval if reuse else layer.idx
+    cnt = vs.vs_count.cpu().numpy()
+    cols, offs, diag = (t.cpu().numpy() for t in (vs.vs_cols, vs.vs_offs, vs.vs_diag))
     blk, bcnt = layer.idx.bs_blk.cpu().numpy(), layer.idx.bs_count.cpu().numpy()
     sets = []
     for item in range(p.n_items):
@@ -31,7 +33,8 @@ def download_sets(layer, cands, choice):
         cand = cands[choice[item]]
         ix = PT.IndexSet(cand=cand, q0=q0, q1=q1)
         if cand.pattern == PT.VERTICAL_SLASH:
-            ix.V, ix.S, ix.D = cols[item, :cnt[item, 0]], offs[item, :cnt[item, 1]], diag[item, :cnt[item, 2]]
+            sl = item * len(cands) + int(choice[item]) if reuse else item
+            ix.V, ix.S, ix.D = cols[sl, :cnt[sl, 0]], offs[sl, :cnt[sl, 1]], diag[sl, :cnt[sl, 2]]
         elif cand.pattern == PT.BLOCK_SPARSE:
             ix.blk = [blk[h * nb + qb, :bcnt[h * nb + qb]] for qb in range(q0 // 64, q1 // 64)]
         sets.append(ix)
