@@ -22,11 +22,22 @@ struct IdxParams {
   rs_cand_stats* stats;
   u64* vblk;          // [n_items][4][nb] block sums of fx(vert)
   float* bs_ws;       // [Hq][nb][nb] fused block scores (materialise mode)
+  u64* keys;          // [n_items][2][n] ranking keys of columns (0) and offsets (1)
+  float* bs_eval_ws;  // [n_items][nb] pooled scores of each segment's last query block
   int32_t* status;
   float scale;
 };
 
-__device__ __forceinline__ u64 fx(float x) { return (u64)__float2ull_rz(x * 4294967296.0f); }
+// floor(x * 2^32) of a non-negative float, exactly, from its bits (no float-to-integer conversion unit involved)
+__device__ __forceinline__ u64 fx(float x) {
+  const uint32_t b = __float_as_uint(x);
+  const int e = (int)((b >> 23) & 0xffu);
+  if (e == 0) return 0ull;                               // zero and subnormals: far below 2^-32
+  const u64 m = (u64)((b & 0x7fffffu) | 0x800000u);      // x = m * 2^(e - 150)
+  const int sh = e - 118;                                // x * 2^32 = m * 2^(e - 118)
+  if (sh >= 0) return m << min(sh, 40);
+  return (sh > -24) ? (m >> (-sh)) : 0ull;
+}
 
 __device__ __forceinline__ u64 line_key(const float* mass, int n, int j) {
   return fx(mass[j]) + fx(mass[(size_t)n + j]) + fx(mass[2 * (size_t)n + j]) + fx(mass[3 * (size_t)n + j]);
@@ -71,6 +82,18 @@ __global__ void rs_vblk_kernel(IdxParams P) {
   if (lane == 0) P.vblk[(size_t)ig * P.nb + kb] = acc;
 }
 
+// ------------------------------------------------------------------------------------------ ranking keys, once per line
+__global__ void __launch_bounds__(256)
+rs_vs_keys_kernel(IdxParams P) {
+  const int item = blockIdx.y >> 1, list = blockIdx.y & 1;
+  const int s = item / P.Hq;
+  const int q1 = P.seg_bounds[s + 1];
+  const int j = blockIdx.x * 256 + threadIdx.x;
+  if (j >= q1) return;
+  const float* mass = (list == 0 ? P.vert : P.slash) + (size_t)item * RS_PROBE_GROUPS * P.n;
+  P.keys[((size_t)item * 2 + list) * P.n + j] = line_key(mass, P.n, j);
+}
+
 // ------------------------------------------------------------------------------------------ exact top-k of a line list
 // grid = (2 lists, jobs).  list 0: vertical columns over [0, q1); list 1: slash offsets over [1, q1) plus offset 0.
 constexpr int kSelThreads = 1024;
@@ -92,7 +115,7 @@ rs_vs_select_kernel(IdxParams P) {
   const int s = item / P.Hq;
   const int q1 = P.seg_bounds[s + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float* mass = (list == 0 ? P.vert : P.slash) + (size_t)item * RS_PROBE_GROUPS * P.n;
+  const u64* keys = P.keys + ((size_t)item * 2 + list) * P.n;
   const int first = (list == 0) ? 0 : 1;                 // first index of the domain
   const int n_dom = q1 - first;
   int k = (list == 0) ? min(cand.b0, q1) : (min(cand.b1, q1) - 1);
@@ -114,7 +137,7 @@ rs_vs_select_kernel(IdxParams P) {
         const int j = base + tid;
         unsigned int digit = 0xffffffffu;
         if (j < n_dom) {
-          const u64 key = line_key(mass, P.n, first + j);
+          const u64 key = keys[first + j];
           if ((key >> (shift + kDigitBits)) == prefix) digit = (unsigned)((key >> shift) & (kBins - 1));
         }
         const unsigned int peers = __match_any_sync(0xffffffffu, digit);
@@ -164,7 +187,7 @@ rs_vs_select_kernel(IdxParams P) {
     const int j = base + lane;
     u64 key = 0;
     const bool in = j < hi;
-    if (in) key = line_key(mass, P.n, first + j);
+    if (in) key = keys[first + j];
     gt += __popc(__ballot_sync(0xffffffffu, in && key > T));
     eq += __popc(__ballot_sync(0xffffffffu, in && key == T));
   }
@@ -179,7 +202,7 @@ rs_vs_select_kernel(IdxParams P) {
     const int j = base + lane;
     u64 key = 0;
     const bool in = j < hi;
-    if (in) key = line_key(mass, P.n, first + j);
+    if (in) key = keys[first + j];
     const bool is_eq = in && key == T;
     const unsigned int beq = __ballot_sync(0xffffffffu, is_eq);
     const bool take = in && (key > T || (is_eq && eq_run + __popc(beq & lt_mask) < k_eq));
@@ -450,6 +473,21 @@ __device__ __forceinline__ float pooled_score(const float* q, const float* k, fl
   return acc * scale;
 }
 
+// Pooled scores of the last query block of every item that has a block-sparse candidate to evaluate.
+__global__ void __launch_bounds__(256)
+rs_bs_eval_scores_kernel(IdxParams P) {
+  __shared__ float qrow[RS_HEAD_DIM];
+  const int item = blockIdx.y;
+  const int s = item / P.Hq, h = item - s * P.Hq, g = h / P.group;
+  const int qb = (P.seg_bounds[s + 1] >> 6) - 1;
+  if (blockIdx.x * 256 >= qb) return;
+  if (threadIdx.x < RS_HEAD_DIM) qrow[threadIdx.x] = P.qpool[((size_t)h * P.nb + qb) * RS_HEAD_DIM + threadIdx.x];
+  __syncthreads();
+  const int kb = blockIdx.x * 256 + threadIdx.x;
+  if (kb < qb)
+    P.bs_eval_ws[(size_t)item * P.nb + kb] = pooled_score(qrow, P.kpool + ((size_t)g * P.nb + kb) * RS_HEAD_DIM, P.scale);
+}
+
 // Evaluation of the block-sparse candidates of one item: the pooled scores of the segment's last query block are
 // computed once, then every block-sparse candidate selects from them (list, coverage, pairs).
 __global__ void __launch_bounds__(256)
@@ -459,7 +497,6 @@ rs_bs_eval_kernel(IdxParams P) {
   __shared__ uint32_t sh[8];
   __shared__ unsigned int wcnt[16];
   __shared__ int32_t sel[1024];
-  __shared__ float qrow[RS_HEAD_DIM];
   __shared__ u64 cov[RS_PROBE_GROUPS];
   const int item = blockIdx.x;
   if (P.stats == nullptr && P.choice != nullptr) return;    // materialise mode without stats: rows are built elsewhere
@@ -467,7 +504,7 @@ rs_bs_eval_kernel(IdxParams P) {
   for (int c = 0; c < P.n_cand; ++c)
     any |= P.lib[c].pattern == RS_BLOCK_SPARSE && (P.choice == nullptr || P.choice[item] == c);
   if (!any) return;
-  const int s = item / P.Hq, h = item - s * P.Hq, g = h / P.group;
+  const int s = item / P.Hq;
   const int q0 = P.seg_bounds[s], q1 = P.seg_bounds[s + 1];
   const int qb = (q1 >> 6) - 1;
   const int tid = threadIdx.x;
@@ -475,10 +512,8 @@ rs_bs_eval_kernel(IdxParams P) {
     const float* row = P.bscore + ((size_t)item * P.nb + qb) * P.nb;
     for (int kb = tid; kb < qb; kb += 256) score[kb] = row[kb];
   } else {
-    if (tid < RS_HEAD_DIM) qrow[tid] = P.qpool[((size_t)h * P.nb + qb) * RS_HEAD_DIM + tid];
-    __syncthreads();
-    for (int kb = tid; kb < qb; kb += 256)
-      score[kb] = pooled_score(qrow, P.kpool + ((size_t)g * P.nb + kb) * RS_HEAD_DIM, P.scale);
+    const float* row = P.bs_eval_ws + (size_t)item * P.nb;
+    for (int kb = tid; kb < qb; kb += 256) score[kb] = row[kb];
   }
   __syncthreads();
   for (int c = 0; c < P.n_cand; ++c) {
@@ -593,17 +628,19 @@ rs_bs_scores_kernel(IdxParams P) {
   }
 }
 
-struct IdxPlan { size_t vblk, bs_ws, total; };
+struct IdxPlan { size_t vblk, bs_ws, keys, bs_eval, total; };
 
 IdxPlan plan(const rs_problem* p, const rs_candidate* lib, int n_cand) {
   IdxPlan w{};
   const size_t nb = (size_t)p->n_keys / 64;
   const size_t items = (size_t)p->n_segments * p->n_q_heads;
-  bool any_bs = false;
-  for (int c = 0; c < n_cand; ++c) any_bs |= (lib[c].pattern == RS_BLOCK_SPARSE);
+  bool any_bs = false, any_vs = false;
+  for (int c = 0; c < n_cand; ++c) { any_bs |= (lib[c].pattern == RS_BLOCK_SPARSE); any_vs |= (lib[c].pattern == RS_VERTICAL_SLASH); }
   size_t off = 0;
   w.vblk = off;  off += rs_align_up(items * RS_PROBE_GROUPS * nb * sizeof(u64), 256);
   w.bs_ws = off; off += any_bs ? rs_align_up((size_t)p->n_q_heads * nb * nb * sizeof(float), 256) : 0;
+  w.keys = off;  off += any_vs ? rs_align_up(items * 2 * (size_t)p->n_keys * sizeof(u64), 256) : 0;
+  w.bs_eval = off; off += any_bs ? rs_align_up(items * nb * sizeof(float), 256) : 0;
   w.total = off;
   return w;
 }
@@ -624,7 +661,7 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   if (choice == nullptr && stats == nullptr) return RS_ERR_INVALID_ARG;
   const int n_items = p->n_segments * p->n_q_heads;
   const int nb = p->n_keys / 64;
-  bool any_vs = false, any_bs = false, any_a = false;
+  bool any_vs = false, any_bs = false;
   for (int c = 0; c < n_cand; ++c) {
     const rs_candidate& cd = lib[c];
     if (cd.pattern < 0 || cd.pattern > 3) return RS_ERR_INVALID_ARG;
@@ -638,7 +675,6 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
       if (cd.b0 < 1 || cd.b0 > 1024) return RS_ERR_INVALID_ARG;
       if (out->kb_cap < (cd.b0 < nb ? cd.b0 : nb)) return RS_ERR_INVALID_ARG;
     } else if (cd.pattern == RS_A_SHAPE) {
-      any_a = true;
       if (cd.b0 < 0 || cd.b1 < 1) return RS_ERR_INVALID_ARG;
       if (stats != nullptr) {
         // coverage of sink + window from column and offset masses needs the two not to overlap on the probe rows
@@ -649,7 +685,6 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
       }
     }
   }
-  (void)any_a;
   if ((any_vs || stats) && (!vert || !slash)) return RS_ERR_INVALID_ARG;
   if (any_bs && bscore == nullptr && (!qpool || !kpool)) return RS_ERR_INVALID_ARG;
   const int n_slots = choice ? n_items : n_items * n_cand;
@@ -673,6 +708,8 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   P.vert = vert; P.slash = slash; P.qpool = qpool; P.kpool = kpool; P.bscore = bscore; P.choice = choice;
   P.out = *out; P.stats = stats; P.vblk = reinterpret_cast<u64*>(wsb + w.vblk);
   P.bs_ws = reinterpret_cast<float*>(wsb + w.bs_ws); P.status = status;
+  P.keys = reinterpret_cast<u64*>(wsb + w.keys);
+  P.bs_eval_ws = reinterpret_cast<float*>(wsb + w.bs_eval);
   P.scale = (float)(1.0 / sqrt((double)RS_HEAD_DIM));
 
   const int n_jobs = n_items * n_cand;
@@ -682,10 +719,13 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
     rs_simple_stats_kernel<<<n_jobs, 256, 0, stream>>>(P);
   }
   if (any_vs && !skip_vs) {
+    rs_vs_keys_kernel<<<dim3((P.n + 255) / 256, 2 * n_items), 256, 0, stream>>>(P);
     rs_vs_select_kernel<<<dim3(2, n_jobs), kSelThreads, 0, stream>>>(P);
     rs_vs_finish_kernel<<<n_jobs, 256, 0, stream>>>(P);
   }
   if (any_bs) {
+    if ((choice == nullptr || stats != nullptr) && bscore == nullptr)
+      rs_bs_eval_scores_kernel<<<dim3((nb + 255) / 256, n_items), 256, 0, stream>>>(P);
     if (choice == nullptr || stats != nullptr)
       rs_bs_eval_kernel<<<n_items, 256, (size_t)nb * sizeof(float), stream>>>(P);
     if (choice != nullptr) {

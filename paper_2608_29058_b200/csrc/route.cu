@@ -11,7 +11,7 @@ namespace {
 
 constexpr int kThreads = 1024;
 constexpr int kMaxItems = 2048;
-constexpr int kCachePairs = 1792;     // (item, candidate) pairs whose risk / cost are kept in shared memory
+constexpr int kCachePairs = 4096;     // (item, candidate) pairs whose risk / cost are kept in shared memory
 
 struct RouteArgs {
   int n_items, n_cand, Hq, Hkv, group, dense_c;
@@ -75,16 +75,18 @@ __device__ __forceinline__ double risk_of(const RouteArgs& A, int item, int c) {
 
 __global__ void __launch_bounds__(kThreads)
 rs_route_kernel(const __grid_constant__ RouteArgs A) {
-  __shared__ int ch[kMaxItems];
-  __shared__ double c_risk[kCachePairs];
-  __shared__ long long c_cost[kCachePairs];
-  __shared__ Sub wbest[32];
+  extern __shared__ unsigned char route_smem[];       // ibest[n_items] | c_risk[cache] | c_cost[cache] | ch[n_items]
+  const int n_cache = (A.n_items * A.n_cand <= kCachePairs) ? A.n_items * A.n_cand : 0;
+  Sub* ibest = reinterpret_cast<Sub*>(route_smem);
+  double* c_risk = reinterpret_cast<double*>(ibest + A.n_items);
+  long long* c_cost = reinterpret_cast<long long*>(c_risk + n_cache);
+  int* ch = reinterpret_cast<int*>(c_cost + n_cache);
   __shared__ long long wsum[32];
   __shared__ long long sh_total;
   __shared__ int sh_feasible, sh_fallback;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_pairs = A.n_items * A.n_cand;
-  const bool cached = n_pairs <= kCachePairs;
+  const bool cached = n_cache > 0;
   if (cached) {
     for (int p = tid; p < n_pairs; p += kThreads) {
       const int it = p / A.n_cand, k = p - it * A.n_cand;
@@ -114,14 +116,13 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
       sh_total = t;
     }
     __syncthreads();
-    // ---- greedy substitutions until the layer budget is met
-    const int max_steps = n_pairs + 1;
-    for (int step = 0; step < max_steps; ++step) {
-      if (sh_total <= A.prm.budget) break;
+    // ---- greedy substitutions until the layer budget is met.  Every item keeps its best substitution in shared
+    // memory; a step only changes one item, so one warp finds the arg-min over items, applies it and refreshes that
+    // item's entry without any block-wide barrier.
+    auto best_of_item = [&](int it, int lane_k0, int stride) -> Sub {
       Sub best; best.ratio = 0.0; best.dT = 0; best.item = -1; best.k = -1;
-      for (int p = tid; p < n_pairs; p += kThreads) {
-        const int it = p / A.n_cand, k = p - it * A.n_cand;
-        const int cur = ch[it];
+      const int cur = ch[it];
+      for (int k = lane_k0; k < A.n_cand; k += stride) {
         const long long dT = costf(it, cur) - costf(it, k);
         if (dT <= 0) continue;
         Sub s;
@@ -129,26 +130,40 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
         s.dT = dT; s.item = it; s.k = k;
         if (better(s, best)) best = s;
       }
-#pragma unroll
-      for (int off = 16; off >= 1; off >>= 1) {
-        const Sub o = shfl_sub(best, off);
-        if (better(o, best)) best = o;
-      }
-      if (lane == 0) wbest[warp] = best;
-      __syncthreads();
-      if (tid == 0) {
-        Sub b = wbest[0];
-        for (int w = 1; w < 32; ++w) if (better(wbest[w], b)) b = wbest[w];
-        if (b.k < 0) {
-          sh_feasible = 0;
-        } else {
-          ch[b.item] = b.k;
-          sh_total -= b.dT;
+      return best;
+    };
+    for (int it = tid; it < A.n_items; it += kThreads) ibest[it] = best_of_item(it, 0, 1);
+    __syncthreads();
+    if (warp == 0) {
+      long long total = sh_total;
+      const int max_steps = n_pairs + 1;
+      for (int step = 0; step < max_steps && total > A.prm.budget; ++step) {
+        Sub best; best.ratio = 0.0; best.dT = 0; best.item = -1; best.k = -1;
+        for (int it = lane; it < A.n_items; it += 32) {
+          const Sub s = ibest[it];
+          if (better(s, best)) best = s;
         }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+          const Sub o = shfl_sub(best, off);
+          if (better(o, best)) best = o;
+        }
+        if (best.k < 0) { if (lane == 0) sh_feasible = 0; break; }
+        if (lane == 0) ch[best.item] = best.k;
+        total -= best.dT;
+        __syncwarp();
+        Sub mine = best_of_item(best.item, lane, 32);
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+          const Sub o = shfl_sub(mine, off);
+          if (better(o, mine)) mine = o;
+        }
+        if (lane == 0) ibest[best.item] = mine;
+        __syncwarp();
       }
-      __syncthreads();
-      if (sh_feasible == 0) break;
+      if (lane == 0) sh_total = total;
     }
+    __syncthreads();
     // ---- fallback walk: larger budget of the family first, then dense
     if (A.prm.use_cert) {
       for (int it = tid; it < A.n_items; it += kThreads) {
@@ -223,6 +238,14 @@ extern "C" int rs_route(const rs_problem* p, const rs_candidate* lib, int n_cand
   if (params->use_cert && params->cert_mode == RS_CERT_ABS && vmax == nullptr) return RS_ERR_INVALID_ARG;
   A.stats = stats; A.cost = cost; A.vmax = vmax; A.prm = *params; A.choice = choice; A.report = report;
   A.status = status;
-  rs_route_kernel<<<1, kThreads, 0, (cudaStream_t)stream_>>>(A);
+  const int n_pairs = n_items * n_cand;
+  const size_t smem = (size_t)n_items * (sizeof(Sub) + sizeof(int)) + (n_pairs <= kCachePairs ? (size_t)n_pairs * 16 : 0) + 16;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(rs_route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess)
+      return RS_ERR_CUDA;
+    attr_set = true;
+  }
+  rs_route_kernel<<<1, kThreads, smem, (cudaStream_t)stream_>>>(A);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }
