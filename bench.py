@@ -44,7 +44,10 @@ def measured_peaks():
 
 # ----------------------------------------------------------------------------------------- workloads
 def workload_spec(name: str, n_override: int | None):
-    from synth import config1_spec, config2_spec, config3_spec
+    from synth import config1_spec, config2_spec, config3_spec, config4_layer_spec
+    if name == "config4":
+        spec = config4_layer_spec(0, n=n_override or 131072, seg_len=(n_override or 131072) // 4)
+        return spec, None, dict(budget_frac=0.15, cert_max=0.05), None
     if name == "config1":
         spec = config1_spec(toeplitz=True, n=n_override or 4096)
         lib = [(2, 256, 512), (0, 0, 0)]
@@ -210,13 +213,20 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="config3", choices=["config1", "config2", "config3"])
+    ap.add_argument("--workload", default="config3", choices=["config1", "config2", "config3", "config4"])
+    ap.add_argument("--layers", type=int, default=32, help="config4: layers of the attention-only stack per step")
+    ap.add_argument("--distinct-layers", type=int, default=2, help="config4: distinct generated layers that are cycled")
+    ap.add_argument("--sweep", action="store_true", help="config-5 sweep: n x budget x forced-dense cells, JSONL output")
     ap.add_argument("--n", type=int, default=None, help="override the sequence length (smaller profiling case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.sweep:
+        return sweep(args)
+    if args.workload == "config4" and args.impl == "ours":
+        return stack(args)
 
     from synth import make_layer
     spec, lib, route_kw, fixed = workload_spec(args.workload, args.n)
@@ -394,6 +404,178 @@ def main():
         "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
     }
     print(json.dumps(out))
+    return 0
+
+
+def _to_dev(bits, dev):
+    import torch
+    return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+
+
+def stack(args):
+    """Config 4: attention-only prefill stack, per-segment rerouting, one attention launch per layer."""
+    import torch
+    import paper_2608_29058_b200 as rs
+    from synth import config4_layer_spec, make_layer
+    rank, world = init_ranks(args.gpus)
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    n = args.n or 131072
+    layers = []
+    for l in range(max(1, args.distinct_layers)):
+        spec = config4_layer_spec(l, n=n, seg_len=n // 4)
+        L = make_layer(spec)
+        layers.append((spec, _to_dev(L["Q"], dev), _to_dev(L["K"], dev), _to_dev(L["V"], dev)))
+    spec0 = layers[0][0]
+    p = rs.Problem(spec0.n_q_heads, spec0.n_kv_heads, n, spec0.seg_bounds())
+    layer = rs.RoutedPrefillLayer(p, None, rs.RouteConfig(budget_frac=0.15, cert_max=0.05), device=dev)
+
+    def step(collect=None):
+        for l in range(args.layers):
+            _, Q, K, V = layers[l % len(layers)]
+            layer.forward(Q, K, V)
+            if collect is not None:
+                collect.append((layer.choice.clone(), layer.stats.clone()))
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    rs.check_status(layer.status, "warm-up")
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    layer.counters.zero_()
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop(t0, time.time())
+    ms_step = e0.elapsed_time(e1) / args.steps
+    rs.check_status(layer.status, "timed region")
+    chunks = int(layer.counters.cpu().numpy()[0]) // args.steps
+    info = []
+    step(info)                       # one untimed pass to read the routes and pair counts of every layer
+    torch.cuda.synchronize()
+    names = {0: "dense", 1: "a_shape", 2: "vertical_slash", 3: "block_sparse"}
+    kinds = [s.kind for s in spec0.segments]
+    pairs, hist = 0, {}
+    for l, (choice, stats) in enumerate(info):
+        ch, st = choice.cpu().numpy(), stats.cpu().numpy()
+        for it in range(p.n_items):
+            pairs += int(st[it, ch[it], 4])
+            sp = layers[l % len(layers)][0]
+            key = sp.segments[it // p.n_q_heads].kind + ":" + names[layer.cands[ch[it]][0]]
+            hist[key] = hist.get(key, 0) + 1
+    f_mask, f_tile = 512.0 * pairs, chunks * (128 * 64 * 512.0)
+    f_dense = float(rs.dense_flops(p.seg_bounds, p.n_q_heads)) * args.layers
+    ms, units = aggregate_over_ranks(ms_step, f_mask, dev)
+    if rank != 0:
+        return 0
+    peaks = measured_peaks()
+    out = {"metric": "effective TFLOP/s of routed sparse prefill attention (FLOPs of selected query-key pairs / stack time)",
+           "value": units / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "bf16", "data": "synthetic",
+           "config": {"workload": f"config4: {args.layers}-layer attention-only stack, Hq=32 Hkv=8 d=128 n={n}, four segments of "
+                                  f"{n // 4} with local / delimiter / needle / diffuse structure (order seeded per layer), per-segment "
+                                  f"online routing; {len(layers)} distinct generated layers cycled", "replicas": args.gpus,
+                      "l2": "inputs exceed L2"},
+           "ms_per_layer": ms / args.layers, "segment_kinds_layer0": kinds, "routes_by_segment_kind": hist,
+           "flops": {"selected_pairs": f_mask, "issued_tiles": f_tile, "dense": f_dense,
+                     "selected_fraction_of_dense": f_mask / f_dense},
+           "roofline": {"kernel": "whole stack (attention dominates)", "bound": "tensor",
+                        "achieved": f_tile / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                        "frac": f_tile / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                        "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "traffic": None},
+           "clocks": clocks, "gpu_launches": 23 * args.layers * args.steps}
+    print(json.dumps(out))
+    return 0
+
+
+def sweep(args):
+    """Config 5: n x latency budget x forced-dense fraction on the config-3 layer; one JSON line per cell (resumable)."""
+    import torch
+    import paper_2608_29058_b200 as rs
+    from synth import config3_spec, make_layer
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    out_dir = os.path.join(ROOT, "gpurun_out")
+    os.makedirs(out_dir, exist_ok=True)
+    path = os.path.join(out_dir, "sweep_config5.jsonl")
+    done = set()
+    if os.path.exists(path):
+        for line in open(path):
+            try:
+                d = json.loads(line)
+                done.add((d["n"], d["budget"], d["forced_dense"]))
+            except Exception:
+                pass
+    peaks = measured_peaks()
+    ns = [args.n] if args.n else [16384, 32768, 65536, 131072]
+    cells = []
+    for n in ns:
+        spec = config3_spec(n)
+        L = make_layer(spec)
+        Q, K, V = _to_dev(L["Q"], dev), _to_dev(L["K"], dev), _to_dev(L["V"], dev)
+        p = rs.Problem(spec.n_q_heads, spec.n_kv_heads, n)
+        layer = rs.RoutedPrefillLayer(p, None, rs.RouteConfig(), device=dev)
+        lse_d = torch.empty((p.n_q_heads, n), dtype=torch.float32, device=dev)
+        O_d = torch.empty_like(layer.O)
+        for _ in range(2):
+            rs.rs_dense_prefill_attn(p, Q, K, V, O_d, lse_d, None, None, layer.ws, layer.status)
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record()
+        for _ in range(2):
+            rs.rs_dense_prefill_attn(p, Q, K, V, O_d, lse_d, None, None, layer.ws, layer.status)
+        d1.record()
+        torch.cuda.synchronize()
+        dense_ms = d0.elapsed_time(d1) / 2
+        del O_d, lse_d
+        perm = np.random.default_rng(260829058 + 5).permutation(p.n_q_heads)
+        for budget in (0.05, 0.10, 0.20, 0.40):
+            for forced in (0.0, 0.25, 0.5, 1.0):
+                if (n, budget, forced) in done:
+                    continue
+                layer.cfg.budget_frac = budget
+                fd = torch.zeros(p.n_items, dtype=torch.int32, device=dev)
+                fd[torch.from_numpy(perm[:int(round(forced * p.n_q_heads))].copy()).to(dev)] = 1
+                for _ in range(max(1, min(args.warmup, 2))):
+                    layer.forward(Q, K, V, forced_dense=fd)
+                torch.cuda.synchronize()
+                layer.counters.zero_()
+                k = max(2, min(args.steps, 3))
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(k):
+                    layer.forward(Q, K, V, forced_dense=fd, record_events=True)
+                e1.record()
+                torch.cuda.synchronize()
+                rs.check_status(layer.status, "sweep cell")
+                ms = e0.elapsed_time(e1) / k
+                stages = layer.stage_ms()
+                ch, st = layer.choice.cpu().numpy(), layer.stats.cpu().numpy()
+                pairs = int(sum(int(st[it, ch[it], 4]) for it in range(p.n_items)))
+                f_mask = 512.0 * pairs
+                f_tile = int(layer.counters.cpu().numpy()[0]) // k * (128 * 64 * 512.0)
+                cell = {"n": n, "budget": budget, "forced_dense": forced, "ms_per_layer": ms, "dense_ms_per_layer": dense_ms,
+                        "speedup_vs_own_dense": dense_ms / ms, "effective_tflops": f_mask / (ms * 1e-3) / 1e12,
+                        "attention_ms": stages["attention"], "overhead_ms": ms - stages["attention"],
+                        "tile_tflops": f_tile / (stages["attention"] * 1e-3) / 1e12,
+                        "roofline_frac": f_tile / (stages["attention"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                        "selected_fraction_of_dense": f_mask / float(rs.dense_flops(p.seg_bounds, p.n_q_heads)),
+                        "n_dense_heads": int(sum(1 for it in range(p.n_items) if layer.cands[ch[it]][0] == 0))}
+                with open(path, "a") as f:
+                    f.write(json.dumps(cell) + "\n")
+                cells.append(cell)
+        del layer, Q, K, V
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "config-5 sweep", "cells_run": len(cells), "cells_file": "gpurun_out/sweep_config5.jsonl",
+                      "peak": peaks["bf16_tflops_sustained"], "data": "synthetic"}))
     return 0
 
 

@@ -189,7 +189,7 @@ def config3_spec(n: int = 131072, seed_offset: int = 3, n_q_heads: int = 32, n_k
 def config4_layer_spec(layer: int, n: int = 131072, seg_len: int = 32768,
                        n_q_heads: int = 32, n_kv_heads: int = 8) -> LayerSpec:
     """One layer of the segmented stack: structure switches every seg_len tokens, order seeded per layer."""
-    spec = config2_spec(n=n, seed_offset=4, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads)
+    spec = config3_spec(n=n, seed_offset=4, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads)
     spec.layer = layer
     kinds = ["local", "delimiter", "needle", "diffuse"]
     order = _rng(spec.seed, layer, _T_MISC, 1002).permutation(len(kinds))
@@ -305,7 +305,7 @@ def make_layer(spec: LayerSpec, heads: Optional[Sequence[int]] = None) -> Dict[s
                 planted += pos.tolist()
             elif s.kind == "delimiter":
                 pos = np.arange(s.start, s.end, 257)
-                kboost[pos] = 4.0
+                kboost[pos] = a_vert[g] if spec.nu is not None else 4.0
                 planted += pos.tolist()
             elif s.kind == "needle":
                 # 16 key vectors, each copied to 8 seeded positions of the segment
