@@ -108,3 +108,45 @@ def test_argument_checks():
     with pytest.raises(rs.RouteSparseError):      # workspace too small
         rs.rs_dense_prefill_attn(p, x, x, x, x, x, None, None, torch.zeros(256, dtype=torch.uint8, device="cuda")[:0]
                                  if False else torch.zeros(256, dtype=torch.uint8, device="cuda")[:128], None)
+
+
+def test_single_block_and_maximum_length():
+    """Degenerate sizes: one 64-row block under every pattern, and the largest supported length (262144 keys)."""
+    L = make_layer(tiny_spec(3, 64, 1, 1))
+    p = rs.Problem(1, 1, 64)
+    Qs, Ks, Vs = f64_heads(L)
+    cands = [C(PT.A_SHAPE, 4, 8), C(PT.VERTICAL_SLASH, 7, 5), C(PT.BLOCK_SPARSE, 1), C(PT.DENSE)]
+    probes = oracle_probe_all(Qs, Ks, p)
+    for c in range(len(cands)):
+        sets = oracle_index_sets(p, cands, [c], probes)
+        lib = c_library(cands)
+        idx = upload_materialised(p, lib, sets)
+        O = torch.zeros((1, 64, 128), dtype=torch.float32, device="cuda")
+        lse = torch.zeros((1, 64), dtype=torch.float32, device="cuda")
+        st = rs.new_status()
+        rs.rs_sparse_prefill_attn(p, dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"]), lib, idx,
+                                  torch.tensor([c], dtype=torch.int32, device="cuda"), O, lse, None, None,
+                                  rs.new_workspace(p, lib), st)
+        rs.check_status(st, "single block")
+        Oo, lo, _ = A.masked_attention(Qs[0], Ks[0], Vs[0], lambda r, nk: PT.mask_rows(sets[0], r, nk))
+        assert_attention_close(O[0].cpu().numpy(), Oo, str(cands[c]))
+    n = 262144
+    L = make_layer(tiny_spec(4, n, 1, 1))
+    p = rs.Problem(1, 1, n)
+    cands = [C(PT.A_SHAPE, 128, 1024), C(PT.DENSE)]
+    lib = c_library(cands)
+    ix = PT.build_indices(cands[0], 0, n)
+    idx = upload_materialised(p, lib, [ix])
+    O = torch.zeros((1, n, 128), dtype=torch.float32, device="cuda")
+    lse = torch.zeros((1, n), dtype=torch.float32, device="cuda")
+    st = rs.new_status()
+    rs.rs_sparse_prefill_attn(p, dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"]), lib, idx,
+                              torch.zeros(1, dtype=torch.int32, device="cuda"), O, lse, None, None, rs.new_workspace(p, lib), st)
+    rs.check_status(st, "maximum length")
+    Qs, Ks, Vs = f64_heads(L)
+    for rows in (np.arange(0, 64), np.arange(100000, 100064), np.arange(n - 64, n)):
+        Oo, lo, _ = A.masked_attention(Qs[0], Ks[0], Vs[0], lambda r, nk: PT.mask_rows(ix, r, nk), rows, chunk=64)
+        assert_attention_close(O[0, rows].cpu().numpy(), Oo, f"rows {rows[0]}")
+        assert np.abs(lse[0, rows].cpu().numpy() - lo).max() < 2e-3
+    with pytest.raises(rs.RouteSparseError):
+        rs.rs_workspace_bytes(rs.Problem(1, 1, 2 * n), None)
