@@ -203,6 +203,13 @@ int rs_certificate(int n_q_heads, int n_kv_heads, int n_keys, const float* lse_s
                    float* m_row, float* cert_row, float* cert_tight, float* m_head, float* cert_head,
                    int32_t* status, void* stream);
 
+/* Self test of the bounded device-side wait every kernel of this library uses (no passage of the paper: the waits
+ * exist because the kernels synchronise TMA, tensor-core and softmax roles through mbarriers).  Launches one small
+ * kernel that waits on a barrier nothing arrives on, with a limit of poll_limit (1 .. 2^20) polls; the wait gives up,
+ * the kernel writes RS_ERR_TIMEOUT and site 99 to `status` (device int32[RS_STATUS_WORDS], required) and ends
+ * normally, leaving the context usable. */
+int rs_selftest_wait_timeout(int32_t* status, unsigned int poll_limit, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -46,7 +46,7 @@ class rs_route_params(C.Structure):
 
 
 EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "rs_build_indices", "rs_route",
-           "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate"]
+           "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate", "rs_selftest_wait_timeout"]
 
 
 def lib_path() -> str:
@@ -218,6 +218,10 @@ def rs_certificate(n_q_heads: int, n_kv_heads: int, n_keys: int, lse_sel, lse_fu
                                  int(rows.numel()), _ptr(vmax), _ptr(onorm), C.c_float(delta_q), _ptr(m_row),
                                  _ptr(cert_row), _ptr(cert_tight), _ptr(m_head), _ptr(cert_head), _ptr(status),
                                  _stream()), "rs_certificate")
+
+
+def rs_selftest_wait_timeout(status, poll_limit: int = 2000):
+    _check(load().rs_selftest_wait_timeout(_ptr(status), C.c_uint(poll_limit), _stream()), "rs_selftest_wait_timeout")
 
 
 def check_status(status: torch.Tensor, what: str = "kernel"):

@@ -113,3 +113,25 @@ extern "C" int rs_workspace_bytes(const rs_problem* p, const rs_candidate* lib, 
   *bytes = rs_align_up(need, 256);
   return RS_OK;
 }
+
+// ------------------------------------------------------------------------------------------ self test of the bounded wait
+namespace {
+__global__ void rs_selftest_wait_kernel(int32_t* status, unsigned int limit) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+  // nothing ever arrives on this barrier: the wait has to give up by itself and the kernel has to end normally
+  if (threadIdx.x == 0 && !mbar_wait(smem_u32(&bar), 0, &abort_flag, limit)) rs_report(status, RS_ERR_TIMEOUT, 99);
+}
+}  // namespace
+
+extern "C" int rs_selftest_wait_timeout(int32_t* status, unsigned int poll_limit, void* stream) {
+  if (status == nullptr || poll_limit == 0 || poll_limit > (1u << 20)) return RS_ERR_INVALID_ARG;
+  rs_selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(status, poll_limit);
+  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+}

@@ -50,13 +50,14 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 // Bounded wait. Returns false when the limit ran out or another role raised `abort_flag`.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t limit = RS_SPIN_LIMIT) {
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     ++spins;
     if ((spins & 0x3ffu) == 0) {
       if (*abort_flag) return false;
-      if (spins > RS_SPIN_LIMIT) return false;
+      if (spins > limit) return false;
     }
   }
   return true;

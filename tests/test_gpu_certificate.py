@@ -30,3 +30,15 @@ def test_certificate_matches_oracle():
         assert np.allclose(tight[h], tg, rtol=1e-4, atol=1e-5)
         assert abs(m_head[h] - mh) < 1e-6 and abs(cert_head[h, 0] - ch) < 1e-4 and abs(cert_head[h, 1] - cm) < 1e-4
     assert np.all(m_row <= 1.0) and np.all(cert_row >= 0)
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A device-side wait that nothing satisfies runs out by itself; the status words say so and the context lives on."""
+    st = rs.new_status()
+    rs.rs_selftest_wait_timeout(st, 2000)
+    torch.cuda.synchronize()
+    words = st.cpu().tolist()
+    assert words[0] == -6 and words[1] == 99
+    with pytest.raises(rs.RouteSparseError, match="bounded device-side wait"):
+        rs.check_status(st, "self test")
+    assert float((torch.ones(4, device="cuda") * 2).sum()) == 8.0       # the device still answers
