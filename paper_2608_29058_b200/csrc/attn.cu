@@ -560,9 +560,15 @@ __global__ void rs_attn_cost_kernel(AttnParams P, int n_work, int* cost, int2* i
   items[wid] = make_int2(item, tile);
 }
 
-// Counting sort by cost, descending (single block).
-__global__ void rs_attn_order_kernel(int n_work, int n_bins, const int* cost, const int2* items, int2* order) {
+// Launch order: KV groups one after the other (the CTAs in flight then stream the same K / V, which keeps them in L2),
+// inside a group heaviest item first.  One block per KV group runs a counting sort by cost over the group's items,
+// which are contiguous in the item enumeration (head-major).
+__global__ void rs_attn_order_kernel(int per_group, int n_bins, const int* cost, const int2* items, int2* order) {
   extern __shared__ int hist[];
+  const int n_work = per_group;
+  cost += (size_t)blockIdx.x * per_group;
+  items += (size_t)blockIdx.x * per_group;
+  order += (size_t)blockIdx.x * per_group;
   for (int i = threadIdx.x; i <= n_bins; i += blockDim.x) hist[i] = 0;
   __syncthreads();
   for (int i = threadIdx.x; i < n_work; i += blockDim.x) atomicAdd(&hist[min(cost[i], n_bins - 1)], 1);
@@ -694,7 +700,7 @@ int launch_attn(const rs_problem* p, const void* Q, const void* K, const void* V
   int2* order = reinterpret_cast<int2*>(wsb + w.order);
   rs_attn_cost_kernel<<<(n_work + 255) / 256, 256, 0, stream>>>(P, n_work, cost, items);
   const int n_bins = (P.n >> 6) + 66;
-  rs_attn_order_kernel<<<1, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work, n_bins, cost, items, order);
+  rs_attn_order_kernel<<<P.Hkv, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work / P.Hkv, n_bins, cost, items, order);
   if (choice != nullptr && any_vs) {
     dim3 grid((P.kv_pad + 15) / 16, w.n_items);
     rs_pack_vertical_kernel<<<grid, 256, 0, stream>>>(P, reinterpret_cast<const __nv_bfloat16*>(K),
@@ -810,7 +816,7 @@ extern "C" int rs_dense_prefill_attn_noalloc(const rs_problem* p, const void* Q,
   // every entry of cost / items / order is rewritten by the two kernels below, so nothing has to be cleared
   rs_attn_cost_kernel<<<(n_work + 255) / 256, 256, 0, stream>>>(P, n_work, cost, items);
   const int n_bins = (P.n >> 6) + 66;
-  rs_attn_order_kernel<<<1, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work, n_bins, cost, items, order);
+  rs_attn_order_kernel<<<P.Hkv, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work / P.Hkv, n_bins, cost, items, order);
   if (cudaFuncSetAttribute(rs_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024) != cudaSuccess)
     return RS_ERR_CUDA;
   // the gathered-column maps are never read by dense tiles; they alias K and V
