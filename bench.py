@@ -216,6 +216,9 @@ def main():
     ap.add_argument("--workload", default="config3", choices=["config1", "config2", "config3", "config4"])
     ap.add_argument("--layers", type=int, default=32, help="config4: layers of the attention-only stack per step")
     ap.add_argument("--distinct-layers", type=int, default=2, help="config4: distinct generated layers that are cycled")
+    ap.add_argument("--cost", default="flops", choices=["flops", "measured"],
+                    help="router cost table: FLOPs of the selected pairs, or kernel times profiled before the timed region")
+    ap.add_argument("--rescue", action="store_true", help="fallback variant: cheapest passing sparse candidate of any family before dense")
     ap.add_argument("--sweep", action="store_true", help="config-5 sweep: n x budget x forced-dense cells, JSONL output")
     ap.add_argument("--n", type=int, default=None, help="override the sequence length (smaller profiling case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -255,7 +258,7 @@ def main():
     to_dev = lambda bits: torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
     Q, K, V = to_dev(L["Q"]), to_dev(L["K"]), to_dev(L["V"])
     p = rs.Problem(spec.n_q_heads, spec.n_kv_heads, spec.n, [int(x) for x in L["seg_bounds"]])
-    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(**route_kw), device=dev)
+    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(rescue_any=args.rescue, **route_kw), device=dev)
     fixed_t = None
     if fixed:
         fixed_t = torch.from_numpy(fixed_choice_for(layer.cands, spec.n_q_heads)).to(dev)
@@ -273,6 +276,21 @@ def main():
         step()
     torch.cuda.synchronize()
     rs.check_status(layer.status, "warm-up")
+    calibration = None
+    if args.cost == "measured" and not fixed:
+        # offline hardware profiling of the library (outside the timed region), then the router uses the measured table
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for _ in range(3):
+            step()
+        f1.record()
+        torch.cuda.synchronize()
+        calibration = layer.profile_costs(Q, K, V)
+        calibration["flop_routed_ms_per_layer"] = f0.elapsed_time(f1) / 3
+        calibration["flop_routed_routes"] = layer.choice.cpu().tolist()
+        for _ in range(args.warmup):
+            step()
+        torch.cuda.synchronize()
 
     # ---- timed region: K steps, CUDA events on the launching stream, per-stage events inside every step
     sampler = ClockSampler(local)
@@ -396,6 +414,7 @@ def main():
         "flops": {"selected_pairs": f_mask, "issued_tiles": f_tile, "dense": f_dense,
                   "selected_fraction_of_dense": f_mask / f_dense},
         "routes": hist, "route_report": layer.route_report() if not fixed else None,
+        "cost_model": args.cost, "calibration": calibration, "fallback_rescue": bool(args.rescue),
         "roofline": {"kernel": "rs_attn_kernel (one launch, all heads)", "bound": "tensor", "achieved": achieved,
                      "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": f"bf16_tflops_sustained, {peaks['source']}",

@@ -102,7 +102,8 @@ typedef struct {
   int32_t use_cert;        /* 0: no fallback step */
   int32_t cert_mode;       /* rs_cert_mode: REL 2(1-m_low), ABS 2(1-m_low) * V_max */
   int32_t expand_first;    /* 1: next larger budget of the family before dense */
-  int32_t reserved;
+  int32_t reserved;        /* rescue_any: 1 = when the family has no larger budget, take the cheapest sparse candidate
+                              of any family whose certificate passes before giving up and going dense */
   const int32_t* forced_dense;  /* device int32[n_items], non-zero = force dense last; may be NULL */
   const int32_t* fixed_choice;  /* device int32[n_items]; when set, bypasses solve and fallback; may be NULL */
 } rs_route_params;

@@ -38,6 +38,7 @@ class RouteParams:
     cert_max: Optional[float] = None  # fallback fires while certificate > cert_max (None: no fallback)
     cert_mode: int = CERT_REL        # REL: 2(1 - m_low);  ABS: 2(1 - m_low) * vmax
     expand_first: bool = True        # try the next larger budget of the family before dense
+    rescue_any: bool = False         # before dense, take the cheapest sparse candidate of any family that passes
     forced_dense: Sequence[int] = field(default_factory=list)   # items forced to dense last
     fixed_choice: Optional[Sequence[int]] = None                 # bypasses the solve and the fallback
 
@@ -130,6 +131,19 @@ def route(lib: List[Candidate], cov_fx: np.ndarray, cost: np.ndarray, vmax: np.n
                         break
                     fired = True
                     nxt = _next_larger(lib, choice[it]) if p.expand_first else None
+                    if nxt is None and p.rescue_any:
+                        # "switches to dense attention if no sparse candidate satisfies the threshold": look at every
+                        # sparse candidate, keep those whose certificate passes, take the cheapest (ties: lower index)
+                        best = None
+                        for k, cand in enumerate(lib):
+                            if cand.pattern == DENSE:
+                                continue
+                            ck = 2.0 * (1.0 - max(0.0, float(M[it, k]) - p.delta_q))
+                            if p.cert_mode == CERT_ABS:
+                                ck = ck * float(np.float32(vmax[it]))
+                            if not ck > p.cert_max and (best is None or int(cost[it, k]) < int(cost[it, best])):
+                                best = k
+                        nxt = best
                     choice[it] = nxt if nxt is not None else dense_c
                 n_fallback += int(fired)
     for it in p.forced_dense:

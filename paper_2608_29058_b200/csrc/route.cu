@@ -177,7 +177,17 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
           if (A.prm.cert_mode == RS_CERT_ABS) cert = __dmul_rn(cert, vm);
           if (!(cert > A.prm.cert_max)) break;
           fired = true;
-          const int nxt = A.prm.expand_first ? A.next_larger[c] : -1;
+          int nxt = A.prm.expand_first ? A.next_larger[c] : -1;
+          if (nxt < 0 && A.prm.reserved != 0) {
+            // rescue: the cheapest sparse candidate of any family whose certificate passes (ties: lower index)
+            for (int k = 0; k < A.n_cand; ++k) {
+              if (A.lib[k].pattern == RS_DENSE) continue;
+              const double mk = fmax(0.0, __dsub_rn(m_hat_of(A, it, k), A.prm.delta_q));
+              double ck = __dmul_rn(2.0, __dsub_rn(1.0, mk));
+              if (A.prm.cert_mode == RS_CERT_ABS) ck = __dmul_rn(ck, vm);
+              if (!(ck > A.prm.cert_max) && (nxt < 0 || costf(it, k) < costf(it, nxt))) nxt = k;
+            }
+          }
           c = (nxt >= 0) ? nxt : A.dense_c;
         }
         ch[it] = c;

@@ -43,6 +43,7 @@ class RouteConfig:
     cert_max: Optional[float] = 0.05   # None disables the fallback step
     cert_mode: int = rs.RS_CERT_REL
     expand_first: bool = True
+    rescue_any: bool = False           # before dense, the cheapest sparse candidate of any family that passes
 
 
 class _IdxView:
@@ -100,6 +101,9 @@ class RoutedPrefillLayer:
         self.prm = rs.rs_route_params()
         self._forced = None
         self.events = None
+        self.cost_table = None      # int64 [n_items, n_cand] measured kernel time (ns); None: FLOPs of the selected pairs
+        self.cost_budget = None     # layer budget in the table's unit
+        self.cost_t_probe = 0
 
     # ------------------------------------------------------------------ steps (each only enqueues kernels)
     def probe(self, Q, K, V):
@@ -112,16 +116,20 @@ class RoutedPrefillLayer:
 
     def route(self, forced_dense: Optional[torch.Tensor] = None):
         c, prm = self.cfg, self.prm
-        prm.budget = int(c.budget_frac * dense_flops(self.p.seg_bounds, self.p.n_q_heads))
-        prm.t_probe = probe_flops(self.p.seg_bounds, self.p.n_q_heads)
+        if self.cost_table is not None:
+            prm.budget, prm.t_probe = int(self.cost_budget), int(self.cost_t_probe)
+        else:
+            prm.budget = int(c.budget_frac * dense_flops(self.p.seg_bounds, self.p.n_q_heads))
+            prm.t_probe = probe_flops(self.p.seg_bounds, self.p.n_q_heads)
         prm.alpha, prm.delta_q = c.alpha, c.delta_q
         prm.use_cert = 0 if c.cert_max is None else 1
         prm.cert_max = 0.0 if c.cert_max is None else c.cert_max
         prm.cert_mode, prm.expand_first = c.cert_mode, int(c.expand_first)
+        prm.reserved = int(c.rescue_any)
         self._forced = forced_dense
         prm.forced_dense = None if forced_dense is None else forced_dense.data_ptr()
         prm.fixed_choice = None
-        rs.rs_route(self.p, self.lib, self.stats, None, self.vmax, prm, self.choice, self.report, self.status)
+        rs.rs_route(self.p, self.lib, self.stats, self.cost_table, self.vmax, prm, self.choice, self.report, self.status)
 
     def materialise(self, reuse_evaluation: bool = False):
         self._reuse_eval = reuse_evaluation and len(self.cands) > 1
@@ -139,6 +147,48 @@ class RoutedPrefillLayer:
         rs.rs_certificate(p.n_q_heads, p.n_kv_heads, p.n_keys, self.lse_sel, self.lse_probe, self.probe_rows,
                           self.vmax[p.n_segments - 1], self.onorm, self.cfg.delta_q, self.m_row, self.cert_row, None,
                           self.m_head, self.cert_head, self.status)
+
+    # ------------------------------------------------------------------ offline calibration (Section 3.5)
+    def profile_costs(self, Q, K, V, reps: int = 3):
+        """Hardware profiling of the pattern library (Section 3.1, 3.5): every candidate runs as the route of all
+        heads and its attention launch is timed (median of `reps`, CUDA events).  The measured time of a candidate is
+        split over the items in proportion to their pair counts and stored as the int64 nanosecond cost table the
+        router reads; the layer budget becomes budget_frac x the dense candidate's measured time and t_probe the
+        measured probe + evaluation time.  Synchronises; meant to run once per (library, length), outside the hot path."""
+        import numpy as np
+        p, n_cand = self.p, len(self.cands)
+        ev = lambda: torch.cuda.Event(enable_timing=True)
+        self.probe(Q, K, V)
+        self.evaluate_candidates()
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        a.record(); self.probe(Q, K, V); self.evaluate_candidates(); b.record()
+        torch.cuda.synchronize()
+        t_probe_ns = a.elapsed_time(b) * 1e6
+        pairs = self.stats.cpu().numpy()[:, :, 4].astype(np.float64)
+        ms = np.zeros(n_cand)
+        saved = self.choice.clone()
+        for c in range(n_cand):
+            self.choice.fill_(c)
+            self.materialise(reuse_evaluation=True)
+            self.attention(Q, K, V)
+            ts = []
+            for _ in range(reps):
+                a, b = ev(), ev()
+                a.record(); self.attention(Q, K, V); b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            ms[c] = float(np.median(ts))
+        self.choice.copy_(saved)
+        table = np.maximum(1, np.rint(ms[None, :] * 1e6 * pairs / pairs.sum(axis=0, keepdims=True))).astype(np.int64)
+        dense_c = [i for i, c in enumerate(self.cands) if c[0] == rs.RS_DENSE][0]
+        self.cost_table = torch.from_numpy(table).to(self.O.device)
+        self.cost_budget = int(self.cfg.budget_frac * ms[dense_c] * 1e6)
+        self.cost_t_probe = int(t_probe_ns)
+        return {"candidate_ms": ms.tolist(), "t_probe_ms": t_probe_ns * 1e-6, "budget_ms": self.cost_budget * 1e-6}
+
+    def use_flop_costs(self):
+        self.cost_table = None
 
     # ------------------------------------------------------------------ whole layer
     def forward(self, Q, K, V, fixed_choice: Optional[torch.Tensor] = None,

@@ -131,3 +131,25 @@ def test_config1_single_head_vertical_slash():
     cfg = rs.RouteConfig(budget_frac=0.6, cert_max=None)
     layer, choice = run_and_check(spec, [0, 4096], cands, cfg, "config1")
     assert choice.tolist() == [0]
+
+
+def test_profiled_cost_table_routes_like_the_oracle():
+    """Measured kernel times as the router's cost table (hardware profiling of Section 3.1 / 3.5): the device
+    decision equals the oracle's on the same table."""
+    cands = [C(PT.A_SHAPE, 8, 128), C(PT.VERTICAL_SLASH, 32, 48), C(PT.BLOCK_SPARSE, 3), C(PT.DENSE)]
+    spec = tiny_spec(71, 2048, 4, 2)
+    L = make_layer(spec)
+    p = rs.Problem(4, 2, 2048)
+    layer = rs.RoutedPrefillLayer(p, [(c.pattern, c.b0, c.b1) for c in cands], rs.RouteConfig(budget_frac=0.5, cert_max=0.9))
+    Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+    info = layer.profile_costs(Q, K, V, reps=2)
+    table = layer.cost_table.cpu().numpy()
+    assert table.shape == (4, 4) and np.all(table >= 1) and len(info["candidate_ms"]) == 4
+    assert abs(table.sum(axis=0)[3] - info["candidate_ms"][3] * 1e6) <= 4          # shares add up to the measured time
+    layer.forward(Q, K, V)
+    rs.check_status(layer.status, "profiled")
+    stats = layer.stats.cpu().numpy()
+    vmax = layer.vmax.cpu().numpy()
+    want, _ = RT.route(cands, stats[:, :, :4].astype(np.uint64), table, np.array([vmax[0, h // 2] for h in range(4)], np.float32),
+                       RT.RouteParams(budget=layer.cost_budget, t_probe=layer.cost_t_probe, cert_max=0.9))
+    assert np.array_equal(layer.choice.cpu().numpy(), want)

@@ -36,6 +36,7 @@ def gpu_route(p, lib, cov, pairs, cost, vmax, **kw):
     prm.use_cert = 0 if kw.get("cert_max") is None else 1
     prm.cert_max = 0.0 if kw.get("cert_max") is None else kw["cert_max"]
     prm.cert_mode = kw.get("cert_mode", rs.RS_CERT_REL); prm.expand_first = int(kw.get("expand_first", True))
+    prm.reserved = int(kw.get("rescue_any", False))
     keep = []
     if kw.get("forced_dense"):
         fd = torch.zeros(cov.shape[0], dtype=torch.int32, device="cuda"); fd[list(kw["forced_dense"])] = 1
@@ -70,12 +71,13 @@ def test_route_is_bit_exact(n_seg, Hq, Hkv):
                   cert_max=[None, 0.3, 0.05, 0.2, None, 2.0][trial],
                   cert_mode=[rs.RS_CERT_REL, rs.RS_CERT_REL, rs.RS_CERT_ABS, rs.RS_CERT_REL, 0, rs.RS_CERT_ABS][trial],
                   expand_first=trial != 3, delta_q=[0, 0.01, 0, 0, 0, 0.1][trial],
-                  forced_dense=[0, n_items - 1] if trial == 1 else None)
+                  forced_dense=[0, n_items - 1] if trial == 1 else None, rescue_any=trial in (2, 5))
         use_cost = None if trial % 2 == 0 else cost
         got, rep = gpu_route(p, LIB, cov, pairs, use_cost, vmax_sg, **kw)
         want, wrep = RT.route(LIB, cov, cost, vmax_item, RT.RouteParams(
             budget=kw["budget"], t_probe=kw["t_probe"], alpha=kw["alpha"], delta_q=kw["delta_q"], cert_max=kw["cert_max"],
-            cert_mode=kw["cert_mode"], expand_first=kw["expand_first"], forced_dense=kw["forced_dense"] or []))
+            cert_mode=kw["cert_mode"], expand_first=kw["expand_first"], forced_dense=kw["forced_dense"] or [],
+            rescue_any=kw["rescue_any"]))
         assert np.array_equal(got, want), (trial, got, want)
         assert rep[0] == wrep.total_cost and rep[2] == wrep.n_fallback and rep[3] == wrep.feasible
         assert abs(rep[1] - wrep.total_risk) < 1e-9

@@ -112,3 +112,16 @@ def test_forced_dense_and_fixed_choice():
     assert choice[1] == DENSE_C and choice[3] == DENSE_C
     choice, rep = RT.route(LIB, cov, cost, np.ones(4, np.float32), RT.RouteParams(budget=1, fixed_choice=[0, 1, 2, 3]))
     assert choice.tolist() == [0, 1, 2, 3] and rep.n_fallback == 0
+
+
+def test_rescue_takes_the_cheapest_passing_candidate_of_any_family():
+    cov = np.zeros((1, len(LIB), 4), dtype=np.uint64)
+    for c, m in enumerate([0.5, 0.6, 0.99, 0.995]):          # A-shape candidates fail, VS and BS pass
+        cov[0, c] = np.uint64(int(m * 16 * 2 ** 32))
+    cost = np.array([[10, 20, 60, 50, 100]], dtype=np.int64)
+    base = RT.RouteParams(budget=15, cert_max=0.05)
+    assert RT.route(LIB, cov, cost, np.float32([1.0]), base)[0].tolist() == [DENSE_C]
+    rescued = RT.RouteParams(budget=15, cert_max=0.05, rescue_any=True)
+    assert RT.route(LIB, cov, cost, np.float32([1.0]), rescued)[0].tolist() == [3]     # block-sparse is cheaper than VS
+    cov[0, 2:4] = np.uint64(int(0.9 * 16 * 2 ** 32))
+    assert RT.route(LIB, cov, cost, np.float32([1.0]), rescued)[0].tolist() == [DENSE_C]
