@@ -142,7 +142,7 @@ def aggregate_over_ranks(ms_local: float, units_local: float, device=None):
 
 
 # ----------------------------------------------------------------------------------------- CPU oracle leg
-def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float = 20.0):
+def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float = 20.0, n_heads: int = 8):
     """Times the oracle's masked attention on sampled query blocks under the routed masks.
 
     Returns (effective TFLOP/s, description, cores, max abs difference to gpu_O on the sampled rows).
@@ -152,8 +152,8 @@ def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float =
     from synth import bf16_bits_to_f64
     G = spec.n_q_heads // spec.n_kv_heads
     nb = spec.n // 64
-    heads = sorted(set(int(h) for h in np.linspace(0, spec.n_q_heads - 1, 4)))
-    blocks = sorted(set([nb // 8, nb // 4, nb // 2, (5 * nb) // 8, (7 * nb) // 8, nb - 1]))
+    heads = sorted(set(int(h) for h in np.linspace(0, spec.n_q_heads - 1, n_heads)))
+    blocks = sorted(set(int(b) for b in np.linspace(nb // 16, nb - 1, 10)))
     t_used, pairs_done, rows_done, worst = 0.0, 0, 0, 0.0
     kv_cache = {}
     for h in heads:
@@ -625,7 +625,7 @@ def reference_arm(args, spec, lib, route_kw, fixed, metric, config):
     for it in range(args.warmup + args.steps):
         t0 = time.perf_counter()
         tf, desc, cores, _ = oracle_sample(Lfull, spec, cands, None, lambda h: sets[h], None,
-                                           budget_s=max(2.0, 60.0 / max(1, args.steps + args.warmup)))
+                                           budget_s=max(2.0, 60.0 / max(1, args.steps + args.warmup)), n_heads=4)
         if it >= args.warmup:
             vals.append(tf); times.append((time.perf_counter() - t0) * 1e3)
     v = float(np.mean(vals))
