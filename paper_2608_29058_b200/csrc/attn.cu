@@ -20,7 +20,7 @@ constexpr int kThreads = 192;
 constexpr int kTileM = 128;
 constexpr int kChunk = 64;
 constexpr int kTmemCols = 256;
-constexpr uint32_t kColS = 0;     // S (fp32, 128 columns); P (bf16 pairs, 64 columns) overwrites its start
+constexpr uint32_t kColS = 0;     // two score buffers (fp32, 64 columns each); bf16 P (32 columns) overwrites a buffer's start
 constexpr uint32_t kColO = 128;   // O (fp32, 128 columns)
 
 constexpr uint32_t F_LO = 1u << 12, F_HI = 1u << 13, F_CAUSAL = 1u << 14, F_EDGE = 1u << 15;
@@ -136,15 +136,19 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   uint32_t* d_bits = hi_bits + 128;
   int* wprefix = reinterpret_cast<int*>(d_bits + 128);
   uint64_t* bars = reinterpret_cast<uint64_t*>(wprefix + 132);
-  volatile int* misc = reinterpret_cast<volatile int*>(bars + 8);   // [0] tmem base, [1] abort, [2] n_block, [3] n_vert
-  const uint32_t bar_q = smem_u32(&bars[0]), bar_kf = smem_u32(&bars[1]), bar_ke = smem_u32(&bars[2]),
-                 bar_vf = smem_u32(&bars[3]), bar_ve = smem_u32(&bars[4]), bar_s = smem_u32(&bars[5]),
-                 bar_p = smem_u32(&bars[6]), bar_o = smem_u32(&bars[7]);
+  volatile int* misc = reinterpret_cast<volatile int*>(bars + 14);   // [0] tmem base, [1] abort, [2] n_block, [3] n_vert
+  // barrier pairs (slot 0 / 1) sit next to each other: address of slot s = base + 8 * s
+  const uint32_t bar_q = smem_u32(&bars[0]), bar_o = smem_u32(&bars[1]), bar_kf = smem_u32(&bars[2]),
+                 bar_ke = smem_u32(&bars[4]), bar_vf = smem_u32(&bars[6]), bar_ve = smem_u32(&bars[8]),
+                 bar_s = smem_u32(&bars[10]), bar_p = smem_u32(&bars[12]);
   volatile int* abort_flag = misc + 1;
 
   if (tid == 0) {
-    mbar_init(bar_q, 1); mbar_init(bar_kf, 1); mbar_init(bar_ke, 1); mbar_init(bar_vf, 1);
-    mbar_init(bar_ve, 1); mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1);
+    mbar_init(bar_q, 1); mbar_init(bar_o, 1);
+    for (uint32_t sl = 0; sl < 2; ++sl) {
+      mbar_init(bar_kf + 8u * sl, 1); mbar_init(bar_ke + 8u * sl, 1); mbar_init(bar_vf + 8u * sl, 1);
+      mbar_init(bar_ve + 8u * sl, 1); mbar_init(bar_s + 8u * sl, 1); mbar_init(bar_p + 8u * sl, 128);
+    }
     misc[1] = 0; misc[2] = 0; misc[3] = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -253,50 +257,45 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   __syncthreads();
   const int n_block = misc[2], n_vert = misc[3];
   const int n_chunks = n_block + n_vert;
-  const int n_pairs = (n_chunks + 1) >> 1;
 
   // =========================================================================================== roles
+  // Everything below is pipelined per 64-key chunk; chunk c uses slot c & 1 of the K / V rings, of the two 64-column
+  // score buffers in TMEM and of the barrier pairs, in phase (c >> 1) & 1.  While the softmax warps work on chunk c the
+  // tensor pipe runs O += P(c-1) V(c-1) and S(c+1) = Q K(c+1)^T, so neither side waits for the other in steady state.
   if (warp == 0) {
     if (lane == 0) {
       // ------------------------------------------------------------------ TMA producer
       bool ok = true;
-      for (int t = 0; t < n_pairs && ok; ++t) {
-        const int nch = min(2, n_chunks - 2 * t);
-        const uint32_t ph = (uint32_t)(t & 1);
-        ok = mbar_wait(bar_ke, ph ^ 1u, abort_flag);
-        if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, 1); break; }
-        mbar_arrive_expect_tx(bar_kf, (uint32_t)nch * 16384u);
-        for (int c = 0; c < nch; ++c) {
-          const int ch = 2 * t + c;
-          const uint32_t dst = base + SmemLayout::k + (uint32_t)c * 8192u;
-          if (ch < n_block) {
-            const int row = g * P.n + (int)(list[ch] & 0xfffu) * kChunk;
-            tma_load_2d(dst, &tmK, bar_kf, 0, row);
-            tma_load_2d(dst + 16384, &tmK, bar_kf, 64, row);
-          } else {
-            const int row = item * P.kv_pad + (ch - n_block) * kChunk;
-            tma_load_2d(dst, &tmKp, bar_kf, 0, row);
-            tma_load_2d(dst + 16384, &tmKp, bar_kf, 64, row);
-          }
+      int site = 1;
+      auto load_chunk = [&](int ch, uint32_t dst, uint32_t bar, const CUtensorMap* tm_blocks, const CUtensorMap* tm_packed) {
+        mbar_arrive_expect_tx(bar, 16384u);
+        if (ch < n_block) {
+          const int row = g * P.n + (int)(list[ch] & 0xfffu) * kChunk;
+          tma_load_2d(dst, tm_blocks, bar, 0, row);
+          tma_load_2d(dst + 16384, tm_blocks, bar, 64, row);
+        } else {
+          const int row = item * P.kv_pad + (ch - n_block) * kChunk;
+          tma_load_2d(dst, tm_packed, bar, 0, row);
+          tma_load_2d(dst + 16384, tm_packed, bar, 64, row);
         }
-        ok = mbar_wait(bar_ve, ph ^ 1u, abort_flag);
-        if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, 2); break; }
-        mbar_arrive_expect_tx(bar_vf, (uint32_t)nch * 16384u);
-        for (int c = 0; c < nch; ++c) {
-          const int ch = 2 * t + c;
-          const uint32_t dst = base + SmemLayout::v + (uint32_t)c * 8192u;
-          if (ch < n_block) {
-            const int row = g * P.n + (int)(list[ch] & 0xfffu) * kChunk;
-            tma_load_2d(dst, &tmV, bar_vf, 0, row);
-            tma_load_2d(dst + 16384, &tmV, bar_vf, 64, row);
-          } else {
-            const int row = item * P.kv_pad + (ch - n_block) * kChunk;
-            tma_load_2d(dst, &tmVp, bar_vf, 0, row);
-            tma_load_2d(dst + 16384, &tmVp, bar_vf, 64, row);
-          }
+      };
+      // order of the loads = order in which their slots come free: K0 K1 V0 K2 V1 K3 ...
+      for (int i = 0; i < n_chunks + 2 && ok; ++i) {
+        if (i >= 2) {
+          const int ch = i - 2;
+          const uint32_t slot = (uint32_t)(ch & 1), ph = (uint32_t)((ch >> 1) & 1);
+          ok = mbar_wait(bar_ve + 8u * slot, ph ^ 1u, abort_flag); site = 2;
+          if (!ok) break;
+          load_chunk(ch, base + SmemLayout::v + slot * 8192u, bar_vf + 8u * slot, &tmV, &tmVp);
+        }
+        if (i < n_chunks) {
+          const uint32_t slot = (uint32_t)(i & 1), ph = (uint32_t)((i >> 1) & 1);
+          ok = mbar_wait(bar_ke + 8u * slot, ph ^ 1u, abort_flag); site = 1;
+          if (!ok) break;
+          load_chunk(i, base + SmemLayout::k + slot * 8192u, bar_kf + 8u * slot, &tmK, &tmKp);
         }
       }
-      if (!ok) *abort_flag = 1;
+      if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, site); *abort_flag = 1; }
     }
   } else if (warp == 1) {
     if (lane == 0) {
@@ -309,58 +308,51 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       const uint32_t q_lo = (uint32_t)q_desc, q_hi = (uint32_t)(q_desc >> 32);
       const uint32_t k_lo = (uint32_t)k_desc, k_hi = (uint32_t)(k_desc >> 32);
       const uint32_t v_lo = (uint32_t)v_desc, v_hi = (uint32_t)(v_desc >> 32);
-      constexpr uint32_t kIdescQK128 = umma_idesc_bf16(128, 128, 0, 0), kIdescQK64 = umma_idesc_bf16(128, 64, 0, 0);
+      constexpr uint32_t kIdescQK = umma_idesc_bf16(128, 64, 0, 0);
       constexpr uint32_t kIdescPV = umma_idesc_bf16(128, 128, 0, 1);
-      auto issue_qk = [&](int nch) {
-        const uint32_t idesc = (nch == 2) ? kIdescQK128 : kIdescQK64;
+      auto issue_qk = [&](uint32_t slot) {      // S[slot] = Q K[slot]^T: 8 steps of 16 head dimensions
+        const uint32_t kb = k_lo + slot * 512u, ds = d_s + slot * 64u;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t off = (uint32_t)(((kk >> 2) * 16384 + (kk & 3) * 32) >> 4);
-          umma_ss2(d_s, q_lo + off, q_hi, k_lo + off, k_hi, idesc, kk > 0 ? 1u : 0u);
+          umma_ss2(ds, q_lo + off, q_hi, kb + off, k_hi, kIdescQK, kk > 0 ? 1u : 0u);
         }
       };
-      auto issue_pv = [&](int nch, bool accumulate) {
-        // 16 keys per step: P columns advance by 8, V rows by 16 (2048 bytes)
-        umma_ts2(d_o, d_s, v_lo, v_hi, kIdescPV, accumulate ? 1u : 0u);
+      auto issue_pv = [&](uint32_t slot, bool accumulate) {   // O += P[slot] V[slot]: 4 steps of 16 keys
+        const uint32_t vb = v_lo + slot * 512u, ps = d_s + slot * 64u;
+        umma_ts2(d_o, ps, vb, v_hi, kIdescPV, accumulate ? 1u : 0u);
 #pragma unroll
-        for (int kk = 1; kk < 4; ++kk) umma_ts2(d_o, d_s + 8u * kk, v_lo + 128u * kk, v_hi, kIdescPV, 1u);
-        if (nch == 2) {
-#pragma unroll
-          for (int kk = 4; kk < 8; ++kk) umma_ts2(d_o, d_s + 8u * kk, v_lo + 128u * kk, v_hi, kIdescPV, 1u);
-        }
+        for (int kk = 1; kk < 4; ++kk) umma_ts2(d_o, ps + 8u * kk, vb + 128u * kk, v_hi, kIdescPV, 1u);
       };
       bool ok = mbar_wait(bar_q, 0, abort_flag);
       int site = 3;
-      for (int t = 0; t < n_pairs && ok; ++t) {
-        const int nch = min(2, n_chunks - 2 * t);
-        const uint32_t ph = (uint32_t)(t & 1);
-        if (t == 0) {
-          ok = mbar_wait(bar_kf, 0, abort_flag); site = 4;
-          if (!ok) break;
-          tc_fence_after();
-          issue_qk(nch);
-          umma_commit(bar_s);
-          umma_commit(bar_ke);
-        }
-        ok = mbar_wait(bar_p, ph, abort_flag); site = 5;
-        if (!ok) break;
-        ok = mbar_wait(bar_vf, ph, abort_flag); site = 6;
+      for (int c = 0; c < 2 && c < n_chunks && ok; ++c) {
+        ok = mbar_wait(bar_kf + 8u * c, 0, abort_flag); site = 4;
         if (!ok) break;
         tc_fence_after();
-        issue_pv(nch, t > 0);
-        umma_commit(bar_ve);
-        if (t + 1 < n_pairs) {
-          const int nch2 = min(2, n_chunks - 2 * (t + 1));
-          ok = mbar_wait(bar_kf, ph ^ 1u, abort_flag); site = 7;
+        issue_qk((uint32_t)c);
+        umma_commit(bar_s + 8u * c);
+        umma_commit(bar_ke + 8u * c);
+      }
+      for (int c = 0; c < n_chunks && ok; ++c) {
+        const uint32_t slot = (uint32_t)(c & 1), ph = (uint32_t)((c >> 1) & 1);
+        ok = mbar_wait(bar_p + 8u * slot, ph, abort_flag); site = 5;
+        if (!ok) break;
+        ok = mbar_wait(bar_vf + 8u * slot, ph, abort_flag); site = 6;
+        if (!ok) break;
+        tc_fence_after();
+        issue_pv(slot, c > 0);
+        umma_commit(bar_ve + 8u * slot);
+        if (c + 2 < n_chunks) {
+          ok = mbar_wait(bar_kf + 8u * slot, ph ^ 1u, abort_flag); site = 7;
           if (!ok) break;
           tc_fence_after();
-          issue_qk(nch2);
-          umma_commit(bar_s);
-          umma_commit(bar_ke);
-        } else {
-          umma_commit(bar_o);
+          issue_qk(slot);
+          umma_commit(bar_s + 8u * slot);
+          umma_commit(bar_ke + 8u * slot);
         }
       }
+      if (ok) umma_commit(bar_o);
       if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, site); *abort_flag = 1; }
     }
   } else {
@@ -403,75 +395,67 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       tmem_st16(dst, pk);
     };
 
-    for (int t = 0; t < n_pairs; ++t) {
-      const int nch = min(2, n_chunks - 2 * t);
-      ok = mbar_wait(bar_s, (uint32_t)(t & 1), abort_flag);
+    // One pass per 64-key chunk: rare chunks are masked in place first, then the scores go to registers (two
+    // 32-column loads per wait), chunk maximum, P = exp2(S * scale*log2e - m) against the running maximum, bf16 P
+    // over the start of the chunk's score buffer.  The maximum only moves when some row of the warp exceeds it by more
+    // than 2^8; then l and O are rescaled, after the product of the previous chunk has left the tensor pipe.
+    for (int ch = 0; ch < n_chunks; ++ch) {
+      const uint32_t slot = (uint32_t)(ch & 1), ph = (uint32_t)((ch >> 1) & 1);
+      const uint32_t t_sc = t_s + slot * 64u;
+      ok = mbar_wait(bar_s + 8u * slot, ph, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      // One pass per 64-key chunk: rare chunks are masked in place first, then the scores go to registers (two
-      // 32-column loads per wait), chunk maximum, P = exp2(S * scale*log2e - m) against the running maximum.  The
-      // maximum only moves when some row of the warp exceeds it by more than 2^8; then l, O and the part of P already
-      // written for this tile are rescaled.
-      for (int c = 0; c < nch; ++c) {
-        const int ch = 2 * t + c;
-        {
-          int mode = -1, j0 = 0, edge = 0, vbase = 0;
-          if (ch < n_block) {
-            const uint32_t e = list[ch];
-            if (!(e & (half ? F_HI : F_LO))) {
-              mode = 0;
-            } else if (e & (F_CAUSAL | F_EDGE)) {
-              mode = 1;
-              j0 = (int)(e & 0xfffu) * kChunk;
-              edge = (e & F_EDGE) ? 1 : 0;
-            }
-          } else {
-            mode = 2;
-            vbase = (ch - n_block) * kChunk;
+      {
+        int mode = -1, j0 = 0, edge = 0, vbase = 0;
+        if (ch < n_block) {
+          const uint32_t e = list[ch];
+          if (!(e & (half ? F_HI : F_LO))) {
+            mode = 0;
+          } else if (e & (F_CAUSAL | F_EDGE)) {
+            mode = 1;
+            j0 = (int)(e & 0xfffu) * kChunk;
+            edge = (e & F_EDGE) ? 1 : 0;
           }
-          if (mode >= 0)
-            rs_mask_chunk(t_s + (uint32_t)c * 64u, mode, i, j0, edge, cand.b0, cand.b1, vcols, vbase, n_vcols, d_bits);
+        } else {
+          mode = 2;
+          vbase = (ch - n_block) * kChunk;
         }
-        tmem_ld32(t_s + (uint32_t)c * 64u, v);
-        tmem_ld32(t_s + (uint32_t)c * 64u + 32u, v2);
-        tc_wait_ld();
-        const float m_chunk = fmaxf(max32(v), max32(v2)) * sl2;
-        const float m_new = fmaxf(m_run, m_chunk);
-        const bool need = m_new > m_run + 8.0f;
-        if (__any_sync(0xffffffffu, need)) {
-          const float alpha = (m_new == NEG_INF) ? 1.0f : fast_exp2(m_run - m_new);
-          l_run *= alpha;
-          m_run = m_new;
+        if (mode >= 0) rs_mask_chunk(t_sc, mode, i, j0, edge, cand.b0, cand.b1, vcols, vbase, n_vcols, d_bits);
+      }
+      tmem_ld32(t_sc, v);
+      tmem_ld32(t_sc + 32u, v2);
+      tc_wait_ld();
+      const float m_chunk = fmaxf(max32(v), max32(v2)) * sl2;
+      const float m_new = fmaxf(m_run, m_chunk);
+      const bool need = m_new > m_run + 8.0f;
+      if (__any_sync(0xffffffffu, need)) {
+        const float alpha = (m_new == NEG_INF) ? 1.0f : fast_exp2(m_run - m_new);
+        l_run *= alpha;
+        m_run = m_new;
+        if (ch > 0) {
+          // O holds the products up to chunk ch - 1; the last of them may still be in flight
+          const uint32_t pslot = (uint32_t)((ch - 1) & 1), pph = (uint32_t)(((ch - 1) >> 1) & 1);
+          ok = mbar_wait(bar_ve + 8u * pslot, pph, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
           uint32_t w32[32];
-          if (t > 0) {
 #pragma unroll 1
-            for (int c4 = 0; c4 < 4; ++c4) {
-              tmem_ld32(t_o + (uint32_t)c4 * 32u, w32);
-              tc_wait_ld();
-#pragma unroll
-              for (int q = 0; q < 32; ++q) w32[q] = __float_as_uint(__uint_as_float(w32[q]) * alpha);
-              tmem_st32(t_o + (uint32_t)c4 * 32u, w32);
-            }
-          }
-          if (c == 1) {        // P of the tile's first chunk was written against the old maximum
-            tmem_ld32(t_s, w32);
+          for (int c4 = 0; c4 < 4; ++c4) {
+            tmem_ld32(t_o + (uint32_t)c4 * 32u, w32);
             tc_wait_ld();
 #pragma unroll
-            for (int q = 0; q < 32; ++q) {
-              const float lo = __uint_as_float(w32[q] << 16) * alpha, hi = __uint_as_float(w32[q] & 0xffff0000u) * alpha;
-              w32[q] = pack_bf16x2(lo, hi);
-            }
-            tmem_st32(t_s, w32);
+            for (int q = 0; q < 32; ++q) w32[q] = __float_as_uint(__uint_as_float(w32[q]) * alpha);
+            tmem_st32(t_o + (uint32_t)c4 * 32u, w32);
           }
           tc_wait_st();
         }
-        const float m_use = (m_run == NEG_INF) ? 0.f : m_run;
-        exp_chunk(v, t_s + (uint32_t)c * 32u, m_use);
-        exp_chunk(v2, t_s + (uint32_t)c * 32u + 16u, m_use);
       }
+      const float m_use = (m_run == NEG_INF) ? 0.f : m_run;
+      exp_chunk(v, t_sc, m_use);
+      exp_chunk(v2, t_sc + 16u, m_use);
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_p);
+      mbar_arrive(bar_p + 8u * slot);
     }
 
     if (ok) ok = mbar_wait(bar_o, 0, abort_flag);
@@ -609,7 +593,7 @@ __global__ void rs_pack_vertical_kernel(AttnParams P, const __nv_bfloat16* K, co
 
 size_t attn_smem_bytes(int n) {
   const int list_cap = (n >> 6) + 64;
-  return 1024 + SmemLayout::end_tiles + ((list_cap * 2 + 15) & ~15) + 3 * 128 * 4 + 132 * 4 + 8 * 8 + 64;
+  return 1024 + SmemLayout::end_tiles + ((list_cap * 2 + 15) & ~15) + 3 * 128 * 4 + 132 * 4 + 14 * 8 + 64;
 }
 
 struct WsPlan { size_t cost, items, order, kpack, vpack, total; int n_work, kv_pad, n_items; };
