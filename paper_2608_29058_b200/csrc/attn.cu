@@ -369,29 +369,50 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     const int* vcols = P.idx.vs_cols + (size_t)vs_slot * P.idx.kv_cap;
     bool ok = true;
     uint32_t v[32], v2[32];
+    auto max3 = [](float a, float b, float c) -> float {
+      float d;
+      asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+      return d;
+    };
     auto max32 = [&](const uint32_t (&x)[32]) -> float {
-      float mx0 = NEG_INF, mx1 = NEG_INF, mx2 = NEG_INF, mx3 = NEG_INF;   // four independent chains
+      float mx0 = max3(__uint_as_float(x[0]), __uint_as_float(x[1]), __uint_as_float(x[2]));
+      float mx1 = max3(__uint_as_float(x[3]), __uint_as_float(x[4]), __uint_as_float(x[5]));
+      float mx2 = max3(__uint_as_float(x[6]), __uint_as_float(x[7]), __uint_as_float(x[8]));
+      float mx3 = max3(__uint_as_float(x[9]), __uint_as_float(x[10]), __uint_as_float(x[11]));
 #pragma unroll
-      for (int q = 0; q < 32; q += 4) {
-        mx0 = fmaxf(mx0, __uint_as_float(x[q]));
-        mx1 = fmaxf(mx1, __uint_as_float(x[q + 1]));
-        mx2 = fmaxf(mx2, __uint_as_float(x[q + 2]));
-        mx3 = fmaxf(mx3, __uint_as_float(x[q + 3]));
+      for (int q = 12; q < 28; q += 8) {
+        mx0 = max3(mx0, __uint_as_float(x[q]), __uint_as_float(x[q + 1]));
+        mx1 = max3(mx1, __uint_as_float(x[q + 2]), __uint_as_float(x[q + 3]));
+        mx2 = max3(mx2, __uint_as_float(x[q + 4]), __uint_as_float(x[q + 5]));
+        mx3 = max3(mx3, __uint_as_float(x[q + 6]), __uint_as_float(x[q + 7]));
       }
-      return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      mx0 = max3(mx0, __uint_as_float(x[28]), __uint_as_float(x[29]));
+      mx1 = max3(mx1, __uint_as_float(x[30]), __uint_as_float(x[31]));
+      return fmaxf(max3(mx0, mx1, mx2), mx3);
     };
     auto exp_chunk = [&](const uint32_t (&x)[32], uint32_t dst, float m_use) {
       uint32_t pk[16];
-      float acc0 = 0.f, acc1 = 0.f;
+      uint64_t acc = 0ull, acc_b = 0ull;     // two packed pairs of fp32 partial sums
+      uint64_t sl2x2, negm2;
+      asm("mov.b64 %0, {%1, %1};" : "=l"(sl2x2) : "f"(sl2));
+      asm("mov.b64 %0, {%1, %1};" : "=l"(negm2) : "f"(-m_use));
 #pragma unroll
       for (int q = 0; q < 16; ++q) {
-        const float p0 = fast_exp2(fmaf(__uint_as_float(x[2 * q]), sl2, -m_use));
-        const float p1 = fast_exp2(fmaf(__uint_as_float(x[2 * q + 1]), sl2, -m_use));
-        acc0 += p0;
-        acc1 += p1;
+        uint64_t s2, t2, p2;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(s2) : "r"(x[2 * q]), "r"(x[2 * q + 1]));
+        asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(t2) : "l"(s2), "l"(sl2x2), "l"(negm2));
+        float t0, t1;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(t0), "=f"(t1) : "l"(t2));
+        const float p0 = fast_exp2(t0), p1 = fast_exp2(t1);
+        asm("mov.b64 %0, {%1, %2};" : "=l"(p2) : "f"(p0), "f"(p1));
+        if (q & 1) { asm("add.rn.f32x2 %0, %1, %2;" : "=l"(acc_b) : "l"(acc_b), "l"(p2)); }
+        else       { asm("add.rn.f32x2 %0, %1, %2;" : "=l"(acc) : "l"(acc), "l"(p2)); }
         pk[q] = pack_bf16x2(p0, p1);
       }
-      l_run += acc0 + acc1;
+      asm("add.rn.f32x2 %0, %1, %2;" : "=l"(acc) : "l"(acc), "l"(acc_b));
+      float a0, a1;
+      asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(acc));
+      l_run += a0 + a1;
       tmem_st16(dst, pk);
     };
 
