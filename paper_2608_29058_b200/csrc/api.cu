@@ -57,6 +57,49 @@ int rs_check_device() {
   return cached[dev];
 }
 
+namespace {
+struct SideStream {
+  std::mutex mu;
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+SideStream g_side[64];
+thread_local int t_side_dev = -1;   // device whose side stream this thread holds between fork and join
+}  // namespace
+
+int rs_side_fork(cudaStream_t main, cudaStream_t* side) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return RS_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return RS_ERR_UNSUPPORTED_DEVICE;
+  SideStream& S = g_side[dev];
+  S.mu.lock();
+  if (S.stream == nullptr) {
+    if (cudaStreamCreateWithFlags(&S.stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&S.fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&S.join, cudaEventDisableTiming) != cudaSuccess) {
+      S.stream = nullptr;
+      S.mu.unlock();
+      return RS_ERR_CUDA;
+    }
+  }
+  if (cudaEventRecord(S.fork, main) != cudaSuccess || cudaStreamWaitEvent(S.stream, S.fork, 0) != cudaSuccess) {
+    S.mu.unlock();
+    return RS_ERR_CUDA;
+  }
+  t_side_dev = dev;
+  *side = S.stream;
+  return RS_OK;
+}
+
+int rs_side_join(cudaStream_t main) {
+  if (t_side_dev < 0) return RS_ERR_INVALID_ARG;
+  SideStream& S = g_side[t_side_dev];
+  t_side_dev = -1;
+  const bool ok = cudaEventRecord(S.join, S.stream) == cudaSuccess && cudaStreamWaitEvent(main, S.join, 0) == cudaSuccess;
+  S.mu.unlock();
+  return ok ? RS_OK : RS_ERR_CUDA;
+}
+
 typedef CUresult (*encode_fn_t)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);

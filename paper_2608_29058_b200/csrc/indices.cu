@@ -716,25 +716,38 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   if (stats != nullptr) {
     const long long warps = (long long)n_items * RS_PROBE_GROUPS * nb;
     rs_vblk_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, stream>>>(P);
-    rs_simple_stats_kernel<<<n_jobs, 256, 0, stream>>>(P);
+  }
+  // The vertical-slash chain (keys, select, D / coverage / pairs) and the block-sparse chain (pooled scores, row
+  // selection) do not read each other's results; both read the block sums above.  The second chain and the closed-form
+  // statistics run on the side stream.
+  const bool two_chains = any_vs && !skip_vs && (any_bs || stats != nullptr);
+  cudaStream_t side = stream;
+  if (two_chains) {
+    rc = rs_side_fork(stream, &side);
+    if (rc != RS_OK) return rc;
   }
   if (any_vs && !skip_vs) {
     rs_vs_keys_kernel<<<dim3((P.n + 255) / 256, 2 * n_items), 256, 0, stream>>>(P);
     rs_vs_select_kernel<<<dim3(2, n_jobs), kSelThreads, 0, stream>>>(P);
     rs_vs_finish_kernel<<<n_jobs, 256, 0, stream>>>(P);
   }
+  if (stats != nullptr) rs_simple_stats_kernel<<<n_jobs, 256, 0, side>>>(P);
   if (any_bs) {
     if ((choice == nullptr || stats != nullptr) && bscore == nullptr)
-      rs_bs_eval_scores_kernel<<<dim3((nb + 255) / 256, n_items), 256, 0, stream>>>(P);
+      rs_bs_eval_scores_kernel<<<dim3((nb + 255) / 256, n_items), 256, 0, side>>>(P);
     if (choice == nullptr || stats != nullptr)
-      rs_bs_eval_kernel<<<n_items, 256, (size_t)nb * sizeof(float), stream>>>(P);
+      rs_bs_eval_kernel<<<n_items, 256, (size_t)nb * sizeof(float), side>>>(P);
     if (choice != nullptr) {
       if (bscore == nullptr) {
         const int nt = (nb + 63) / 64;
-        rs_bs_scores_kernel<<<dim3(nt, nt, P.Hq), 256, 0, stream>>>(P);
+        rs_bs_scores_kernel<<<dim3(nt, nt, P.Hq), 256, 0, side>>>(P);
       }
-      rs_bs_rows_kernel<<<dim3(nb, P.Hq), 256, (size_t)nb * sizeof(float), stream>>>(P);
+      rs_bs_rows_kernel<<<dim3(nb, P.Hq), 256, (size_t)nb * sizeof(float), side>>>(P);
     }
+  }
+  if (two_chains) {
+    rc = rs_side_join(stream);
+    if (rc != RS_OK) return rc;
   }
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }

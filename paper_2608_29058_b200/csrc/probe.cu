@@ -476,18 +476,23 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
       return RS_ERR_CUDA;
     attr_set = true;
   }
+  // the pooled means and the value norms only read Q, K, V: they run beside the two probe passes
+  cudaStream_t side = nullptr;
+  rc = rs_side_fork(stream, &side);
+  if (rc != RS_OK) return rc;
+  const long long nb = p->n_keys / 64;
+  if (qpool) rs_pool_kernel<<<(unsigned)(P.Hq * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(Q), qpool, P.Hq * nb);
+  if (kpool) rs_pool_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(K), kpool, P.Hkv * nb);
+  if (vmax) {
+    float* blockmax = reinterpret_cast<float*>(wsb + w.blockmax);
+    rs_vnorm_block_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(V), blockmax, P.Hkv * nb);
+    rs_vmax_kernel<<<P.n_seg * P.Hkv, 256, 0, side>>>(P, blockmax, vmax);
+  }
   dim3 grid(w.n_splits, w.n_units);
   rs_probe_kernel<1><<<grid, kThreads, Smem::total, stream>>>(tmQ, tmK, P);
   rs_probe_merge_kernel<<<w.n_units, kRows, 0, stream>>>(P);
   rs_probe_kernel<2><<<grid, kThreads, Smem::total, stream>>>(tmQ, tmK, P);
-
-  const long long nb = p->n_keys / 64;
-  if (qpool) rs_pool_kernel<<<(unsigned)(P.Hq * nb), 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(Q), qpool, P.Hq * nb);
-  if (kpool) rs_pool_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(K), kpool, P.Hkv * nb);
-  if (vmax) {
-    float* blockmax = reinterpret_cast<float*>(wsb + w.blockmax);
-    rs_vnorm_block_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, stream>>>(reinterpret_cast<const __nv_bfloat16*>(V), blockmax, P.Hkv * nb);
-    rs_vmax_kernel<<<P.n_seg * P.Hkv, 256, 0, stream>>>(P, blockmax, vmax);
-  }
+  rc = rs_side_join(stream);
+  if (rc != RS_OK) return rc;
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }
