@@ -18,7 +18,8 @@ constexpr int kHC = 4;                 // head slots per CTA (4 x 64 = 256 probe
 constexpr int kRows = kHC * RS_PROBE_ROWS;
 constexpr int kKeyTile = 128;
 constexpr int kStages = 3;
-constexpr int kThreads = 320;          // warp 0 TMA, warp 1 MMA, warps 2..9 compute
+constexpr int kThreads1 = 320;         // pass 1: warp 0 TMA, warp 1 MMA, warps 2..9 compute
+constexpr int kThreads2 = 576;         // pass 2: warp 0 TMA, warp 1 MMA, warps 2..17 compute
 constexpr uint32_t kTmemCols = 512;
 
 struct ProbeParams {
@@ -37,7 +38,7 @@ struct ProbeParams {
 struct Smem {
   static constexpr uint32_t qp = 0;                       // 2 halves x 256 rows x 128 B
   static constexpr uint32_t k = 65536;                    // kStages x (2 halves x 128 rows x 128 B)
-  static constexpr uint32_t x = k + kStages * 32768;      // pass 2: [2 column halves][2 buffers][16][128] fp32
+  static constexpr uint32_t x = k + kStages * 32768;      // pass 2: [16 compute warps][16 rows][32 keys] fp32
   static constexpr uint32_t lse = x + 32768;              // 256 floats
   static constexpr uint32_t bars = lse + 1024;            // mbarriers
   static constexpr uint32_t misc = bars + 128;
@@ -49,7 +50,7 @@ __device__ __forceinline__ void named_bar_sync(int id, int count) {
 }
 
 template <int PASS>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(PASS == 1 ? kThreads1 : kThreads2, 1)
 rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ ProbeParams P) {
   extern __shared__ uint8_t smem_raw[];
@@ -57,6 +58,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (base - raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr int kThreads = PASS == 1 ? kThreads1 : kThreads2;
 
   // unit = (segment, kv head, head chunk); blockIdx.x = split of the key range
   const int unit = blockIdx.y;
@@ -85,7 +87,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (tid == 0) {
     mbar_init(bar_q, 1);
     for (int i = 0; i < kStages; ++i) { mbar_init(bar_full[i], 1); mbar_init(bar_empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull[i], 1); mbar_init(bar_tempty[i], 256); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull[i], 1); mbar_init(bar_tempty[i], kThreads - 64); }
     misc[1] = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
@@ -177,7 +179,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     // ------------------------------------------------------------------ compute warps
     const int cw = warp - 2;                 // 0..7
     const int quad = warp & 3;               // TMEM lane quadrant this warp may touch
-    const int part = cw >> 2;                // pass 1: head pair; pass 2: column half
+    const int part = cw >> 2;                // pass 1: head pair
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const float sl2 = P.scale_log2e;
     uint32_t v[32];
@@ -222,9 +224,61 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         P.partial[((size_t)unit * P.n_splits + blockIdx.x) * kRows + hh * 64 + (r & 63)] = make_float2(m_run, l_run);
       }
     } else {
+      // Sixteen warps: warp (quad, hh) owns 32 keys of the tile (its TMEM lanes) and the 64 probe rows of head slot hh.
+      // Per probe group: 16 probabilities per key, their sum is the column mass; the diagonal mass is a skewed sum
+      // over the warp's own 16 x 32 tile in shared memory (bin u = l - r + 15, offset o = obase - u).  Bins fed by
+      // this warp alone are stored, the 15 bins on either side also get an addend from the neighbouring 32 keys
+      // and are accumulated with atomics (two addends onto zero: the order does not change the sum).
+      const int hh = cw >> 2;                         // head slot
       const int l128 = quad * 32 + lane;              // key inside the tile
-      float* xs = reinterpret_cast<float*>(sm + Smem::x) + part * (2 * 16 * 128);
-      int iter = 0;
+      float* xw = reinterpret_cast<float*>(sm + Smem::x) + cw * (16 * 32);
+      const bool live = hh < n_heads;
+      // Row r of the warp's tile is read rotated by (lane + r + 17) mod 32: for r >= 15 - lane that is key
+      // lane - 15 + r (bin u = lane), otherwise key lane + 17 + r (bin u = lane + 32, lanes 0..14 only), so one
+      // conflict-free read per row serves both bins of a lane.
+      int rot[16];
+#pragma unroll
+      for (int r = 0; r < 16; ++r) rot[r] = r * 32 + ((lane + r + 17) & 31);
+      const int k_lo = 15 - lane;                     // rows r >= k_lo feed bin u = lane
+      auto group = [&](const uint32_t (&v16)[16], int grp, int j, int j0, bool masked) {
+        const int ig = i_first + grp * 16;            // first row of the group
+        const float4* l4 = reinterpret_cast<const float4*>(s_lse + hh * 64 + grp * 16);
+        float lse16[16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 t4 = l4[q];
+          lse16[4 * q] = t4.x; lse16[4 * q + 1] = t4.y; lse16[4 * q + 2] = t4.z; lse16[4 * q + 3] = t4.w;
+        }
+        float vsum = 0.f;
+        __syncwarp();                                 // the previous group's rotated reads are done
+#pragma unroll
+        for (int r = 0; r < 16; ++r) {
+          float p = fast_exp2(fmaf(__uint_as_float(v16[r]), sl2, -lse16[r]));
+          if (masked && j > ig + r) p = 0.f;
+          vsum += p;
+          xw[r * 32 + lane] = p;
+        }
+        const size_t out = (((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS + grp) * (size_t)P.n;
+        if (live && j < q1) P.vert[out + j] = vsum;
+        __syncwarp();
+        float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+        for (int r = 0; r < 16; ++r) {
+          const float x = xw[rot[r]];
+          if (r >= k_lo) acc0 += x; else acc1 += x;
+        }
+        // bin u <-> offset o = obase - u; bins 15..31 are fed by this warp's keys alone
+        const int obase = ig - (j0 + quad * 32) + 15;
+        if (live) {
+          const int o0 = obase - lane;
+          if (o0 >= 0) {
+            if (lane >= 15) P.slash[out + o0] = acc0;
+            else atomicAdd(&P.slash[out + o0], acc0);
+          }
+          const int o1 = o0 - 32;
+          if (lane < 15 && o1 >= 0) atomicAdd(&P.slash[out + o1], acc1);
+        }
+      };
       for (int t = t0; t < t1; ++t) {
         const int it = t - t0, b = it & 1;
         ok = mbar_wait(bar_tfull[b], (uint32_t)(it >> 1) & 1u, abort_flag);
@@ -232,63 +286,14 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tc_fence_after();
         const int j0 = t * kKeyTile;
         const int j = j0 + l128;
-        const bool need_mask = j0 + kKeyTile - 1 > i_first;
+        const bool need_mask = j0 + kKeyTile - 1 > i_first;   // only the tiles that reach the probe rows
 #pragma unroll 1
-        for (int q = 0; q < 8; ++q, ++iter) {         // (head slot, probe group) pairs of this column half
-          const int hh = part * 2 + (q >> 2), grp = q & 3;
-          float* xb = xs + (iter & 1) * (16 * 128);
+        for (int grp = 0; grp < RS_PROBE_GROUPS; ++grp) {
           uint32_t v16[16];
-          {
-            uint32_t* d = v16;
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-                "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-                : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]), "=r"(d[4]), "=r"(d[5]), "=r"(d[6]), "=r"(d[7]),
-                  "=r"(d[8]), "=r"(d[9]), "=r"(d[10]), "=r"(d[11]), "=r"(d[12]), "=r"(d[13]), "=r"(d[14]), "=r"(d[15])
-                : "r"(tmem + lane_addr + (uint32_t)(b * 256 + hh * 64 + grp * 16))
-                : "memory");
-          }
+          tmem_ld16(tmem + lane_addr + (uint32_t)(b * 256 + hh * 64 + grp * 16), v16);
           tc_wait_ld();
-          const int ig = i_first + grp * 16;          // first row of the group
-          float vsum = 0.f;
-#pragma unroll
-          for (int r = 0; r < 16; ++r) {
-            float p = fast_exp2(fmaf(__uint_as_float(v16[r]), sl2, -s_lse[hh * 64 + grp * 16 + r]));
-            if (need_mask && j > ig + r) p = 0.f;
-            vsum += p;
-            xb[r * 128 + l128] = p;
-          }
-          const bool live = hh < n_heads;
-          const size_t out = (((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS + grp) * (size_t)P.n;
-          if (live && j < q1) P.vert[out + j] = vsum;
-          named_bar_sync(1 + part, 128);
-          // skewed sums: u = l - r + 15 in [0, 142]; offset o = (ig - j0 + 15) - u
-          const int obase = ig - j0 + 15;
-          {
-            const int u = l128;
-            float acc = 0.f;
-#pragma unroll
-            for (int r = 0; r < 16; ++r) {
-              const int l = u - 15 + r;
-              if (l >= 0) acc += xb[r * 128 + l];
-            }
-            const int o = obase - u;
-            if (live && o >= 0) {
-              if (u >= 15) P.slash[out + o] = acc;      // all 16 rows of the group inside this tile
-              else atomicAdd(&P.slash[out + o], acc);   // shared with the neighbouring tile (two addends)
-            }
-          }
-          if (l128 < 15) {
-            const int u = 128 + l128;
-            float acc = 0.f;
-#pragma unroll
-            for (int r = 0; r < 16; ++r) {
-              const int l = u - 15 + r;
-              if (l < 128) acc += xb[r * 128 + l];
-            }
-            const int o = obase - u;
-            if (live && o >= 0) atomicAdd(&P.slash[out + o], acc);
-          }
+          if (need_mask) group(v16, grp, j, j0, true);
+          else group(v16, grp, j, j0, false);
         }
         tc_fence_before();
         mbar_arrive(bar_tempty[b]);
@@ -476,22 +481,24 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
       return RS_ERR_CUDA;
     attr_set = true;
   }
-  // the pooled means and the value norms only read Q, K, V: they run beside the two probe passes
+  // The pooled means and the value norms only read Q, K, V: they run beside the two probe passes, on the side
+  // stream.  Pass 1 is enqueued first so that its CTAs (one per SM, most of the shared memory) are resident before
+  // the small streaming CTAs fill what is left; the other way round the streaming kernels would run alone.
   cudaStream_t side = nullptr;
   rc = rs_side_fork(stream, &side);
   if (rc != RS_OK) return rc;
+  dim3 grid(w.n_splits, w.n_units);
+  rs_probe_kernel<1><<<grid, kThreads1, Smem::total, stream>>>(tmQ, tmK, P);
   const long long nb = p->n_keys / 64;
-  if (qpool) rs_pool_kernel<<<(unsigned)(P.Hq * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(Q), qpool, P.Hq * nb);
   if (kpool) rs_pool_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(K), kpool, P.Hkv * nb);
   if (vmax) {
     float* blockmax = reinterpret_cast<float*>(wsb + w.blockmax);
     rs_vnorm_block_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(V), blockmax, P.Hkv * nb);
     rs_vmax_kernel<<<P.n_seg * P.Hkv, 256, 0, side>>>(P, blockmax, vmax);
   }
-  dim3 grid(w.n_splits, w.n_units);
-  rs_probe_kernel<1><<<grid, kThreads, Smem::total, stream>>>(tmQ, tmK, P);
+  if (qpool) rs_pool_kernel<<<(unsigned)(P.Hq * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(Q), qpool, P.Hq * nb);
   rs_probe_merge_kernel<<<w.n_units, kRows, 0, stream>>>(P);
-  rs_probe_kernel<2><<<grid, kThreads, Smem::total, stream>>>(tmQ, tmK, P);
+  rs_probe_kernel<2><<<grid, kThreads2, Smem::total, stream>>>(tmQ, tmK, P);
   rc = rs_side_join(stream);
   if (rc != RS_OK) return rc;
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
