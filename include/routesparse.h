@@ -204,6 +204,29 @@ int rs_certificate(int n_q_heads, int n_kv_heads, int n_keys, const float* lse_s
                    float* m_row, float* cert_row, float* cert_tight, float* m_head, float* cert_head,
                    int32_t* status, void* stream);
 
+/* Shared attention probe of Eq. 3 (Section 3.2) in its general form: r sampled query rows per (segment, head) against
+ * keys pooled over blocks of width g, S = Q[I] pool_g(K)^T / sqrt(d), soft-maxed over the visible key blocks, and the
+ * three descriptors of Section 3.2.  The paper leaves open what this library fixes as follows: a key block is visible
+ * to row i when its first key is <= i and is pooled (arithmetic mean) over its visible keys only; the agreement
+ * descriptor is 1 - total-variation distance between the mean signatures of the first two row subsets, the signature
+ * of a row being its mass re-binned into [key block 0] + [relative block offsets 0..15] + [everything else].
+ *   rows        device int32[n_seg][r], row ids inside the segment (r <= 64); the caller chooses the mixture of
+ *               recent, uniformly spaced and boundary-adjacent positions
+ *   g           pooling width, a divisor of 64
+ *   sub_bounds  HOST int32[n_sub + 1], 0 = b_0 < ... < b_n_sub = r: the row subsets (n_sub <= 4)
+ *   A           device fp32 [n_seg][n_q_heads][r][n_keys / g] out: probabilities (0 on invisible blocks)
+ *   lse         device fp32 [n_seg][n_q_heads][r] out
+ *   colmass     device fp32 [n_seg][n_q_heads][n_sub][n_keys / g] out: sum over the subset's rows of A[i][kb]
+ *   diagmass    same shape, indexed by relative block offset: sum over the subset's rows of A[i][i / g - delta]
+ *   descr       device fp32 [n_seg][n_q_heads][4] out: entropy (mean of H_i / log max(2, visible_i)), local-band
+ *               mass (blocks whose first key lies within 1024 of the row), agreement, mean number of visible blocks
+ *   scratch     device fp32, rs_probe_pooled_scratch_floats() elements
+ * Query heads per KV head must be <= 4.  Errors as for the other calls; nothing is allocated. */
+int rs_probe_pooled_scratch_floats(const rs_problem* p, int r, size_t* n_floats);
+int rs_probe_pooled(const rs_problem* p, const void* Q, const void* K, const int32_t* rows, int r, int g,
+                    const int32_t* sub_bounds, int n_sub, float* A, float* lse, float* colmass, float* diagmass,
+                    float* descr, float* scratch, int32_t* status, void* stream);
+
 /* Self test of the bounded device-side wait every kernel of this library uses (no passage of the paper: the waits
  * exist because the kernels synchronise TMA, tensor-core and softmax roles through mbarriers).  Launches one small
  * kernel that waits on a barrier nothing arrives on, with a limit of poll_limit (1 .. 2^20) polls; the wait gives up,

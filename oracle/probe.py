@@ -77,3 +77,108 @@ def value_norms(V: np.ndarray, q1: int):
     """vnorm[j] = ||v_j||_2 for j < q1 and their maximum V_max (Eq. 5), float32."""
     vn = np.sqrt((V[:q1] * V[:q1]).sum(axis=1))
     return vn.astype(np.float32), np.float32(vn.max())
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Eq. 3 in its general form: r sampled query rows (a deterministic mixture of recent, uniformly spaced and
+# boundary-adjacent positions) against keys pooled over blocks of width g, and the three descriptors of
+# Section 3.2 (entropy, local-band concentration, agreement between the recent and the uniform group).
+# The paper fixes neither the proportions of the mixture, nor how a key block that straddles the causal
+# boundary is pooled, nor the formula of the agreement; the choices below are this build's reading:
+#   * rows: the last r_recent rows of the segment, r_boundary rows right after the segment start, and r_uniform
+#     rows spread evenly (midpoints of equal strata) over what lies between;
+#   * a key block is visible to row i when its first key is <= i, and it is pooled (arithmetic mean) over its
+#     visible keys only, so no future key enters a logit;
+#   * agreement = 1 - total-variation distance between the two groups' mean "signatures", the signature of a row
+#     being its mass re-binned into [key block 0] + [relative block offsets 0..15] + [everything else]
+#     (position-independent, so rows at different depths can be compared).
+SIG_LOCAL = 16
+
+
+def mixture_rows(q0: int, q1: int, r_recent: int = 32, r_uniform: int = 16, r_boundary: int = 16) -> np.ndarray:
+    """Row ids of the mixture, in the order recent, uniform, boundary (each ascending); all distinct."""
+    span = (q1 - q0) - r_recent - r_boundary
+    if span < r_uniform:
+        raise ValueError("segment too short for this mixture")
+    recent = np.arange(q1 - r_recent, q1)
+    uniform = q0 + r_boundary + ((2 * np.arange(r_uniform) + 1) * span) // (2 * r_uniform)
+    boundary = np.arange(q0, q0 + r_boundary)
+    return np.concatenate([recent, uniform, boundary]).astype(np.int64)
+
+
+@dataclass
+class PooledProbeResult:
+    A: np.ndarray          # [r, nbg] float64 softmax rows over pooled key blocks (0 on invisible blocks)
+    lse: np.ndarray        # [r] float64
+    colmass: np.ndarray    # [n_sub, nbg] sum over the subset's rows of A[i, kb]
+    diagmass: np.ndarray   # [n_sub, nbg] sum over the subset's rows of A[i, i // g - delta], indexed by delta
+    entropy: float         # mean over rows of H_i / log(max(2, visible_i)), in [0, 1]
+    local_conc: float      # mean over rows of the mass of blocks whose first key is within 1024 of the row
+    agreement: float       # 1 - TV(signature of subset 0, signature of subset 1); 1.0 with fewer than two subsets
+
+
+def pooled_logits(Q: np.ndarray, K: np.ndarray, rows: np.ndarray, g: int, q1: int) -> np.ndarray:
+    """S[t, kb] = q_i . mean(K[kb*g .. min(kb*g+g-1, i)]) / sqrt(d) for visible blocks, -inf otherwise."""
+    d = Q.shape[1]
+    nbg = q1 // g
+    S = np.full((len(rows), nbg), -np.inf, dtype=np.float64)
+    Kf = K[:q1].astype(np.float64)
+    full = Kf.reshape(nbg, g, d).mean(axis=1)
+    for t, i in enumerate(rows):
+        q = Q[i].astype(np.float64)
+        kb_d = i // g
+        S[t, :kb_d] = full[:kb_d] @ q
+        S[t, kb_d] = Kf[kb_d * g:i + 1].mean(axis=0) @ q
+    return S * (1.0 / np.sqrt(float(d)))
+
+
+def row_signature(a: np.ndarray, i: int, g: int) -> np.ndarray:
+    """Mass of one probe row re-binned into [block 0] + [relative offsets 0..15] + [rest] (18 bins)."""
+    sig = np.zeros(SIG_LOCAL + 2, dtype=np.float64)
+    kb_d = i // g
+    for kb in range(kb_d + 1):
+        delta = kb_d - kb
+        if delta < SIG_LOCAL:
+            sig[1 + delta] += a[kb]
+        elif kb == 0:
+            sig[0] += a[kb]
+        else:
+            sig[SIG_LOCAL + 1] += a[kb]
+    return sig
+
+
+def pooled_probe(Q: np.ndarray, K: np.ndarray, rows: np.ndarray, g: int, q1: int, sub_bounds) -> PooledProbeResult:
+    rows = np.asarray(rows, dtype=np.int64)
+    S = pooled_logits(Q, K, rows, g, q1)
+    mx = S.max(axis=1, keepdims=True)
+    lse = mx[:, 0] + np.log(np.exp(S - mx).sum(axis=1))
+    A = np.exp(S - lse[:, None])
+    nbg = q1 // g
+    n_sub = len(sub_bounds) - 1
+    col = np.zeros((n_sub, nbg), dtype=np.float64)
+    diag = np.zeros((n_sub, nbg), dtype=np.float64)
+    sig = np.zeros((n_sub, SIG_LOCAL + 2), dtype=np.float64)
+    ent, loc = 0.0, 0.0
+    for s in range(n_sub):
+        for t in range(sub_bounds[s], sub_bounds[s + 1]):
+            i = int(rows[t])
+            kb_d = i // g
+            col[s] += A[t]
+            diag[s, :kb_d + 1] += A[t, kb_d::-1]
+            sig[s] += row_signature(A[t], i, g)
+    for t, i in enumerate(rows):
+        vis = int(i) // g + 1
+        a = A[t, :vis]
+        with np.errstate(divide="ignore", invalid="ignore"):
+            h = -np.where(a > 0, a * np.log(a), 0.0).sum()
+        ent += h / np.log(max(2, vis))
+        first = np.arange(vis) * g
+        loc += a[int(i) - first < LOCAL_BAND].sum()
+    r = len(rows)
+    agreement = 1.0
+    if n_sub >= 2:
+        s0 = sig[0] / max(1, sub_bounds[1] - sub_bounds[0])
+        s1 = sig[1] / max(1, sub_bounds[2] - sub_bounds[1])
+        agreement = 1.0 - 0.5 * float(np.abs(s0 - s1).sum())
+    return PooledProbeResult(A=A, lse=lse, colmass=col, diagmass=diag, entropy=ent / r, local_conc=loc / r,
+                             agreement=agreement)

@@ -46,7 +46,8 @@ class rs_route_params(C.Structure):
 
 
 EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "rs_build_indices", "rs_route",
-           "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate", "rs_selftest_wait_timeout"]
+           "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate",
+           "rs_selftest_wait_timeout", "rs_probe_pooled", "rs_probe_pooled_scratch_floats"]
 
 
 def lib_path() -> str:
@@ -220,6 +221,34 @@ def rs_certificate(n_q_heads: int, n_kv_heads: int, n_keys: int, lse_sel, lse_fu
                                  _stream()), "rs_certificate")
 
 
+def rs_probe_pooled_scratch_floats(p: Problem, r: int) -> int:
+    out = C.c_size_t(0)
+    _check(load().rs_probe_pooled_scratch_floats(C.byref(p.c), int(r), C.byref(out)), "rs_probe_pooled_scratch_floats")
+    return int(out.value)
+
+
+def mixture_rows(q0: int, q1: int, r_recent: int = 32, r_uniform: int = 16, r_boundary: int = 16):
+    """Row ids of the probe's query mixture (Section 3.2) for the segment [q0, q1), in the order recent, uniform,
+    boundary: the last r_recent rows, r_uniform rows at the midpoints of equal strata of what lies between the two
+    other groups, and the r_boundary rows right after the segment start.  Plain index arithmetic on the host."""
+    span = (q1 - q0) - r_recent - r_boundary
+    if span < r_uniform:
+        raise ValueError("segment too short for this mixture")
+    rows = list(range(q1 - r_recent, q1))
+    rows += [q0 + r_boundary + ((2 * k + 1) * span) // (2 * r_uniform) for k in range(r_uniform)]
+    rows += list(range(q0, q0 + r_boundary))
+    return rows
+
+
+def rs_probe_pooled(p: Problem, Q, K, rows, g: int, sub_bounds, A, lse, colmass, diagmass, descr, scratch, status):
+    """rows: device int32 [n_seg][r]; sub_bounds: host list of n_sub + 1 ints."""
+    r = int(rows.shape[-1])
+    sb = (C.c_int32 * len(sub_bounds))(*[int(x) for x in sub_bounds])
+    _check(load().rs_probe_pooled(C.byref(p.c), _ptr(Q), _ptr(K), _ptr(rows), r, int(g), sb, len(sub_bounds) - 1,
+                                  _ptr(A), _ptr(lse), _ptr(colmass), _ptr(diagmass), _ptr(descr), _ptr(scratch),
+                                  _ptr(status), _stream()), "rs_probe_pooled")
+
+
 def rs_selftest_wait_timeout(status, poll_limit: int = 2000):
     _check(load().rs_selftest_wait_timeout(_ptr(status), C.c_uint(poll_limit), _stream()), "rs_selftest_wait_timeout")
 
@@ -233,4 +262,5 @@ def check_status(status: torch.Tensor, what: str = "kernel"):
 
 __all__ = [n for n in dir() if n.startswith(("rs_", "RS_")) or n in
            ("Problem", "IndexSet", "make_library", "new_status", "new_workspace", "check_status", "load", "lib_path",
+            "mixture_rows",
             "RouteSparseError", "EXPORTS")]

@@ -148,6 +148,33 @@ class RoutedPrefillLayer:
                           self.vmax[p.n_segments - 1], self.onorm, self.cfg.delta_q, self.m_row, self.cert_row, None,
                           self.m_head, self.cert_head, self.status)
 
+    # ------------------------------------------------------------------ Eq. 3 in its general form + descriptors
+    def pooled_probe(self, Q, K, g: int = 64, mixture=(32, 16, 16)):
+        """Mixture-of-rows probe against keys pooled over width g (Eq. 3) and the three descriptors of Section 3.2.
+        Returns the descriptor tensor [n_seg][Hq][4] (entropy, local-band mass, agreement between the recent and the
+        uniform rows, mean number of visible blocks); probabilities and block masses stay in self.pp."""
+        p = self.p
+        key = (g, tuple(mixture))
+        if getattr(self, "_pp_key", None) != key:
+            dev = self.O.device
+            r = sum(mixture)
+            f32 = dict(dtype=torch.float32, device=dev)
+            rows = [rs.mixture_rows(p.seg_bounds[s], p.seg_bounds[s + 1], *mixture) for s in range(p.n_segments)]
+            nbg = p.n_keys // g
+            self.pp = dict(rows=torch.tensor(rows, dtype=torch.int32, device=dev),
+                           sub=[0, mixture[0], mixture[0] + mixture[1], r],
+                           A=torch.empty((p.n_segments, p.n_q_heads, r, nbg), **f32),
+                           lse=torch.empty((p.n_segments, p.n_q_heads, r), **f32),
+                           col=torch.empty((p.n_segments, p.n_q_heads, 3, nbg), **f32),
+                           diag=torch.empty((p.n_segments, p.n_q_heads, 3, nbg), **f32),
+                           descr=torch.empty((p.n_segments, p.n_q_heads, 4), **f32),
+                           scratch=torch.empty(rs.rs_probe_pooled_scratch_floats(p, r), **f32))
+            self._pp_key = key
+        pp = self.pp
+        rs.rs_probe_pooled(p, Q, K, pp["rows"], g, pp["sub"], pp["A"], pp["lse"], pp["col"], pp["diag"], pp["descr"],
+                           pp["scratch"], self.status)
+        return pp["descr"]
+
     # ------------------------------------------------------------------ offline calibration (Section 3.5)
     def profile_costs(self, Q, K, V, reps: int = 3):
         """Hardware profiling of the pattern library (Section 3.1, 3.5): every candidate runs as the route of all

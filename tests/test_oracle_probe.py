@@ -67,3 +67,92 @@ def test_descriptors_on_known_distributions():
     rows = np.arange(2048 - 64, 2048)
     assert abs(pr.entropy - np.log(rows + 1).mean()) < 1e-9
     assert abs(pr.local_conc - (1024 / (rows + 1)).mean()) < 1e-9
+
+
+# ------------------------------------------------------------------ Eq. 3 in its general form (mixture rows, pooled keys)
+def test_mixture_rows_are_distinct_ordered_and_inside_the_segment():
+    for q0, q1 in ((0, 4096), (1024, 3072), (320, 384), (0, 64)):
+        rows = P.mixture_rows(q0, q1)
+        assert len(rows) == 64 and len(set(rows.tolist())) == 64
+        assert rows.min() >= q0 and rows.max() == q1 - 1
+        assert np.array_equal(rows[:32], np.arange(q1 - 32, q1))          # recent
+        assert np.array_equal(rows[48:], np.arange(q0, q0 + 16))          # boundary-adjacent
+        assert np.all(np.diff(rows[32:48]) > 0) and rows[32] >= q0 + 16 and rows[47] < q1 - 32
+    # strata midpoints: the uniform rows of a long segment are evenly spaced
+    rows = P.mixture_rows(0, 4096 + 48)
+    assert set(np.diff(rows[32:48]).tolist()) == {256}
+
+
+def test_pooled_probe_with_width_one_is_the_exact_probe():
+    Q, K, _ = _head(seed=9, n=384)
+    for q1 in (384, 256):
+        pp = P.pooled_probe(Q, K, np.arange(q1 - 64, q1), 1, q1, [0, 16, 32, 48, 64])
+        pr = P.probe_rows(Q, K, q1)
+        assert np.allclose(pp.A, pr.P, atol=1e-12)
+        assert np.allclose(pp.colmass, pr.vert, atol=1e-6) and np.allclose(pp.diagmass, pr.slash, atol=1e-6)
+        assert np.allclose(pp.lse, pr.lse, atol=1e-5)
+        assert abs(pp.local_conc - pr.local_conc) < 1e-9
+
+
+def test_pooled_logit_is_the_mean_of_the_visible_per_key_logits():
+    Q, K, _ = _head(seed=10, n=256)
+    rows = np.array([255, 130, 77, 8, 3])
+    g = 8
+    S = P.pooled_logits(Q, K, rows, g, 256)
+    for t, i in enumerate(rows):
+        per_key = (K[:i + 1] @ Q[i]) / np.sqrt(128.0)                     # brute force, key by key
+        for kb in range(256 // g):
+            vis = per_key[kb * g:min(kb * g + g, i + 1)]
+            if len(vis) == 0:
+                assert S[t, kb] == -np.inf
+            else:
+                assert abs(S[t, kb] - vis.mean()) < 1e-10
+
+
+def test_pooled_probe_on_identical_keys_is_uniform():
+    rng = np.random.default_rng(5)
+    n, g = 512, 16
+    Q = rng.standard_normal((n, 128))
+    K = np.tile(rng.standard_normal((1, 128)), (n, 1))
+    rows = P.mixture_rows(0, n)
+    pp = P.pooled_probe(Q, K, rows, g, n, [0, 32, 48, 64])
+    for t, i in enumerate(rows):
+        vis = i // g + 1
+        assert np.allclose(pp.A[t, :vis], 1.0 / vis, atol=1e-12) and np.all(pp.A[t, vis:] == 0)
+    # normalised entropy of a uniform row is 1 when it sees at least two blocks, 0 when it sees one
+    want = np.mean([1.0 if i // g + 1 >= 2 else 0.0 for i in rows])
+    assert abs(pp.entropy - want) < 1e-12
+    # local-band mass of a uniform row = share of its visible blocks whose first key lies within 1024 of the row
+    local = [sum(1 for kb in range(i // g + 1) if i - kb * g < 1024) / (i // g + 1) for i in rows]
+    assert abs(pp.local_conc - np.mean(local)) < 1e-12
+
+
+def test_pooled_probe_invariants():
+    Q, K, _ = _head(seed=11, n=1024)
+    rows = P.mixture_rows(0, 1024)
+    for g in (8, 64):
+        pp = P.pooled_probe(Q, K, rows, g, 1024, [0, 32, 48, 64])
+        assert np.allclose(pp.A.sum(axis=1), 1.0, atol=1e-12)
+        assert np.allclose(pp.colmass.sum(axis=1), [32, 16, 16]) and np.allclose(pp.diagmass.sum(axis=1), [32, 16, 16])
+        assert 0.0 <= pp.entropy <= 1.0 and 0.0 <= pp.local_conc <= 1.0 + 1e-12 and 0.0 <= pp.agreement <= 1.0
+        for t, i in enumerate(rows[:4]):
+            assert abs(P.row_signature(pp.A[t], int(i), g).sum() - 1.0) < 1e-12
+    # two subsets made of the same rows agree completely
+    same = np.concatenate([rows[:16], rows[:16]])
+    pp = P.pooled_probe(Q, K, same, 8, 1024, [0, 16, 32])
+    assert abs(pp.agreement - 1.0) < 1e-12
+    # a local head (recent and uniform rows both attend to their own neighbourhood) agrees more than a head whose
+    # recent rows look at the neighbourhood and whose earlier rows look at key block 0
+    n, g = 1024, 8
+    Kl = np.zeros((n, 128)); Ql = np.zeros((n, 128))
+    for j in range(n):
+        Kl[j, j % 128] = 30.0
+        Ql[j, j % 128] = 30.0                                             # row i likes keys j = i mod 128: a slash pattern
+    a_local = P.pooled_probe(Ql, Kl, rows, g, n, [0, 32, 48, 64]).agreement
+    Qm = Ql.copy()
+    Qm[:n - 32] = 0.0
+    Qm[:n - 32, 0] = 30.0                                                 # earlier rows like dim 0 = keys 0, 128, ...
+    Km = Kl.copy()
+    Km[1:, 0] = 0.0                                                       # ... of which only key 0 is left
+    a_mixed = P.pooled_probe(Qm, Km, rows, g, n, [0, 32, 48, 64]).agreement
+    assert a_local > a_mixed + 0.2
