@@ -96,7 +96,7 @@ typedef enum { RS_CERT_ABS = 0, RS_CERT_REL = 1 } rs_cert_mode;
 typedef struct {
   int64_t budget;          /* T_l of Eq. 8, same integer unit as cost */
   int64_t t_probe;         /* t_probe of Eq. 8 */
-  double alpha;            /* weight of u in Eq. 4 (beta = 0: training-free router) */
+  double alpha;            /* weight of u in Eq. 4 */
   double delta_q;          /* m_low = max(0, m_hat - delta_q) */
   double cert_max;         /* fallback fires while certificate > cert_max */
   int32_t use_cert;        /* 0: no fallback step */
@@ -106,6 +106,9 @@ typedef struct {
                               of any family whose certificate passes before giving up and going dense */
   const int32_t* forced_dense;  /* device int32[n_items], non-zero = force dense last; may be NULL */
   const int32_t* fixed_choice;  /* device int32[n_items]; when set, bypasses solve and fallback; may be NULL */
+  const double* e;         /* device double[n_items][n_cand]: calibrated error predictor e of Eq. 4 (rs_regressor_eval);
+                              NULL or beta == 0: the training-free router */
+  double beta;             /* weight of e in Eq. 4 */
 } rs_route_params;
 
 typedef struct { int64_t total_cost; double total_risk; int32_t n_fallback; int32_t feasible; } rs_route_report;
@@ -226,6 +229,25 @@ int rs_probe_pooled_scratch_floats(const rs_problem* p, int r, size_t* n_floats)
 int rs_probe_pooled(const rs_problem* p, const void* Q, const void* K, const int32_t* rows, int r, int g,
                     const int32_t* sub_bounds, int n_sub, float* A, float* lse, float* colmass, float* diagmass,
                     float* descr, float* scratch, int32_t* status, void* stream);
+
+/* Calibrated predictor e of Eq. 4 (Section 3.3: "a small monotone regressor fitted offline from dense calibration
+ * runs; it consumes only the probe descriptors and candidate metadata").  The form used here, this library's choice:
+ *   z(item, c) = w0 (1 - m_hat) + w1 u + w2 entropy + w3 (1 - local) + w4 (1 - agreement) + w5 (1 - pairs / dense pairs)
+ *   e(item, c) = table value of the last breakpoint z_k <= z (0 below the first; a non-decreasing step function),
+ * with w >= 0 and a non-decreasing table, so e is monotone in every feature.  Dense candidates get e = 0.
+ * All arithmetic is IEEE double, one rounding per operation, in the order written above.
+ *   stats  device rs_cand_stats[n_items][n_cand] (rs_build_indices);  descr  device fp32 [n_items][4] (rs_probe_pooled)
+ *   w      HOST double[6];  bp_z, bp_e  HOST double[n_bp] (n_bp <= 64, bp_z ascending)
+ *   e_out  device double[n_items][n_cand] */
+int rs_regressor_eval(const rs_problem* p, const rs_candidate* lib, int n_cand, const rs_cand_stats* stats,
+                      const float* descr, const double* w, const double* bp_z, const double* bp_e, int n_bp,
+                      double* e_out, int32_t* status, void* stream);
+
+/* Dense audit of Section 3.5: row-wise output error between two attention outputs of the same shape,
+ *   err[i] = || Oa_i - Ob_i ||_2,  norm_a[i] = || Oa_i ||_2   (fp32 accumulation over the 128 dimensions)
+ * Oa, Ob: [n_rows][128] bf16 (o_dtype 0) or fp32 (o_dtype 1); err, norm_a (may be NULL): device fp32[n_rows]. */
+int rs_output_error(long long n_rows, const void* Oa, const void* Ob, int o_dtype, float* err, float* norm_a,
+                    int32_t* status, void* stream);
 
 /* Self test of the bounded device-side wait every kernel of this library uses (no passage of the paper: the waits
  * exist because the kernels synchronise TMA, tensor-core and softmax roles through mbarriers).  Launches one small

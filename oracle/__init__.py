@@ -17,5 +17,12 @@ Parts and what pins them (tests/test_oracle_*.py):
                                                                   as a lower bound.  The exact substitution order is this
                                                                   build's reading: "parity unpinned".
   certificate.certificate        Eq. 5.                           Pinned: equality case, L1 identity, bound on every row.
+  probe.pooled_probe             Eq. 3, general form + descriptors. Pinned: width 1 == exact probe, per-key brute force,
+                                                                  identical keys -> uniform rows.  The mixture, the pooling
+                                                                  of a straddling block and the agreement formula are this
+                                                                  build's reading: beyond those "parity unpinned".
+  calibration.*                  Section 3.5, predictor e of Eq. 4. Pinned: isotonic fit == scikit-learn's, quantile by
+                                                                  counting, monotonicity.  The feature set is this build's
+                                                                  reading: "parity unpinned".
 """
-from . import attention, certificate, patterns, probe, routing  # noqa: F401
+from . import attention, calibration, certificate, patterns, probe, routing  # noqa: F401

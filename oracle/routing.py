@@ -33,7 +33,9 @@ CERT_ABS, CERT_REL = 0, 1
 class RouteParams:
     budget: int                      # T_l, same integer unit as cost
     t_probe: int = 0
-    alpha: float = 1.0               # weight of the probe-subset disagreement u (beta = 0: training-free router)
+    alpha: float = 1.0               # weight of the probe-subset disagreement u
+    beta: float = 0.0                # weight of the calibrated error predictor e (0: training-free router)
+    e: Optional[np.ndarray] = None   # [items, n_cand] float64 predictor values (calibration.regressor_eval)
     delta_q: float = 0.0             # one-sided residual quantile: m_low = max(0, m_hat - delta_q)
     cert_max: Optional[float] = None  # fallback fires while certificate > cert_max (None: no fallback)
     cert_mode: int = CERT_REL        # REL: 2(1 - m_low);  ABS: 2(1 - m_low) * vmax
@@ -51,8 +53,8 @@ class RouteReport:
     feasible: int
 
 
-def risks(lib: List[Candidate], cov_fx: np.ndarray, alpha: float):
-    """R[item][c] = (1 - m_hat) + alpha * u (Eq. 4 with beta = 0); dense has m_hat = 1, u = 0, R = 0."""
+def risks(lib: List[Candidate], cov_fx: np.ndarray, alpha: float, beta: float = 0.0, e: Optional[np.ndarray] = None):
+    """R[item][c] = (1 - m_hat) + alpha * u + beta * e (Eq. 4); dense has m_hat = 1, u = 0, e = 0, R = 0."""
     n_items, n_cand = cov_fx.shape[0], len(lib)
     R = np.zeros((n_items, n_cand), dtype=np.float64)
     M = np.ones((n_items, n_cand), dtype=np.float64)
@@ -63,6 +65,8 @@ def risks(lib: List[Candidate], cov_fx: np.ndarray, alpha: float):
             m_hat, u = m_hat_from_fx(cov_fx[it, c])
             M[it, c] = m_hat
             R[it, c] = (1.0 - m_hat) + alpha * u
+            if e is not None and beta != 0.0:
+                R[it, c] = R[it, c] + beta * float(e[it, c])
     return R, M
 
 
@@ -112,7 +116,7 @@ def route(lib: List[Candidate], cov_fx: np.ndarray, cost: np.ndarray, vmax: np.n
     """Full routing of one layer. cov_fx[items, n_cand, 4] uint64, cost[items, n_cand] int64, vmax[items] fp32."""
     n_items = cov_fx.shape[0]
     dense_c = _dense_index(lib)
-    R, M = risks(lib, cov_fx, p.alpha)
+    R, M = risks(lib, cov_fx, p.alpha, p.beta, p.e)
     n_fallback = 0
     if p.fixed_choice is not None:
         choice = [int(c) for c in p.fixed_choice]

@@ -42,12 +42,13 @@ class rs_route_params(C.Structure):
     _fields_ = [("budget", C.c_int64), ("t_probe", C.c_int64), ("alpha", C.c_double), ("delta_q", C.c_double),
                 ("cert_max", C.c_double), ("use_cert", C.c_int32), ("cert_mode", C.c_int32),
                 ("expand_first", C.c_int32), ("reserved", C.c_int32),
-                ("forced_dense", C.c_void_p), ("fixed_choice", C.c_void_p)]
+                ("forced_dense", C.c_void_p), ("fixed_choice", C.c_void_p), ("e", C.c_void_p), ("beta", C.c_double)]
 
 
 EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "rs_build_indices", "rs_route",
            "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate",
-           "rs_selftest_wait_timeout", "rs_probe_pooled", "rs_probe_pooled_scratch_floats"]
+           "rs_selftest_wait_timeout", "rs_probe_pooled", "rs_probe_pooled_scratch_floats", "rs_regressor_eval",
+           "rs_output_error"]
 
 
 def lib_path() -> str:
@@ -247,6 +248,23 @@ def rs_probe_pooled(p: Problem, Q, K, rows, g: int, sub_bounds, A, lse, colmass,
     _check(load().rs_probe_pooled(C.byref(p.c), _ptr(Q), _ptr(K), _ptr(rows), r, int(g), sb, len(sub_bounds) - 1,
                                   _ptr(A), _ptr(lse), _ptr(colmass), _ptr(diagmass), _ptr(descr), _ptr(scratch),
                                   _ptr(status), _stream()), "rs_probe_pooled")
+
+
+def rs_regressor_eval(p: Problem, lib, stats, descr, w, bp_z, bp_e, e_out, status):
+    """w: 6 host floats; bp_z / bp_e: host lists (breakpoints of the step function); e_out: device float64."""
+    wd = (C.c_double * 6)(*[float(x) for x in w])
+    n_bp = len(bp_z)
+    bz = (C.c_double * max(1, n_bp))(*[float(x) for x in bp_z])
+    be = (C.c_double * max(1, n_bp))(*[float(x) for x in bp_e])
+    _check(load().rs_regressor_eval(C.byref(p.c), lib, len(lib), _ptr(stats), _ptr(descr), wd, bz, be, n_bp,
+                                    _ptr(e_out), _ptr(status), _stream()), "rs_regressor_eval")
+
+
+def rs_output_error(Oa, Ob, err, norm_a, status):
+    n_rows = Oa.numel() // 128
+    o_dtype = 1 if Oa.dtype == torch.float32 else 0
+    _check(load().rs_output_error(C.c_longlong(n_rows), _ptr(Oa), _ptr(Ob), o_dtype, _ptr(err), _ptr(norm_a),
+                                  _ptr(status), _stream()), "rs_output_error")
 
 
 def rs_selftest_wait_timeout(status, poll_limit: int = 2000):

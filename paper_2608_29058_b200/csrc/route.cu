@@ -70,7 +70,9 @@ __device__ __forceinline__ double risk_of(const RouteArgs& A, int item, int c) {
     mn = fmin(mn, mg);
   }
   const double u = __dsub_rn(mx, mn);
-  return __dadd_rn(__dsub_rn(1.0, m_hat_of(A, item, c)), __dmul_rn(A.prm.alpha, u));
+  double r = __dadd_rn(__dsub_rn(1.0, m_hat_of(A, item, c)), __dmul_rn(A.prm.alpha, u));
+  if (A.prm.e != nullptr && A.prm.beta != 0.0) r = __dadd_rn(r, __dmul_rn(A.prm.beta, A.prm.e[(size_t)item * A.n_cand + c]));
+  return r;
 }
 
 __global__ void __launch_bounds__(kThreads)

@@ -41,6 +41,9 @@ def gpu_route(p, lib, cov, pairs, cost, vmax, **kw):
     if kw.get("forced_dense"):
         fd = torch.zeros(cov.shape[0], dtype=torch.int32, device="cuda"); fd[list(kw["forced_dense"])] = 1
         prm.forced_dense = fd.data_ptr(); keep.append(fd)
+    if kw.get("e") is not None:
+        et = torch.from_numpy(np.ascontiguousarray(kw["e"], dtype=np.float64)).cuda()
+        prm.e = et.data_ptr(); prm.beta = float(kw.get("beta", 0.0)); keep.append(et)
     if kw.get("fixed_choice") is not None:
         fc = torch.tensor(kw["fixed_choice"], dtype=torch.int32, device="cuda")
         prm.fixed_choice = fc.data_ptr(); keep.append(fc)
@@ -94,3 +97,57 @@ def test_fixed_choice_and_ties():
     assert got.tolist() == [1, 0, 1, 0] and rep[3] == 1
     got, rep = gpu_route(p, lib, cov, pairs, None, np.ones((1, 2), np.float32), budget=1)
     assert got.tolist() == [0, 0, 0, 0] and rep[3] == 0
+
+
+def test_route_with_the_calibrated_predictor_is_bit_exact():
+    """Eq. 4 with beta > 0: e comes from rs_regressor_eval (checked bit for bit against the oracle's predictor) and
+    enters the risk; decisions and the reported risk are those of the oracle."""
+    from oracle import calibration as CAL
+    rng = np.random.default_rng(77)
+    n_seg, Hq, Hkv = 2, 8, 2
+    p = rs.Problem(Hq, Hkv, 1024, [0, 384, 1024])
+    n_items = n_seg * Hq
+    cov, pairs = instance(rng, n_items, LIB)
+    for it in range(n_items):                     # pair counts below the segment's dense count, as real statistics are
+        q0, q1 = p.seg_bounds[it // Hq], p.seg_bounds[it // Hq + 1]
+        dense = (q1 * (q1 + 1) - q0 * (q0 + 1)) // 2
+        pairs[it] = rng.integers(dense // 50, dense, len(LIB)); pairs[it, -1] = dense
+    descr = rng.uniform(0, 1, (n_items, 4)).astype(np.float32)
+    w = [1.0, 0.5, 0.25, 0.125, 0.3, 0.07]
+    bp_z = np.array([0.05, 0.3, 0.55, 0.9, 1.4]); bp_e = np.array([0.0, 0.02, 0.1, 0.1, 0.6])
+    stats = np.zeros((n_items, len(LIB), 5), dtype=np.int64)
+    stats[:, :, :4] = cov.astype(np.int64); stats[:, :, 4] = pairs
+    e_dev = torch.full((n_items, len(LIB)), -1.0, dtype=torch.float64, device="cuda")
+    rs.rs_regressor_eval(p, c_library(LIB), torch.from_numpy(stats).cuda(), torch.from_numpy(descr).cuda(), w, bp_z, bp_e,
+                         e_dev, rs.new_status())
+    seg_of = [(p.seg_bounds[it // Hq], p.seg_bounds[it // Hq + 1]) for it in range(n_items)]
+    e_want = CAL.regressor_eval(LIB, cov, pairs, descr, seg_of, w, bp_z, bp_e)
+    assert np.array_equal(e_dev.cpu().numpy(), e_want)
+    assert len(np.unique(e_want)) >= 3            # the instance exercises several steps of the table
+    cost = 512 * pairs
+    vmax_sg = rng.uniform(1, 4, (n_seg, Hkv)).astype(np.float32)
+    vmax_item = np.array([vmax_sg[it // Hq, (it % Hq) // (Hq // Hkv)] for it in range(n_items)], np.float32)
+    for beta, budget_frac in ((0.0, 0.2), (1.0, 0.2), (4.0, 0.1), (0.5, 0.5)):
+        kw = dict(budget=int(cost[:, -1].sum() * budget_frac), t_probe=1000, alpha=1.0, cert_max=0.4, e=e_want, beta=beta)
+        got, rep = gpu_route(p, LIB, cov, pairs, cost, vmax_sg, **kw)
+        want, wrep = RT.route(LIB, cov, cost, vmax_item, RT.RouteParams(budget=kw["budget"], t_probe=1000, alpha=1.0,
+                                                                         cert_max=0.4, beta=beta, e=e_want))
+        assert np.array_equal(got, want), beta
+        assert rep[0] == wrep.total_cost and rep[1] == wrep.total_risk and rep[2] == wrep.n_fallback
+    # the predictor changes decisions on this instance
+    a, _ = gpu_route(p, LIB, cov, pairs, cost, vmax_sg, budget=int(cost[:, -1].sum() * 0.2), alpha=1.0)
+    b, _ = gpu_route(p, LIB, cov, pairs, cost, vmax_sg, budget=int(cost[:, -1].sum() * 0.2), alpha=1.0, e=e_want, beta=4.0)
+    assert not np.array_equal(a, b)
+
+
+def test_output_error_rows():
+    rng = np.random.default_rng(3)
+    a = torch.from_numpy(rng.standard_normal((3, 70, 128)).astype(np.float32)).cuda()
+    b = a + torch.from_numpy((0.01 * rng.standard_normal((3, 70, 128))).astype(np.float32)).cuda()
+    for dt in (torch.float32, torch.bfloat16):
+        x, y = a.to(dt), b.to(dt)
+        err = torch.zeros(210, device="cuda"); nrm = torch.zeros(210, device="cuda")
+        rs.rs_output_error(x, y, err, nrm, rs.new_status())
+        xd, yd = x.double().cpu().numpy().reshape(210, 128), y.double().cpu().numpy().reshape(210, 128)
+        assert np.allclose(err.cpu().numpy(), np.sqrt(((xd - yd) ** 2).sum(axis=1)), rtol=1e-5, atol=1e-7)
+        assert np.allclose(nrm.cpu().numpy(), np.sqrt((xd ** 2).sum(axis=1)), rtol=1e-5)
