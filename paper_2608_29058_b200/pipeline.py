@@ -44,6 +44,7 @@ class RouteConfig:
     cert_mode: int = rs.RS_CERT_REL
     expand_first: bool = True
     rescue_any: bool = False           # before dense, the cheapest sparse candidate of any family that passes
+    beta: float = 0.0                  # weight of the calibrated predictor e of Eq. 4 (needs use_calibration())
 
 
 class _IdxView:
@@ -101,6 +102,8 @@ class RoutedPrefillLayer:
         self.prm = rs.rs_route_params()
         self._forced = None
         self.events = None
+        self.regressor = None       # dict(w, bp_z, bp_e, g) from calibrate(); used when cfg.beta > 0
+        self.e_risk = torch.zeros((p.n_items, len(self.cands)), dtype=torch.float64, device=device)
         self.cost_table = None      # int64 [n_items, n_cand] measured kernel time (ns); None: FLOPs of the selected pairs
         self.cost_budget = None     # layer budget in the table's unit
         self.cost_t_probe = 0
@@ -126,6 +129,9 @@ class RoutedPrefillLayer:
         prm.cert_max = 0.0 if c.cert_max is None else c.cert_max
         prm.cert_mode, prm.expand_first = c.cert_mode, int(c.expand_first)
         prm.reserved = int(c.rescue_any)
+        use_e = self.regressor is not None and c.beta > 0.0
+        prm.e = self.e_risk.data_ptr() if use_e else None
+        prm.beta = float(c.beta) if use_e else 0.0
         self._forced = forced_dense
         prm.forced_dense = None if forced_dense is None else forced_dense.data_ptr()
         prm.fixed_choice = None
@@ -179,7 +185,7 @@ class RoutedPrefillLayer:
     def profile_costs(self, Q, K, V, reps: int = 3):
         """Hardware profiling of the pattern library (Section 3.1, 3.5): every candidate runs as the route of all
         heads and its attention launch is timed (median of `reps`, CUDA events).  The measured time of a candidate is
-        split over the items in proportion to their pair counts and stored as the int64 nanosecond cost table the
+        (the maximum is reported as its tail latency) is split over the items in proportion to their pair counts and stored as the int64 nanosecond cost table the
         router reads; the layer budget becomes budget_frac x the dense candidate's measured time and t_probe the
         measured probe + evaluation time.  Synchronises; meant to run once per (library, length), outside the hot path."""
         import numpy as np
@@ -193,7 +199,7 @@ class RoutedPrefillLayer:
         torch.cuda.synchronize()
         t_probe_ns = a.elapsed_time(b) * 1e6
         pairs = self.stats.cpu().numpy()[:, :, 4].astype(np.float64)
-        ms = np.zeros(n_cand)
+        ms, tail = np.zeros(n_cand), np.zeros(n_cand)     # median and tail (maximum of the repetitions)
         saved = self.choice.clone()
         for c in range(n_cand):
             self.choice.fill_(c)
@@ -206,16 +212,32 @@ class RoutedPrefillLayer:
                 torch.cuda.synchronize()
                 ts.append(a.elapsed_time(b))
             ms[c] = float(np.median(ts))
+            tail[c] = float(np.max(ts))
         self.choice.copy_(saved)
         table = np.maximum(1, np.rint(ms[None, :] * 1e6 * pairs / pairs.sum(axis=0, keepdims=True))).astype(np.int64)
         dense_c = [i for i, c in enumerate(self.cands) if c[0] == rs.RS_DENSE][0]
         self.cost_table = torch.from_numpy(table).to(self.O.device)
         self.cost_budget = int(self.cfg.budget_frac * ms[dense_c] * 1e6)
         self.cost_t_probe = int(t_probe_ns)
-        return {"candidate_ms": ms.tolist(), "t_probe_ms": t_probe_ns * 1e-6, "budget_ms": self.cost_budget * 1e-6}
+        return {"candidate_ms": ms.tolist(), "candidate_ms_tail": tail.tolist(), "t_probe_ms": t_probe_ns * 1e-6,
+                "budget_ms": self.cost_budget * 1e-6}
 
     def use_flop_costs(self):
         self.cost_table = None
+
+    def use_calibration(self, calib: dict, beta: Optional[float] = None):
+        """Installs the result of calibrate(): the one-sided residual quantile delta_q and the predictor e of Eq. 4."""
+        self.cfg.delta_q = float(calib["delta_q"])
+        self.regressor = dict(calib["regressor"])
+        if beta is not None:
+            self.cfg.beta = float(beta)
+
+    def predict_error(self, Q, K):
+        """Descriptors (pooled mixture probe) and the predictor e for every (item, candidate); needs evaluate_candidates()."""
+        r = self.regressor
+        descr = self.pooled_probe(Q, K, g=int(r["g"]))
+        rs.rs_regressor_eval(self.p, self.lib, self.stats, descr, r["w"], r["bp_z"], r["bp_e"], self.e_risk, self.status)
+        return self.e_risk
 
     # ------------------------------------------------------------------ whole layer
     def forward(self, Q, K, V, fixed_choice: Optional[torch.Tensor] = None,
@@ -228,6 +250,8 @@ class RoutedPrefillLayer:
         mark(1)
         if fixed_choice is None:
             self.evaluate_candidates()
+            if self.regressor is not None and self.cfg.beta > 0.0:
+                self.predict_error(Q, K)
             mark(2)
             self.route(forced_dense)
         else:
