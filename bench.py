@@ -219,6 +219,11 @@ def main():
     ap.add_argument("--cost", default="flops", choices=["flops", "measured"],
                     help="router cost table: FLOPs of the selected pairs, or kernel times profiled before the timed region")
     ap.add_argument("--rescue", action="store_true", help="fallback variant: cheapest passing sparse candidate of any family before dense")
+    ap.add_argument("--calibration", type=str, default=None,
+                    help="JSON written by `python -m paper_2608_29058_b200.calibrate`: installs delta_q and the predictor e")
+    ap.add_argument("--beta", type=float, default=0.0, help="weight of the calibrated predictor e in Eq. 4 (needs --calibration)")
+    ap.add_argument("--launch-ablation", action="store_true",
+                    help="also time the attention stage as one launch per KV group and as one launch per head")
     ap.add_argument("--sweep", action="store_true", help="config-5 sweep: n x budget x forced-dense cells, JSONL output")
     ap.add_argument("--n", type=int, default=None, help="override the sequence length (smaller profiling case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -259,6 +264,13 @@ def main():
     Q, K, V = to_dev(L["Q"]), to_dev(L["K"]), to_dev(L["V"])
     p = rs.Problem(spec.n_q_heads, spec.n_kv_heads, spec.n, [int(x) for x in L["seg_bounds"]])
     layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(rescue_any=args.rescue, **route_kw), device=dev)
+    risk_calibration = None
+    if args.calibration:
+        with open(args.calibration) as f:
+            calib = json.loads(f.read())
+        layer.use_calibration(calib, beta=args.beta)
+        risk_calibration = {"file": os.path.basename(args.calibration), "delta_q": calib["delta_q"], "beta": args.beta,
+                            "q": calib.get("q"), "calibrated_at_n": calib.get("n")}
     fixed_t = None
     if fixed:
         fixed_t = torch.from_numpy(fixed_choice_for(layer.cands, spec.n_q_heads)).to(dev)
@@ -348,6 +360,27 @@ def main():
         dense_ms = d0.elapsed_time(d1) / reps
         del O_d, lse_d
 
+    # ---- launch ablation (Section 3.4 / Table 3: grouping heads into one launch against per-group / per-head launches)
+    launch_ablation = None
+    if args.launch_ablation and p.n_segments == 1:
+        def timed(fn, reps=3):
+            fn()
+            torch.cuda.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record()
+            for _ in range(reps):
+                fn()
+            a1.record()
+            torch.cuda.synchronize()
+            return a0.elapsed_time(a1) / reps
+        group = p.n_q_heads // p.n_kv_heads
+        launch_ablation = {
+            "single_launch_ms": timed(lambda: layer.attention(Q, K, V)),
+            "per_kv_group_ms": timed(lambda: layer.attention_split(Q, K, V, group)),
+            "per_head_ms": timed(lambda: layer.attention_split(Q, K, V, 1)),
+            "launches": {"single": 1, "per_kv_group": p.n_kv_heads, "per_head": p.n_q_heads},
+            "note": "attention stage only, same routes and index arrays; every launch also runs its own work-list kernels"}
+
     # ---- end to end through the public call with pinned host buffers
     e2e = None
     if not args.no_e2e:
@@ -414,7 +447,8 @@ def main():
         "flops": {"selected_pairs": f_mask, "issued_tiles": f_tile, "dense": f_dense,
                   "selected_fraction_of_dense": f_mask / f_dense},
         "routes": hist, "route_report": layer.route_report() if not fixed else None,
-        "cost_model": args.cost, "calibration": calibration, "fallback_rescue": bool(args.rescue),
+        "cost_model": args.cost, "calibration": calibration, "risk_calibration": risk_calibration, "launch_ablation": launch_ablation,
+        "fallback_rescue": bool(args.rescue),
         "roofline": {"kernel": "rs_attn_kernel (one launch, all heads)", "bound": "tensor", "achieved": achieved,
                      "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": f"bf16_tflops_sustained, {peaks['source']}",

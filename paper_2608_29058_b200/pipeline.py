@@ -148,6 +148,38 @@ class RoutedPrefillLayer:
         rs.rs_sparse_prefill_attn(self.p, Q, K, V, self.lib, idx, self.choice, self.O, self.lse_sel, self.onorm,
                                   self.counters, self.ws, self.status)
 
+    def attention_split(self, Q, K, V, heads_per_launch: int):
+        """The same attention work as attention(), issued as one launch per group of `heads_per_launch` consecutive
+        query heads (a KV group, or a single head) instead of one launch for all heads: the launch-fragmentation
+        ablation of Section 3.4 / Table 3.  Single-segment problems only; every launch is the ordinary
+        rs_sparse_prefill_attn call on slices of the layer's tensors and index arrays."""
+        p = self.p
+        assert p.n_segments == 1, "attention_split covers single-segment problems"
+        Hq, Hkv, n = p.n_q_heads, p.n_kv_heads, p.n_keys
+        group = Hq // Hkv
+        assert heads_per_launch in (1, group) or heads_per_launch % group == 0
+        nb, n_cand = n // 64, len(self.cands)
+        full = self._idx_hybrid if self._reuse_eval else self.idx.c
+        eval_layout = self._reuse_eval
+        if not hasattr(self, "_sub_problems"):
+            self._sub_problems = {}
+        for h0 in range(0, Hq, heads_per_launch):
+            hn = heads_per_launch
+            kv0, kvn = h0 // group, max(1, hn // group)
+            key = (hn, kvn)
+            if key not in self._sub_problems:
+                self._sub_problems[key] = rs.Problem(hn, kvn, n)
+            sp = self._sub_problems[key]
+            slot0 = h0 * n_cand if eval_layout else h0           # first vertical-slash slot of the slice
+            n_slots = hn * n_cand if eval_layout else hn
+            sub = rs.rs_index_set(n_slots, full.kv_cap, full.ks_cap, full.nd_cap, hn * nb, full.kb_cap,
+                                  full.vs_cols + 4 * slot0 * full.kv_cap, full.vs_offs + 4 * slot0 * full.ks_cap,
+                                  full.vs_diag + 4 * slot0 * full.nd_cap, full.vs_count + 16 * slot0,
+                                  full.bs_blk + 4 * h0 * nb * full.kb_cap, full.bs_count + 4 * h0 * nb)
+            rs.rs_sparse_prefill_attn(sp, Q[h0:h0 + hn], K[kv0:kv0 + kvn], V[kv0:kv0 + kvn], self.lib, _IdxView(sub),
+                                      self.choice[h0:h0 + hn], self.O[h0:h0 + hn], self.lse_sel[h0:h0 + hn],
+                                      self.onorm[h0:h0 + hn], self.counters, self.ws, self.status)
+
     def certificate(self):
         p = self.p
         rs.rs_certificate(p.n_q_heads, p.n_kv_heads, p.n_keys, self.lse_sel, self.lse_probe, self.probe_rows,

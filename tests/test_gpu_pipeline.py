@@ -153,3 +153,27 @@ def test_profiled_cost_table_routes_like_the_oracle():
     want, _ = RT.route(cands, stats[:, :, :4].astype(np.uint64), table, np.array([vmax[0, h // 2] for h in range(4)], np.float32),
                        RT.RouteParams(budget=layer.cost_budget, t_probe=layer.cost_t_probe, cert_max=0.9))
     assert np.array_equal(layer.choice.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("online", [True, False])
+def test_split_launches_give_the_single_launch_result(online):
+    """Launch ablation: one launch per KV group / per head computes exactly what the single launch computes."""
+    n, Hq, Hkv = 1152, 8, 2
+    L = make_layer(tiny_spec(91, n, Hq, Hkv))
+    Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+    p = rs.Problem(Hq, Hkv, n)
+    lib = [(rs.RS_A_SHAPE, 64, 128), (rs.RS_VERTICAL_SLASH, 48, 160), (rs.RS_VERTICAL_SLASH, 96, 320),
+           (rs.RS_BLOCK_SPARSE, 4, 0), (rs.RS_DENSE, 0, 0)]
+    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(budget_frac=0.5, cert_max=None))
+    if online:
+        layer.forward(Q, K, V)
+    else:                                              # every pattern present, index arrays in the materialised layout
+        fixed = torch.tensor([0, 1, 2, 3, 4, 3, 2, 1], dtype=torch.int32, device="cuda")
+        layer.forward(Q, K, V, fixed_choice=fixed)
+    rs.check_status(layer.status, "single launch")
+    want_O, want_lse = layer.O.clone(), layer.lse_sel.clone()
+    for heads in (Hq // Hkv, 1):
+        layer.O.zero_(); layer.lse_sel.zero_()
+        layer.attention_split(Q, K, V, heads)
+        rs.check_status(layer.status, "split launches")
+        assert torch.equal(layer.O, want_O) and torch.equal(layer.lse_sel, want_lse), heads
