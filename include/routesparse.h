@@ -109,6 +109,9 @@ typedef struct {
   const double* e;         /* device double[n_items][n_cand]: calibrated error predictor e of Eq. 4 (rs_regressor_eval);
                               NULL or beta == 0: the training-free router */
   double beta;             /* weight of e in Eq. 4 */
+  int32_t backfill;        /* 1: after the greedy solve, spend what is left of the budget on the substitutions with
+                              the largest risk decrease per unit of added cost that still fit (before the fallback) */
+  int32_t reserved2;       /* 0 */
 } rs_route_params;
 
 typedef struct { int64_t total_cost; double total_risk; int32_t n_fallback; int32_t feasible; } rs_route_report;

@@ -41,6 +41,7 @@ class RouteParams:
     cert_mode: int = CERT_REL        # REL: 2(1 - m_low);  ABS: 2(1 - m_low) * vmax
     expand_first: bool = True        # try the next larger budget of the family before dense
     rescue_any: bool = False         # before dense, take the cheapest sparse candidate of any family that passes
+    backfill: bool = False           # spend leftover budget on the best risk decrease per added cost (before fallback)
     forced_dense: Sequence[int] = field(default_factory=list)   # items forced to dense last
     fixed_choice: Optional[Sequence[int]] = None                 # bypasses the solve and the fallback
 
@@ -104,6 +105,32 @@ def greedy_solve(R: np.ndarray, cost: np.ndarray, dense_c: int, budget: int, t_p
     return choice, total, feasible
 
 
+def backfill(choice: List[int], total: int, R: np.ndarray, cost: np.ndarray, budget: int):
+    """Greedy back-fill: while some substitution to a more expensive, less risky candidate still fits the budget, apply
+    the one with the largest risk decrease per unit of added cost (ties: cheaper, lower item, lower candidate).
+    The paper does not describe this pass; it is this build's extension of the greedy heuristic."""
+    n_items, n_cand = R.shape
+    while True:
+        best = None
+        for it in range(n_items):
+            cur = choice[it]
+            for k in range(n_cand):
+                dT = int(cost[it, k]) - int(cost[it, cur])
+                if dT <= 0 or total + dT > budget:
+                    continue
+                dR = float(R[it, k]) - float(R[it, cur])
+                if not dR < 0.0:
+                    continue
+                key = (dR / float(dT), dT, it, k)
+                if best is None or key < best:
+                    best = key
+        if best is None:
+            return choice, total
+        _, dT, it, k = best
+        choice[it] = k
+        total += dT
+
+
 def _next_larger(lib: List[Candidate], c: int) -> Optional[int]:
     """Index of the next entry of the same family after c (library lists a family by increasing budget)."""
     for k in range(c + 1, len(lib)):
@@ -122,7 +149,9 @@ def route(lib: List[Candidate], cov_fx: np.ndarray, cost: np.ndarray, vmax: np.n
         choice = [int(c) for c in p.fixed_choice]
         feasible = 1
     else:
-        choice, _, feasible = greedy_solve(R, cost, dense_c, int(p.budget), int(p.t_probe))
+        choice, total, feasible = greedy_solve(R, cost, dense_c, int(p.budget), int(p.t_probe))
+        if p.backfill and feasible:
+            choice, total = backfill(choice, total, R, cost, int(p.budget))
         if p.cert_max is not None:
             for it in range(n_items):
                 fired = False

@@ -163,6 +163,42 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
         if (lane == 0) ibest[best.item] = mine;
         __syncwarp();
       }
+      // ---- back-fill: what is left of the budget goes to the substitutions with the largest risk decrease per unit
+      // of added cost that still fit (ties: cheaper, lower item, lower candidate)
+      if (A.prm.backfill != 0 && total <= A.prm.budget) {
+        for (int step = 0; step < max_steps; ++step) {
+          const long long slack = A.prm.budget - total;
+          Sub best; best.ratio = 0.0; best.dT = 0; best.item = -1; best.k = -1;
+          auto better_up = [](const Sub& a, const Sub& b) -> bool {
+            if (a.k < 0) return false;
+            if (b.k < 0) return true;
+            if (a.ratio != b.ratio) return a.ratio < b.ratio;
+            if (a.dT != b.dT) return a.dT < b.dT;
+            if (a.item != b.item) return a.item < b.item;
+            return a.k < b.k;
+          };
+          for (int it = lane; it < A.n_items; it += 32) {
+            const int cur = ch[it];
+            for (int k = 0; k < A.n_cand; ++k) {
+              const long long dT = costf(it, k) - costf(it, cur);
+              if (dT <= 0 || dT > slack) continue;
+              const double dR = __dsub_rn(riskf(it, k), riskf(it, cur));
+              if (!(dR < 0.0)) continue;
+              Sub s2; s2.ratio = __ddiv_rn(dR, (double)dT); s2.dT = dT; s2.item = it; s2.k = k;
+              if (better_up(s2, best)) best = s2;
+            }
+          }
+#pragma unroll
+          for (int off = 16; off >= 1; off >>= 1) {
+            const Sub o = shfl_sub(best, off);
+            if (better_up(o, best)) best = o;
+          }
+          if (best.k < 0) break;
+          if (lane == 0) ch[best.item] = best.k;
+          total += best.dT;
+          __syncwarp();
+        }
+      }
       if (lane == 0) sh_total = total;
     }
     __syncthreads();

@@ -45,6 +45,7 @@ class RouteConfig:
     expand_first: bool = True
     rescue_any: bool = False           # before dense, the cheapest sparse candidate of any family that passes
     beta: float = 0.0                  # weight of the calibrated predictor e of Eq. 4 (needs use_calibration())
+    backfill: bool = False             # spend leftover budget on the best risk decrease per added cost
 
 
 class _IdxView:
@@ -129,6 +130,7 @@ class RoutedPrefillLayer:
         prm.cert_max = 0.0 if c.cert_max is None else c.cert_max
         prm.cert_mode, prm.expand_first = c.cert_mode, int(c.expand_first)
         prm.reserved = int(c.rescue_any)
+        prm.backfill = int(c.backfill)
         use_e = self.regressor is not None and c.beta > 0.0
         prm.e = self.e_risk.data_ptr() if use_e else None
         prm.beta = float(c.beta) if use_e else 0.0

@@ -37,6 +37,7 @@ def gpu_route(p, lib, cov, pairs, cost, vmax, **kw):
     prm.cert_max = 0.0 if kw.get("cert_max") is None else kw["cert_max"]
     prm.cert_mode = kw.get("cert_mode", rs.RS_CERT_REL); prm.expand_first = int(kw.get("expand_first", True))
     prm.reserved = int(kw.get("rescue_any", False))
+    prm.backfill = int(kw.get("backfill", False))
     keep = []
     if kw.get("forced_dense"):
         fd = torch.zeros(cov.shape[0], dtype=torch.int32, device="cuda"); fd[list(kw["forced_dense"])] = 1
@@ -151,3 +152,27 @@ def test_output_error_rows():
         xd, yd = x.double().cpu().numpy().reshape(210, 128), y.double().cpu().numpy().reshape(210, 128)
         assert np.allclose(err.cpu().numpy(), np.sqrt(((xd - yd) ** 2).sum(axis=1)), rtol=1e-5, atol=1e-7)
         assert np.allclose(nrm.cpu().numpy(), np.sqrt((xd ** 2).sum(axis=1)), rtol=1e-5)
+
+
+def test_backfill_is_bit_exact_and_never_worse():
+    rng = np.random.default_rng(5)
+    p = rs.Problem(32, 8, 512)
+    improved = 0
+    for trial in range(6):
+        cov, pairs = instance(rng, 32, LIB)
+        cost = 512 * pairs
+        vmax_sg = np.ones((1, 8), dtype=np.float32)
+        budget = int(cost[:, -1].sum() * [0.1, 0.2, 0.3, 0.5, 0.05, 0.15][trial])
+        base, brep = gpu_route(p, LIB, cov, pairs, cost, vmax_sg, budget=budget, alpha=1.0)
+        got, rep = gpu_route(p, LIB, cov, pairs, cost, vmax_sg, budget=budget, alpha=1.0, backfill=True)
+        want, wrep = RT.route(LIB, cov, cost, np.ones(32, np.float32), RT.RouteParams(budget=budget, backfill=True))
+        assert np.array_equal(got, want) and rep[0] == wrep.total_cost and rep[1] == wrep.total_risk
+        assert rep[0] <= budget and rep[1] <= brep[1] and rep[0] >= brep[0]
+        improved += int(rep[1] < brep[1])
+        # nothing that fits is left
+        R, _ = RT.risks(LIB, cov, 1.0)
+        for it in range(32):
+            for k in range(len(LIB)):
+                dT = int(cost[it, k]) - int(cost[it, got[it]])
+                assert not (dT > 0 and rep[0] + dT <= budget and R[it, k] < R[it, got[it]])
+    assert improved >= 1

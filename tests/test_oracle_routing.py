@@ -125,3 +125,32 @@ def test_rescue_takes_the_cheapest_passing_candidate_of_any_family():
     assert RT.route(LIB, cov, cost, np.float32([1.0]), rescued)[0].tolist() == [3]     # block-sparse is cheaper than VS
     cov[0, 2:4] = np.uint64(int(0.9 * 16 * 2 ** 32))
     assert RT.route(LIB, cov, cost, np.float32([1.0]), rescued)[0].tolist() == [DENSE_C]
+
+
+def test_backfill_uses_leftover_budget_without_exceeding_it():
+    from oracle.routing import RouteParams, backfill, greedy_solve, risks, route
+    rng = np.random.default_rng(12)
+    lib = PT.default_library()
+    for trial in range(5):
+        n_items = 6
+        cov = np.zeros((n_items, len(lib), 4), dtype=np.uint64)
+        cost = np.zeros((n_items, len(lib)), dtype=np.int64)
+        for it in range(n_items):
+            for c, cand in enumerate(lib):
+                base = rng.uniform(0.3, 1.0) if cand.pattern != PT.DENSE else 1.0
+                cov[it, c] = np.full(4, int(base * 16 * 2 ** 32), dtype=np.uint64)
+                cost[it, c] = rng.integers(100, 5000) if cand.pattern != PT.DENSE else 10000
+        budget = int(cost[:, -1].sum() * 0.3)
+        R, _ = risks(lib, cov, 1.0)
+        ch, total, feas = greedy_solve(R, cost, len(lib) - 1, budget, 0)
+        r0 = sum(R[i, ch[i]] for i in range(n_items))
+        ch2, total2 = backfill(list(ch), total, R, cost, budget)
+        r1 = sum(R[i, ch2[i]] for i in range(n_items))
+        assert total2 <= budget and total2 >= total and r1 <= r0
+        assert total2 == sum(int(cost[i, ch2[i]]) for i in range(n_items))
+        for i in range(n_items):                                   # nothing that fits and lowers the risk is left
+            for k in range(len(lib)):
+                dT = int(cost[i, k]) - int(cost[i, ch2[i]])
+                assert not (dT > 0 and total2 + dT <= budget and R[i, k] < R[i, ch2[i]])
+        got, rep = route(lib, cov, cost, np.ones(n_items, np.float32), RouteParams(budget=budget, backfill=True))
+        assert list(got) == ch2 and rep.total_cost == total2
