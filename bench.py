@@ -224,6 +224,8 @@ def main():
     ap.add_argument("--beta", type=float, default=0.0, help="weight of the calibrated predictor e in Eq. 4 (needs --calibration)")
     ap.add_argument("--launch-ablation", action="store_true",
                     help="also time the attention stage as one launch per KV group and as one launch per head")
+    ap.add_argument("--ablations", action="store_true",
+                    help="router ablations of the paper's Table 3 on the config-3 layer, JSONL output")
     ap.add_argument("--sweep", action="store_true", help="config-5 sweep: n x budget x forced-dense cells, JSONL output")
     ap.add_argument("--n", type=int, default=None, help="override the sequence length (smaller profiling case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -233,6 +235,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.sweep:
         return sweep(args)
+    if args.ablations:
+        return ablations(args)
     if args.workload == "config4" and args.impl == "ours":
         return stack(args)
 
@@ -547,6 +551,98 @@ def stack(args):
                         "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "traffic": None},
            "clocks": clocks, "gpu_launches": 23 * args.layers * args.steps}
     print(json.dumps(out))
+    return 0
+
+
+def ablations(args):
+    """The router ablations of the paper's Table 3, on the config-3 layer: time per layer, fallback rate, share of the
+    dense pairs computed and, in place of task scores (no model, no datasets here), the exactly retained attention mass
+    on the audited probe rows: mean over heads, mean of the worst tenth of the heads, minimum."""
+    import torch
+    import paper_2608_29058_b200 as rs
+    from synth import config3_spec, make_layer
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    n = args.n or 131072
+    out_dir = os.path.join(ROOT, "gpurun_out")
+    os.makedirs(out_dir, exist_ok=True)
+    path = os.path.join(out_dir, f"ablations_config3_n{n}.jsonl")
+    spec = config3_spec(n)
+    L = make_layer(spec)
+    Q, K, V = _to_dev(L["Q"], dev), _to_dev(L["K"], dev), _to_dev(L["V"], dev)
+    p = rs.Problem(spec.n_q_heads, spec.n_kv_heads, n)
+    full_lib = rs.default_library()
+    one_budget = [full_lib[1], full_lib[5], full_lib[9], full_lib[12]]     # second budget of each family + dense
+    base = dict(budget_frac=0.15, cert_max=0.05)
+    # routes of another input of the same recipe, applied unchanged ("no input routing")
+    Lc = make_layer(config3_spec(n, seed_offset=5000))
+    cal_layer = rs.RoutedPrefillLayer(p, None, rs.RouteConfig(**base), device=dev)
+    cal_layer.forward(_to_dev(Lc["Q"], dev), _to_dev(Lc["K"], dev), _to_dev(Lc["V"], dev))
+    static_routes = cal_layer.choice.clone()
+    del cal_layer, Lc
+    variants = [
+        ("full", None, rs.RouteConfig(**base), {}),
+        ("no input routing (routes of another input)", None, rs.RouteConfig(**base), {"fixed": static_routes}),
+        ("no uncertainty score (alpha = 0)", None, rs.RouteConfig(alpha=0.0, **base), {}),
+        ("no dense fallback", None, rs.RouteConfig(budget_frac=0.15, cert_max=None), {}),
+        ("one fixed budget per family", one_budget, rs.RouteConfig(**base), {}),
+        ("profiled latency table instead of FLOPs", None, rs.RouteConfig(**base), {"measured": True}),
+        ("per-head launches", None, rs.RouteConfig(**base), {"per_head": True}),
+        ("fallback rescue (any family before dense)", None, rs.RouteConfig(rescue_any=True, **base), {}),
+        ("greedy back-fill of leftover budget", None, rs.RouteConfig(backfill=True, **base), {}),
+    ]
+    rows = []
+    with open(path, "w") as f:
+        for name, lib, cfg, opt in variants:
+            layer = rs.RoutedPrefillLayer(p, lib, cfg, device=dev)
+            fixed = opt.get("fixed")
+            if opt.get("measured"):
+                layer.forward(Q, K, V)
+                layer.profile_costs(Q, K, V)
+            for _ in range(2):
+                layer.forward(Q, K, V, fixed_choice=fixed)
+            torch.cuda.synchronize()
+            k = 3
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(k):
+                layer.forward(Q, K, V, fixed_choice=fixed, record_events=True)
+            e1.record()
+            torch.cuda.synchronize()
+            rs.check_status(layer.status, name)
+            ms = e0.elapsed_time(e1) / k
+            st = layer.stage_ms()
+            if opt.get("per_head"):
+                a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                layer.attention_split(Q, K, V, 1)
+                a0.record()
+                for _ in range(k):
+                    layer.attention_split(Q, K, V, 1)
+                a1.record()
+                torch.cuda.synchronize()
+                ms = ms - st["attention"] + a0.elapsed_time(a1) / k
+            choice = layer.choice.cpu().numpy()
+            m_head = np.sort(layer.m_head.cpu().numpy().astype(np.float64))
+            worst = max(1, len(m_head) // 10)
+            pairs = layer.stats.cpu().numpy()[:, :, 4]
+            dense_c = [i for i, c in enumerate(layer.cands) if c[0] == rs.RS_DENSE][0]
+            if fixed is None and (pairs.sum() > 0):
+                frac = float(sum(pairs[i, choice[i]] for i in range(p.n_items)) / pairs[:, dense_c].sum())
+            else:
+                frac = None
+            rep = layer.route_report() if fixed is None else {"n_fallback": 0}
+            row = {"variant": name, "n": n, "ms_per_layer": ms, "fallback_pct": 100.0 * rep["n_fallback"] / p.n_items,
+                   "dense_heads": int((choice == dense_c).sum()), "pairs_fraction_of_dense": frac,
+                   "retained_mass_mean": float(m_head.mean()), "retained_mass_worst_decile": float(m_head[:worst].mean()),
+                   "retained_mass_min": float(m_head[0]), "stage_ms": st}
+            f.write(json.dumps(row) + "\n")
+            f.flush()
+            rows.append(row)
+            del layer
+            torch.cuda.empty_cache()
+    print(json.dumps({"ablations": [{k: r[k] for k in ("variant", "ms_per_layer", "fallback_pct", "dense_heads",
+                                                       "retained_mass_mean", "retained_mass_worst_decile")} for r in rows],
+                      "file": os.path.relpath(path, ROOT)}))
     return 0
 
 
