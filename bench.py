@@ -226,6 +226,8 @@ def main():
                     help="also time the attention stage as one launch per KV group and as one launch per head")
     ap.add_argument("--ablations", action="store_true",
                     help="router ablations of the paper's Table 3 on the config-3 layer, JSONL output")
+    ap.add_argument("--graph", action="store_true",
+                    help="also time the layer replayed from a CUDA graph (whole pass captured once; for launch-bound sizes)")
     ap.add_argument("--sweep", action="store_true", help="config-5 sweep: n x budget x forced-dense cells, JSONL output")
     ap.add_argument("--n", type=int, default=None, help="override the sequence length (smaller profiling case)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -364,6 +366,23 @@ def main():
         dense_ms = d0.elapsed_time(d1) / reps
         del O_d, lse_d
 
+    # ---- the same layer pass replayed from a CUDA graph (no host work between the launches)
+    graph_ms = None
+    if args.graph:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step()
+        g.replay()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(args.steps):
+            g.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        rs.check_status(layer.status, "graph replay")
+        graph_ms = g0.elapsed_time(g1) / args.steps
+
     # ---- launch ablation (Section 3.4 / Table 3: grouping heads into one launch against per-group / per-head launches)
     launch_ablation = None
     if args.launch_ablation and p.n_segments == 1:
@@ -452,6 +471,7 @@ def main():
                   "selected_fraction_of_dense": f_mask / f_dense},
         "routes": hist, "route_report": layer.route_report() if not fixed else None,
         "cost_model": args.cost, "calibration": calibration, "risk_calibration": risk_calibration, "launch_ablation": launch_ablation,
+        "cuda_graph_ms_per_layer": graph_ms,
         "fallback_rescue": bool(args.rescue),
         "roofline": {"kernel": "rs_attn_kernel (one launch, all heads)", "bound": "tensor", "achieved": achieved,
                      "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,

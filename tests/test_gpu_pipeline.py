@@ -177,3 +177,30 @@ def test_split_launches_give_the_single_launch_result(online):
         layer.attention_split(Q, K, V, heads)
         rs.check_status(layer.status, "split launches")
         assert torch.equal(layer.O, want_O) and torch.equal(layer.lse_sel, want_lse), heads
+
+
+def test_layer_replays_from_a_cuda_graph():
+    """The whole layer pass (probe, evaluation, routing on the device, materialisation, attention, certificate; the
+    side-stream fork / join inside the probe and index calls included) can be captured once and replayed: no host
+    decision sits between the steps."""
+    n, Hq, Hkv = 1024, 4, 2
+    L = make_layer(tiny_spec(93, n, Hq, Hkv))
+    Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+    p = rs.Problem(Hq, Hkv, n, [0, 384, 1024])
+    lib = [(rs.RS_A_SHAPE, 64, 128), (rs.RS_VERTICAL_SLASH, 48, 160), (rs.RS_BLOCK_SPARSE, 4, 0), (rs.RS_DENSE, 0, 0)]
+    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(budget_frac=0.5, cert_max=0.6))
+    layer.forward(Q, K, V)                              # eager: also does the one-time kernel attribute set-up
+    torch.cuda.synchronize()
+    rs.check_status(layer.status, "eager layer")
+    want_O, want_choice, want_m = layer.O.clone(), layer.choice.clone(), layer.m_head.clone()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        layer.forward(Q, K, V)
+    for other_seed in (94, 93):                         # new inputs in the same buffers, then the first ones again
+        L2 = make_layer(tiny_spec(other_seed, n, Hq, Hkv))
+        Q.copy_(dev_bf16(L2["Q"])); K.copy_(dev_bf16(L2["K"])); V.copy_(dev_bf16(L2["V"]))
+        layer.O.zero_(); layer.choice.fill_(-1)
+        g.replay()
+        torch.cuda.synchronize()
+        rs.check_status(layer.status, "replayed layer")
+    assert torch.equal(layer.choice, want_choice) and torch.equal(layer.O, want_O) and torch.equal(layer.m_head, want_m)
