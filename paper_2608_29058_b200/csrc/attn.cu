@@ -23,6 +23,7 @@ constexpr int kTmemCols = 256;
 constexpr uint32_t kColS = 0;     // two score buffers (fp32, 64 columns each); bf16 P (32 columns) overwrites a buffer's start
 constexpr uint32_t kColO = 128;   // O (fp32, 128 columns)
 
+constexpr int kMaskChunks = 128;   // gathered-column chunks with precomputed keep masks (8192 columns); beyond: per element
 constexpr uint32_t F_LO = 1u << 12, F_HI = 1u << 13, F_CAUSAL = 1u << 14, F_EDGE = 1u << 15;
 
 struct AttnParams {
@@ -62,8 +63,12 @@ __device__ __forceinline__ uint32_t range_mask(int lo, int hi, int w) {
 // pays one uniform branch and nothing else.
 //   mode 0: every column to -inf;  mode 1: keep j <= i (and, with `edge`, j < n_sink or i - j < window);
 //   mode 2: gathered columns: keep vcols[vbase + x] <= i unless a block diagonal of D already covers that key.
+//   mode 3: gathered columns with the keep decisions of this row half precomputed per tile: bit x of `keep` says
+//           column x survives (valid, not covered by D, not in a later block); bit x of `diag` says the column lies
+//           in the row's own key block, where j <= i still has to be tested.
 __device__ __noinline__ void rs_mask_chunk(uint32_t taddr, int mode, int i, int j0, int edge, int n_sink, int window,
-                                           const int* vcols, int vbase, int n_vcols, const uint32_t* d_bits) {
+                                           const int* vcols, int vbase, int n_vcols, const uint32_t* d_bits,
+                                           unsigned long long keep = 0ull, unsigned long long diag = 0ull) {
   const uint32_t NEG = 0xff800000u;
   uint32_t x[32];
 #pragma unroll 1
@@ -81,6 +86,16 @@ __device__ __noinline__ void rs_mask_chunk(uint32_t taddr, int mode, int i, int 
         bool keep = j <= i;
         if (edge) keep = keep && (j < n_sink || i - j < window);
         if (!keep) x[q] = NEG;
+      }
+    } else if (mode == 3) {
+      const uint32_t kp = (uint32_t)(keep >> cb), dg = (uint32_t)(diag >> cb);
+#pragma unroll
+      for (int q = 0; q < 32; ++q)
+        if (!((kp >> q) & 1u)) x[q] = NEG;
+      if (dg != 0u) {
+#pragma unroll
+        for (int q = 0; q < 32; ++q)
+          if (((dg >> q) & 1u) && __ldg(vcols + vbase + cb + q) > i) x[q] = NEG;
       }
     } else {
       const int qb_i = i >> 6;
@@ -137,6 +152,10 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   int* wprefix = reinterpret_cast<int*>(d_bits + 128);
   uint64_t* bars = reinterpret_cast<uint64_t*>(wprefix + 132);
   volatile int* misc = reinterpret_cast<volatile int*>(bars + 14);   // [0] tmem base, [1] abort, [2] n_block, [3] n_vert
+  // keep / own-block masks of the gathered-column chunks: [chunk][row half]
+  unsigned long long* vkeep = reinterpret_cast<unsigned long long*>(sm + SmemLayout::end_tiles + ((list_cap * 2 + 15) & ~15) +
+                                                                      3 * 128 * 4 + 132 * 4 + 14 * 8 + 64);
+  unsigned long long* vdiag = vkeep + 2 * kMaskChunks;
   // barrier pairs (slot 0 / 1) sit next to each other: address of slot s = base + 8 * s
   const uint32_t bar_q = smem_u32(&bars[0]), bar_o = smem_u32(&bars[1]), bar_kf = smem_u32(&bars[2]),
                  bar_ke = smem_u32(&bars[4]), bar_vf = smem_u32(&bars[6]), bar_ve = smem_u32(&bars[8]),
@@ -257,6 +276,35 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   __syncthreads();
   const int n_block = misc[2], n_vert = misc[3];
   const int n_chunks = n_block + n_vert;
+  if (n_vert > 0) {
+    // Per gathered-column chunk and row half: which columns survive for every row of the half (valid entry, key
+    // block not after the half's block, not already covered by a block diagonal of D) and which of them lie in the
+    // half's own key block.  A chunk whose 64 columns all survive outside the own block needs no mask at all.
+    const int* vc = P.idx.vs_cols + (size_t)vs_slot * P.idx.kv_cap;
+    const int n_piece = min(n_vert, kMaskChunks) * 2;          // 32-column pieces, one per warp iteration
+    for (int piece = warp; piece < n_piece; piece += kThreads / 32) {
+      const int vi = piece * 32 + lane;
+      const bool valid = vi < n_vcols;
+      const int j = valid ? vc[vi] : 0;
+      uint32_t kp[2], dg[2];
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {
+        const int dlt = qb0 + hf - (j >> 6);
+        const bool covered = dlt >= 0 && ((d_bits[dlt >> 5] >> (dlt & 31)) & 1u);
+        const bool keep = valid && dlt >= 0 && !covered;
+        kp[hf] = __ballot_sync(0xffffffffu, keep);
+        dg[hf] = __ballot_sync(0xffffffffu, keep && dlt == 0);
+      }
+      if (lane == 0) {
+        uint32_t* k32 = reinterpret_cast<uint32_t*>(vkeep);
+        uint32_t* d32 = reinterpret_cast<uint32_t*>(vdiag);
+        const int chunk = piece >> 1, part = piece & 1;
+        k32[(chunk * 2 + 0) * 2 + part] = kp[0]; k32[(chunk * 2 + 1) * 2 + part] = kp[1];
+        d32[(chunk * 2 + 0) * 2 + part] = dg[0]; d32[(chunk * 2 + 1) * 2 + part] = dg[1];
+      }
+    }
+    __syncthreads();
+  }
 
   // =========================================================================================== roles
   // Everything below is pipelined per 64-key chunk; chunk c uses slot c & 1 of the K / V rings, of the two 64-column
@@ -428,6 +476,7 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
       tc_fence_after();
       {
         int mode = -1, j0 = 0, edge = 0, vbase = 0;
+        unsigned long long vk = 0ull, vd = 0ull;
         if (ch < n_block) {
           const uint32_t e = list[ch];
           if (!(e & (half ? F_HI : F_LO))) {
@@ -438,10 +487,17 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             edge = (e & F_EDGE) ? 1 : 0;
           }
         } else {
-          mode = 2;
-          vbase = (ch - n_block) * kChunk;
+          const int vch = ch - n_block;
+          vbase = vch * kChunk;
+          if (vch < kMaskChunks) {
+            vk = vkeep[vch * 2 + half];
+            vd = vdiag[vch * 2 + half];
+            mode = (vk == ~0ull && vd == 0ull) ? -1 : 3;
+          } else {
+            mode = 2;
+          }
         }
-        if (mode >= 0) rs_mask_chunk(t_sc, mode, i, j0, edge, cand.b0, cand.b1, vcols, vbase, n_vcols, d_bits);
+        if (mode >= 0) rs_mask_chunk(t_sc, mode, i, j0, edge, cand.b0, cand.b1, vcols, vbase, n_vcols, d_bits, vk, vd);
       }
       tmem_ld32(t_sc, v);
       tmem_ld32(t_sc + 32u, v2);
@@ -614,7 +670,7 @@ __global__ void rs_pack_vertical_kernel(AttnParams P, const __nv_bfloat16* K, co
 
 size_t attn_smem_bytes(int n) {
   const int list_cap = (n >> 6) + 64;
-  return 1024 + SmemLayout::end_tiles + ((list_cap * 2 + 15) & ~15) + 3 * 128 * 4 + 132 * 4 + 14 * 8 + 64;
+  return 1024 + SmemLayout::end_tiles + ((list_cap * 2 + 15) & ~15) + 3 * 128 * 4 + 132 * 4 + 14 * 8 + 64 + 4 * kMaskChunks * 8;
 }
 
 struct WsPlan { size_t cost, items, order, kpack, vpack, total; int n_work, kv_pad, n_items; };
