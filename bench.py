@@ -410,26 +410,30 @@ def main():
         Qh, Kh, Vh = (torch.from_numpy(L[k].view(np.int16)).view(torch.bfloat16).pin_memory() for k in ("Q", "K", "V"))
         Oh = torch.empty(tuple(layer.O.shape), dtype=layer.O.dtype).pin_memory()
         bufs = (Q, K, V)
-        # fixed routes need the route tensor inside forward: bind it through a small closure
+        # Every step copies its Q, K, V from pinned host memory and its O back; the copies of neighbouring steps overlap
+        # with the kernels (three streams, two device buffer sets).
+        pipe = rs.StreamedPrefill(layer)
         def e2e_step():
-            Q.copy_(Qh, non_blocking=True); K.copy_(Kh, non_blocking=True); V.copy_(Vh, non_blocking=True)
-            layer.forward(Q, K, V, fixed_choice=fixed_t)
-            Oh.copy_(layer.O, non_blocking=True)
+            pipe.submit(Qh, Kh, Vh, Oh, fixed_choice=fixed_t)
         e2e_step()
+        pipe.finish()
         sync_all()
-        k_e2e = max(2, min(args.steps, 3))
+        k_e2e = max(4, min(args.steps, 20))      # the first copy in and the last copy out are not hidden: short runs show them
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record()
         for _ in range(k_e2e):
             e2e_step()
+        pipe.finish()
         g1.record()
         sync_all()
+        rs.check_status(layer.status, "end-to-end steps")
         ms_e2e, units_e2e = aggregate_over_ranks(g0.elapsed_time(g1) / k_e2e, f_mask, dev)
         h2d = sum(int(t.numel() * t.element_size()) for t in (Qh, Kh, Vh))
         d2h = int(Oh.numel() * Oh.element_size())
         e2e = {"value": units_e2e / (ms_e2e * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
-        del Qh, Kh, Vh
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "overlap": "copies of neighbouring steps overlap the kernels (3 streams, 2 buffer sets); every step copies its own inputs and output"}
+        del Qh, Kh, Vh, pipe
 
     if rank != 0:
         return 0

@@ -328,3 +328,59 @@ def prefill_from_host(layer: RoutedPrefillLayer, Q_host: torch.Tensor, K_host: t
     O = layer.forward(Qd, Kd, Vd)
     O_host.copy_(O, non_blocking=True)
     return O_host
+
+
+class StreamedPrefill:
+    """Layer passes fed from pinned HOST buffers with the copies overlapped with the kernels: three streams (host to
+    device, compute, device to host) and two device buffer sets, so that while pass k computes, the inputs of pass k + 1
+    arrive and the output of pass k - 1 leaves.  Every pass still copies its own Q, K, V in and its own O out; only the
+    order on the copy engines and the SMs is pipelined.  submit() enqueues one pass and returns immediately; finish()
+    makes the caller's current stream wait for everything submitted."""
+
+    def __init__(self, layer: RoutedPrefillLayer, n_buffers: int = 2):
+        self.layer = layer
+        dev = layer.O.device
+        p = layer.p
+        shape_q = (p.n_q_heads, p.n_keys, 128)
+        shape_kv = (p.n_kv_heads, p.n_keys, 128)
+        bf = dict(dtype=torch.bfloat16, device=dev)
+        self.n = n_buffers
+        self.Q = [torch.empty(shape_q, **bf) for _ in range(n_buffers)]
+        self.K = [torch.empty(shape_kv, **bf) for _ in range(n_buffers)]
+        self.V = [torch.empty(shape_kv, **bf) for _ in range(n_buffers)]
+        self.O = [layer.O] + [torch.empty_like(layer.O) for _ in range(n_buffers - 1)]
+        self.s_in, self.s_run, self.s_out = (torch.cuda.Stream(device=dev) for _ in range(3))
+        ev = lambda: [torch.cuda.Event() for _ in range(n_buffers)]
+        self.in_done, self.run_done, self.out_done = ev(), ev(), ev()
+        self.k = 0
+
+    def submit(self, Q_host, K_host, V_host, O_host, **forward_kw):
+        b = self.k % self.n
+        first_use = self.k < self.n
+        cur = torch.cuda.current_stream()
+        with torch.cuda.stream(self.s_in):
+            self.s_in.wait_stream(cur) if self.k == 0 else None
+            if not first_use:
+                self.s_in.wait_event(self.run_done[b])          # the pass that last read this input set is done
+            self.Q[b].copy_(Q_host, non_blocking=True)
+            self.K[b].copy_(K_host, non_blocking=True)
+            self.V[b].copy_(V_host, non_blocking=True)
+            self.in_done[b].record(self.s_in)
+        with torch.cuda.stream(self.s_run):
+            self.s_run.wait_event(self.in_done[b])
+            if not first_use:
+                self.s_run.wait_event(self.out_done[b])         # the output buffer has been copied out
+            self.layer.O = self.O[b]
+            self.layer.forward(self.Q[b], self.K[b], self.V[b], **forward_kw)
+            self.run_done[b].record(self.s_run)
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.run_done[b])
+            O_host.copy_(self.O[b], non_blocking=True)
+            self.out_done[b].record(self.s_out)
+        self.k += 1
+
+    def finish(self):
+        cur = torch.cuda.current_stream()
+        for s in (self.s_in, self.s_run, self.s_out):
+            cur.wait_stream(s)
+        self.layer.O = self.O[0]

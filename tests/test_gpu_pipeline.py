@@ -204,3 +204,27 @@ def test_layer_replays_from_a_cuda_graph():
         torch.cuda.synchronize()
         rs.check_status(layer.status, "replayed layer")
     assert torch.equal(layer.choice, want_choice) and torch.equal(layer.O, want_O) and torch.equal(layer.m_head, want_m)
+
+
+def test_streamed_host_passes_match_the_plain_call():
+    """Overlapped host-buffer passes (StreamedPrefill) return, for every pass, what the plain call returns."""
+    n, Hq, Hkv = 1024, 4, 2
+    p = rs.Problem(Hq, Hkv, n)
+    lib = [(rs.RS_A_SHAPE, 64, 128), (rs.RS_VERTICAL_SLASH, 48, 160), (rs.RS_BLOCK_SPARSE, 4, 0), (rs.RS_DENSE, 0, 0)]
+    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(budget_frac=0.4, cert_max=0.5))
+    hosts, want = [], []
+    for seed in (71, 72, 73, 74, 75):
+        L = make_layer(tiny_spec(seed, n, Hq, Hkv))
+        Qh, Kh, Vh = (torch.from_numpy(L[k].view(np.int16)).view(torch.bfloat16).pin_memory() for k in ("Q", "K", "V"))
+        hosts.append((Qh, Kh, Vh, torch.zeros((Hq, n, 128), dtype=torch.bfloat16).pin_memory()))
+        layer.forward(Qh.cuda(), Kh.cuda(), Vh.cuda())
+        torch.cuda.synchronize()
+        want.append(layer.O.cpu().clone())
+    pipe = rs.StreamedPrefill(layer)
+    for Qh, Kh, Vh, Oh in hosts:
+        pipe.submit(Qh, Kh, Vh, Oh)
+    pipe.finish()
+    torch.cuda.synchronize()
+    rs.check_status(layer.status, "streamed passes")
+    for k, (_, _, _, Oh) in enumerate(hosts):
+        assert torch.equal(Oh, want[k]), k
