@@ -95,61 +95,111 @@ rs_vs_keys_kernel(IdxParams P) {
 }
 
 // ------------------------------------------------------------------------------------------ exact top-k of a line list
-// grid = (2 lists, jobs).  list 0: vertical columns over [0, q1); list 1: slash offsets over [1, q1) plus offset 0.
+// grid = (2 lists, items, groups of up to kSelMaxC vertical-slash candidates).  list 0: vertical columns over [0, q1);
+// list 1: slash offsets over [1, q1) plus offset 0.  One block serves every budget of the item in the same passes
+// over the keys: the radix digits are histogrammed once per distinct prefix (the first digit once for all budgets),
+// and one counting sweep plus one writing sweep produce all the ordered lists.
 constexpr int kSelThreads = 1024;
 constexpr int kDigitBits = 13;
 constexpr int kBins = 1 << kDigitBits;
+constexpr int kSelMaxC = 2;       // budgets served by one block: two keeps 2 x items x 2 blocks in flight and halves the key passes
+constexpr int kSelBatch = 8;      // independent key loads in flight per thread
 
 __global__ void __launch_bounds__(kSelThreads)
 rs_vs_select_kernel(IdxParams P) {
-  __shared__ unsigned int hist[kBins];
+  extern __shared__ unsigned int sel_hist[];             // [unique prefixes <= kSelMaxC][kBins]
   __shared__ unsigned int wsum[32];
-  __shared__ u64 sh_prefix;
-  __shared__ unsigned int sh_k;
-  __shared__ unsigned int w_gt[32], w_eq[32];
-  int item, c, slot;
-  if (!job_of(P, blockIdx.y, item, c, slot)) return;
-  const rs_candidate cand = P.lib[c];
-  if (cand.pattern != RS_VERTICAL_SLASH) return;
-  const int list = blockIdx.x;
+  __shared__ u64 sh_prefix[kSelMaxC];
+  __shared__ unsigned int sh_k[kSelMaxC];
+  __shared__ unsigned int w_gt[kSelMaxC][32], w_eq[kSelMaxC][32];
+  const int list = blockIdx.x, item = blockIdx.y;
+  // the vertical-slash candidates this block serves
+  int cand_id[kSelMaxC] = {}, slot_id[kSelMaxC] = {}, kk[kSelMaxC] = {};
+  int nC = 0;
+  {
+    int seen = 0;
+    for (int c = 0; c < P.n_cand; ++c) {
+      if (P.lib[c].pattern != RS_VERTICAL_SLASH) continue;
+      if (P.choice != nullptr && P.choice[item] != c) continue;
+      if (seen / kSelMaxC == (int)blockIdx.z && nC < kSelMaxC) {
+        const int sl = (P.choice != nullptr) ? item : item * P.n_cand + c;
+        _Pragma("unroll") for (int e = 0; e < kSelMaxC; ++e) if (e == nC) { cand_id[e] = c; slot_id[e] = sl; }
+        ++nC;
+      }
+      ++seen;
+    }
+  }
+  if (nC == 0) return;
   const int s = item / P.Hq;
   const int q1 = P.seg_bounds[s + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const u64* keys = P.keys + ((size_t)item * 2 + list) * P.n;
   const int first = (list == 0) ? 0 : 1;                 // first index of the domain
   const int n_dom = q1 - first;
-  int k = (list == 0) ? min(cand.b0, q1) : (min(cand.b1, q1) - 1);
-  if (k < 0) k = 0;
-  if (k > n_dom) k = n_dom;
-  int32_t* out = (list == 0) ? (P.out.vs_cols + (size_t)slot * P.out.kv_cap) : (P.out.vs_offs + (size_t)slot * P.out.ks_cap);
+  _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+    const rs_candidate cand = P.lib[cand_id[c]];
+    int k = (list == 0) ? min(cand.b0, q1) : (min(cand.b1, q1) - 1);
+    if (k < 0) k = 0;
+    if (k > n_dom) k = n_dom;
+    kk[c] = k;
+  }
   const int cap = (list == 0) ? P.out.kv_cap : P.out.ks_cap;
 
-  u64 T = ~0ull;           // threshold key: everything above is taken, k_eq ties in index order
-  unsigned int k_eq = 0;
-  if (k > 0) {
-    if (tid == 0) { sh_prefix = 0; sh_k = (unsigned)k; }
-    for (int pass = 2; pass >= 0; --pass) {
-      for (int i = tid; i < kBins; i += kSelThreads) hist[i] = 0;
-      __syncthreads();
-      const u64 prefix = sh_prefix;
-      const int shift = pass * kDigitBits;
-      for (int base = 0; base < n_dom; base += kSelThreads) {
-        const int j = base + tid;
-        unsigned int digit = 0xffffffffu;
-        if (j < n_dom) {
-          const u64 key = keys[first + j];
-          if ((key >> (shift + kDigitBits)) == prefix) digit = (unsigned)((key >> shift) & (kBins - 1));
-        }
-        const unsigned int peers = __match_any_sync(0xffffffffu, digit);
-        if (digit != 0xffffffffu && lane == (__ffs(peers) - 1)) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+  // ---- thresholds: T[c] = key of the k-th entry in "key descending" order, k_eq[c] = how many of its ties are taken
+  if (tid < nC) { sh_prefix[tid] = 0; sh_k[tid] = (unsigned)kk[tid]; }
+  __syncthreads();
+  for (int pass = 2; pass >= 0; --pass) {
+    const int shift = pass * kDigitBits;
+    // candidates with the same prefix share a histogram: hsel[c] = index of the first candidate with that prefix
+    u64 pre[kSelMaxC];
+    int hsel[kSelMaxC];
+    int n_hist = 0;
+    _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+      pre[c] = sh_prefix[c];
+      hsel[c] = -1;
+      if (kk[c] == 0) continue;
+      _Pragma("unroll") for (int d = 0; d < kSelMaxC; ++d)
+        if (d < c && hsel[c] < 0 && kk[d] > 0 && pre[d] == pre[c]) hsel[c] = hsel[d];
+      if (hsel[c] < 0) hsel[c] = n_hist++;
+    }
+    for (int i = tid; i < n_hist * kBins; i += kSelThreads) sel_hist[i] = 0;
+    __syncthreads();
+    // eight independent loads per thread are in flight before any is used: the sweep is latency-bound otherwise
+    for (int base = 0; base < n_dom; base += kSelThreads * kSelBatch) {
+      u64 keyb[kSelBatch];
+      bool inb[kSelBatch];
+#pragma unroll
+      for (int u = 0; u < kSelBatch; ++u) {
+        const int j = base + u * kSelThreads + tid;
+        inb[u] = j < n_dom;
+        keyb[u] = inb[u] ? keys[first + j] : 0ull;
       }
-      __syncthreads();
-      // each thread owns 8 consecutive bins, highest bins first
+#pragma unroll
+      for (int u = 0; u < kSelBatch; ++u) {
+        const u64 hi = keyb[u] >> (shift + kDigitBits);
+        const unsigned int dig = (unsigned)((keyb[u] >> shift) & (kBins - 1));
+        int done_hist = -1;                              // histograms are numbered in candidate order
+        _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+          if (hsel[c] <= done_hist) continue;            // shared with an earlier candidate (or k = 0: hsel = -1)
+          done_hist = hsel[c];
+          unsigned int digit = (inb[u] && hi == pre[c]) ? dig : 0xffffffffu;
+          if (__ballot_sync(0xffffffffu, digit != 0xffffffffu) == 0u) continue;   // nobody in this warp is in the bin
+          const unsigned int peers = __match_any_sync(0xffffffffu, digit);
+          if (digit != 0xffffffffu && lane == (__ffs(peers) - 1))
+            atomicAdd(&sel_hist[hsel[c] * kBins + digit], (unsigned)__popc(peers));
+        }
+      }
+    }
+    __syncthreads();
+    // per candidate: locate the bin that holds its k-th entry (each thread owns 8 consecutive bins, highest first)
+    _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+      if (kk[c] == 0) continue;                          // uniform over the block
+      const unsigned int* hist = sel_hist + hsel[c] * kBins;
       const int b0 = kBins - 8 * (tid + 1);
       unsigned int loc[8], lsum = 0;
 #pragma unroll
       for (int i = 0; i < 8; ++i) { loc[i] = hist[b0 + i]; lsum += loc[i]; }
-      unsigned int incl = lsum;           // inclusive scan over threads (thread 0 owns the top bins)
+      unsigned int incl = lsum;                          // inclusive scan over threads (thread 0 owns the top bins)
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
         const unsigned int t = __shfl_up_sync(0xffffffffu, incl, off);
@@ -159,15 +209,15 @@ rs_vs_select_kernel(IdxParams P) {
       __syncthreads();
       unsigned int before = 0;
       for (int w = 0; w < warp; ++w) before += wsum[w];
-      const unsigned int above = before + incl - lsum;    // entries in bins above this thread's bins
-      const unsigned int kk = sh_k;
+      const unsigned int above = before + incl - lsum;   // entries in bins above this thread's bins
+      const unsigned int kq = sh_k[c];
       __syncthreads();
-      if (above < kk && kk <= above + lsum) {
+      if (above < kq && kq <= above + lsum) {
         unsigned int acc = above;
         for (int i = 7; i >= 0; --i) {
-          if (acc + loc[i] >= kk) {
-            sh_prefix = (prefix << kDigitBits) | (u64)(b0 + i);
-            sh_k = kk - acc;
+          if (acc + loc[i] >= kq) {
+            sh_prefix[c] = (pre[c] << kDigitBits) | (u64)(b0 + i);
+            sh_k[c] = kq - acc;
             break;
           }
           acc += loc[i];
@@ -175,48 +225,84 @@ rs_vs_select_kernel(IdxParams P) {
       }
       __syncthreads();
     }
-    T = sh_prefix;
-    k_eq = sh_k;
+  }
+  u64 T[kSelMaxC];
+  unsigned int k_eq[kSelMaxC];
+  _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+    T[c] = (kk[c] > 0) ? sh_prefix[c] : ~0ull;           // k = 0: nothing is above or equal
+    k_eq[c] = (kk[c] > 0) ? sh_k[c] : 0u;
   }
 
-  // ordered compaction: warp w walks the contiguous range [w * chunk, (w + 1) * chunk)
+  // ---- ordered compaction: warp w walks the contiguous range [w * chunk, (w + 1) * chunk)
   const int chunk = (((n_dom + 31) / 32) + 31) / 32 * 32;
   const int lo = warp * chunk, hi = min(n_dom, lo + chunk);
-  unsigned int gt = 0, eq = 0;
-  for (int base = lo; base < hi; base += 32) {
-    const int j = base + lane;
-    u64 key = 0;
-    const bool in = j < hi;
-    if (in) key = keys[first + j];
-    gt += __popc(__ballot_sync(0xffffffffu, in && key > T));
-    eq += __popc(__ballot_sync(0xffffffffu, in && key == T));
-  }
-  if (lane == 0) { w_gt[warp] = gt; w_eq[warp] = eq; }
-  __syncthreads();
-  unsigned int gt_before = 0, eq_before = 0;
-  for (int w = 0; w < warp; ++w) { gt_before += w_gt[w]; eq_before += w_eq[w]; }
-  unsigned int pos = gt_before + min(k_eq, eq_before) + (list == 1 ? 1u : 0u);
-  unsigned int eq_run = eq_before;
-  const unsigned int lt_mask = (1u << lane) - 1u;
-  for (int base = lo; base < hi; base += 32) {
-    const int j = base + lane;
-    u64 key = 0;
-    const bool in = j < hi;
-    if (in) key = keys[first + j];
-    const bool is_eq = in && key == T;
-    const unsigned int beq = __ballot_sync(0xffffffffu, is_eq);
-    const bool take = in && (key > T || (is_eq && eq_run + __popc(beq & lt_mask) < k_eq));
-    const unsigned int bt = __ballot_sync(0xffffffffu, take);
-    if (take) {
-      const unsigned int p = pos + __popc(bt & lt_mask);
-      if ((int)p < cap) out[p] = first + j;
+  unsigned int gt[kSelMaxC], eq[kSelMaxC];
+  _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) { gt[c] = 0; eq[c] = 0; }
+  for (int base = lo; base < hi; base += 32 * kSelBatch) {
+    u64 keyb[kSelBatch];
+    bool inb[kSelBatch];
+#pragma unroll
+    for (int u = 0; u < kSelBatch; ++u) {
+      const int j = base + u * 32 + lane;
+      inb[u] = j < hi;
+      keyb[u] = inb[u] ? keys[first + j] : 0ull;
     }
-    pos += __popc(bt);
-    eq_run += __popc(beq);
+#pragma unroll
+    for (int u = 0; u < kSelBatch; ++u) {
+      _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+        gt[c] += __popc(__ballot_sync(0xffffffffu, inb[u] && keyb[u] > T[c]));
+        eq[c] += __popc(__ballot_sync(0xffffffffu, inb[u] && keyb[u] == T[c]));
+      }
+    }
+  }
+  if (lane == 0)
+    _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) { w_gt[c][warp] = gt[c]; w_eq[c][warp] = eq[c]; }
+  __syncthreads();
+  unsigned int pos[kSelMaxC], eq_run[kSelMaxC];
+  _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+    unsigned int gt_before = 0, eq_before = 0;
+    for (int w = 0; w < warp; ++w) { gt_before += w_gt[c][w]; eq_before += w_eq[c][w]; }
+    pos[c] = gt_before + min(k_eq[c], eq_before) + (list == 1 ? 1u : 0u);
+    eq_run[c] = eq_before;
+  }
+  const unsigned int lt_mask = (1u << lane) - 1u;
+  for (int base = lo; base < hi; base += 32 * kSelBatch) {
+    u64 keyb[kSelBatch];
+    bool inb[kSelBatch];
+#pragma unroll
+    for (int u = 0; u < kSelBatch; ++u) {
+      const int j = base + u * 32 + lane;
+      inb[u] = j < hi;
+      keyb[u] = inb[u] ? keys[first + j] : 0ull;
+    }
+#pragma unroll
+    for (int u = 0; u < kSelBatch; ++u) {
+      const int j = base + u * 32 + lane;
+      _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+        const bool is_eq = inb[u] && keyb[u] == T[c];
+        const unsigned int beq = __ballot_sync(0xffffffffu, is_eq);
+        const bool take = inb[u] && (keyb[u] > T[c] || (is_eq && eq_run[c] + __popc(beq & lt_mask) < k_eq[c]));
+        const unsigned int bt = __ballot_sync(0xffffffffu, take);
+        if (take) {
+          const unsigned int p = pos[c] + __popc(bt & lt_mask);
+          int32_t* out = (list == 0) ? (P.out.vs_cols + (size_t)slot_id[c] * P.out.kv_cap)
+                                     : (P.out.vs_offs + (size_t)slot_id[c] * P.out.ks_cap);
+          if ((int)p < cap) out[p] = first + j;
+        }
+        pos[c] += __popc(bt);
+        eq_run[c] += __popc(beq);
+      }
+    }
   }
   if (tid == 0) {
-    if (list == 1) { out[0] = 0; P.out.vs_count[4 * slot + 1] = k + 1; }
-    else P.out.vs_count[4 * slot + 0] = k;
+    _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+      if (list == 1) {
+        P.out.vs_offs[(size_t)slot_id[c] * P.out.ks_cap] = 0;
+        P.out.vs_count[4 * slot_id[c] + 1] = kk[c] + 1;
+      } else {
+        P.out.vs_count[4 * slot_id[c] + 0] = kk[c];
+      }
+    }
   }
 }
 
@@ -260,11 +346,20 @@ rs_vs_finish_kernel(IdxParams P) {
   if (tid < RS_PROBE_GROUPS) cov[tid] = 0;
   if (tid == 0) extra_pairs = 0;
   __syncthreads();
-  for (int i = tid; i < n_offs; i += blockDim.x) {
-    const int o = offs[i];
-    const int d0 = o >> 6, d1 = (o + 63) >> 6;
-    if (d0 < nbs) atomicOr(&dbits[d0 >> 5], 1u << (d0 & 31));
-    if (d1 < nbs) atomicOr(&dbits[d1 >> 5], 1u << (d1 & 31));
+  for (int base = 0; base < n_offs; base += 8 * (int)blockDim.x) {     // eight independent loads in flight per thread
+    int ob[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = base + u * (int)blockDim.x + tid;
+      ob[u] = (i < n_offs) ? offs[i] : -1;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (ob[u] < 0) continue;
+      const int d0 = ob[u] >> 6, d1 = (ob[u] + 63) >> 6;
+      if (d0 < nbs) atomicOr(&dbits[d0 >> 5], 1u << (d0 & 31));
+      if (d1 < nbs) atomicOr(&dbits[d1 >> 5], 1u << (d1 & 31));
+    }
   }
   __syncthreads();
   if (tid == 0) {
@@ -301,27 +396,43 @@ rs_vs_finish_kernel(IdxParams P) {
   // pairs: verticals not covered by a block diagonal of their query block
   u64 vp = 0;
   const bool has0 = (dbits[0] & 1u) != 0;
-  for (int i = tid; i < n_cols; i += blockDim.x) {
-    const int j = cols[i];
-    const int kbj = j >> 6;
-    const int d = qb_star - kbj;
-    if (!((dbits[d >> 5] >> (d & 31)) & 1u)) {
+  // number of block diagonals of D with delta <= x, from the per-word prefix counts
+  auto d_upto = [&](int x) -> int {
+    if (x < 0) return 0;
+    const int w = x >> 5;
+    return wpre[w] + __popc(dbits[w] & (0xffffffffu >> (31 - (x & 31))));
+  };
+  for (int base = 0; base < n_cols; base += 4 * (int)blockDim.x) {      // four independent load chains per thread
+    int jb[4];
 #pragma unroll
-      for (int g = 0; g < RS_PROBE_GROUPS; ++g) part[g] += fx(vert[(size_t)g * P.n + j]);
+    for (int u = 0; u < 4; ++u) {
+      const int i = base + u * (int)blockDim.x + tid;
+      jb[u] = (i < n_cols) ? cols[i] : -1;
     }
-    // query blocks qb in [max(kbj, qb_lo), nbs): delta = qb - kbj
-    if (kbj >= qb_lo && !has0) vp += (u64)((kbj + 1) * 64 - j);
-    const int d_lo = max(1, qb_lo - kbj), d_hi = qb_star - kbj;       // deltas >= 1 of the other query blocks
-    if (d_hi >= d_lo) {
-      int covered = 0;                                                 // |D intersect [d_lo, d_hi]|
-      const int w_lo = d_lo >> 5, w_hi = d_hi >> 5;
-      for (int w = w_lo; w <= w_hi; ++w) {
-        uint32_t bits = dbits[w];
-        if (w == w_lo) bits &= 0xffffffffu << (d_lo & 31);
-        if (w == w_hi) bits &= 0xffffffffu >> (31 - (d_hi & 31));
-        covered += __popc(bits);
+    float vb[4][RS_PROBE_GROUPS];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = max(jb[u], 0);
+#pragma unroll
+      for (int g = 0; g < RS_PROBE_GROUPS; ++g) vb[u][g] = vert[(size_t)g * P.n + j];
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = jb[u];
+      if (j < 0) continue;
+      const int kbj = j >> 6;
+      const int d = qb_star - kbj;
+      if (!((dbits[d >> 5] >> (d & 31)) & 1u)) {
+#pragma unroll
+        for (int g = 0; g < RS_PROBE_GROUPS; ++g) part[g] += fx(vb[u][g]);
       }
-      vp += 64ull * (u64)(d_hi - d_lo + 1 - covered);
+      // query blocks qb in [max(kbj, qb_lo), nbs): delta = qb - kbj
+      if (kbj >= qb_lo && !has0) vp += (u64)((kbj + 1) * 64 - j);
+      const int d_lo = max(1, qb_lo - kbj), d_hi = qb_star - kbj;     // deltas >= 1 of the other query blocks
+      if (d_hi >= d_lo) {
+        const int covered = d_upto(d_hi) - d_upto(d_lo - 1);          // |D intersect [d_lo, d_hi]|
+        vp += 64ull * (u64)(d_hi - d_lo + 1 - covered);
+      }
     }
   }
 #pragma unroll
@@ -728,7 +839,19 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   }
   if (any_vs && !skip_vs) {
     rs_vs_keys_kernel<<<dim3((P.n + 255) / 256, 2 * n_items), 256, 0, stream>>>(P);
-    rs_vs_select_kernel<<<dim3(2, n_jobs), kSelThreads, 0, stream>>>(P);
+    {
+      int n_vs = 0;
+      for (int c = 0; c < n_cand; ++c) n_vs += (lib[c].pattern == RS_VERTICAL_SLASH);
+      const int groups = choice ? 1 : (n_vs + kSelMaxC - 1) / kSelMaxC;
+      const size_t sel_smem = (size_t)(choice ? 1 : kSelMaxC) * kBins * sizeof(unsigned int);
+      static bool sel_attr = false;
+      if (!sel_attr) {
+        if (cudaFuncSetAttribute(rs_vs_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(kSelMaxC * kBins * sizeof(unsigned int))) != cudaSuccess) return RS_ERR_CUDA;
+        sel_attr = true;
+      }
+      rs_vs_select_kernel<<<dim3(2, n_items, groups), kSelThreads, sel_smem, stream>>>(P);
+    }
     rs_vs_finish_kernel<<<n_jobs, 256, 0, stream>>>(P);
   }
   if (stats != nullptr) rs_simple_stats_kernel<<<n_jobs, 256, 0, side>>>(P);
