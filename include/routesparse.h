@@ -131,8 +131,9 @@ int rs_workspace_bytes(const rs_problem* p, const rs_candidate* lib, int n_cand,
  * plus the pooled signals of the coarse block candidates and the value norms of Eq. 5:
  *   qpool [n_q_heads][n_keys/64][d], kpool [n_kv_heads][n_keys/64][d]  64-row means (fp32)
  *   vmax  [n_seg][n_kv_heads]   max_j ||v_j||_2 over j < segment end             (fp32)
- * vert and slash are fully overwritten.  descr (may be NULL) is reserved for the entropy /
- * local-concentration descriptors. */
+ * vert and slash are fully overwritten.  descr (may be NULL): [n_seg][n_q_heads][2], two of the descriptors of
+ * Section 3.2 on the exact probe rows: entropy (mean over the 64 rows of -sum_j p ln p, in nats) and local-band
+ * concentration (mean over the rows of the mass of keys with i - j < 1024). */
 int rs_probe(const rs_problem* p, const void* Q, const void* K, const void* V,
              float* vert, float* slash, float* lse_probe, float* qpool, float* kpool, float* vmax,
              float* descr, void* ws, size_t ws_bytes, int32_t* status, void* stream);

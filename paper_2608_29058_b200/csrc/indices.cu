@@ -831,6 +831,18 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   // The vertical-slash chain (keys, select, D / coverage / pairs) and the block-sparse chain (pooled scores, row
   // selection) do not read each other's results; both read the block sums above.  The second chain and the closed-form
   // statistics run on the side stream.
+  // launch shape of the select kernel; its attribute is set before the fork so that no error path sits between the
+  // fork and the join below
+  int n_vs = 0;
+  for (int c = 0; c < n_cand; ++c) n_vs += (lib[c].pattern == RS_VERTICAL_SLASH);
+  const int sel_groups = choice ? 1 : (n_vs + kSelMaxC - 1) / kSelMaxC;
+  const size_t sel_smem = (size_t)(choice ? 1 : kSelMaxC) * kBins * sizeof(unsigned int);
+  static bool sel_attr = false;
+  if (!sel_attr) {
+    if (cudaFuncSetAttribute(rs_vs_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(kSelMaxC * kBins * sizeof(unsigned int))) != cudaSuccess) return RS_ERR_CUDA;
+    sel_attr = true;
+  }
   const bool two_chains = any_vs && !skip_vs && (any_bs || stats != nullptr);
   cudaStream_t side = stream;
   if (two_chains) {
@@ -839,19 +851,7 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   }
   if (any_vs && !skip_vs) {
     rs_vs_keys_kernel<<<dim3((P.n + 255) / 256, 2 * n_items), 256, 0, stream>>>(P);
-    {
-      int n_vs = 0;
-      for (int c = 0; c < n_cand; ++c) n_vs += (lib[c].pattern == RS_VERTICAL_SLASH);
-      const int groups = choice ? 1 : (n_vs + kSelMaxC - 1) / kSelMaxC;
-      const size_t sel_smem = (size_t)(choice ? 1 : kSelMaxC) * kBins * sizeof(unsigned int);
-      static bool sel_attr = false;
-      if (!sel_attr) {
-        if (cudaFuncSetAttribute(rs_vs_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(kSelMaxC * kBins * sizeof(unsigned int))) != cudaSuccess) return RS_ERR_CUDA;
-        sel_attr = true;
-      }
-      rs_vs_select_kernel<<<dim3(2, n_items, groups), kSelThreads, sel_smem, stream>>>(P);
-    }
+    rs_vs_select_kernel<<<dim3(2, n_items, sel_groups), kSelThreads, sel_smem, stream>>>(P);
     rs_vs_finish_kernel<<<n_jobs, 256, 0, stream>>>(P);
   }
   if (stats != nullptr) rs_simple_stats_kernel<<<n_jobs, 256, 0, side>>>(P);

@@ -14,6 +14,7 @@
 
 namespace {
 
+constexpr int RS_LOCAL_BAND = 1024;     // keys with i - j below this count as the row's local band
 constexpr int kHC = 4;                 // head slots per CTA (4 x 64 = 256 probe rows)
 constexpr int kRows = kHC * RS_PROBE_ROWS;
 constexpr int kKeyTile = 128;
@@ -26,9 +27,10 @@ struct ProbeParams {
   int n, Hq, Hkv, group, n_seg, n_hc;  // n_hc = head chunks per KV head = ceil(group / 4)
   int seg_bounds[RS_MAX_SEGMENTS + 1];
   int n_splits;
-  float2* partial;    // [n_seg*Hkv*n_hc][n_splits][256] (max, sum) in the exp2 domain
+  float4* partial;    // [n_seg*Hkv*n_hc][n_splits][256] (max, sum, sum of p * score, sum of p inside the local band), exp2 domain
   float* lse2;        // [n_seg*Hkv*n_hc][256] log-sum-exp * log2(e)
   float* lse_probe;   // [Hq][n_seg][64]
+  float* descr;       // [n_seg][Hq][2] entropy and local-band mass, means over the 64 probe rows (may be NULL)
   float* vert;        // [n_seg][Hq][4][n]
   float* slash;       // [n_seg][Hq][4][n]
   int32_t* status;
@@ -103,7 +105,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (t0 >= t1) {   // nothing to do for this split (uniform across the CTA)
     if (PASS == 1) {
       for (int i = tid; i < kRows; i += kThreads)
-        P.partial[((size_t)unit * P.n_splits + blockIdx.x) * kRows + i] = make_float2(-INFINITY, 0.f);
+        P.partial[((size_t)unit * P.n_splits + blockIdx.x) * kRows + i] = make_float4(-INFINITY, 0.f, 0.f, 0.f);
     }
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
@@ -189,7 +191,9 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int r = quad * 32 + lane;                 // row inside the head pair (0..127)
       const int hh = part * 2 + (r >> 6);             // head slot
       const int i = i_first + (r & 63);               // global query row
+      const bool want_descr = P.descr != nullptr;
       float m_run = -INFINITY, l_run = 0.f;
+      float a_run = 0.f, loc_run = 0.f;               // sum of p * score and local-band sum of p (descriptors)
       for (int t = t0; t < t1; ++t) {
         const int it = t - t0, b = it & 1;
         ok = mbar_wait(bar_tfull[b], (uint32_t)(it >> 1) & 1u, abort_flag);
@@ -197,6 +201,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tc_fence_after();
         const int j0 = t * kKeyTile;
         const bool need_mask = j0 + kKeyTile - 1 > i_first;
+        const bool near = j0 + kKeyTile - 1 > i_first - RS_LOCAL_BAND;   // tile reaches into some row's local band
 #pragma unroll 1
         for (int c4 = 0; c4 < 4; ++c4) {
           tmem_ld32(tmem + lane_addr + (uint32_t)(b * 256 + part * 128 + c4 * 32), v);
@@ -209,19 +214,34 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             v[x] = __float_as_uint(sv);
             mx = fmaxf(mx, sv);
           }
-          if (mx > m_run) { l_run *= fast_exp2(m_run - mx); m_run = mx; }
+          if (mx > m_run) {
+            const float sc = fast_exp2(m_run - mx);
+            l_run *= sc; a_run *= sc; loc_run *= sc;
+            m_run = mx;
+          }
           if (m_run > -INFINITY) {
-            float acc = 0.f;
+            float acc = 0.f, acc_a = 0.f, acc_l = 0.f;
+            if (want_descr) {
 #pragma unroll
-            for (int x = 0; x < 32; ++x) acc += fast_exp2(__uint_as_float(v[x]) - m_run);
-            l_run += acc;
+              for (int x = 0; x < 32; ++x) {
+                const float sv = __uint_as_float(v[x]);
+                const float pe = fast_exp2(sv - m_run);
+                acc += pe;
+                acc_a = fmaf(pe, fmaxf(sv, -1e30f), acc_a);          // masked entries: pe = 0, keep the product finite
+                if (near && i - (j0 + c4 * 32 + x) < RS_LOCAL_BAND) acc_l += pe;
+              }
+            } else {
+#pragma unroll
+              for (int x = 0; x < 32; ++x) acc += fast_exp2(__uint_as_float(v[x]) - m_run);
+            }
+            l_run += acc; a_run += acc_a; loc_run += acc_l;
           }
         }
         tc_fence_before();
         mbar_arrive(bar_tempty[b]);
       }
       if (ok) {
-        P.partial[((size_t)unit * P.n_splits + blockIdx.x) * kRows + hh * 64 + (r & 63)] = make_float2(m_run, l_run);
+        P.partial[((size_t)unit * P.n_splits + blockIdx.x) * kRows + hh * 64 + (r & 63)] = make_float4(m_run, l_run, a_run, loc_run);
       }
     } else {
       // Sixteen warps: warp (quad, hh) owns 32 keys of the tile (its TMEM lanes) and the 64 probe rows of head slot hh.
@@ -315,19 +335,37 @@ __global__ void rs_probe_merge_kernel(ProbeParams P) {
   const int g = (unit / P.n_hc) % P.Hkv;
   const int s = unit / (P.n_hc * P.Hkv);
   const int hh = row >> 6;
-  const float2* part = P.partial + (size_t)unit * P.n_splits * kRows + row;
+  const float4* part = P.partial + (size_t)unit * P.n_splits * kRows + row;
   float m = -INFINITY;
   for (int k = 0; k < P.n_splits; ++k) m = fmaxf(m, part[(size_t)k * kRows].x);
-  float l = 0.f;
+  float l = 0.f, a = 0.f, loc = 0.f;
   for (int k = 0; k < P.n_splits; ++k) {
-    const float2 pk = part[(size_t)k * kRows];
-    if (pk.x > -INFINITY) l += pk.y * exp2f(pk.x - m);
+    const float4 pk = part[(size_t)k * kRows];
+    if (pk.x > -INFINITY) {
+      const float sc = exp2f(pk.x - m);
+      l += pk.y * sc; a += pk.z * sc; loc += pk.w * sc;
+    }
   }
   const float lse2 = m + log2f(l);
   P.lse2[(size_t)unit * kRows + row] = lse2;
-  if (hc * kHC + hh < P.group) {
+  const bool live = hc * kHC + hh < P.group;
+  if (live) {
     const int h = g * P.group + hc * kHC + hh;
     P.lse_probe[((size_t)h * P.n_seg + s) * RS_PROBE_ROWS + (row & 63)] = lse2 * 0.6931471805599453f;
+  }
+  if (P.descr != nullptr) {
+    // H_i = -sum p ln p = ln 2 * (lse2 - E_p[score2]); local mass = local sum / l; then the mean over the head's 64 rows
+    __shared__ float sh[kRows][2];
+    sh[row][0] = 0.6931471805599453f * (lse2 - a / l);
+    sh[row][1] = loc / l;
+    __syncthreads();
+    if ((row & 63) == 0 && live) {
+      float e = 0.f, lc = 0.f;
+      for (int r = 0; r < 64; ++r) { e += sh[row + r][0]; lc += sh[row + r][1]; }
+      const int h = g * P.group + hc * kHC + hh;
+      P.descr[((size_t)s * P.Hq + h) * 2 + 0] = e * (1.0f / 64.0f);
+      P.descr[((size_t)s * P.Hq + h) * 2 + 1] = lc * (1.0f / 64.0f);
+    }
   }
 }
 
@@ -429,7 +467,7 @@ ProbePlan plan(const rs_problem* p) {
   if (splits > 64) splits = 64;
   w.n_splits = splits;
   size_t off = 0;
-  w.partial = off;  off += rs_align_up((size_t)w.n_units * splits * kRows * sizeof(float2), 256);
+  w.partial = off;  off += rs_align_up((size_t)w.n_units * splits * kRows * sizeof(float4), 256);
   w.lse2 = off;     off += rs_align_up((size_t)w.n_units * kRows * sizeof(float), 256);
   w.blockmax = off; off += rs_align_up((size_t)p->n_kv_heads * (p->n_keys / 64) * sizeof(float), 256);
   w.total = off;
@@ -443,7 +481,6 @@ size_t rs_probe_workspace_bytes(const rs_problem* p) { return plan(p).total; }
 extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const void* V, float* vert, float* slash,
                         float* lse_probe, float* qpool, float* kpool, float* vmax, float* descr, void* ws,
                         size_t ws_bytes, int32_t* status, void* stream_) {
-  (void)descr;
   int rc = rs_check_problem(p);
   if (rc != RS_OK) return rc;
   if (!Q || !K || !V || !vert || !slash || !lse_probe || !ws) return RS_ERR_INVALID_ARG;
@@ -461,7 +498,8 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
   P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = P.Hq / P.Hkv;
   P.n_seg = p->n_segments; P.n_hc = w.n_hc; P.n_splits = w.n_splits;
   for (int s = 0; s <= p->n_segments; ++s) P.seg_bounds[s] = p->seg_bounds[s];
-  P.partial = reinterpret_cast<float2*>(wsb + w.partial);
+  P.partial = reinterpret_cast<float4*>(wsb + w.partial);
+  P.descr = descr;
   P.lse2 = reinterpret_cast<float*>(wsb + w.lse2);
   P.lse_probe = lse_probe; P.vert = vert; P.slash = slash; P.status = status;
   P.scale_log2e = (float)(1.4426950408889634 / sqrt((double)RS_HEAD_DIM));

@@ -65,3 +65,25 @@ def test_probe_is_deterministic():
     a, b = run_probe(L, p), run_probe(L, p)
     for k in a:
         assert np.array_equal(a[k], b[k]), k
+
+
+def test_probe_descriptors_match_oracle():
+    """descr output of rs_probe: entropy and local-band mass of the exact probe rows (Section 3.2)."""
+    for n, Hq, Hkv, bounds in ((2304, 4, 2, None), (1088, 4, 2, [0, 320, 1088]), (2048 + 1280, 2, 1, None)):
+        L = make_layer(tiny_spec(55 + n, n, Hq, Hkv))
+        p = rs.Problem(Hq, Hkv, n, bounds or [0, n])
+        Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+        S = p.n_segments
+        f32 = dict(dtype=torch.float32, device="cuda")
+        vert = torch.zeros((S, Hq, 4, n), **f32); slash = torch.zeros((S, Hq, 4, n), **f32)
+        lse = torch.zeros((Hq, S, 64), **f32); descr = torch.full((S, Hq, 2), -1.0, **f32)
+        st = rs.new_status()
+        rs.rs_probe(p, Q, K, V, vert, slash, lse, None, None, None, descr, rs.new_workspace(p, None), st)
+        rs.check_status(st, "probe with descriptors")
+        got = descr.cpu().numpy()
+        Qs, Ks, _ = f64_heads(L)
+        for s in range(S):
+            for h in range(Hq):
+                pr = OP.probe_rows(Qs[h], Ks[h // (Hq // Hkv)], p.seg_bounds[s + 1])
+                assert abs(got[s, h, 0] - pr.entropy) < 2e-3 * max(1.0, pr.entropy), (n, s, h, got[s, h, 0], pr.entropy)
+                assert abs(got[s, h, 1] - pr.local_conc) < 1e-3, (n, s, h, got[s, h, 1], pr.local_conc)
