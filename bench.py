@@ -226,6 +226,8 @@ def main():
                     help="also time the attention stage as one launch per KV group and as one launch per head")
     ap.add_argument("--ablations", action="store_true",
                     help="router ablations of the paper's Table 3 on the config-3 layer, JSONL output")
+    ap.add_argument("--mixture", action="store_true",
+                    help="u of Eq. 4 = disagreement among the recent / uniform / boundary rows of the query mixture (pooled probe)")
     ap.add_argument("--graph", action="store_true",
                     help="also time the layer replayed from a CUDA graph (whole pass captured once; for launch-bound sizes)")
     ap.add_argument("--sweep", action="store_true", help="config-5 sweep: n x budget x forced-dense cells, JSONL output")
@@ -269,7 +271,7 @@ def main():
     to_dev = lambda bits: torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
     Q, K, V = to_dev(L["Q"]), to_dev(L["K"]), to_dev(L["V"])
     p = rs.Problem(spec.n_q_heads, spec.n_kv_heads, spec.n, [int(x) for x in L["seg_bounds"]])
-    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(rescue_any=args.rescue, **route_kw), device=dev)
+    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(rescue_any=args.rescue, mixture_u=args.mixture, **route_kw), device=dev)
     risk_calibration = None
     if args.calibration:
         with open(args.calibration) as f:
@@ -476,7 +478,7 @@ def main():
         "routes": hist, "route_report": layer.route_report() if not fixed else None,
         "cost_model": args.cost, "calibration": calibration, "risk_calibration": risk_calibration, "launch_ablation": launch_ablation,
         "cuda_graph_ms_per_layer": graph_ms,
-        "fallback_rescue": bool(args.rescue),
+        "fallback_rescue": bool(args.rescue), "mixture_uncertainty": bool(args.mixture),
         "roofline": {"kernel": "rs_attn_kernel (one launch, all heads)", "bound": "tensor", "achieved": achieved,
                      "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": f"bf16_tflops_sustained, {peaks['source']}",
@@ -614,6 +616,8 @@ def ablations(args):
         ("per-head launches", None, rs.RouteConfig(**base), {"per_head": True}),
         ("fallback rescue (any family before dense)", None, rs.RouteConfig(rescue_any=True, **base), {}),
         ("greedy back-fill of leftover budget", None, rs.RouteConfig(backfill=True, **base), {}),
+        ("uncertainty from recent / uniform / boundary rows (query mixture)", None, rs.RouteConfig(mixture_u=True, **base), {}),
+        ("the same with alpha = 4", None, rs.RouteConfig(mixture_u=True, alpha=4.0, **base), {}),
     ]
     rows = []
     with open(path, "w") as f:

@@ -112,6 +112,11 @@ typedef struct {
   int32_t backfill;        /* 1: after the greedy solve, spend what is left of the budget on the substitutions with
                               the largest risk decrease per unit of added cost that still fit (before the fallback) */
   int32_t reserved2;       /* 0 */
+  const uint64_t* cov_mix; /* device uint64[n_items][n_cand][4] from rs_mixture_coverage, or NULL.  When set, u of Eq. 4
+                              is the disagreement among the row subsets of the query mixture, max_b m_b - min_b m_b with
+                              m_b = cov_mix[..][b] / (mix_rows[b] * 2^32), instead of the spread over the four groups of
+                              the last 64 rows */
+  int32_t mix_rows[4];     /* rows per subset (0 = subset unused) */
 } rs_route_params;
 
 typedef struct { int64_t total_cost; double total_risk; int32_t n_fallback; int32_t feasible; } rs_route_report;
@@ -233,6 +238,21 @@ int rs_probe_pooled_scratch_floats(const rs_problem* p, int r, size_t* n_floats)
 int rs_probe_pooled(const rs_problem* p, const void* Q, const void* K, const int32_t* rows, int r, int g,
                     const int32_t* sub_bounds, int n_sub, float* A, float* lse, float* colmass, float* diagmass,
                     float* descr, float* scratch, int32_t* status, void* stream);
+
+/* Coverage of every candidate's mask on the rows of the query mixture (Section 3.2), the input of the "disagreement
+ * among probe subsets" u of Eq. 4.  A comes from rs_probe_pooled at g = 64 (key blocks = the pattern blocks); the mass of
+ * a key block is split evenly over its visible keys, so row i of candidate c collects
+ *   sum over key blocks kb of  floor(A[i][kb] * 2^32) * num_c(i, kb) / den(i, kb)      (integer arithmetic)
+ * with den = visible keys of the block (j <= i) and num = how many of them the candidate's mask row i selects
+ * (A-shape: closed form; vertical-slash: all if the block diagonal is in D, else the selected columns of the block;
+ * block-sparse: all if the block is among the top-k_b pooled scores of the row's query block; dense: all).
+ *   idx_eval   the evaluation-layout index set written by rs_build_indices(choice = NULL)
+ *   covmix     device uint64 [n_items][n_cand][4] out: the sums per row subset (cleared by the call)
+ * rows, r, sub_bounds, n_sub as for rs_probe_pooled. */
+int rs_mixture_coverage(const rs_problem* p, const rs_candidate* lib, int n_cand, const float* A,
+                        const int32_t* rows, int r, const int32_t* sub_bounds, int n_sub,
+                        const rs_index_set* idx_eval, const float* qpool, const float* kpool,
+                        uint64_t* covmix, int32_t* status, void* stream);
 
 /* Calibrated predictor e of Eq. 4 (Section 3.3: "a small monotone regressor fitted offline from dense calibration
  * runs; it consumes only the probe descriptors and candidate metadata").  The form used here, this library's choice:

@@ -241,3 +241,24 @@ def default_library() -> List[Candidate]:
     lib += [Candidate(BLOCK_SPARSE, kb) for kb in (50, 100, 200, 400)]
     lib += [Candidate(DENSE)]
     return lib
+
+
+def mixture_coverage_fx(ix: IndexSet, a_row: np.ndarray, i: int, n_keys: int) -> int:
+    """Coverage of mask row i under the pooled probe's block resolution (Section 3.2 mixture rows): the probability of
+    every visible key block (a_row, float32, 64 keys per block) is split evenly over the block's visible keys, and the
+    row collects floor(a * 2^32) * (selected visible keys) // (visible keys) per block.  Plain definition: the mask row
+    itself is built and counted key by key."""
+    m = mask_rows(ix, np.array([i]), n_keys)[0]
+    m = m & (np.arange(n_keys) <= i)
+    total = 0
+    for kb in range(i // B + 1):
+        lo, hi = kb * B, min(kb * B + B - 1, i)
+        num = int(m[lo:hi + 1].sum())
+        total += int(fx(np.float32(a_row[kb]))) * num // (hi - lo + 1)
+    return total
+
+
+def mixture_u(covmix: np.ndarray, rows_per_subset) -> float:
+    """max_b m_b - min_b m_b with m_b = covmix[b] / (rows_b * 2^32) over the subsets in use."""
+    ms = [float(int(covmix[b])) / (float(r) * float(FX_ONE)) for b, r in enumerate(rows_per_subset) if r > 0]
+    return max(ms) - min(ms)

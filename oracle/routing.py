@@ -42,6 +42,7 @@ class RouteParams:
     expand_first: bool = True        # try the next larger budget of the family before dense
     rescue_any: bool = False         # before dense, take the cheapest sparse candidate of any family that passes
     backfill: bool = False           # spend leftover budget on the best risk decrease per added cost (before fallback)
+    u_mix: Optional[np.ndarray] = None   # [items, n_cand] disagreement among the mixture's row subsets (replaces u)
     forced_dense: Sequence[int] = field(default_factory=list)   # items forced to dense last
     fixed_choice: Optional[Sequence[int]] = None                 # bypasses the solve and the fallback
 
@@ -54,7 +55,8 @@ class RouteReport:
     feasible: int
 
 
-def risks(lib: List[Candidate], cov_fx: np.ndarray, alpha: float, beta: float = 0.0, e: Optional[np.ndarray] = None):
+def risks(lib: List[Candidate], cov_fx: np.ndarray, alpha: float, beta: float = 0.0, e: Optional[np.ndarray] = None,
+          u_mix: Optional[np.ndarray] = None):
     """R[item][c] = (1 - m_hat) + alpha * u + beta * e (Eq. 4); dense has m_hat = 1, u = 0, e = 0, R = 0."""
     n_items, n_cand = cov_fx.shape[0], len(lib)
     R = np.zeros((n_items, n_cand), dtype=np.float64)
@@ -64,6 +66,8 @@ def risks(lib: List[Candidate], cov_fx: np.ndarray, alpha: float, beta: float = 
             if cand.pattern == DENSE:
                 continue
             m_hat, u = m_hat_from_fx(cov_fx[it, c])
+            if u_mix is not None:
+                u = float(u_mix[it, c])
             M[it, c] = m_hat
             R[it, c] = (1.0 - m_hat) + alpha * u
             if e is not None and beta != 0.0:
@@ -143,7 +147,7 @@ def route(lib: List[Candidate], cov_fx: np.ndarray, cost: np.ndarray, vmax: np.n
     """Full routing of one layer. cov_fx[items, n_cand, 4] uint64, cost[items, n_cand] int64, vmax[items] fp32."""
     n_items = cov_fx.shape[0]
     dense_c = _dense_index(lib)
-    R, M = risks(lib, cov_fx, p.alpha, p.beta, p.e)
+    R, M = risks(lib, cov_fx, p.alpha, p.beta, p.e, p.u_mix)
     n_fallback = 0
     if p.fixed_choice is not None:
         choice = [int(c) for c in p.fixed_choice]

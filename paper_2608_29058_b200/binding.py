@@ -43,13 +43,13 @@ class rs_route_params(C.Structure):
                 ("cert_max", C.c_double), ("use_cert", C.c_int32), ("cert_mode", C.c_int32),
                 ("expand_first", C.c_int32), ("reserved", C.c_int32),
                 ("forced_dense", C.c_void_p), ("fixed_choice", C.c_void_p), ("e", C.c_void_p), ("beta", C.c_double),
-                ("backfill", C.c_int32), ("reserved2", C.c_int32)]
+                ("backfill", C.c_int32), ("reserved2", C.c_int32), ("cov_mix", C.c_void_p), ("mix_rows", C.c_int32 * 4)]
 
 
 EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "rs_build_indices", "rs_route",
            "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate",
            "rs_selftest_wait_timeout", "rs_probe_pooled", "rs_probe_pooled_scratch_floats", "rs_regressor_eval",
-           "rs_output_error"]
+           "rs_output_error", "rs_mixture_coverage"]
 
 
 def lib_path() -> str:
@@ -249,6 +249,15 @@ def rs_probe_pooled(p: Problem, Q, K, rows, g: int, sub_bounds, A, lse, colmass,
     _check(load().rs_probe_pooled(C.byref(p.c), _ptr(Q), _ptr(K), _ptr(rows), r, int(g), sb, len(sub_bounds) - 1,
                                   _ptr(A), _ptr(lse), _ptr(colmass), _ptr(diagmass), _ptr(descr), _ptr(scratch),
                                   _ptr(status), _stream()), "rs_probe_pooled")
+
+
+def rs_mixture_coverage(p: Problem, lib, A, rows, sub_bounds, idx_eval, qpool, kpool, covmix, status):
+    """A: pooled-probe probabilities at g = 64; rows: device int32 [n_seg][r]; covmix: device int64/uint64 [items][cands][4]."""
+    r = int(rows.shape[-1])
+    sb = (C.c_int32 * len(sub_bounds))(*[int(x) for x in sub_bounds])
+    _check(load().rs_mixture_coverage(C.byref(p.c), lib, len(lib), _ptr(A), _ptr(rows), r, sb, len(sub_bounds) - 1,
+                                      C.byref(idx_eval.c), _ptr(qpool), _ptr(kpool), _ptr(covmix), _ptr(status),
+                                      _stream()), "rs_mixture_coverage")
 
 
 def rs_regressor_eval(p: Problem, lib, stats, descr, w, bp_z, bp_e, e_out, status):

@@ -739,6 +739,102 @@ rs_bs_scores_kernel(IdxParams P) {
   }
 }
 
+// ------------------------------------------------------------------------------------------ mixture coverage
+// Coverage of every candidate's mask on the rows of the query mixture (Section 3.2, Eq. 4: "u measures disagreement
+// among probe subsets").  The pooled probe resolves key blocks of 64, so the mass of a block is split evenly over its
+// visible keys: row i of candidate c collects  sum_kb  fx(A[i][kb]) * num_c(i, kb) / den(i, kb)  with den the number of
+// visible keys of the block (j <= i) and num how many of them the candidate's mask row selects; integer arithmetic, so
+// the sums do not depend on the order of evaluation.  One block per (probe row, item); candidates in a loop.
+struct MixArgs {
+  const float* A;          // [n_seg][Hq][r][nb] probabilities of the pooled probe at g = 64
+  const int32_t* rows;     // [n_seg][r]
+  int r, n_sub;
+  int sub_bounds[5];
+  u64* covmix;             // [n_items][n_cand][4]
+};
+
+__device__ __forceinline__ int interval_len(int lo, int hi) { return hi >= lo ? hi - lo + 1 : 0; }
+
+__global__ void __launch_bounds__(256)
+rs_mix_cov_kernel(IdxParams P, MixArgs M) {
+  extern __shared__ float mix_smem[];                    // score[nb] | vcnt[nb] | list[kb_cap]
+  float* score = mix_smem;
+  int* vcnt = reinterpret_cast<int*>(mix_smem + P.nb);
+  int32_t* blist = reinterpret_cast<int32_t*>(vcnt + P.nb);
+  __shared__ uint32_t dbits[128];
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t sh[8];
+  __shared__ unsigned int wcnt[16];
+  __shared__ u64 red[8];
+  __shared__ float qrow[RS_HEAD_DIM];
+  const int t = blockIdx.x, item = blockIdx.y;
+  const int s = item / P.Hq, h = item - s * P.Hq, g = h / P.group;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int i = M.rows[s * M.r + t];
+  const int qb_i = i >> 6;
+  int sub = 0;
+  while (sub + 1 < M.n_sub && t >= M.sub_bounds[sub + 1]) ++sub;
+  const float* a = M.A + (((size_t)s * P.Hq + h) * M.r + t) * (size_t)P.nb;
+  bool have_scores = false;
+  for (int c = 0; c < P.n_cand; ++c) {
+    const rs_candidate cand = P.lib[c];
+    const int slot = item * P.n_cand + c;
+    u64 part = 0;
+    if (cand.pattern == RS_DENSE) {
+      for (int kb = tid; kb <= qb_i; kb += 256) part += fx(a[kb]);
+    } else if (cand.pattern == RS_A_SHAPE) {
+      const int n_sink = cand.b0, w = cand.b1;
+      for (int kb = tid; kb <= qb_i; kb += 256) {
+        const int lo = kb * 64, hi = min(lo + 63, i);
+        const int s_hi = min(hi, n_sink - 1), w_lo = max(lo, i - w + 1);
+        const int num = interval_len(lo, s_hi) + interval_len(w_lo, hi) - interval_len(w_lo, s_hi);
+        part += fx(a[kb]) * (u64)num / (u64)(hi - lo + 1);
+      }
+    } else if (cand.pattern == RS_VERTICAL_SLASH) {
+      const int n_cols = P.out.vs_count[4 * slot + 0], n_diag = P.out.vs_count[4 * slot + 2];
+      const int32_t* cols = P.out.vs_cols + (size_t)slot * P.out.kv_cap;
+      const int32_t* diag = P.out.vs_diag + (size_t)slot * P.out.nd_cap;
+      __syncthreads();
+      for (int x = tid; x < 128; x += 256) dbits[x] = 0;
+      for (int kb = tid; kb <= qb_i; kb += 256) vcnt[kb] = 0;
+      __syncthreads();
+      for (int x = tid; x < n_diag; x += 256) { const int d = diag[x]; atomicOr(&dbits[d >> 5], 1u << (d & 31)); }
+      for (int x = tid; x < n_cols; x += 256) { const int j = cols[x]; if (j <= i) atomicAdd(&vcnt[j >> 6], 1); }
+      __syncthreads();
+      for (int kb = tid; kb <= qb_i; kb += 256) {
+        const int lo = kb * 64, hi = min(lo + 63, i);
+        const int d = qb_i - kb;
+        const int den = hi - lo + 1;
+        const int num = ((dbits[d >> 5] >> (d & 31)) & 1u) ? den : vcnt[kb];
+        part += fx(a[kb]) * (u64)num / (u64)den;
+      }
+    } else {   // block-sparse: the row's query block selects like the materialising kernel does
+      __syncthreads();
+      if (!have_scores) {
+        if (tid < RS_HEAD_DIM) qrow[tid] = P.qpool[((size_t)h * P.nb + qb_i) * RS_HEAD_DIM + tid];
+        __syncthreads();
+        for (int kb = tid; kb < qb_i; kb += 256)
+          score[kb] = pooled_score(qrow, P.kpool + ((size_t)g * P.nb + kb) * RS_HEAD_DIM, P.scale);
+        have_scores = true;
+        __syncthreads();
+      }
+      const int k_b = min(cand.b0, P.out.kb_cap);
+      const int cnt = select_row(score, qb_i, min(k_b, qb_i + 1) - 1, qb_i, blist, P.out.kb_cap, hist, sh, wcnt);
+      for (int x = tid; x < cnt; x += 256) part += fx(a[blist[x]]);
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+    __syncthreads();
+    if (lane == 0) red[warp] = part;
+    __syncthreads();
+    if (tid == 0) {
+      u64 tot = 0;
+      for (int w8 = 0; w8 < 8; ++w8) tot += red[w8];
+      atomicAdd(&M.covmix[(size_t)slot * 4 + sub], tot);
+    }
+  }
+}
+
 struct IdxPlan { size_t vblk, bs_ws, keys, bs_eval, total; };
 
 IdxPlan plan(const rs_problem* p, const rs_candidate* lib, int n_cand) {
@@ -872,5 +968,51 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
     rc = rs_side_join(stream);
     if (rc != RS_OK) return rc;
   }
+  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+}
+
+extern "C" int rs_mixture_coverage(const rs_problem* p, const rs_candidate* lib, int n_cand, const float* A,
+                                   const int32_t* rows, int r, const int32_t* sub_bounds, int n_sub,
+                                   const rs_index_set* idx_eval, const float* qpool, const float* kpool,
+                                   uint64_t* covmix, int32_t* status, void* stream_) {
+  int rc = rs_check_problem(p);
+  if (rc != RS_OK) return rc;
+  if (!lib || n_cand <= 0 || n_cand > RS_MAX_CANDIDATES || !A || !rows || !sub_bounds || !idx_eval || !covmix)
+    return RS_ERR_INVALID_ARG;
+  if (r < 1 || r > 64 || n_sub < 1 || n_sub > 4 || sub_bounds[0] != 0 || sub_bounds[n_sub] != r) return RS_ERR_INVALID_ARG;
+  const int n_items = p->n_segments * p->n_q_heads;
+  const int nb = p->n_keys / 64;
+  bool any_vs = false, any_bs = false;
+  for (int c = 0; c < n_cand; ++c) {
+    any_vs |= lib[c].pattern == RS_VERTICAL_SLASH;
+    any_bs |= lib[c].pattern == RS_BLOCK_SPARSE;
+  }
+  if (any_vs && idx_eval->n_vs_slots < n_items * n_cand) return RS_ERR_INVALID_ARG;   // needs the evaluation layout
+  if (any_bs && (!qpool || !kpool)) return RS_ERR_INVALID_ARG;
+  rc = rs_check_device();
+  if (rc != RS_OK) return rc;
+  (void)status;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  IdxParams P{};
+  P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = P.Hq / P.Hkv; P.n_seg = p->n_segments;
+  P.n_cand = n_cand; P.nb = nb;
+  for (int s = 0; s <= p->n_segments; ++s) P.seg_bounds[s] = p->seg_bounds[s];
+  for (int c = 0; c < n_cand; ++c) P.lib[c] = lib[c];
+  P.qpool = qpool; P.kpool = kpool; P.out = *idx_eval;
+  P.scale = (float)(1.0 / sqrt((double)RS_HEAD_DIM));
+  MixArgs M{};
+  M.A = A; M.rows = rows; M.r = r; M.n_sub = n_sub;
+  for (int k = 0; k <= n_sub; ++k) M.sub_bounds[k] = sub_bounds[k];
+  M.covmix = reinterpret_cast<u64*>(covmix);
+  if (cudaMemsetAsync(covmix, 0, (size_t)n_items * n_cand * 4 * sizeof(uint64_t), stream) != cudaSuccess) return RS_ERR_CUDA;
+  const size_t smem = (size_t)nb * 8 + (size_t)(idx_eval->kb_cap > 0 ? idx_eval->kb_cap : 1) * 4;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(rs_mix_cov_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
+      return RS_ERR_CUDA;
+    attr_set = true;
+  }
+  if (smem > 64 * 1024) return RS_ERR_UNSUPPORTED_SHAPE;
+  rs_mix_cov_kernel<<<dim3(r, n_items), 256, smem, stream>>>(P, M);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }

@@ -69,7 +69,22 @@ __device__ __forceinline__ double risk_of(const RouteArgs& A, int item, int c) {
     mx = fmax(mx, mg);
     mn = fmin(mn, mg);
   }
-  const double u = __dsub_rn(mx, mn);
+  double u = __dsub_rn(mx, mn);
+  if (A.prm.cov_mix != nullptr) {
+    // disagreement among the row subsets of the query mixture
+    const uint64_t* cm = A.prm.cov_mix + ((size_t)item * A.n_cand + c) * 4;
+    double hi = 0.0, lo = 2.0;
+    bool any = false;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      if (A.prm.mix_rows[b] <= 0) continue;
+      const double mb = (double)cm[b] / ((double)A.prm.mix_rows[b] * 4294967296.0);
+      hi = fmax(hi, mb);
+      lo = fmin(lo, mb);
+      any = true;
+    }
+    if (any) u = __dsub_rn(hi, lo);
+  }
   double r = __dadd_rn(__dsub_rn(1.0, m_hat_of(A, item, c)), __dmul_rn(A.prm.alpha, u));
   if (A.prm.e != nullptr && A.prm.beta != 0.0) r = __dadd_rn(r, __dmul_rn(A.prm.beta, A.prm.e[(size_t)item * A.n_cand + c]));
   return r;

@@ -46,6 +46,7 @@ class RouteConfig:
     rescue_any: bool = False           # before dense, the cheapest sparse candidate of any family that passes
     beta: float = 0.0                  # weight of the calibrated predictor e of Eq. 4 (needs use_calibration())
     backfill: bool = False             # spend leftover budget on the best risk decrease per added cost
+    mixture_u: bool = False            # u of Eq. 4 from the recent / uniform / boundary rows of the query mixture
 
 
 class _IdxView:
@@ -103,6 +104,7 @@ class RoutedPrefillLayer:
         self.prm = rs.rs_route_params()
         self._forced = None
         self.events = None
+        self.covmix = torch.zeros((p.n_items, len(self.cands), 4), dtype=torch.int64, device=device)
         self.regressor = None       # dict(w, bp_z, bp_e, g) from calibrate(); used when cfg.beta > 0
         self.e_risk = torch.zeros((p.n_items, len(self.cands)), dtype=torch.float64, device=device)
         self.cost_table = None      # int64 [n_items, n_cand] measured kernel time (ns); None: FLOPs of the selected pairs
@@ -131,6 +133,13 @@ class RoutedPrefillLayer:
         prm.cert_mode, prm.expand_first = c.cert_mode, int(c.expand_first)
         prm.reserved = int(c.rescue_any)
         prm.backfill = int(c.backfill)
+        if c.mixture_u and getattr(self, "_pp_key", None) is not None:
+            prm.cov_mix = self.covmix.data_ptr()
+            sub = self.pp["sub"]
+            for b in range(4):
+                prm.mix_rows[b] = (sub[b + 1] - sub[b]) if b + 1 < len(sub) else 0
+        else:
+            prm.cov_mix = None
         use_e = self.regressor is not None and c.beta > 0.0
         prm.e = self.e_risk.data_ptr() if use_e else None
         prm.beta = float(c.beta) if use_e else 0.0
@@ -266,6 +275,15 @@ class RoutedPrefillLayer:
         if beta is not None:
             self.cfg.beta = float(beta)
 
+    def mixture_coverage(self, Q, K):
+        """Coverage of every candidate on the rows of the query mixture (pooled probe at g = 64), the input of the
+        subset-disagreement u of Eq. 4; needs evaluate_candidates()."""
+        self.pooled_probe(Q, K, g=64)
+        pp = self.pp
+        rs.rs_mixture_coverage(self.p, self.lib, pp["A"], pp["rows"], pp["sub"], self.idx_eval, self.qpool, self.kpool,
+                               self.covmix, self.status)
+        return self.covmix
+
     def predict_error(self, Q, K):
         """Descriptors (pooled mixture probe) and the predictor e for every (item, candidate); needs evaluate_candidates()."""
         r = self.regressor
@@ -284,6 +302,8 @@ class RoutedPrefillLayer:
         mark(1)
         if fixed_choice is None:
             self.evaluate_candidates()
+            if self.cfg.mixture_u:
+                self.mixture_coverage(Q, K)
             if self.regressor is not None and self.cfg.beta > 0.0:
                 self.predict_error(Q, K)
             mark(2)

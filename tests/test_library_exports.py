@@ -42,7 +42,7 @@ def test_host_side_calls_without_a_gpu():
 
 def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(rs.rs_candidate) == 16
-    assert ctypes.sizeof(rs.rs_route_params) == 96
+    assert ctypes.sizeof(rs.rs_route_params) == 120
     assert ctypes.sizeof(rs.rs_index_set) == 24 + 6 * 8
     assert rs.rs_route_params.forced_dense.offset == 56
 

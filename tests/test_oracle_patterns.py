@@ -166,3 +166,28 @@ def test_default_library_shape():
     lib = PT.default_library()
     assert len(lib) == 13 and lib[-1].pattern == PT.DENSE
     assert [c.pattern for c in lib].count(PT.VERTICAL_SLASH) == 4
+
+
+def test_mixture_coverage_closed_cases():
+    """Coverage of mask rows at the pooled probe's block resolution: dense collects everything, a window that ends on
+    block boundaries collects exactly its blocks, a half-covered block collects half of its mass."""
+    from oracle.patterns import A_SHAPE, DENSE, VERTICAL_SLASH, Candidate, build_indices, fx, mixture_coverage_fx, mixture_u
+    n = 512
+    a = np.zeros(n // 64, dtype=np.float32)
+    a[:] = [0.25, 0.03125, 0.125, 0.0625, 0.03125, 0.125, 0.125, 0.25]
+    i = 447                                                         # last row of block 6: blocks 0..6 fully visible
+    dense = build_indices(Candidate(DENSE), 0, n)
+    assert mixture_coverage_fx(dense, a, i, n) == int(fx(a[:7]).sum())
+    win = build_indices(Candidate(A_SHAPE, 64, 128), 0, n)          # sink = block 0, window = keys 320..447 = blocks 5, 6
+    assert mixture_coverage_fx(win, a, i, n) == int(fx(a[[0, 5, 6]]).sum())
+    half = build_indices(Candidate(A_SHAPE, 32, 96), 0, n)          # half of block 0, keys 352..447 = half of block 5 + block 6
+    assert mixture_coverage_fx(half, a, i, n) == int(fx(a[0])) * 32 // 64 + int(fx(a[5])) * 32 // 64 + int(fx(a[6]))
+    # a row in the middle of a block: window = keys 74..201 = 54 keys of block 1, block 2, the 10 visible keys of block 3
+    i2 = 64 * 3 + 9
+    assert mixture_coverage_fx(win, a, i2, n) == int(fx(a[0])) + int(fx(a[1])) * 54 // 64 + int(fx(a[2])) + int(fx(a[3]))
+    # vertical-slash: columns count individually, block diagonals cover whole blocks
+    from oracle.patterns import IndexSet
+    vs = IndexSet(cand=Candidate(VERTICAL_SLASH, 2, 2), q0=0, q1=n, V=np.array([70, 71]), S=np.array([0, 1]),
+                  D=np.array([0, 1]))                           # two columns in block 1, block diagonals 0 and 1
+    assert mixture_coverage_fx(vs, a, i, n) == int(fx(a[1])) * 2 // 64 + int(fx(a[5])) + int(fx(a[6]))
+    assert abs(mixture_u(np.array([2 ** 32 * 16, 2 ** 32 * 8, 2 ** 32 * 12, 0], dtype=np.uint64), [32, 16, 16, 0]) - 0.25) < 1e-15
