@@ -577,10 +577,19 @@ __device__ int select_row(const float* score, int m, int take, int qb, int32_t* 
   return take + 1;
 }
 
+// k is read as 16-byte vectors (rows of the pooled arrays are 512-byte aligned); the products are still accumulated
+// one after the other in the order t = 0..127, so every kernel that calls this gets the same bits.
 __device__ __forceinline__ float pooled_score(const float* q, const float* k, float scale) {
   float acc = 0.f;
-#pragma unroll 8
-  for (int t = 0; t < RS_HEAD_DIM; ++t) acc = fmaf(q[t], k[t], acc);
+  const float4* k4 = reinterpret_cast<const float4*>(k);
+#pragma unroll 4
+  for (int t = 0; t < RS_HEAD_DIM / 4; ++t) {
+    const float4 kv = k4[t];
+    acc = fmaf(q[4 * t], kv.x, acc);
+    acc = fmaf(q[4 * t + 1], kv.y, acc);
+    acc = fmaf(q[4 * t + 2], kv.z, acc);
+    acc = fmaf(q[4 * t + 3], kv.w, acc);
+  }
   return acc * scale;
 }
 
@@ -755,82 +764,161 @@ struct MixArgs {
 
 __device__ __forceinline__ int interval_len(int lo, int hi) { return hi >= lo ? hi - lo + 1 : 0; }
 
+constexpr int kMixMaxVS = 4, kMixMaxBS = 4;      // vertical-slash / block-sparse candidates per library served here
+
+// One block per run of consecutive mixture rows that share a query block and a subset (the recent rows, the
+// boundary rows, every uniform row); the other blocks of the grid leave at once.  Prologue: per vertical-slash
+// candidate the block-diagonal bitmap and the number of selected columns per key block, per block-sparse candidate the
+// membership bitmap of the query block's selection.  Then one sweep over (row, key block) feeds all candidates.
 __global__ void __launch_bounds__(256)
 rs_mix_cov_kernel(IdxParams P, MixArgs M) {
-  extern __shared__ float mix_smem[];                    // score[nb] | vcnt[nb] | list[kb_cap]
+  extern __shared__ float mix_smem[];
+  // score[nb] | blist[kb_cap] | vcnt[kMixMaxVS][nb] | dbits[kMixMaxVS][128] | member[kMixMaxBS][nb / 32 + 1] | diagcols[kMixMaxVS][64]
   float* score = mix_smem;
-  int* vcnt = reinterpret_cast<int*>(mix_smem + P.nb);
-  int32_t* blist = reinterpret_cast<int32_t*>(vcnt + P.nb);
-  __shared__ uint32_t dbits[128];
+  int32_t* blist = reinterpret_cast<int32_t*>(score + P.nb);
+  int* vcnt = reinterpret_cast<int*>(blist + P.out.kb_cap);
+  uint32_t* dbits = reinterpret_cast<uint32_t*>(vcnt + kMixMaxVS * P.nb);
+  const int mw = P.nb / 32 + 1;
+  uint32_t* member = dbits + kMixMaxVS * 128;
+  int* diagcols = reinterpret_cast<int*>(member + kMixMaxBS * mw);
+  __shared__ int n_diagcols[kMixMaxVS];
   __shared__ uint32_t hist[256];
   __shared__ uint32_t sh[8];
   __shared__ unsigned int wcnt[16];
   __shared__ u64 red[8];
   __shared__ float qrow[RS_HEAD_DIM];
-  const int t = blockIdx.x, item = blockIdx.y;
+  const int t0 = blockIdx.x, item = blockIdx.y;
   const int s = item / P.Hq, h = item - s * P.Hq, g = h / P.group;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int i = M.rows[s * M.r + t];
-  const int qb_i = i >> 6;
+  const int32_t* rows = M.rows + s * M.r;
   int sub = 0;
-  while (sub + 1 < M.n_sub && t >= M.sub_bounds[sub + 1]) ++sub;
-  const float* a = M.A + (((size_t)s * P.Hq + h) * M.r + t) * (size_t)P.nb;
-  bool have_scores = false;
+  while (sub + 1 < M.n_sub && t0 >= M.sub_bounds[sub + 1]) ++sub;
+  const int qb_i = rows[t0] >> 6;
+  if (t0 > M.sub_bounds[sub] && (rows[t0 - 1] >> 6) == qb_i) return;      // not the first row of its run
+  int t1 = t0 + 1;
+  while (t1 < M.sub_bounds[sub + 1] && (rows[t1] >> 6) == qb_i) ++t1;
+  // a long run (the 32 recent rows) is shared by the blocks of grid.z: block z takes rows t0 + z, t0 + z + gridDim.z, ..
+  if (t0 + (int)blockIdx.z >= t1) return;
+
+  // ---- prologue
+  int vs_of[kMixMaxVS], bs_of[kMixMaxBS];
+  int n_vs = 0, n_bs = 0;
   for (int c = 0; c < P.n_cand; ++c) {
-    const rs_candidate cand = P.lib[c];
-    const int slot = item * P.n_cand + c;
-    u64 part = 0;
-    if (cand.pattern == RS_DENSE) {
-      for (int kb = tid; kb <= qb_i; kb += 256) part += fx(a[kb]);
-    } else if (cand.pattern == RS_A_SHAPE) {
-      const int n_sink = cand.b0, w = cand.b1;
-      for (int kb = tid; kb <= qb_i; kb += 256) {
-        const int lo = kb * 64, hi = min(lo + 63, i);
-        const int s_hi = min(hi, n_sink - 1), w_lo = max(lo, i - w + 1);
-        const int num = interval_len(lo, s_hi) + interval_len(w_lo, hi) - interval_len(w_lo, s_hi);
-        part += fx(a[kb]) * (u64)num / (u64)(hi - lo + 1);
-      }
-    } else if (cand.pattern == RS_VERTICAL_SLASH) {
-      const int n_cols = P.out.vs_count[4 * slot + 0], n_diag = P.out.vs_count[4 * slot + 2];
-      const int32_t* cols = P.out.vs_cols + (size_t)slot * P.out.kv_cap;
-      const int32_t* diag = P.out.vs_diag + (size_t)slot * P.out.nd_cap;
-      __syncthreads();
-      for (int x = tid; x < 128; x += 256) dbits[x] = 0;
-      for (int kb = tid; kb <= qb_i; kb += 256) vcnt[kb] = 0;
-      __syncthreads();
-      for (int x = tid; x < n_diag; x += 256) { const int d = diag[x]; atomicOr(&dbits[d >> 5], 1u << (d & 31)); }
-      for (int x = tid; x < n_cols; x += 256) { const int j = cols[x]; if (j <= i) atomicAdd(&vcnt[j >> 6], 1); }
-      __syncthreads();
-      for (int kb = tid; kb <= qb_i; kb += 256) {
-        const int lo = kb * 64, hi = min(lo + 63, i);
-        const int d = qb_i - kb;
-        const int den = hi - lo + 1;
-        const int num = ((dbits[d >> 5] >> (d & 31)) & 1u) ? den : vcnt[kb];
-        part += fx(a[kb]) * (u64)num / (u64)den;
-      }
-    } else {   // block-sparse: the row's query block selects like the materialising kernel does
-      __syncthreads();
-      if (!have_scores) {
-        if (tid < RS_HEAD_DIM) qrow[tid] = P.qpool[((size_t)h * P.nb + qb_i) * RS_HEAD_DIM + tid];
-        __syncthreads();
-        for (int kb = tid; kb < qb_i; kb += 256)
-          score[kb] = pooled_score(qrow, P.kpool + ((size_t)g * P.nb + kb) * RS_HEAD_DIM, P.scale);
-        have_scores = true;
-        __syncthreads();
-      }
-      const int k_b = min(cand.b0, P.out.kb_cap);
-      const int cnt = select_row(score, qb_i, min(k_b, qb_i + 1) - 1, qb_i, blist, P.out.kb_cap, hist, sh, wcnt);
-      for (int x = tid; x < cnt; x += 256) part += fx(a[blist[x]]);
-    }
+    if (P.lib[c].pattern == RS_VERTICAL_SLASH && n_vs < kMixMaxVS) {
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) part += __shfl_xor_sync(0xffffffffu, part, off);
+      for (int e = 0; e < kMixMaxVS; ++e) if (e == n_vs) vs_of[e] = c;
+      ++n_vs;
+    }
+    if (P.lib[c].pattern == RS_BLOCK_SPARSE && n_bs < kMixMaxBS) {
+#pragma unroll
+      for (int e = 0; e < kMixMaxBS; ++e) if (e == n_bs) bs_of[e] = c;
+      ++n_bs;
+    }
+  }
+  for (int x = tid; x < kMixMaxVS * P.nb; x += 256) vcnt[x] = 0;
+  for (int x = tid; x < kMixMaxVS * 128; x += 256) dbits[x] = 0;
+  for (int x = tid; x < kMixMaxBS * mw; x += 256) member[x] = 0;
+  if (tid < kMixMaxVS) n_diagcols[tid] = 0;
+  __syncthreads();
+#pragma unroll
+  for (int v = 0; v < kMixMaxVS; ++v) {
+    if (v >= n_vs) continue;
+    const int slot = item * P.n_cand + vs_of[v];
+    const int n_cols = P.out.vs_count[4 * slot + 0], n_diag = P.out.vs_count[4 * slot + 2];
+    const int32_t* cols = P.out.vs_cols + (size_t)slot * P.out.kv_cap;
+    const int32_t* diag = P.out.vs_diag + (size_t)slot * P.out.nd_cap;
+    for (int x = tid; x < n_diag; x += 256) { const int d = diag[x]; atomicOr(&dbits[v * 128 + (d >> 5)], 1u << (d & 31)); }
+    for (int x = tid; x < n_cols; x += 256) {
+      const int j = cols[x];
+      const int kb = j >> 6;
+      if (kb < qb_i) atomicAdd(&vcnt[v * P.nb + kb], 1);
+      else if (kb == qb_i) { const int at = atomicAdd(&n_diagcols[v], 1); diagcols[v * 64 + at] = j; }   // tested per row
+    }
+  }
+  if (n_bs > 0 && qb_i == (P.seg_bounds[s + 1] >> 6) - 1) {
+    // the segment's last query block: the evaluation already selected for it (evaluation layout, slot = item, candidate)
+#pragma unroll
+    for (int b = 0; b < kMixMaxBS; ++b) {
+      if (b >= n_bs) continue;
+      const size_t slot = (size_t)item * P.n_cand + bs_of[b];
+      const int cnt = P.out.bs_count[slot];
+      const int32_t* bl = P.out.bs_blk + slot * P.out.kb_cap;
+      for (int x = tid; x < cnt; x += 256) { const int kb = bl[x]; atomicOr(&member[b * mw + (kb >> 5)], 1u << (kb & 31)); }
+    }
+  } else if (n_bs > 0) {
+    if (tid < RS_HEAD_DIM) qrow[tid] = P.qpool[((size_t)h * P.nb + qb_i) * RS_HEAD_DIM + tid];
     __syncthreads();
-    if (lane == 0) red[warp] = part;
+    for (int kb = tid; kb < qb_i; kb += 256)
+      score[kb] = pooled_score(qrow, P.kpool + ((size_t)g * P.nb + kb) * RS_HEAD_DIM, P.scale);
+    __syncthreads();
+#pragma unroll
+    for (int b = 0; b < kMixMaxBS; ++b) {
+      if (b >= n_bs) continue;
+      const int k_b = min(P.lib[bs_of[b]].b0, P.out.kb_cap);
+      const int cnt = select_row(score, qb_i, min(k_b, qb_i + 1) - 1, qb_i, blist, P.out.kb_cap, hist, sh, wcnt);
+      for (int x = tid; x < cnt; x += 256) { const int kb = blist[x]; atomicOr(&member[b * mw + (kb >> 5)], 1u << (kb & 31)); }
+      __syncthreads();
+    }
+  }
+  __syncthreads();
+
+  // ---- one sweep over (row, key block) for all candidates
+  u64 part[RS_MAX_CANDIDATES];
+#pragma unroll
+  for (int c = 0; c < RS_MAX_CANDIDATES; ++c) part[c] = 0;
+  for (int t = t0 + (int)blockIdx.z; t < t1; t += (int)gridDim.z) {
+    const int i = rows[t];
+    const float* a = M.A + (((size_t)s * P.Hq + h) * M.r + t) * (size_t)P.nb;
+    for (int kb = tid; kb <= qb_i; kb += 256) {
+      const u64 af = fx(a[kb]);
+      if (af == 0) continue;
+      const int lo = kb * 64, hi = min(lo + 63, i);
+      const u64 den = (u64)(hi - lo + 1);
+      int iv = 0, ib = 0;
+#pragma unroll
+      for (int c = 0; c < RS_MAX_CANDIDATES; ++c) {
+        if (c >= P.n_cand) continue;
+        const rs_candidate cand = P.lib[c];
+        u64 num;
+        if (cand.pattern == RS_DENSE) {
+          num = den;
+        } else if (cand.pattern == RS_A_SHAPE) {
+          const int s_hi = min(hi, cand.b0 - 1), w_lo = max(lo, i - cand.b1 + 1);
+          num = (u64)(interval_len(lo, s_hi) + interval_len(w_lo, hi) - interval_len(w_lo, s_hi));
+        } else if (cand.pattern == RS_VERTICAL_SLASH) {
+          const int v = iv++;
+          if (v >= kMixMaxVS) { num = 0; }
+          else {
+            const int d = qb_i - kb;
+            if ((dbits[v * 128 + (d >> 5)] >> (d & 31)) & 1u) num = den;
+            else if (kb < qb_i) num = (u64)vcnt[v * P.nb + kb];
+            else {
+              int cntd = 0;
+              for (int x = 0; x < n_diagcols[v]; ++x) cntd += (diagcols[v * 64 + x] <= i);
+              num = (u64)cntd;
+            }
+          }
+        } else {
+          const int b = ib++;
+          num = (b < kMixMaxBS && ((member[b * mw + (kb >> 5)] >> (kb & 31)) & 1u)) ? den : 0;
+        }
+        part[c] += (den == 64) ? ((af * num) >> 6) : (af * num / den);      // 64-bit division only on the row's own block
+      }
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < RS_MAX_CANDIDATES; ++c) {
+    if (c >= P.n_cand) continue;
+    u64 v = part[c];
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
     __syncthreads();
     if (tid == 0) {
       u64 tot = 0;
       for (int w8 = 0; w8 < 8; ++w8) tot += red[w8];
-      atomicAdd(&M.covmix[(size_t)slot * 4 + sub], tot);
+      atomicAdd(&M.covmix[((size_t)item * P.n_cand + c) * 4 + sub], tot);
     }
   }
 }
@@ -1005,7 +1093,11 @@ extern "C" int rs_mixture_coverage(const rs_problem* p, const rs_candidate* lib,
   for (int k = 0; k <= n_sub; ++k) M.sub_bounds[k] = sub_bounds[k];
   M.covmix = reinterpret_cast<u64*>(covmix);
   if (cudaMemsetAsync(covmix, 0, (size_t)n_items * n_cand * 4 * sizeof(uint64_t), stream) != cudaSuccess) return RS_ERR_CUDA;
-  const size_t smem = (size_t)nb * 8 + (size_t)(idx_eval->kb_cap > 0 ? idx_eval->kb_cap : 1) * 4;
+  int n_vs = 0, n_bs = 0;
+  for (int c = 0; c < n_cand; ++c) { n_vs += lib[c].pattern == RS_VERTICAL_SLASH; n_bs += lib[c].pattern == RS_BLOCK_SPARSE; }
+  if (n_vs > kMixMaxVS || n_bs > kMixMaxBS) return RS_ERR_UNSUPPORTED_SHAPE;
+  const size_t smem = (size_t)nb * 4 + (size_t)idx_eval->kb_cap * 4 + (size_t)kMixMaxVS * nb * 4 + kMixMaxVS * 128 * 4 +
+                      (size_t)kMixMaxBS * (nb / 32 + 1) * 4 + kMixMaxVS * 64 * 4;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(rs_mix_cov_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
@@ -1013,6 +1105,6 @@ extern "C" int rs_mixture_coverage(const rs_problem* p, const rs_candidate* lib,
     attr_set = true;
   }
   if (smem > 64 * 1024) return RS_ERR_UNSUPPORTED_SHAPE;
-  rs_mix_cov_kernel<<<dim3(r, n_items), 256, smem, stream>>>(P, M);
+  rs_mix_cov_kernel<<<dim3(r, n_items, 4), 256, smem, stream>>>(P, M);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }
