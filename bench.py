@@ -334,6 +334,9 @@ def main():
 
     names = ["probe", "evaluate", "route", "materialise", "attention", "certificate"]
     stages = {nm: float(np.mean([ev[i].elapsed_time(ev[i + 1]) for ev in stage_events])) for i, nm in enumerate(names)}
+    step_ms = [ev[0].elapsed_time(ev[6]) for ev in stage_events]      # per-step device time (first to last stage event)
+    step_stats = {"median": float(np.median(step_ms)), "p95": float(np.percentile(step_ms, 95)),
+                  "min": float(np.min(step_ms)), "max": float(np.max(step_ms)), "n": len(step_ms)}
     counters = layer.counters.cpu().numpy()
     chunks_per_step = int(counters[0]) // args.steps
     choice = layer.choice.cpu().numpy()
@@ -469,7 +472,7 @@ def main():
         "metric": metric, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "config": config,
-        "ms_per_layer": ms, "dense_ms_per_layer": dense_ms,
+        "ms_per_layer": ms, "ms_per_step_stats": step_stats, "dense_ms_per_layer": dense_ms,
         "speedup_vs_own_dense": (dense_ms / ms) if dense_ms else None,
         "dense_tflops": (f_dense / (dense_ms * 1e-3) / 1e12) if dense_ms else None,
         "stage_ms": stages, "overhead_over_attention": overhead_ms / attn_ms,

@@ -21,6 +21,9 @@ Parts and what pins them (tests/test_oracle_*.py):
                                                                   identical keys -> uniform rows.  The mixture, the pooling
                                                                   of a straddling block and the agreement formula are this
                                                                   build's reading: beyond those "parity unpinned".
+  patterns.mixture_coverage_fx   coverage on the mixture's rows.   Pinned: closed cases (whole blocks, half blocks, columns).
+                                                                  The even split of a block's mass over its visible keys
+                                                                  is this build's reading: "parity unpinned".
   calibration.*                  Section 3.5, predictor e of Eq. 4. Pinned: isotonic fit == scikit-learn's, quantile by
                                                                   counting, monotonicity.  The feature set is this build's
                                                                   reading: "parity unpinned".
