@@ -74,6 +74,11 @@ def fixed_choice_for(lib, n_q_heads):
 
 
 # ----------------------------------------------------------------------------------------- clocks
+# DRAM bytes of the attention launch measured with ncu (one-pass metrics, full-size workload, clocks untouched); the
+# algorithmic minimum of the config-3 launch is Q + K + V + O + row outputs = 2.71e9 bytes.
+ATTN_DRAM_BYTES_PER_LAUNCH = {("config3", 131072, "flops", False, False): 3.20e9 + 1.08e9}
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -485,7 +490,10 @@ def main():
         "roofline": {"kernel": "rs_attn_kernel (one launch, all heads)", "bound": "tensor", "achieved": achieved,
                      "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": f"bf16_tflops_sustained, {peaks['source']}",
-                     "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "traffic": None,
+                     "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
+                     "traffic": ATTN_DRAM_BYTES_PER_LAUNCH.get((args.workload, spec.n, args.cost, bool(args.rescue), bool(args.mixture))),
+                     "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of this launch from a one-pass ncu capture of this "
+                                     "workload (profiles/rs_attn_kernel_config3_n16384.md); null for workloads that were not captured",
                      "note": "achieved = 512 FLOP x 128 x 64 pairs per issued chunk / attention-call time (CUDA events)"},
         "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
     }
