@@ -141,7 +141,17 @@ int rs_workspace_bytes(const rs_problem* p, const rs_candidate* lib, int n_cand,
  * concentration (mean over the rows of the mass of keys with i - j < 1024). */
 int rs_probe(const rs_problem* p, const void* Q, const void* K, const void* V,
              float* vert, float* slash, float* lse_probe, float* qpool, float* kpool, float* vmax,
-             float* descr, void* ws, size_t ws_bytes, int32_t* status, void* stream);
+             float* descr, int flags, void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* rs_probe flag: fill only the rows of qpool that candidate evaluation reads (the last query block of every segment)
+ * and leave the rest to rs_pool_queries once the routes are known; reading all of Q for the pooled means is the
+ * largest single stream of the probe (1 GB at 128K) and only heads routed to block-sparse need it. */
+#define RS_PROBE_QPOOL_LAST_ONLY 1
+
+/* 64-row means of Q (the rows of qpool rs_probe left out) for the heads whose routed candidate is block-sparse.
+ * choice: device int32[n_items] (NULL: every head).  qpool as for rs_probe. */
+int rs_pool_queries(const rs_problem* p, const void* Q, const rs_candidate* lib, int n_cand, const int32_t* choice,
+                    float* qpool, int32_t* status, void* stream);
 
 /* Candidate index construction and coverage (Section 3.1, 3.2; step 2 of the procedure table).
  * Ranking keys are the integers sum_g floor(mass_g * 2^32); order is key descending, index ascending.

@@ -49,7 +49,7 @@ class rs_route_params(C.Structure):
 EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "rs_build_indices", "rs_route",
            "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate",
            "rs_selftest_wait_timeout", "rs_probe_pooled", "rs_probe_pooled_scratch_floats", "rs_regressor_eval",
-           "rs_output_error", "rs_mixture_coverage"]
+           "rs_output_error", "rs_mixture_coverage", "rs_pool_queries"]
 
 
 def lib_path() -> str:
@@ -176,10 +176,20 @@ def new_workspace(p: Problem, lib, device="cuda") -> torch.Tensor:
     return torch.empty(max(256, rs_workspace_bytes(p, lib)), dtype=torch.uint8, device=device)
 
 
-def rs_probe(p: Problem, Q, K, V, vert, slash, lse_probe, qpool, kpool, vmax, descr, ws, status):
+RS_PROBE_QPOOL_LAST_ONLY = 1
+
+
+def rs_probe(p: Problem, Q, K, V, vert, slash, lse_probe, qpool, kpool, vmax, descr, ws, status, flags: int = 0):
     _check(load().rs_probe(C.byref(p.c), _ptr(Q), _ptr(K), _ptr(V), _ptr(vert), _ptr(slash), _ptr(lse_probe),
-                           _ptr(qpool), _ptr(kpool), _ptr(vmax), _ptr(descr), _ptr(ws), C.c_size_t(ws.numel()),
-                           _ptr(status), _stream()), "rs_probe")
+                           _ptr(qpool), _ptr(kpool), _ptr(vmax), _ptr(descr), int(flags), _ptr(ws),
+                           C.c_size_t(ws.numel()), _ptr(status), _stream()), "rs_probe")
+
+
+def rs_pool_queries(p: Problem, Q, lib, choice, qpool, status):
+    """64-row means of Q for the heads routed to block-sparse (choice None: every head)."""
+    n = 0 if lib is None else len(lib)
+    _check(load().rs_pool_queries(C.byref(p.c), _ptr(Q), lib, n, _ptr(choice), _ptr(qpool), _ptr(status), _stream()),
+           "rs_pool_queries")
 
 
 def rs_build_indices(p: Problem, lib, vert, slash, qpool, kpool, bscore, choice, out: IndexSet, stats, ws, status):

@@ -23,6 +23,8 @@ constexpr int kThreads1 = 320;         // pass 1: warp 0 TMA, warp 1 MMA, warps 
 constexpr int kThreads2 = 576;         // pass 2: warp 0 TMA, warp 1 MMA, warps 2..17 compute
 constexpr uint32_t kTmemCols = 512;
 
+struct rs_candidate_list { int32_t pattern[RS_MAX_CANDIDATES]; };
+
 struct ProbeParams {
   int n, Hq, Hkv, group, n_seg, n_hc;  // n_hc = head chunks per KV head = ceil(group / 4)
   int seg_bounds[RS_MAX_SEGMENTS + 1];
@@ -478,8 +480,106 @@ ProbePlan plan(const rs_problem* p) {
 
 size_t rs_probe_workspace_bytes(const rs_problem* p) { return plan(p).total; }
 
+namespace {
+
+// 64-row mean of one block (all 256 threads of the CTA); same arithmetic and summation order as rs_pool_kernel.
+__device__ __forceinline__ void pool_block(const __nv_bfloat16* __restrict__ X, float* __restrict__ out, long long blk,
+                                           float (*red)[128 + 4]) {
+  const int rg = threadIdx.x >> 4, cc = threadIdx.x & 15;
+  const uint4* src = reinterpret_cast<const uint4*>(X + (size_t)blk * 64 * RS_HEAD_DIM);
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint4 u = __ldg(src + (size_t)(rg + 16 * k) * 16 + cc);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      acc[2 * e] += __uint_as_float(w[e] << 16);
+      acc[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 8; ++e) red[rg][cc * 8 + e] = acc[e];
+  __syncthreads();
+  if (threadIdx.x < 128) {
+    float sum = 0.f;
+#pragma unroll
+    for (int r = 0; r < 16; ++r) sum += red[r][threadIdx.x];
+    out[(size_t)blk * RS_HEAD_DIM + threadIdx.x] = sum * (1.0f / 64.0f);
+  }
+}
+
+// 64-row means of the Q blocks that are asked for: with `choice`, the blocks of heads routed to block-sparse; with
+// last_only, the last block of every segment.  Same arithmetic and summation order as rs_pool_kernel.
+__global__ void __launch_bounds__(256)
+rs_pool_q_select_kernel(ProbeParams P, const __nv_bfloat16* __restrict__ Q, float* __restrict__ out, rs_candidate_list L,
+                        const int32_t* __restrict__ choice, int last_only) {
+  __shared__ float red[16][128 + 4];
+  const int nb = P.n >> 6;
+  int h, qb;
+  if (last_only) {
+    h = blockIdx.x % P.Hq;
+    qb = (P.seg_bounds[blockIdx.x / P.Hq + 1] >> 6) - 1;
+  } else {
+    h = blockIdx.y;
+    qb = blockIdx.x;
+    int s = 0;
+    while (s + 1 < P.n_seg && qb * 64 >= P.seg_bounds[s + 1]) ++s;
+    if (choice != nullptr && L.pattern[choice[s * P.Hq + h]] != RS_BLOCK_SPARSE) return;
+  }
+  pool_block(Q, out, (long long)h * nb + qb, red);
+}
+
+// The same for a run of kPoolRun consecutive query blocks per CTA: with a choice most heads are not routed to
+// block-sparse, and tens of thousands of CTAs that leave at once still cost a tenth of a millisecond to launch.
+constexpr int kPoolRun = 32;
+__global__ void __launch_bounds__(256)
+rs_pool_q_routed_kernel(ProbeParams P, const __nv_bfloat16* __restrict__ Q, float* __restrict__ out, rs_candidate_list L,
+                        const int32_t* __restrict__ choice) {
+  __shared__ float red[16][128 + 4];
+  const int nb = P.n >> 6;
+  const int h = blockIdx.y;
+  int s = -1;
+  bool want = false;
+  for (int qb = blockIdx.x * kPoolRun; qb < min(nb, (int)(blockIdx.x + 1) * kPoolRun); ++qb) {
+    if (s < 0 || qb * 64 >= P.seg_bounds[s + 1]) {          // the route is looked up once per segment of the run
+      s = max(s, 0);
+      while (s + 1 < P.n_seg && qb * 64 >= P.seg_bounds[s + 1]) ++s;
+      want = choice == nullptr || L.pattern[choice[s * P.Hq + h]] == RS_BLOCK_SPARSE;
+    }
+    if (!want) continue;                                    // uniform over the CTA
+    pool_block(Q, out, (long long)h * nb + qb, red);
+    __syncthreads();
+  }
+}
+
+
+}  // namespace
+
+extern "C" int rs_pool_queries(const rs_problem* p, const void* Q, const rs_candidate* lib, int n_cand,
+                               const int32_t* choice, float* qpool, int32_t* status, void* stream_) {
+  (void)status;
+  int rc = rs_check_problem(p);
+  if (rc != RS_OK) return rc;
+  if (!Q || !qpool || n_cand < 0 || n_cand > RS_MAX_CANDIDATES || (choice != nullptr && (!lib || n_cand == 0)))
+    return RS_ERR_INVALID_ARG;
+  rc = rs_check_device();
+  if (rc != RS_OK) return rc;
+  ProbeParams P{};
+  P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = P.Hq / P.Hkv; P.n_seg = p->n_segments;
+  for (int s = 0; s <= p->n_segments; ++s) P.seg_bounds[s] = p->seg_bounds[s];
+  rs_candidate_list L{};
+  bool any_bs = choice == nullptr;
+  for (int c = 0; c < n_cand; ++c) { L.pattern[c] = lib[c].pattern; any_bs |= lib[c].pattern == RS_BLOCK_SPARSE; }
+  if (!any_bs) return RS_OK;                            // no block-sparse candidate: nothing can be routed to it
+  const int nb = P.n >> 6;
+  rs_pool_q_routed_kernel<<<dim3((nb + kPoolRun - 1) / kPoolRun, P.Hq), 256, 0, (cudaStream_t)stream_>>>(
+      P, reinterpret_cast<const __nv_bfloat16*>(Q), qpool, L, choice);
+  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+}
+
 extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const void* V, float* vert, float* slash,
-                        float* lse_probe, float* qpool, float* kpool, float* vmax, float* descr, void* ws,
+                        float* lse_probe, float* qpool, float* kpool, float* vmax, float* descr, int flags, void* ws,
                         size_t ws_bytes, int32_t* status, void* stream_) {
   int rc = rs_check_problem(p);
   if (rc != RS_OK) return rc;
@@ -534,7 +634,13 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
     rs_vnorm_block_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(V), blockmax, P.Hkv * nb);
     rs_vmax_kernel<<<P.n_seg * P.Hkv, 256, 0, side>>>(P, blockmax, vmax);
   }
-  if (qpool) rs_pool_kernel<<<(unsigned)(P.Hq * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(Q), qpool, P.Hq * nb);
+  if (qpool && (flags & RS_PROBE_QPOOL_LAST_ONLY)) {
+    rs_candidate_list none{};
+    rs_pool_q_select_kernel<<<(unsigned)(P.n_seg * P.Hq), 256, 0, side>>>(P, reinterpret_cast<const __nv_bfloat16*>(Q), qpool,
+                                                                           none, nullptr, 1);
+  } else if (qpool) {
+    rs_pool_kernel<<<(unsigned)(P.Hq * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(Q), qpool, P.Hq * nb);
+  }
   rs_probe_merge_kernel<<<w.n_units, kRows, 0, stream>>>(P);
   rs_probe_kernel<2><<<grid, kThreads2, Smem::total, stream>>>(tmQ, tmK, P);
   rc = rs_side_join(stream);

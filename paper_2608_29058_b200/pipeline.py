@@ -112,9 +112,14 @@ class RoutedPrefillLayer:
         self.cost_t_probe = 0
 
     # ------------------------------------------------------------------ steps (each only enqueues kernels)
-    def probe(self, Q, K, V):
+    def probe(self, Q, K, V, lazy_qpool: bool = False):
+        """lazy_qpool: pool only the Q rows candidate evaluation reads; pool_routed_queries() adds the rest for the
+        heads that end up routed to block-sparse (reading all of Q is the largest stream of the probe)."""
         rs.rs_probe(self.p, Q, K, V, self.vert, self.slash, self.lse_probe, self.qpool, self.kpool, self.vmax, None,
-                    self.ws, self.status)
+                    self.ws, self.status, flags=rs.RS_PROBE_QPOOL_LAST_ONLY if lazy_qpool else 0)
+
+    def pool_routed_queries(self, Q):
+        rs.rs_pool_queries(self.p, Q, self.lib, self.choice, self.qpool, self.status)
 
     def evaluate_candidates(self):
         rs.rs_build_indices(self.p, self.lib, self.vert, self.slash, self.qpool, self.kpool, None, None,
@@ -298,7 +303,8 @@ class RoutedPrefillLayer:
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(7)] if record_events else None
         mark = (lambda i: ev[i].record()) if record_events else (lambda i: None)
         mark(0)
-        self.probe(Q, K, V)
+        lazy = not self.cfg.mixture_u        # the mixture coverage reads pooled queries of blocks all over the segment
+        self.probe(Q, K, V, lazy_qpool=lazy)
         mark(1)
         if fixed_choice is None:
             self.evaluate_candidates()
@@ -312,6 +318,8 @@ class RoutedPrefillLayer:
             self.choice.copy_(fixed_choice)
             mark(2)
         mark(3)
+        if lazy:
+            self.pool_routed_queries(Q)
         self.materialise(reuse_evaluation=fixed_choice is None)
         mark(4)
         self.attention(Q, K, V)

@@ -62,8 +62,10 @@ def test_config3_full_size_online_routing():
         vert, slash = layer.vert[0, h].cpu().numpy(), layer.slash[0, h].cpu().numpy()
         assert _close(vert, pr.vert) and _close(slash, pr.slash), h
         assert np.abs(layer.lse_probe[h, 0].cpu().numpy() - pr.lse).max() < 1e-3
+        # the layer pools queries lazily: the block candidate evaluation reads (the last one) is there after the probe,
+        # the others only for heads routed to block-sparse
         qp = layer.qpool[h].cpu().numpy()
-        assert np.allclose(qp[::97], OP.pool_mean(Qf)[::97], rtol=1e-5, atol=1e-6)
+        assert np.allclose(qp[-1], OP.pool_mean(Qf)[-1], rtol=1e-5, atol=1e-6)
         # candidate statistics and chosen lists from the GPU's own probe scores: bit-exact
         for c, cand in enumerate(cands):
             if cand.pattern == PT.BLOCK_SPARSE:

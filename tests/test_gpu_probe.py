@@ -87,3 +87,38 @@ def test_probe_descriptors_match_oracle():
                 pr = OP.probe_rows(Qs[h], Ks[h // (Hq // Hkv)], p.seg_bounds[s + 1])
                 assert abs(got[s, h, 0] - pr.entropy) < 2e-3 * max(1.0, pr.entropy), (n, s, h, got[s, h, 0], pr.entropy)
                 assert abs(got[s, h, 1] - pr.local_conc) < 1e-3, (n, s, h, got[s, h, 1], pr.local_conc)
+
+
+def test_lazy_query_pooling_equals_full_pooling_where_it_is_read():
+    """RS_PROBE_QPOOL_LAST_ONLY fills the last query block of every segment; rs_pool_queries adds every block of the
+    heads routed to block-sparse; together they hold the same bits as the full pooling wherever anything reads them."""
+    n, Hq, Hkv = 1088, 4, 2
+    L = make_layer(tiny_spec(17, n, Hq, Hkv))
+    p = rs.Problem(Hq, Hkv, n, [0, 320, 1088])
+    full = run_probe(L, p)["qpool"]
+    Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+    f32 = dict(dtype=torch.float32, device="cuda")
+    S = p.n_segments
+    vert = torch.zeros((S, Hq, 4, n), **f32); slash = torch.zeros((S, Hq, 4, n), **f32); lse = torch.zeros((Hq, S, 64), **f32)
+    qpool = torch.full((Hq, n // 64, 128), 123.0, **f32)
+    st = rs.new_status()
+    rs.rs_probe(p, Q, K, V, vert, slash, lse, qpool, None, None, None, rs.new_workspace(p, None), st,
+                flags=rs.RS_PROBE_QPOOL_LAST_ONLY)
+    got = qpool.cpu().numpy()
+    for s in range(S):
+        qb = p.seg_bounds[s + 1] // 64 - 1
+        assert np.array_equal(got[:, qb], full[:, qb])
+    assert np.all(got[:, 0] == 123.0)                                   # untouched elsewhere
+    lib = rs.make_library([(rs.RS_A_SHAPE, 64, 128), (rs.RS_BLOCK_SPARSE, 3, 0), (rs.RS_DENSE, 0, 0)])
+    # items = (segment, head): heads 1 and 2 go block-sparse in segment 0, head 3 in segment 1
+    choice = torch.tensor([0, 1, 1, 2, 0, 2, 0, 1], dtype=torch.int32, device="cuda")
+    rs.rs_pool_queries(p, Q, lib, choice, qpool, st)
+    rs.check_status(st, "lazy pooling")
+    got = qpool.cpu().numpy()
+    seg0 = slice(0, 320 // 64); seg1 = slice(320 // 64, n // 64)
+    for h in (1, 2):
+        assert np.array_equal(got[h, seg0], full[h, seg0])
+    assert np.array_equal(got[3, seg1], full[3, seg1])
+    assert np.all(got[0, 1:4] == 123.0) and np.all(got[3, 0:4] == 123.0)   # heads not routed to block-sparse stay untouched
+    rs.rs_pool_queries(p, Q, None, None, qpool, st)                     # no choice: every head
+    assert np.array_equal(qpool.cpu().numpy(), full)
