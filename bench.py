@@ -471,8 +471,19 @@ def main():
         hist[key] = hist.get(key, 0) + 1
     any_vs = any(c[0] == 2 for c in layer.cands)
     any_bs = any(c[0] == 3 for c in layer.cands)
-    launches_per_step = (7 + (0 if fixed else 2 + 2 * any_vs + any_bs + 1) + 2 * any_vs + 2 * any_bs
-                         + 3 + any_vs + 1)      # probe, evaluate + route, materialise, attention, certificate
+    # kernels of this library per layer pass, stage by stage (memsets and torch copies are not counted)
+    n_probe = 3 + 3 + 1                                   # two passes + merge; K pooling, value norms, V_max; Q pooling
+    if fixed:
+        n_eval, n_route = 0, 0
+        n_mat = 3 * any_vs + 2 * any_bs                   # keys / select / finish; fused scores / rows
+    else:
+        n_eval = 2 + 3 * any_vs + 2 * any_bs              # block sums, closed-form stats; VS chain; BS evaluation
+        n_eval += 4 if args.mixture else 0                # pooled probe (3) + mixture coverage
+        n_eval += (0 if args.mixture else 3) + 1 if (args.calibration and args.beta > 0) else 0   # pooled probe + predictor
+        n_route = 1
+        n_mat = 2 * any_bs                                # the evaluation's vertical-slash lists are reused
+    n_mat += 0 if (args.mixture and not fixed) else int(any_bs)     # queries of the heads routed to block-sparse
+    launches_per_step = n_probe + n_eval + n_route + n_mat + (3 + any_vs) + 1   # + attention (4 with packing) + certificate
     out = {
         "metric": metric, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
