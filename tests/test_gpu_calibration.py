@@ -92,3 +92,20 @@ def test_calibrated_router_matches_the_oracle():
         budget=int(0.35 * rs.dense_flops(p.seg_bounds, p.n_q_heads)), t_probe=rs.probe_flops(p.seg_bounds, p.n_q_heads),
         alpha=1.0, delta_q=calib["delta_q"], cert_max=0.5, beta=2.0, e=e))
     assert np.array_equal(got, want)
+
+
+def test_calibration_command_line_on_synthetic_layers(tmp_path, capsys):
+    """The offline calibration entry point end to end (seeded config-3 / config-4 recipe layers at a small length)."""
+    import json
+    out = tmp_path / "calibration.json"
+    assert CALIB.main(["--n", "8192", "--layers", "1", "--held-out", "1", "--q", "0.9", "--out", str(out)]) == 0
+    res = json.loads(out.read_text())
+    assert res["n"] == 8192 and res["n_records"] == 32 * 12
+    assert 0.0 <= res["delta_q"] < 1.0 and res["coverage_in_domain"]["mass"] >= 0.9
+    assert res["coverage_in_domain"]["rows_exact_mass"] == 1.0          # Eq. 5 with the exact mass holds on every row
+    for dom in ("same_recipe", "segmented"):
+        assert res[f"coverage_held_out_{dom}"]["n"] > 0
+    # the result installs into a layer
+    layer = rs.RoutedPrefillLayer(rs.Problem(32, 8, 8192), None, rs.RouteConfig())
+    layer.use_calibration(res, beta=1.0)
+    assert layer.cfg.delta_q == res["delta_q"] and layer.cfg.beta == 1.0
