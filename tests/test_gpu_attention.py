@@ -150,3 +150,32 @@ def test_single_block_and_maximum_length():
         assert np.abs(lse[0, rows].cpu().numpy() - lo).max() < 2e-3
     with pytest.raises(rs.RouteSparseError):
         rs.rs_workspace_bytes(rs.Problem(1, 1, 2 * n), None)
+
+
+def test_many_vertical_columns_cover_both_mask_paths():
+    """A vertical-slash head with more gathered columns than the per-tile keep masks cover (128 chunks = 8192 columns):
+    the first chunks use the precomputed masks, the rest the per-element path; columns inside block diagonals are
+    de-duplicated, columns after a row are invisible.  Checked on sampled rows against the oracle under the same mask."""
+    n = 16384
+    L = make_layer(tiny_spec(29, n, 1, 1))
+    p = rs.Problem(1, 1, n)
+    rng = np.random.default_rng(9)
+    cand = C(PT.VERTICAL_SLASH, 9000, 3)
+    V_cols = np.sort(rng.choice(n, 9000, replace=False)).astype(np.int32)
+    S_offs = np.array([0, 70, 5000], dtype=np.int32)
+    D = np.unique(np.concatenate([S_offs // 64, (S_offs + 63) // 64])).astype(np.int32)
+    ix = PT.IndexSet(cand=cand, q0=0, q1=n, V=V_cols, S=S_offs, D=D)
+    lib = c_library([cand, C(PT.DENSE)])
+    idx = upload_materialised(p, lib, [ix])
+    Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+    O = torch.zeros((1, n, 128), dtype=torch.float32, device="cuda")
+    lse = torch.zeros((1, n), dtype=torch.float32, device="cuda")
+    st = rs.new_status()
+    rs.rs_sparse_prefill_attn(p, Q, K, V, lib, idx, torch.zeros(1, dtype=torch.int32, device="cuda"), O, lse, None, None,
+                              rs.new_workspace(p, lib), st)
+    rs.check_status(st, "many verticals")
+    Qs, Ks, Vs = f64_heads(L)
+    rows = np.concatenate([np.arange(0, 128), np.arange(5000, 5128), np.arange(9984, 10112), np.arange(n - 128, n)])
+    Oo, lo, _ = A.masked_attention(Qs[0], Ks[0], Vs[0], lambda r, nk: PT.mask_rows(ix, r, nk), rows)
+    assert_attention_close(O[0].cpu().numpy()[rows], Oo, "many verticals")
+    assert np.abs(lse[0].cpu().numpy()[rows] - lo).max() < 2e-3
