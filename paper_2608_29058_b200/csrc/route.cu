@@ -149,12 +149,61 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
       }
       return best;
     };
-    for (int it = tid; it < A.n_items; it += kThreads) ibest[it] = best_of_item(it, 0, 1);
+    // An item's sequence of substitutions depends on that item alone, so when the tables fit in shared memory every
+    // item's whole sequence is worked out first, one thread per item (that is where the divisions are); the serial part
+    // is then a merge: take the best head of all sequences, pop it, until the budget is met.
+    Sub* queue = reinterpret_cast<Sub*>(ch + A.n_items + (A.n_items & 1));      // [n_items][n_cand], 8-byte aligned
+    int* qpos = reinterpret_cast<int*>(queue + (cached ? n_pairs : 0));         // [n_items] next entry, [n_items] length
+    int* qlen = qpos + A.n_items;
+    if (cached) {
+      for (int it = tid; it < A.n_items; it += kThreads) {
+        int cur = A.dense_c, len = 0;
+        for (int guard = 0; guard < A.n_cand; ++guard) {
+          Sub best; best.ratio = 0.0; best.dT = 0; best.item = -1; best.k = -1;
+          for (int k = 0; k < A.n_cand; ++k) {
+            const long long dT = costf(it, cur) - costf(it, k);
+            if (dT <= 0) continue;
+            Sub s2;
+            s2.ratio = __ddiv_rn(__dsub_rn(riskf(it, k), riskf(it, cur)), (double)dT);
+            s2.dT = dT; s2.item = it; s2.k = k;
+            if (better(s2, best)) best = s2;
+          }
+          if (best.k < 0) break;
+          queue[it * A.n_cand + len++] = best;
+          cur = best.k;
+        }
+        qpos[it] = 0;
+        qlen[it] = len;
+      }
+    } else {
+      for (int it = tid; it < A.n_items; it += kThreads) ibest[it] = best_of_item(it, 0, 1);
+    }
     __syncthreads();
     if (warp == 0) {
       long long total = sh_total;
       const int max_steps = n_pairs + 1;
-      for (int step = 0; step < max_steps && total > A.prm.budget; ++step) {
+      if (cached) {
+        for (int step = 0; step < max_steps && total > A.prm.budget; ++step) {
+          Sub best; best.ratio = 0.0; best.dT = 0; best.item = -1; best.k = -1;
+          for (int it = lane; it < A.n_items; it += 32) {
+            const int qp = qpos[it];
+            if (qp < qlen[it]) {
+              const Sub s2 = queue[it * A.n_cand + qp];
+              if (better(s2, best)) best = s2;
+            }
+          }
+#pragma unroll
+          for (int off = 16; off >= 1; off >>= 1) {
+            const Sub o = shfl_sub(best, off);
+            if (better(o, best)) best = o;
+          }
+          if (best.k < 0) { if (lane == 0) sh_feasible = 0; break; }
+          if (lane == 0) { ch[best.item] = best.k; qpos[best.item] += 1; }
+          total -= best.dT;
+          __syncwarp();
+        }
+      }
+      for (int step = 0; !cached && step < max_steps && total > A.prm.budget; ++step) {
         Sub best; best.ratio = 0.0; best.dT = 0; best.item = -1; best.k = -1;
         for (int it = lane; it < A.n_items; it += 32) {
           const Sub s = ibest[it];
@@ -302,10 +351,11 @@ extern "C" int rs_route(const rs_problem* p, const rs_candidate* lib, int n_cand
   A.stats = stats; A.cost = cost; A.vmax = vmax; A.prm = *params; A.choice = choice; A.report = report;
   A.status = status;
   const int n_pairs = n_items * n_cand;
-  const size_t smem = (size_t)n_items * (sizeof(Sub) + sizeof(int)) + (n_pairs <= kCachePairs ? (size_t)n_pairs * 16 : 0) + 16;
+  const size_t smem = (size_t)n_items * (sizeof(Sub) + sizeof(int)) + (n_pairs <= kCachePairs ? (size_t)n_pairs * (16 + sizeof(Sub)) : 0) +
+                      (size_t)n_items * 8 + 32;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(rs_route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(rs_route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
       return RS_ERR_CUDA;
     attr_set = true;
   }
