@@ -11,6 +11,7 @@ namespace {
 
 constexpr int kThreads = 1024;
 constexpr int kMaxItems = 2048;
+constexpr int kSortPairs = 2048;      // up to this many pairs the merge of the sequences is a parallel sort
 constexpr int kCachePairs = 4096;     // (item, candidate) pairs whose risk / cost are kept in shared memory
 
 struct RouteArgs {
@@ -155,9 +156,12 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
     Sub* queue = reinterpret_cast<Sub*>(ch + A.n_items + (A.n_items & 1));      // [n_items][n_cand], 8-byte aligned
     int* qpos = reinterpret_cast<int*>(queue + (cached ? n_pairs : 0));         // [n_items] next entry, [n_items] length
     int* qlen = qpos + A.n_items;
+    const bool sorted_path = cached && n_pairs <= kSortPairs;
+    uint32_t* sidx = reinterpret_cast<uint32_t*>(qlen + A.n_items);             // [2048] (item << 8 | position), sorted
+    unsigned char* mrun = reinterpret_cast<unsigned char*>(sidx + (sorted_path ? kSortPairs : 0));   // [n_pairs]
     if (cached) {
       for (int it = tid; it < A.n_items; it += kThreads) {
-        int cur = A.dense_c, len = 0;
+        int cur = A.dense_c, len = 0, m_at = 0;
         for (int guard = 0; guard < A.n_cand; ++guard) {
           Sub best; best.ratio = 0.0; best.dT = 0; best.item = -1; best.k = -1;
           for (int k = 0; k < A.n_cand; ++k) {
@@ -169,7 +173,12 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
             if (better(s2, best)) best = s2;
           }
           if (best.k < 0) break;
-          queue[it * A.n_cand + len++] = best;
+          queue[it * A.n_cand + len] = best;
+          if (sorted_path) {                    // position of the largest key so far: an entry cannot be taken before it
+            if (len == 0 || better(queue[it * A.n_cand + m_at], best)) m_at = len;
+            mrun[it * A.n_cand + len] = (unsigned char)m_at;
+          }
+          ++len;
           cur = best.k;
         }
         qpos[it] = 0;
@@ -179,10 +188,62 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
       for (int it = tid; it < A.n_items; it += kThreads) ibest[it] = best_of_item(it, 0, 1);
     }
     __syncthreads();
+    if (sorted_path) {
+      // The merge takes, at every step, the smallest head.  An entry whose key is smaller than an earlier key of its own
+      // sequence is taken right after that earlier entry, so the merged order is the order of the running maxima of
+      // the keys (entries of one item by position): a sort, then one walk until the budget is met.
+      __shared__ int sh_entries;
+      if (tid == 0) {
+        int acc = 0;
+        for (int it = 0; it < A.n_items; ++it) { qpos[it] = acc; acc += qlen[it]; }
+        sh_entries = acc;
+      }
+      __syncthreads();
+      const int n_entries = sh_entries;
+      int n_pad = 1;
+      while (n_pad < n_entries) n_pad <<= 1;
+      for (int x = tid; x < n_pad; x += kThreads) sidx[x] = 0xffffffffu;
+      __syncthreads();
+      for (int it = tid; it < A.n_items; it += kThreads)
+        for (int j = 0; j < qlen[it]; ++j) sidx[qpos[it] + j] = ((uint32_t)it << 8) | (uint32_t)j;
+      __syncthreads();
+      auto before = [&](uint32_t a, uint32_t b) -> bool {        // a strictly before b in the merged order
+        if (a == 0xffffffffu) return false;
+        if (b == 0xffffffffu) return true;
+        const int ia = (int)(a >> 8), ja = (int)(a & 255u), ib = (int)(b >> 8), jb = (int)(b & 255u);
+        if (ia == ib) return ja < jb;
+        return better(queue[ia * A.n_cand + mrun[ia * A.n_cand + ja]], queue[ib * A.n_cand + mrun[ib * A.n_cand + jb]]);
+      };
+      for (int k2 = 2; k2 <= n_pad; k2 <<= 1) {
+        for (int j2 = k2 >> 1; j2 > 0; j2 >>= 1) {
+          for (int x = tid; x < n_pad; x += kThreads) {
+            const int y = x ^ j2;
+            if (y > x) {
+              const uint32_t a = sidx[x], b = sidx[y];
+              const bool up = (x & k2) == 0;
+              if (up ? before(b, a) : before(a, b)) { sidx[x] = b; sidx[y] = a; }
+            }
+          }
+          __syncthreads();
+        }
+      }
+      if (tid == 0) {
+        long long total = sh_total;
+        int x = 0;
+        for (; x < n_entries && total > A.prm.budget; ++x) {
+          const Sub e = queue[(sidx[x] >> 8) * A.n_cand + (sidx[x] & 255u)];
+          ch[e.item] = e.k;
+          total -= e.dT;
+        }
+        if (total > A.prm.budget) sh_feasible = 0;
+        sh_total = total;
+      }
+      __syncthreads();
+    }
     if (warp == 0) {
       long long total = sh_total;
       const int max_steps = n_pairs + 1;
-      if (cached) {
+      if (cached && !sorted_path) {
         for (int step = 0; step < max_steps && total > A.prm.budget; ++step) {
           Sub best; best.ratio = 0.0; best.dT = 0; best.item = -1; best.k = -1;
           for (int it = lane; it < A.n_items; it += 32) {
@@ -352,7 +413,7 @@ extern "C" int rs_route(const rs_problem* p, const rs_candidate* lib, int n_cand
   A.status = status;
   const int n_pairs = n_items * n_cand;
   const size_t smem = (size_t)n_items * (sizeof(Sub) + sizeof(int)) + (n_pairs <= kCachePairs ? (size_t)n_pairs * (16 + sizeof(Sub)) : 0) +
-                      (size_t)n_items * 8 + 32;
+                      (size_t)n_items * 8 + 32 + (n_pairs <= kSortPairs ? (size_t)kSortPairs * 4 + n_pairs : 0);
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(rs_route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)

@@ -176,3 +176,28 @@ def test_backfill_is_bit_exact_and_never_worse():
                 dT = int(cost[it, k]) - int(cost[it, got[it]])
                 assert not (dT > 0 and rep[0] + dT <= budget and R[it, k] < R[it, got[it]])
     assert improved >= 1
+
+
+def test_route_with_many_ties_and_non_monotone_sequences():
+    """Coarsely quantised coverages and costs: many substitutions share a ratio, many items' sequences are not monotone;
+    the device solve (sequences precomputed per item, merged by a sort of running maxima) must still take exactly the
+    substitutions of the oracle's step-by-step greedy loop."""
+    rng = np.random.default_rng(2024)
+    for n_seg, Hq, Hkv in ((5, 32, 8), (1, 32, 8), (3, 8, 2)):
+        p = rs.Problem(Hq, Hkv, 64 * n_seg * 2, [128 * s for s in range(n_seg + 1)])
+        n_items = n_seg * Hq
+        for trial in range(4):
+            cov = np.zeros((n_items, len(LIB), 4), dtype=np.uint64)
+            pairs = np.zeros((n_items, len(LIB)), dtype=np.int64)
+            for it in range(n_items):
+                for c, cand in enumerate(LIB):
+                    lvl = rng.integers(2, 9) if cand.pattern != PT.DENSE else 8          # coverage in eighths
+                    cov[it, c] = np.uint64(lvl * 2 * 2 ** 32)
+                    pairs[it, c] = 1000 * rng.integers(1, 12) if cand.pattern != PT.DENSE else 20000
+            cost = 512 * pairs
+            vmax_sg = np.ones((n_seg, Hkv), dtype=np.float32)
+            budget = int(cost[:, -1].sum() * [0.08, 0.2, 0.45, 0.02][trial])
+            got, rep = gpu_route(p, LIB, cov, pairs, cost, vmax_sg, budget=budget, alpha=1.0, backfill=trial == 2)
+            want, wrep = RT.route(LIB, cov, cost, np.ones(n_items, np.float32), RT.RouteParams(budget=budget, backfill=trial == 2))
+            assert np.array_equal(got, want), (n_seg, trial)
+            assert rep[0] == wrep.total_cost and rep[1] == wrep.total_risk and rep[3] == wrep.feasible

@@ -154,3 +154,55 @@ def test_backfill_uses_leftover_budget_without_exceeding_it():
                 assert not (dT > 0 and total2 + dT <= budget and R[i, k] < R[i, ch2[i]])
         got, rep = route(lib, cov, cost, np.ones(n_items, np.float32), RouteParams(budget=budget, backfill=True))
         assert list(got) == ch2 and rep.total_cost == total2
+
+
+def test_greedy_order_is_the_order_of_running_maxima():
+    """The step-by-step greedy loop takes the substitutions in the order obtained by sorting every item's own sequence
+    entries by the running maximum of their keys (entries of one item by position): an entry whose key is smaller than
+    an earlier key of its sequence is taken right after that earlier entry.  (The device solve relies on this.)"""
+    from oracle.routing import greedy_solve, risks
+    rng = np.random.default_rng(77)
+    lib = PT.default_library()
+    dense_c = len(lib) - 1
+    for trial in range(8):
+        n_items = 9
+        cov = np.zeros((n_items, len(lib), 4), dtype=np.uint64)
+        cost = np.zeros((n_items, len(lib)), dtype=np.int64)
+        for it in range(n_items):
+            for c, cand in enumerate(lib):
+                lvl = rng.integers(2, 9) if cand.pattern != PT.DENSE else 8
+                cov[it, c] = np.uint64(lvl * 2 * 2 ** 32)
+                cost[it, c] = 1000 * rng.integers(1, 12) if cand.pattern != PT.DENSE else 20000
+        R, _ = risks(lib, cov, 1.0)
+        # every item's sequence from dense, key = (ratio, -dT, item, k)
+        entries = []
+        for it in range(n_items):
+            cur, seq = dense_c, []
+            while True:
+                best = None
+                for k in range(len(lib)):
+                    dT = int(cost[it, cur]) - int(cost[it, k])
+                    if dT <= 0:
+                        continue
+                    key = ((float(R[it, k]) - float(R[it, cur])) / float(dT), -dT, it, k)
+                    if best is None or key < best:
+                        best = key
+                if best is None:
+                    break
+                seq.append(best)
+                cur = best[3]
+            run = None
+            for j, key in enumerate(seq):
+                run = key if run is None or key > run else run
+                entries.append((run, j, key))
+        order = [e[2] for e in sorted(entries, key=lambda e: (e[0], e[1]))]
+        for frac in (0.05, 0.2, 0.5):
+            budget = int(cost[:, dense_c].sum() * frac)
+            choice, total, feas = greedy_solve(R, cost, dense_c, budget, 0)
+            ch2, tot2 = [dense_c] * n_items, int(cost[:, dense_c].sum())
+            for key in order:
+                if tot2 <= budget:
+                    break
+                ch2[key[2]] = key[3]
+                tot2 += key[1]
+            assert ch2 == choice and tot2 == total, (trial, frac)
