@@ -124,6 +124,13 @@ typedef struct { int64_t total_cost; double total_risk; int32_t n_fallback; int3
 const char* rs_error_string(int code);
 int rs_version(void);
 
+/* Streams and graphs.  Every call below only enqueues work on the caller's stream; rs_probe and rs_build_indices also
+ * use one internal side stream per device for kernels that do not depend on each other, forked from and joined back
+ * into the caller's stream with events, so the caller still sees one ordered piece of work and the calls can be
+ * captured into a CUDA graph.  The first call of an entry point on a device sets kernel attributes and creates that
+ * side stream: make it outside any capture.  Calls from several host threads on one device are serialised while they
+ * hold the side stream. */
+
 /* Bytes of scratch that any hot-path call below needs for this problem and library (host computation). */
 int rs_workspace_bytes(const rs_problem* p, const rs_candidate* lib, int n_cand, size_t* bytes);
 
