@@ -147,7 +147,7 @@ def aggregate_over_ranks(ms_local: float, units_local: float, device=None):
 
 
 # ----------------------------------------------------------------------------------------- CPU oracle leg
-def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float = 20.0, n_heads: int = 8):
+def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float = 20.0, n_heads: int = 8, n_blocks: int = 20):
     """Times the oracle's masked attention on sampled query blocks under the routed masks.
 
     Returns (effective TFLOP/s, description, cores, max abs difference to gpu_O on the sampled rows).
@@ -158,7 +158,7 @@ def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float =
     G = spec.n_q_heads // spec.n_kv_heads
     nb = spec.n // 64
     heads = sorted(set(int(h) for h in np.linspace(0, spec.n_q_heads - 1, n_heads)))
-    blocks = sorted(set(int(b) for b in np.linspace(nb // 16, nb - 1, 10)))
+    blocks = sorted(set(int(b) for b in np.linspace(nb // 16, nb - 1, n_blocks)))
     t_used, pairs_done, rows_done, worst = 0.0, 0, 0, 0.0
     kv_cache = {}
     for h in heads:
