@@ -28,7 +28,7 @@ struct rs_candidate_list { int32_t pattern[RS_MAX_CANDIDATES]; };
 struct ProbeParams {
   int n, Hq, Hkv, group, n_seg, n_hc;  // n_hc = head chunks per KV head = ceil(group / 4)
   int seg_bounds[RS_MAX_SEGMENTS + 1];
-  int n_splits;
+  int n_splits, per;
   float4* partial;    // [n_seg*Hkv*n_hc][n_splits][256] (max, sum, sum of p * score, sum of p inside the local band), exp2 domain
   float* lse2;        // [n_seg*Hkv*n_hc][256] log-sum-exp * log2(e)
   float* lse_probe;   // [Hq][n_seg][64]
@@ -73,7 +73,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int h0 = g * P.group + hc * kHC;
   const int n_heads = min(kHC, P.group - hc * kHC);
   const int n_tiles = (q1 + kKeyTile - 1) / kKeyTile;
-  const int per = (n_tiles + P.n_splits - 1) / P.n_splits;
+  const int per = P.per;                      // key tiles per CTA, the same for every unit
   const int t0 = blockIdx.x * per, t1 = min(n_tiles, t0 + per);
   const int i_first = q1 - RS_PROBE_ROWS;   // first probe row
 
@@ -455,18 +455,24 @@ __global__ void rs_vmax_kernel(ProbeParams P, const float* blockmax, float* vmax
   }
 }
 
-struct ProbePlan { size_t partial, lse2, blockmax, total; int n_units, n_splits, n_hc; };
+struct ProbePlan { size_t partial, lse2, blockmax, total; int n_units, n_splits, n_hc, per; };
 
 ProbePlan plan(const rs_problem* p) {
   ProbePlan w{};
   const int group = p->n_q_heads / p->n_kv_heads;
   w.n_hc = (group + kHC - 1) / kHC;
   w.n_units = p->n_segments * p->n_kv_heads * w.n_hc;
-  int splits = (2 * 148 + w.n_units - 1) / w.n_units;
+  // Every CTA gets about the same number of key tiles: segments that end early have fewer tiles and use fewer CTAs
+  // (two CTAs' worth of work per SM in total).
+  const int per_seg_units = p->n_kv_heads * w.n_hc;
+  long long total_tiles = 0;
+  for (int s = 0; s < p->n_segments; ++s) total_tiles += (long long)per_seg_units * ((p->seg_bounds[s + 1] + kKeyTile - 1) / kKeyTile);
   const int max_tiles = (p->n_keys + kKeyTile - 1) / kKeyTile;
-  if (splits > max_tiles) splits = max_tiles;
-  if (splits < 1) splits = 1;
-  if (splits > 64) splits = 64;
+  int per = (int)((total_tiles + 2 * 148 - 1) / (2 * 148));
+  if (per < 1) per = 1;
+  if ((max_tiles + per - 1) / per > 64) per = (max_tiles + 63) / 64;
+  const int splits = (max_tiles + per - 1) / per;
+  w.per = per;
   w.n_splits = splits;
   size_t off = 0;
   w.partial = off;  off += rs_align_up((size_t)w.n_units * splits * kRows * sizeof(float4), 256);
@@ -596,7 +602,7 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
 
   ProbeParams P{};
   P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = P.Hq / P.Hkv;
-  P.n_seg = p->n_segments; P.n_hc = w.n_hc; P.n_splits = w.n_splits;
+  P.n_seg = p->n_segments; P.n_hc = w.n_hc; P.n_splits = w.n_splits; P.per = w.per;
   for (int s = 0; s <= p->n_segments; ++s) P.seg_bounds[s] = p->seg_bounds[s];
   P.partial = reinterpret_cast<float4*>(wsb + w.partial);
   P.descr = descr;
