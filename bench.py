@@ -215,7 +215,7 @@ def download_sets(layer, cands, choice):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config3", choices=["config1", "config2", "config3", "config4"])
@@ -640,6 +640,8 @@ def ablations(args):
         ("greedy back-fill of leftover budget", None, rs.RouteConfig(backfill=True, **base), {}),
         ("uncertainty from recent / uniform / boundary rows (query mixture)", None, rs.RouteConfig(mixture_u=True, **base), {}),
         ("the same with alpha = 4", None, rs.RouteConfig(mixture_u=True, alpha=4.0, **base), {}),
+        ("layer-level router: one candidate for all heads", None, rs.RouteConfig(global_pattern=True, **base), {}),
+        ("layer-level router without fallback", None, rs.RouteConfig(global_pattern=True, budget_frac=0.15, cert_max=None), {}),
     ]
     rows = []
     with open(path, "w") as f:

@@ -111,7 +111,9 @@ typedef struct {
   double beta;             /* weight of e in Eq. 4 */
   int32_t backfill;        /* 1: after the greedy solve, spend what is left of the budget on the substitutions with
                               the largest risk decrease per unit of added cost that still fit (before the fallback) */
-  int32_t reserved2;       /* 0 */
+  int32_t global_pattern;  /* 1: the layer-level comparison router of Section 4 (baselines): every item takes the
+                              same candidate, the feasible one with the smallest summed risk (ties: cheaper, lower
+                              index); the greedy solve and the back-fill are skipped, the fallback still runs */
   const uint64_t* cov_mix; /* device uint64[n_items][n_cand][4] from rs_mixture_coverage, or NULL.  When set, u of Eq. 4
                               is the disagreement among the row subsets of the query mixture, max_b m_b - min_b m_b with
                               m_b = cov_mix[..][b] / (mix_rows[b] * 2^32), instead of the spread over the four groups of

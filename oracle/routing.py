@@ -43,6 +43,7 @@ class RouteParams:
     rescue_any: bool = False         # before dense, take the cheapest sparse candidate of any family that passes
     backfill: bool = False           # spend leftover budget on the best risk decrease per added cost (before fallback)
     u_mix: Optional[np.ndarray] = None   # [items, n_cand] disagreement among the mixture's row subsets (replaces u)
+    global_pattern: bool = False     # comparison router of Section 4: one candidate for the whole layer
     forced_dense: Sequence[int] = field(default_factory=list)   # items forced to dense last
     fixed_choice: Optional[Sequence[int]] = None                 # bypasses the solve and the fallback
 
@@ -109,6 +110,25 @@ def greedy_solve(R: np.ndarray, cost: np.ndarray, dense_c: int, budget: int, t_p
     return choice, total, feasible
 
 
+def global_solve(R: np.ndarray, cost: np.ndarray, budget: int, t_probe: int):
+    """The layer-level router the paper compares against (Section 4, baselines): Eq. 6-8 with the extra constraint that
+    every item takes the same candidate.  Among the candidates whose summed cost meets the budget the one with the
+    smallest summed risk wins (ties: cheaper, lower index); if none does, the cheapest one is taken and the result is
+    marked infeasible.  Risks are summed in item order, one rounding per addition."""
+    n_items, n_cand = R.shape
+    best = None                                       # (infeasible, risk or 0, cost, c)
+    for c in range(n_cand):
+        tot = int(t_probe) + sum(int(cost[it, c]) for it in range(n_items))
+        risk = 0.0
+        for it in range(n_items):
+            risk += float(R[it, c])
+        key = (0, risk, tot, c) if tot <= budget else (1, 0.0, tot, c)
+        if best is None or key < best:
+            best = key
+    infeasible, _, tot, c = best
+    return [c] * n_items, tot, 1 - infeasible
+
+
 def backfill(choice: List[int], total: int, R: np.ndarray, cost: np.ndarray, budget: int):
     """Greedy back-fill: while some substitution to a more expensive, less risky candidate still fits the budget, apply
     the one with the largest risk decrease per unit of added cost (ties: cheaper, lower item, lower candidate).
@@ -153,8 +173,11 @@ def route(lib: List[Candidate], cov_fx: np.ndarray, cost: np.ndarray, vmax: np.n
         choice = [int(c) for c in p.fixed_choice]
         feasible = 1
     else:
-        choice, total, feasible = greedy_solve(R, cost, dense_c, int(p.budget), int(p.t_probe))
-        if p.backfill and feasible:
+        if p.global_pattern:
+            choice, total, feasible = global_solve(R, cost, int(p.budget), int(p.t_probe))
+        else:
+            choice, total, feasible = greedy_solve(R, cost, dense_c, int(p.budget), int(p.t_probe))
+        if p.backfill and feasible and not p.global_pattern:
             choice, total = backfill(choice, total, R, cost, int(p.budget))
         if p.cert_max is not None:
             for it in range(n_items):

@@ -43,7 +43,7 @@ class rs_route_params(C.Structure):
                 ("cert_max", C.c_double), ("use_cert", C.c_int32), ("cert_mode", C.c_int32),
                 ("expand_first", C.c_int32), ("reserved", C.c_int32),
                 ("forced_dense", C.c_void_p), ("fixed_choice", C.c_void_p), ("e", C.c_void_p), ("beta", C.c_double),
-                ("backfill", C.c_int32), ("reserved2", C.c_int32), ("cov_mix", C.c_void_p), ("mix_rows", C.c_int32 * 4)]
+                ("backfill", C.c_int32), ("global_pattern", C.c_int32), ("cov_mix", C.c_void_p), ("mix_rows", C.c_int32 * 4)]
 
 
 EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "rs_build_indices", "rs_route",

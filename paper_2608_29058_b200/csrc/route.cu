@@ -121,6 +121,48 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
     for (int it = tid; it < A.n_items; it += kThreads) ch[it] = A.prm.fixed_choice[it];
     __syncthreads();
   } else {
+    const bool global_pattern = A.prm.global_pattern != 0;
+    if (global_pattern) {
+      // Layer-level comparison router: every item takes the same candidate.  Lane c of warp 0 sums candidate c's cost
+      // and risk over the items (risk in item order, one rounding per addition); the feasible candidate with the
+      // smallest risk wins (ties: cheaper, lower index), else the cheapest one and the result is marked infeasible.
+      if (warp == 0) {
+        int b_inf = 2, b_c = -1;
+        double b_risk = 0.0;
+        long long b_cost = 0;
+        for (int c = lane; c < A.n_cand; c += 32) {
+          long long tot = A.prm.t_probe;
+          double risk = 0.0;
+          for (int it = 0; it < A.n_items; ++it) {
+            tot += costf(it, c);
+            risk = __dadd_rn(risk, riskf(it, c));
+          }
+          const int inf = tot <= A.prm.budget ? 0 : 1;
+          if (inf) risk = 0.0;
+          const bool take = b_c < 0 || inf < b_inf || (inf == b_inf && (risk < b_risk || (risk == b_risk && tot < b_cost)));
+          if (take) { b_inf = inf; b_risk = risk; b_cost = tot; b_c = c; }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+          const int o_inf = __shfl_xor_sync(0xffffffffu, b_inf, off), o_c = __shfl_xor_sync(0xffffffffu, b_c, off);
+          const double o_risk = __shfl_xor_sync(0xffffffffu, b_risk, off);
+          const long long o_cost = __shfl_xor_sync(0xffffffffu, b_cost, off);
+          bool take = false;
+          if (o_c >= 0) {
+            if (b_c < 0) take = true;
+            else if (o_inf != b_inf) take = o_inf < b_inf;
+            else if (o_risk != b_risk) take = o_risk < b_risk;
+            else if (o_cost != b_cost) take = o_cost < b_cost;
+            else take = o_c < b_c;
+          }
+          if (take) { b_inf = o_inf; b_risk = o_risk; b_cost = o_cost; b_c = o_c; }
+        }
+        for (int it = lane; it < A.n_items; it += 32) ch[it] = b_c;
+        if (lane == 0) { sh_total = b_cost; sh_feasible = b_inf ? 0 : 1; }
+      }
+      __syncthreads();
+    }
+    if (!global_pattern) {
     for (int it = tid; it < A.n_items; it += kThreads) ch[it] = A.dense_c;
     long long part = 0;
     for (int it = tid; it < A.n_items; it += kThreads) part += costf(it, A.dense_c);
@@ -327,6 +369,7 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
       if (lane == 0) sh_total = total;
     }
     __syncthreads();
+    }   // !global_pattern
     // ---- fallback walk: larger budget of the family first, then dense
     if (A.prm.use_cert) {
       for (int it = tid; it < A.n_items; it += kThreads) {

@@ -47,6 +47,7 @@ class RouteConfig:
     beta: float = 0.0                  # weight of the calibrated predictor e of Eq. 4 (needs use_calibration())
     backfill: bool = False             # spend leftover budget on the best risk decrease per added cost
     mixture_u: bool = False            # u of Eq. 4 from the recent / uniform / boundary rows of the query mixture
+    global_pattern: bool = False       # comparison router: one candidate for the whole layer (Section 4, baselines)
 
 
 class _IdxView:
@@ -138,6 +139,7 @@ class RoutedPrefillLayer:
         prm.cert_mode, prm.expand_first = c.cert_mode, int(c.expand_first)
         prm.reserved = int(c.rescue_any)
         prm.backfill = int(c.backfill)
+        prm.global_pattern = int(c.global_pattern)
         if c.mixture_u and getattr(self, "_pp_key", None) is not None:
             prm.cov_mix = self.covmix.data_ptr()
             sub = self.pp["sub"]

@@ -38,6 +38,7 @@ def gpu_route(p, lib, cov, pairs, cost, vmax, **kw):
     prm.cert_mode = kw.get("cert_mode", rs.RS_CERT_REL); prm.expand_first = int(kw.get("expand_first", True))
     prm.reserved = int(kw.get("rescue_any", False))
     prm.backfill = int(kw.get("backfill", False))
+    prm.global_pattern = int(kw.get("global_pattern", False))
     keep = []
     if kw.get("forced_dense"):
         fd = torch.zeros(cov.shape[0], dtype=torch.int32, device="cuda"); fd[list(kw["forced_dense"])] = 1
@@ -201,3 +202,27 @@ def test_route_with_many_ties_and_non_monotone_sequences():
             want, wrep = RT.route(LIB, cov, cost, np.ones(n_items, np.float32), RT.RouteParams(budget=budget, backfill=trial == 2))
             assert np.array_equal(got, want), (n_seg, trial)
             assert rep[0] == wrep.total_cost and rep[1] == wrep.total_risk and rep[3] == wrep.feasible
+
+
+@pytest.mark.parametrize("n_seg,Hq,Hkv", [(1, 32, 8), (4, 32, 8), (64, 32, 8)])
+def test_layer_level_router_is_bit_exact(n_seg, Hq, Hkv):
+    """One candidate for the whole layer: same decision, cost, risk (bit for bit) and fallback count as the oracle,
+    on the shared-memory path and (2048 items) on the path that reads the tables from global memory."""
+    rng = np.random.default_rng(900 + n_seg)
+    p = rs.Problem(Hq, Hkv, 64 * n_seg * 2, [128 * s for s in range(n_seg + 1)])
+    n_items = n_seg * Hq
+    for trial in range(5):
+        cov, pairs = instance(rng, n_items, LIB)
+        cost = 512 * pairs
+        vmax_sg = np.ones((n_seg, Hkv), dtype=np.float32)
+        dense_total = int(cost[:, -1].sum())
+        budget = int(dense_total * [0.05, 0.2, 0.5, 1.0, 0.0001][trial])
+        cert_max = [None, 0.3, None, 0.3, None][trial]
+        got, rep = gpu_route(p, LIB, cov, pairs, cost, vmax_sg, budget=budget, t_probe=77, global_pattern=True,
+                             cert_max=cert_max)
+        want, wrep = RT.route(LIB, cov, cost, np.ones(n_items, np.float32),
+                              RT.RouteParams(budget=budget, t_probe=77, global_pattern=True, cert_max=cert_max))
+        assert np.array_equal(got, want)
+        assert rep == (wrep.total_cost, wrep.total_risk, wrep.n_fallback, wrep.feasible)
+        if cert_max is None:
+            assert len(set(got.tolist())) == 1

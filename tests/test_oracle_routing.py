@@ -206,3 +206,32 @@ def test_greedy_order_is_the_order_of_running_maxima():
                 ch2[key[2]] = key[3]
                 tot2 += key[1]
             assert ch2 == choice and tot2 == total, (trial, frac)
+
+
+def test_global_router_is_the_best_constant_assignment():
+    """One candidate for the whole layer (the layer-level comparison router of Section 4): the exhaustive optimum over
+    the constant assignments, never better than the exhaustive optimum over all assignments."""
+    rng = np.random.default_rng(7)
+    n_feasible = 0
+    for trial in range(60):
+        cov, cost = _instance(rng)
+        budget = int(rng.integers(60, 420))
+        choice, rep = RT.route(LIB, cov, cost, np.ones(4, np.float32),
+                               RT.RouteParams(budget=budget, t_probe=5, global_pattern=True))
+        assert len(set(choice.tolist())) == 1
+        R, _ = RT.risks(LIB, cov, 1.0)
+        constant = [(sum(R[i, c] for i in range(4)), 5 + int(cost[:, c].sum()), c) for c in range(len(LIB))
+                    if 5 + int(cost[:, c].sum()) <= budget]
+        if not constant:
+            assert rep.feasible == 0 and int(cost[:, choice[0]].sum()) == min(int(cost[:, c].sum()) for c in range(len(LIB)))
+            continue
+        n_feasible += 1
+        assert rep.feasible == 1 and rep.total_cost <= budget
+        assert choice[0] == min(constant)[2]
+        best = RT.exhaustive_optimum(R, cost, budget, 5)
+        assert rep.total_risk >= best[0] - 1e-12
+    assert n_feasible > 20
+    # dense fits: the layer stays dense; nothing fits: cheapest candidate, marked infeasible
+    cov, cost = _instance(rng)
+    choice, rep = RT.route(LIB, cov, cost, np.ones(4, np.float32), RT.RouteParams(budget=405, t_probe=5, global_pattern=True))
+    assert np.all(choice == DENSE_C) and rep.total_risk == 0.0
