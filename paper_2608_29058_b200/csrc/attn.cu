@@ -16,6 +16,8 @@
 
 namespace {
 
+rs_smem_attr g_attn_smem;          // dynamic shared memory opt-in of rs_attn_kernel, per device
+
 constexpr int kThreads = 192;
 constexpr int kTileM = 128;
 constexpr int kChunk = 64;
@@ -768,12 +770,7 @@ int launch_attn(const rs_problem* p, const void* Q, const void* K, const void* V
                                                       reinterpret_cast<const __nv_bfloat16*>(V), Kp, Vp);
   }
   const size_t smem = attn_smem_bytes(P.n);
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(rs_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024) != cudaSuccess)
-      return RS_ERR_CUDA;
-    attr_set = true;
-  }
+  if (rs_ensure_dynamic_smem(g_attn_smem, rs_attn_kernel, 116 * 1024) != RS_OK) return RS_ERR_CUDA;
   rs_attn_kernel<<<n_work, kThreads, smem, stream>>>(tmQ, tmK, tmV, tmKp, tmVp, P);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }
@@ -878,8 +875,7 @@ extern "C" int rs_dense_prefill_attn_noalloc(const rs_problem* p, const void* Q,
   rs_attn_cost_kernel<<<(n_work + 255) / 256, 256, 0, stream>>>(P, n_work, cost, items);
   const int n_bins = (P.n >> 6) + 66;
   rs_attn_order_kernel<<<P.Hkv, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work / P.Hkv, n_bins, cost, items, order);
-  if (cudaFuncSetAttribute(rs_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024) != cudaSuccess)
-    return RS_ERR_CUDA;
+  if (rs_ensure_dynamic_smem(g_attn_smem, rs_attn_kernel, 116 * 1024) != RS_OK) return RS_ERR_CUDA;
   // the gathered-column maps are never read by dense tiles; they alias K and V
   rs_attn_kernel<<<n_work, kThreads, attn_smem_bytes(P.n), stream>>>(tmQ, tmK, tmV, tmK, tmV, P);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/routesparse.h"
 
 #define RS_MAX_SEGMENTS 64
@@ -217,3 +219,17 @@ int rs_side_join(cudaStream_t main);
 int rs_check_problem(const rs_problem* p);
 int rs_check_device();
 static inline size_t rs_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) is a per-device setting: it is applied once per (kernel, device)
+// and remembered in a bit mask indexed by the device ordinal.  Safe to call from several threads.
+struct rs_smem_attr { std::atomic<unsigned long long> done{0ull}; };
+template <typename Kernel>
+static inline int rs_ensure_dynamic_smem(rs_smem_attr& a, Kernel kernel, int bytes) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return RS_ERR_CUDA;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (dev < 64 && (a.done.load(std::memory_order_acquire) & bit)) return RS_OK;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return RS_ERR_CUDA;
+  if (dev < 64) a.done.fetch_or(bit, std::memory_order_release);
+  return RS_OK;
+}

@@ -1021,12 +1021,9 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   for (int c = 0; c < n_cand; ++c) n_vs += (lib[c].pattern == RS_VERTICAL_SLASH);
   const int sel_groups = choice ? 1 : (n_vs + kSelMaxC - 1) / kSelMaxC;
   const size_t sel_smem = (size_t)(choice ? 1 : kSelMaxC) * kBins * sizeof(unsigned int);
-  static bool sel_attr = false;
-  if (!sel_attr) {
-    if (cudaFuncSetAttribute(rs_vs_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)(kSelMaxC * kBins * sizeof(unsigned int))) != cudaSuccess) return RS_ERR_CUDA;
-    sel_attr = true;
-  }
+  static rs_smem_attr sel_attr;
+  if (rs_ensure_dynamic_smem(sel_attr, rs_vs_select_kernel, (int)(kSelMaxC * kBins * sizeof(unsigned int))) != RS_OK)
+    return RS_ERR_CUDA;
   const bool two_chains = any_vs && !skip_vs && (any_bs || stats != nullptr);
   cudaStream_t side = stream;
   if (two_chains) {
@@ -1098,12 +1095,8 @@ extern "C" int rs_mixture_coverage(const rs_problem* p, const rs_candidate* lib,
   if (n_vs > kMixMaxVS || n_bs > kMixMaxBS) return RS_ERR_UNSUPPORTED_SHAPE;
   const size_t smem = (size_t)nb * 4 + (size_t)idx_eval->kb_cap * 4 + (size_t)kMixMaxVS * nb * 4 + kMixMaxVS * 128 * 4 +
                       (size_t)kMixMaxBS * (nb / 32 + 1) * 4 + kMixMaxVS * 64 * 4;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(rs_mix_cov_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
-      return RS_ERR_CUDA;
-    attr_set = true;
-  }
+  static rs_smem_attr mix_attr;
+  if (rs_ensure_dynamic_smem(mix_attr, rs_mix_cov_kernel, 64 * 1024) != RS_OK) return RS_ERR_CUDA;
   if (smem > 64 * 1024) return RS_ERR_UNSUPPORTED_SHAPE;
   rs_mix_cov_kernel<<<dim3(r, n_items, 4), 256, smem, stream>>>(P, M);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;

@@ -618,13 +618,10 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
   if (rs_make_tmap_bf16_2d(&tmQ, Q, (uint64_t)P.Hq * P.n, RS_HEAD_DIM, 64, 64) ||
       rs_make_tmap_bf16_2d(&tmK, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kKeyTile, 64))
     return RS_ERR_CUDA;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(rs_probe_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::total) != cudaSuccess ||
-        cudaFuncSetAttribute(rs_probe_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Smem::total) != cudaSuccess)
-      return RS_ERR_CUDA;
-    attr_set = true;
-  }
+  static rs_smem_attr attr_pass1, attr_pass2;
+  if (rs_ensure_dynamic_smem(attr_pass1, rs_probe_kernel<1>, (int)Smem::total) != RS_OK ||
+      rs_ensure_dynamic_smem(attr_pass2, rs_probe_kernel<2>, (int)Smem::total) != RS_OK)
+    return RS_ERR_CUDA;
   // The pooled means and the value norms only read Q, K, V: they run beside the two probe passes, on the side
   // stream.  Pass 1 is enqueued first so that its CTAs (one per SM, most of the shared memory) are resident before
   // the small streaming CTAs fill what is left; the other way round the streaming kernels would run alone.

@@ -281,12 +281,8 @@ extern "C" int rs_probe_pooled(const rs_problem* p, const void* Q, const void* K
   per = (per + kKB - 1) / kKB * kKB;
   ctas = (nbg + per - 1) / per;
   const size_t smem = 128 * 256 * 2 + kKB * 128 * 4;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(rs_pp_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return RS_ERR_CUDA;
-    attr_set = true;
-  }
+  static rs_smem_attr logits_attr;
+  if (rs_ensure_dynamic_smem(logits_attr, rs_pp_logits_kernel, (int)smem) != RS_OK) return RS_ERR_CUDA;
   rs_pp_logits_kernel<<<dim3(ctas, P.n_seg * P.Hkv), 256, smem, stream>>>(P, per);
   rs_pp_softmax_kernel<<<dim3(r, P.n_seg * P.Hq), 256, 0, stream>>>(P);
   rs_pp_reduce_kernel<<<dim3((nbg + 255) / 256, P.n_seg * P.Hq), 256, 0, stream>>>(P);

@@ -457,12 +457,8 @@ extern "C" int rs_route(const rs_problem* p, const rs_candidate* lib, int n_cand
   const int n_pairs = n_items * n_cand;
   const size_t smem = (size_t)n_items * (sizeof(Sub) + sizeof(int)) + (n_pairs <= kCachePairs ? (size_t)n_pairs * (16 + sizeof(Sub)) : 0) +
                       (size_t)n_items * 8 + 32 + (n_pairs <= kSortPairs ? (size_t)kSortPairs * 4 + n_pairs : 0);
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(rs_route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-      return RS_ERR_CUDA;
-    attr_set = true;
-  }
+  static rs_smem_attr route_attr;
+  if (rs_ensure_dynamic_smem(route_attr, rs_route_kernel, 200 * 1024) != RS_OK) return RS_ERR_CUDA;
   rs_route_kernel<<<1, kThreads, smem, (cudaStream_t)stream_>>>(A);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }
