@@ -148,6 +148,7 @@ extern "C" int rs_workspace_bytes(const rs_problem* p, const rs_candidate* lib, 
   int max_kv = 0;
   for (int c = 0; c < n_cand; ++c)
     if (lib[c].pattern == RS_VERTICAL_SLASH && lib[c].b0 > max_kv) max_kv = lib[c].b0;
+  if (max_kv > p->n_keys) max_kv = p->n_keys;
   size_t need = rs_attn_workspace_bytes(p, max_kv);
   size_t b = rs_probe_workspace_bytes(p);
   if (b > need) need = b;

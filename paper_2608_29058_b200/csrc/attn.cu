@@ -714,6 +714,7 @@ int launch_attn(const rs_problem* p, const void* Q, const void* K, const void* V
     if (lib[c].pattern == RS_A_SHAPE && (lib[c].b1 < 1 || lib[c].b0 < 0)) return RS_ERR_INVALID_ARG;
     if (lib[c].pattern < 0 || lib[c].pattern > 3) return RS_ERR_INVALID_ARG;
   }
+  if (max_kv > p->n_keys) max_kv = p->n_keys;      // a column list never holds more than n_keys entries
   bool vs_eval_layout = false;
   if (choice != nullptr && any_vs) {
     const int n_items_ = p->n_segments * p->n_q_heads;

@@ -228,3 +228,44 @@ def test_streamed_host_passes_match_the_plain_call():
     rs.check_status(layer.status, "streamed passes")
     for k, (_, _, _, Oh) in enumerate(hosts):
         assert torch.equal(Oh, want[k]), k
+
+
+def test_budgets_larger_than_the_sequence():
+    """One 64-row block with vertical-slash budgets beyond the number of keys: the lists are clamped to the keys that exist."""
+    cands = [C(PT.VERTICAL_SLASH, 8, 139), C(PT.VERTICAL_SLASH, 119, 140), C(PT.BLOCK_SPARSE, 4), C(PT.DENSE)]
+    run_and_check(tiny_spec(80, 64, 4, 2), [0, 64], cands, rs.RouteConfig(budget_frac=0.6, cert_max=0.8), "one block")
+
+
+def _random_case(seed):
+    """Random geometry, segments, candidate library and router settings for the stage-by-stage comparison."""
+    rng = np.random.default_rng(seed)
+    Hkv = int(rng.choice([1, 2, 4]))
+    Hq = Hkv * int(rng.choice([1, 2, 4]))
+    nb = int(rng.integers(1, 24))
+    n_seg = int(rng.integers(1, min(4, nb) + 1))
+    cuts = sorted(rng.choice(np.arange(1, nb), size=n_seg - 1, replace=False).tolist()) if n_seg > 1 else []
+    bounds = [0] + [64 * c for c in cuts] + [64 * nb]
+    cands = [C(PT.A_SHAPE, int(rng.integers(0, 100)), int(rng.integers(1, 400))) for _ in range(int(rng.integers(0, 3)))]
+    cands.sort(key=lambda c: c.b0 + c.b1)
+    # candidate evaluation needs sink and window disjoint on the probe rows of every segment
+    cands = [c for c in cands if all(c.b1 >= q1 or q1 - 64 - c.b1 + 1 >= c.b0 for q1 in bounds[1:])]
+    kv = ks = 0
+    for a, b in sorted((int(rng.integers(1, 200)), int(rng.integers(1, 300))) for _ in range(int(rng.integers(0, 4)))):
+        kv, ks = max(kv + 1, a), max(ks + 1, b)           # budgets nested inside the family
+        cands.append(C(PT.VERTICAL_SLASH, kv, ks))
+    for kb in sorted(set(int(x) for x in rng.integers(1, 12, size=int(rng.integers(0, 3))))):
+        cands.append(C(PT.BLOCK_SPARSE, kb))
+    cands.append(C(PT.DENSE))
+    cfg = rs.RouteConfig(budget_frac=float(rng.uniform(0.05, 0.9)), alpha=float(rng.choice([0.0, 1.0, 2.5])),
+                         delta_q=float(rng.choice([0.0, 0.02])), cert_max=[None, 0.05, 0.3, 0.8][int(rng.integers(0, 4))],
+                         cert_mode=int(rng.choice([rs.RS_CERT_REL, rs.RS_CERT_ABS])), expand_first=bool(rng.integers(0, 2)))
+    spec = tiny_spec(1000 + seed, 64 * nb, Hq, Hkv, toeplitz=bool(rng.integers(0, 2)), n_vert=int(rng.integers(0, 6)))
+    return spec, bounds, cands, cfg
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_small_layers(seed):
+    """Seeded random cases of the whole path (ragged segment lengths, one-block segments, budgets beyond the segment,
+    libraries without some family, every router setting), each checked stage by stage like the fixed cases above."""
+    spec, bounds, cands, cfg = _random_case(seed)
+    run_and_check(spec, bounds, cands, cfg, f"random {seed}")
