@@ -169,7 +169,11 @@ int rs_pool_queries(const rs_problem* p, const void* Q, const rs_candidate* lib,
  *   (qpool . kpool / sqrt(d); `bscore` [n_items][n_keys/64][n_keys/64], indexed by global query block,
  *   replaces the fused product when not NULL).
  * choice == NULL: evaluate every candidate of every item (lists + stats, see rs_index_set).
- * choice != NULL (device int32[n_items]): materialise only the chosen candidate of each item. */
+ * choice != NULL (device int32[n_items]): materialise only the chosen candidate of each item.
+ * Limits: every segment needs at least 64 rows (the probe rows), and with stats != NULL an A-shape candidate whose sink
+ * columns and window overlap on the probe rows of some segment (window < segment end and segment end - 64 - window + 1 <
+ * sink columns) is refused with RS_ERR_UNSUPPORTED_SHAPE: the joint coverage of the two parts cannot be had from the
+ * column and offset masses alone.  Budgets larger than a segment are clamped to what exists. */
 int rs_build_indices(const rs_problem* p, const rs_candidate* lib, int n_cand,
                      const float* vert, const float* slash, const float* qpool, const float* kpool,
                      const float* bscore, const int32_t* choice,
@@ -291,6 +295,40 @@ int rs_regressor_eval(const rs_problem* p, const rs_candidate* lib, int n_cand, 
  * Oa, Ob: [n_rows][128] bf16 (o_dtype 0) or fp32 (o_dtype 1); err, norm_a (may be NULL): device fp32[n_rows]. */
 int rs_output_error(long long n_rows, const void* Oa, const void* Ob, int o_dtype, float* err, float* norm_a,
                     int32_t* status, void* stream);
+
+/* The whole hot path of one layer in one call (the procedure table of Section 3.4): rs_probe (pooling all of Q
+ * deferred), rs_build_indices in evaluation mode, rs_route, rs_pool_queries, rs_build_indices for the routed
+ * block-sparse rows, one rs_sparse_prefill_attn launch, rs_certificate on the probe rows.  Host code only: it
+ * enqueues those calls on `stream` in that order with the arguments below; the routes never leave the device, so the
+ * call returns before any kernel has run and can be captured into a CUDA graph.  Results are the same, bit for bit,
+ * as issuing the seven calls one by one.
+ *   params      as for rs_route.  params->fixed_choice != NULL skips candidate evaluation (stats are not written) and
+ *               runs the given routes; otherwise routing is online and idx_eval must be in the evaluation layout
+ *   cost        as for rs_route (NULL: 512 x selected pairs)
+ *   b           device buffers, all owned by the caller; shapes as documented at the call that fills them.
+ *               descr, report, onorm, counters, probe_rows (with m_row, cert_row, m_head, cert_head) may be NULL;
+ *               without probe_rows or onorm the certificate step is skipped.  probe_rows: the last 64 rows of every
+ *               segment, segment after segment (the layout of lse_probe); vmax of the last segment bounds Eq. 5
+ *   ws          one workspace of rs_workspace_bytes() bytes serves every step
+ * Errors: the first failing step's code; kernels of earlier steps stay enqueued. */
+typedef struct {
+  float *vert, *slash, *lse_probe, *qpool, *kpool, *vmax, *descr;
+  rs_cand_stats* stats;
+  rs_index_set idx_eval;       /* evaluation layout (n_vs_slots = n_items * n_cand) */
+  rs_index_set idx;            /* materialised layout */
+  int32_t* choice;             /* [n_items] out */
+  rs_route_report* report;
+  void* O; int32_t o_dtype;    /* 0: bf16, 1: fp32 */
+  int32_t n_probe_rows;
+  float *lse_sel, *onorm;
+  uint64_t* counters;
+  const int32_t* probe_rows;
+  float *m_row, *cert_row, *m_head, *cert_head;
+} rs_layer_buffers;
+int rs_routed_prefill_layer(const rs_problem* p, const void* Q, const void* K, const void* V,
+                            const rs_candidate* lib, int n_cand, const rs_route_params* params,
+                            const int64_t* cost, const rs_layer_buffers* b, void* ws, size_t ws_bytes,
+                            int32_t* status, void* stream);
 
 /* Self test of the bounded device-side wait every kernel of this library uses (no passage of the paper: the waits
  * exist because the kernels synchronise TMA, tensor-core and softmax roles through mbarriers).  Launches one small

@@ -46,10 +46,19 @@ class rs_route_params(C.Structure):
                 ("backfill", C.c_int32), ("global_pattern", C.c_int32), ("cov_mix", C.c_void_p), ("mix_rows", C.c_int32 * 4)]
 
 
+class rs_layer_buffers(C.Structure):
+    _fields_ = [("vert", C.c_void_p), ("slash", C.c_void_p), ("lse_probe", C.c_void_p), ("qpool", C.c_void_p),
+                ("kpool", C.c_void_p), ("vmax", C.c_void_p), ("descr", C.c_void_p), ("stats", C.c_void_p),
+                ("idx_eval", rs_index_set), ("idx", rs_index_set), ("choice", C.c_void_p), ("report", C.c_void_p),
+                ("O", C.c_void_p), ("o_dtype", C.c_int32), ("n_probe_rows", C.c_int32), ("lse_sel", C.c_void_p),
+                ("onorm", C.c_void_p), ("counters", C.c_void_p), ("probe_rows", C.c_void_p), ("m_row", C.c_void_p),
+                ("cert_row", C.c_void_p), ("m_head", C.c_void_p), ("cert_head", C.c_void_p)]
+
+
 EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "rs_build_indices", "rs_route",
            "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate",
            "rs_selftest_wait_timeout", "rs_probe_pooled", "rs_probe_pooled_scratch_floats", "rs_regressor_eval",
-           "rs_output_error", "rs_mixture_coverage", "rs_pool_queries"]
+           "rs_output_error", "rs_mixture_coverage", "rs_pool_queries", "rs_routed_prefill_layer"]
 
 
 def lib_path() -> str:
@@ -201,6 +210,13 @@ def rs_build_indices(p: Problem, lib, vert, slash, qpool, kpool, bscore, choice,
 def rs_route(p: Problem, lib, stats, cost, vmax, params: rs_route_params, choice, report, status):
     _check(load().rs_route(C.byref(p.c), lib, len(lib), _ptr(stats), _ptr(cost), _ptr(vmax), C.byref(params),
                            _ptr(choice), _ptr(report), _ptr(status), _stream()), "rs_route")
+
+
+def rs_routed_prefill_layer(p: Problem, Q, K, V, lib, params: rs_route_params, cost, bufs: rs_layer_buffers, ws, status):
+    """The whole layer pass in one library call (probe, evaluation, routing, materialisation, attention, certificate)."""
+    _check(load().rs_routed_prefill_layer(C.byref(p.c), _ptr(Q), _ptr(K), _ptr(V), lib, len(lib), C.byref(params),
+                                          _ptr(cost), C.byref(bufs), _ptr(ws), C.c_size_t(ws.numel()), _ptr(status),
+                                          _stream()), "rs_routed_prefill_layer")
 
 
 def rs_sparse_prefill_attn(p: Problem, Q, K, V, lib, idx: IndexSet, choice, O, lse_sel, onorm, counters, ws, status):

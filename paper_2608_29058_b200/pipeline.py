@@ -103,6 +103,8 @@ class RoutedPrefillLayer:
         self.m_head = torch.empty((Hq,), **f32)
         self.cert_head = torch.empty((Hq, 2), **f32)
         self.prm = rs.rs_route_params()
+        self.one_call = True        # forward() = one rs_routed_prefill_layer call where that entry point covers the pass
+        self._bufs = None
         self._forced = None
         self.events = None
         self.covmix = torch.zeros((p.n_items, len(self.cands), 4), dtype=torch.int64, device=device)
@@ -111,6 +113,20 @@ class RoutedPrefillLayer:
         self.cost_table = None      # int64 [n_items, n_cand] measured kernel time (ns); None: FLOPs of the selected pairs
         self.cost_budget = None     # layer budget in the table's unit
         self.cost_t_probe = 0
+
+    def _layer_buffers(self):
+        if self._bufs is None:
+            b = rs.rs_layer_buffers()
+            for name in ("vert", "slash", "lse_probe", "qpool", "kpool", "vmax", "stats", "choice", "report", "O",
+                         "lse_sel", "onorm", "counters", "probe_rows", "m_row", "cert_row", "m_head", "cert_head"):
+                setattr(b, name, getattr(self, name).data_ptr())
+            b.descr = None
+            b.idx_eval, b.idx = self.idx_eval.c, self.idx.c
+            b.o_dtype = 1 if self.O.dtype == torch.float32 else 0
+            b.n_probe_rows = int(self.probe_rows.numel())
+            self._bufs = b
+        self._bufs.O = self.O.data_ptr()          # StreamedPrefill rotates the output buffer between passes
+        return self._bufs
 
     # ------------------------------------------------------------------ steps (each only enqueues kernels)
     def probe(self, Q, K, V, lazy_qpool: bool = False):
@@ -126,7 +142,7 @@ class RoutedPrefillLayer:
         rs.rs_build_indices(self.p, self.lib, self.vert, self.slash, self.qpool, self.kpool, None, None,
                             self.idx_eval, self.stats, self.ws, self.status)
 
-    def route(self, forced_dense: Optional[torch.Tensor] = None):
+    def _fill_route_params(self, forced_dense: Optional[torch.Tensor] = None):
         c, prm = self.cfg, self.prm
         if self.cost_table is not None:
             prm.budget, prm.t_probe = int(self.cost_budget), int(self.cost_t_probe)
@@ -153,6 +169,10 @@ class RoutedPrefillLayer:
         self._forced = forced_dense
         prm.forced_dense = None if forced_dense is None else forced_dense.data_ptr()
         prm.fixed_choice = None
+        return prm
+
+    def route(self, forced_dense: Optional[torch.Tensor] = None):
+        prm = self._fill_route_params(forced_dense)
         rs.rs_route(self.p, self.lib, self.stats, self.cost_table, self.vmax, prm, self.choice, self.report, self.status)
 
     def materialise(self, reuse_evaluation: bool = False):
@@ -302,6 +322,19 @@ class RoutedPrefillLayer:
     def forward(self, Q, K, V, fixed_choice: Optional[torch.Tensor] = None,
                 forced_dense: Optional[torch.Tensor] = None, record_events: bool = False) -> torch.Tensor:
         """Routed sparse prefill attention of one layer; returns O (device). Nothing synchronises."""
+        staged = (record_events or self.cfg.mixture_u or (self.regressor is not None and self.cfg.beta > 0.0)
+                  or not self.one_call)
+        if not staged:
+            # the whole pass as one library call; the staged path below issues the same calls one by one (needed for
+            # per-stage timing and for the steps the one-call entry point does not cover: mixture coverage, predictor e)
+            prm = self._fill_route_params(forced_dense if fixed_choice is None else None)
+            prm.fixed_choice = None if fixed_choice is None else fixed_choice.data_ptr()
+            rs.rs_routed_prefill_layer(self.p, Q, K, V, self.lib, prm, self.cost_table, self._layer_buffers(), self.ws,
+                                       self.status)
+            prm.fixed_choice = None
+            self._reuse_eval = fixed_choice is None and len(self.cands) > 1
+            self.events = None
+            return self.O
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(7)] if record_events else None
         mark = (lambda i: ev[i].record()) if record_events else (lambda i: None)
         mark(0)

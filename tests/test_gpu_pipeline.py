@@ -269,3 +269,28 @@ def test_random_small_layers(seed):
     libraries without some family, every router setting), each checked stage by stage like the fixed cases above."""
     spec, bounds, cands, cfg = _random_case(seed)
     run_and_check(spec, bounds, cands, cfg, f"random {seed}")
+
+
+@pytest.mark.parametrize("online", [True, False])
+def test_one_call_layer_equals_the_staged_calls(online):
+    """rs_routed_prefill_layer enqueues the same seven calls the staged path issues one by one: every output is
+    bit-identical, with online routing and with given routes."""
+    n, Hq, Hkv = 1280, 8, 2
+    L = make_layer(tiny_spec(73, n, Hq, Hkv))
+    p = rs.Problem(Hq, Hkv, n, [0, 512, 1280])
+    cands = [(rs.RS_A_SHAPE, 8, 128), (rs.RS_VERTICAL_SLASH, 32, 48), (rs.RS_VERTICAL_SLASH, 64, 96),
+             (rs.RS_BLOCK_SPARSE, 3, 0), (rs.RS_BLOCK_SPARSE, 6, 0), (rs.RS_DENSE, 0, 0)]
+    Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+    fixed = None if online else torch.tensor([i % len(cands) for i in range(p.n_items)], dtype=torch.int32, device="cuda")
+    outs = []
+    for one_call in (False, True):
+        layer = rs.RoutedPrefillLayer(p, cands, rs.RouteConfig(budget_frac=0.4, cert_max=0.5))
+        layer.one_call = one_call
+        layer.forward(Q, K, V, fixed_choice=fixed)
+        rs.check_status(layer.status, f"one_call={one_call}")
+        outs.append([t.clone() for t in (layer.O, layer.lse_sel, layer.onorm, layer.choice, layer.m_row, layer.m_head,
+                                         layer.cert_head, layer.counters)] + ([layer.stats.clone(), layer.report.clone()] if online else []))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    if online:
+        assert len(set(outs[0][3].tolist())) > 1
