@@ -128,3 +128,63 @@ def test_config2_full_size_fixed_routes():
             n_diff = sum(len(np.setxor1d(a, b)) for a, b in zip(sets[h].blk, ref))
             assert n_diff <= 0.002 * 100 * (n // 64)          # only near-ties of the fp32 fused scores may differ
     _check_sampled_attention(L, spec, layer, sets, heads, [1, 255, 511])
+
+
+def test_config4_full_size_segmented_layer():
+    """One layer of the segmented 128K recipe (four segments of 32K with different planted structure, per-segment
+    routing, one launch): probe and candidate statistics of sampled (segment, head) items, the routing of all 128 items,
+    and the attention output on sampled query blocks of every segment (first, interior and last block)."""
+    from synth import config4_layer_spec
+    spec = config4_layer_spec(0, n=131072, seg_len=32768)
+    L = make_layer(spec)
+    n, Hq, Hkv = spec.n, spec.n_q_heads, spec.n_kv_heads
+    bounds = spec.seg_bounds()
+    p = rs.Problem(Hq, Hkv, n, bounds)
+    layer = rs.RoutedPrefillLayer(p, None, rs.RouteConfig(budget_frac=0.15, cert_max=0.05))
+    Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+    layer.forward(Q, K, V)
+    rs.check_status(layer.status, "config 4")
+    cands = PT.default_library()
+    choice = layer.choice.cpu().numpy()
+    stats = layer.stats.cpu().numpy()
+    cov, pairs = stats[:, :, :4].astype(np.uint64), stats[:, :, 4]
+    G = Hq // Hkv
+    sampled = [(0, 3), (1, 12), (2, 22), (3, 31)]                     # (segment, head)
+    for s, h in sampled:
+        q0, q1 = bounds[s], bounds[s + 1]
+        item = s * Hq + h
+        Qf, Kf = bf16_bits_to_f64(L["Q"][h]), bf16_bits_to_f64(L["K"][h // G])
+        pr = OP.probe_rows(Qf, Kf, q1)
+        vert, slash = layer.vert[s, h].cpu().numpy(), layer.slash[s, h].cpu().numpy()
+        assert _close(vert[:, :q1], pr.vert) and _close(slash[:, :q1], pr.slash), (s, h)
+        assert np.all(vert[:, q1:] == 0)
+        assert np.abs(layer.lse_probe[h, s].cpu().numpy() - pr.lse).max() < 1e-3
+        for c, cand in enumerate(cands):
+            if cand.pattern == PT.BLOCK_SPARSE:
+                assert pairs[item, c] == sum((min(cand.b0, qb + 1) - 1) * 4096 + 2080 for qb in range(q0 // 64, q1 // 64))
+                continue
+            ix = PT.build_indices(cand, q0, q1, vert[:, :q1], slash[:, :q1], None)
+            assert pairs[item, c] == PT.pairs(ix), (s, h, cand)
+            if cand.pattern != PT.DENSE:
+                assert cov[item, c].tolist() == PT.coverage_fx(ix, vert[:, :q1], slash[:, :q1]).tolist(), (s, h, cand)
+    vmax = layer.vmax.cpu().numpy()
+    vmax_item = np.array([vmax[it // Hq, (it % Hq) // G] for it in range(p.n_items)], np.float32)
+    want, wrep = RT.route(cands, cov, 512 * pairs, vmax_item, RT.RouteParams(
+        budget=int(0.15 * rs.dense_flops(p.seg_bounds, Hq)), t_probe=rs.probe_flops(p.seg_bounds, Hq), cert_max=0.05))
+    assert np.array_equal(choice, want)
+    rep = layer.route_report()
+    assert rep["total_cost"] == wrep.total_cost and rep["n_fallback"] == wrep.n_fallback
+    assert len(set(choice.tolist())) > 2                              # the segments really get different routes
+    sets = download_sets(layer, cands, choice)
+    O = layer.O
+    for s, h in sampled:
+        q0, q1 = bounds[s], bounds[s + 1]
+        ix = sets[s * Hq + h]
+        Qf, Kf, Vf = (bf16_bits_to_f64(L["Q"][h]), bf16_bits_to_f64(L["K"][h // G]), bf16_bits_to_f64(L["V"][h // G]))
+        for qb in (q0 // 64, (q0 + q1) // 128 + 1, q1 // 64 - 1):
+            rows = np.arange(64 * qb, 64 * qb + 64)
+            Om, lo, _ = A.masked_attention(Qf, Kf, Vf, lambda r, nk: PT.mask_rows(ix, r, nk), rows, chunk=64)
+            got = O[h, 64 * qb:64 * qb + 64].float().cpu().numpy()
+            err = np.abs(got - Om)
+            assert err.max() <= 2e-2 + 2.0 ** -9 * np.abs(Om).max() and err.mean() <= 5e-3, (s, h, qb, err.max())
+            assert np.abs(layer.lse_sel[h, 64 * qb:64 * qb + 64].cpu().numpy() - lo).max() < 2e-3
