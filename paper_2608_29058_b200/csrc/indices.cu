@@ -26,6 +26,7 @@ struct IdxParams {
   float* bs_eval_ws;  // [n_items][nb] pooled scores of each segment's last query block
   int32_t* status;
   float scale;
+  int bs_rows_first;  // first query block served by rs_bs_rows_kernel (the shorter rows go to the warp-per-row kernel)
 };
 
 // floor(x * 2^32) of a non-negative float, exactly, from its bits (no float-to-integer conversion unit involved)
@@ -676,7 +677,7 @@ rs_bs_rows_kernel(IdxParams P) {
   __shared__ uint32_t hist[256];
   __shared__ uint32_t sh[8];
   __shared__ unsigned int wcnt[16];
-  const int qb = blockIdx.x, h = blockIdx.y;
+  const int qb = P.bs_rows_first + blockIdx.x, h = blockIdx.y;
   const int s = seg_of_block(P, qb);
   const int item = s * P.Hq + h;
   const rs_candidate cand = P.lib[P.choice[item]];
@@ -691,6 +692,77 @@ rs_bs_rows_kernel(IdxParams P) {
   const int cnt = select_row(score, qb, min(k_b, qb + 1) - 1, qb, P.out.bs_blk + orow * P.out.kb_cap, P.out.kb_cap,
                              hist, sh, wcnt);
   if (tid == 0) P.out.bs_count[orow] = cnt;
+}
+
+// The same selection for query blocks with at most 1024 candidate key blocks, one warp per query block: every lane
+// keeps its strided share of the row's ranking keys in registers, the take-th largest key is built bit by bit from
+// the top (a count over the row per bit), then an ordered compaction by ballots writes the ascending list.  Same
+// order as select_row (key descending, index ascending), without block-wide barriers.
+constexpr int kWarpRowMax = 1024;
+
+__global__ void __launch_bounds__(256)
+rs_bs_rows_warp_kernel(IdxParams P, int qb_end) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qb = blockIdx.x * 8 + warp, h = blockIdx.y;
+  if (qb >= qb_end) return;
+  const int s = seg_of_block(P, qb);
+  const int item = s * P.Hq + h;
+  const rs_candidate cand = P.lib[P.choice[item]];
+  if (cand.pattern != RS_BLOCK_SPARSE) return;
+  const float* row = (P.bscore != nullptr) ? P.bscore + ((size_t)item * P.nb + qb) * P.nb
+                                           : P.bs_ws + ((size_t)h * P.nb + qb) * P.nb;
+  const int m = qb;                                   // candidates: key blocks 0 .. qb - 1
+  const size_t orow = (size_t)h * P.nb + qb;
+  int32_t* out = P.out.bs_blk + orow * P.out.kb_cap;
+  const int cap = P.out.kb_cap;
+  const int take = min(min(min(cand.b0, cap), qb + 1) - 1, m);
+  uint32_t key[kWarpRowMax / 32];
+#pragma unroll
+  for (int c = 0; c < kWarpRowMax / 32; ++c) {
+    const int i = c * 32 + lane;
+    key[c] = (i < m) ? f32_order_key(row[i]) : 0u;    // finite scores have keys > 0: the padding is never counted
+  }
+  uint32_t T = 0u;
+  int k_eq = 0;
+  if (take > 0) {
+    for (int b = 31; b >= 0; --b) {
+      const uint32_t Tc = T | (1u << b);
+      int cnt = 0;
+#pragma unroll
+      for (int c = 0; c < kWarpRowMax / 32; ++c)
+        if (c * 32 < m) cnt += (key[c] >= Tc) ? 1 : 0;
+      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      if (cnt >= take) T = Tc;
+    }
+    int gt = 0;
+#pragma unroll
+    for (int c = 0; c < kWarpRowMax / 32; ++c)
+      if (c * 32 < m) gt += (key[c] > T) ? 1 : 0;
+    k_eq = take - __reduce_add_sync(0xffffffffu, gt);
+  }
+  const unsigned int lt_mask = (1u << lane) - 1u;
+  int pos = 0, eq_run = 0;
+#pragma unroll
+  for (int c = 0; c < kWarpRowMax / 32; ++c) {
+    if (c * 32 < m && take > 0) {
+      const int i = c * 32 + lane;
+      const bool in = i < m;
+      const bool is_eq = in && key[c] == T;
+      const unsigned int beq = __ballot_sync(0xffffffffu, is_eq);
+      const bool tk = in && (key[c] > T || (is_eq && eq_run + __popc(beq & lt_mask) < k_eq));
+      const unsigned int bt = __ballot_sync(0xffffffffu, tk);
+      if (tk) {
+        const int p = pos + __popc(bt & lt_mask);
+        if (p < cap) out[p] = i;
+      }
+      pos += __popc(bt);
+      eq_run += __popc(beq);
+    }
+  }
+  if (lane == 0) {
+    if (take < cap) out[take] = qb;                   // the diagonal block is the largest index: list stays ascending
+    P.out.bs_count[orow] = take + 1;
+  }
 }
 
 // Fused pooled scores for the items routed to block-sparse: 64 x 64 tiles of qpool[h] kpool[g]^T / sqrt(d),
@@ -1046,7 +1118,13 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
         const int nt = (nb + 63) / 64;
         rs_bs_scores_kernel<<<dim3(nt, nt, P.Hq), 256, 0, side>>>(P);
       }
-      rs_bs_rows_kernel<<<dim3(nb, P.Hq), 256, (size_t)nb * sizeof(float), side>>>(P);
+      // short rows one warp each; rows with more than 1024 candidate blocks one thread block each
+      const int n_short = nb < kWarpRowMax + 1 ? nb : kWarpRowMax + 1;       // query blocks 0 .. 1024
+      rs_bs_rows_warp_kernel<<<dim3((n_short + 7) / 8, P.Hq), 256, 0, side>>>(P, n_short);
+      if (nb > n_short) {
+        P.bs_rows_first = n_short;
+        rs_bs_rows_kernel<<<dim3(nb - n_short, P.Hq), 256, (size_t)nb * sizeof(float), side>>>(P);
+      }
     }
   }
   if (two_chains) {
