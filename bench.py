@@ -339,6 +339,8 @@ def main():
 
     names = ["probe", "evaluate", "route", "materialise", "attention", "certificate"]
     stages = {nm: float(np.mean([ev[i].elapsed_time(ev[i + 1]) for ev in stage_events])) for i, nm in enumerate(names)}
+    # medians as well: one slow event pair (a clock change between two stage events) shifts the mean of a 0.01 ms stage
+    stages_med = {nm: float(np.median([ev[i].elapsed_time(ev[i + 1]) for ev in stage_events])) for i, nm in enumerate(names)}
     step_ms = [ev[0].elapsed_time(ev[6]) for ev in stage_events]      # per-step device time (first to last stage event)
     step_stats = {"median": float(np.median(step_ms)), "p95": float(np.percentile(step_ms, 95)),
                   "min": float(np.min(step_ms)), "max": float(np.max(step_ms)), "n": len(step_ms)}
@@ -492,6 +494,8 @@ def main():
         "speedup_vs_own_dense": (dense_ms / ms) if dense_ms else None,
         "dense_tflops": (f_dense / (dense_ms * 1e-3) / 1e12) if dense_ms else None,
         "stage_ms": stages, "overhead_over_attention": overhead_ms / attn_ms,
+        "stage_ms_median": stages_med,
+        "overhead_over_attention_median": (sum(stages_med.values()) - stages_med["attention"]) / stages_med["attention"],
         "flops": {"selected_pairs": f_mask, "issued_tiles": f_tile, "dense": f_dense,
                   "selected_fraction_of_dense": f_mask / f_dense},
         "routes": hist, "route_report": layer.route_report() if not fixed else None,
