@@ -4,5 +4,5 @@ The product is the C-ABI library built from csrc/ (see include/routesparse.h); t
 Python binding over it.  PyTorch is used for device memory and streams only.
 """
 from .binding import *  # noqa: F401,F403
-from .pipeline import (RoutedPrefillLayer, RouteConfig, StreamedPrefill, default_library, dense_flops, probe_flops,
+from .pipeline import (GraphedPrefill, RoutedPrefillLayer, RouteConfig, StreamedPrefill, default_library, dense_flops, probe_flops,
                        prefill_from_host)  # noqa: F401,E402

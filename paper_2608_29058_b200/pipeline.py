@@ -393,6 +393,31 @@ def prefill_from_host(layer: RoutedPrefillLayer, Q_host: torch.Tensor, K_host: t
     return O_host
 
 
+class GraphedPrefill:
+    """A layer pass captured once into a CUDA graph and replayed: for launch-bound sizes (a 4K layer takes 0.26 ms issued
+    call by call and 0.13 ms replayed).  The graph reads the Q, K, V buffers it was captured with, so run() copies new
+    inputs into those buffers (device to device) unless it is handed the very same tensors; the routes are recomputed on
+    the device at every replay.  The first, eager pass also does the one-time per-device kernel set-up, which must stay
+    outside the capture."""
+
+    def __init__(self, layer: RoutedPrefillLayer, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, **forward_kw):
+        self.layer, self.Q, self.K, self.V = layer, Q, K, V
+        layer.forward(Q, K, V, **forward_kw)
+        torch.cuda.synchronize()
+        rs.check_status(layer.status, "eager pass before the capture")
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            layer.forward(Q, K, V, **forward_kw)
+
+    def run(self, Q: Optional[torch.Tensor] = None, K: Optional[torch.Tensor] = None,
+            V: Optional[torch.Tensor] = None) -> torch.Tensor:
+        for dst, src in ((self.Q, Q), (self.K, K), (self.V, V)):
+            if src is not None and src.data_ptr() != dst.data_ptr():
+                dst.copy_(src, non_blocking=True)
+        self.graph.replay()
+        return self.layer.O
+
+
 class StreamedPrefill:
     """Layer passes fed from pinned HOST buffers with the copies overlapped with the kernels: three streams (host to
     device, compute, device to host) and two device buffer sets, so that while pass k computes, the inputs of pass k + 1

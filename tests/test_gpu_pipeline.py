@@ -294,3 +294,23 @@ def test_one_call_layer_equals_the_staged_calls(online):
         assert torch.equal(a, b)
     if online:
         assert len(set(outs[0][3].tolist())) > 1
+
+
+def test_graphed_prefill_replays_with_new_inputs():
+    """GraphedPrefill: inputs handed to run() are copied into the captured buffers; every replay routes anew and gives
+    what the plain call gives."""
+    n, Hq, Hkv = 768, 4, 2
+    p = rs.Problem(Hq, Hkv, n)
+    lib = [(rs.RS_A_SHAPE, 64, 128), (rs.RS_VERTICAL_SLASH, 48, 160), (rs.RS_BLOCK_SPARSE, 4, 0), (rs.RS_DENSE, 0, 0)]
+    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(budget_frac=0.5, cert_max=0.6))
+    ref = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(budget_frac=0.5, cert_max=0.6))
+    L0 = make_layer(tiny_spec(201, n, Hq, Hkv))
+    gp = rs.GraphedPrefill(layer, dev_bf16(L0["Q"]), dev_bf16(L0["K"]), dev_bf16(L0["V"]))
+    for seed in (202, 203, 201):
+        L = make_layer(tiny_spec(seed, n, Hq, Hkv))
+        Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+        O = gp.run(Q, K, V)
+        want = ref.forward(Q, K, V)
+        torch.cuda.synchronize()
+        rs.check_status(layer.status, f"replay {seed}")
+        assert torch.equal(O, want) and torch.equal(layer.choice, ref.choice) and torch.equal(layer.m_head, ref.m_head)
