@@ -314,3 +314,34 @@ def test_graphed_prefill_replays_with_new_inputs():
         torch.cuda.synchronize()
         rs.check_status(layer.status, f"replay {seed}")
         assert torch.equal(O, want) and torch.equal(layer.choice, ref.choice) and torch.equal(layer.m_head, ref.m_head)
+
+
+def test_two_layers_on_two_streams():
+    """Two layers issued from two streams at the same time share the library's per-device side stream (forked from and
+    joined into each caller's stream with events): both get what they get when they run alone."""
+    n, Hq, Hkv = 1024, 4, 2
+    p = rs.Problem(Hq, Hkv, n, [0, 448, 1024])
+    lib = [(rs.RS_A_SHAPE, 64, 128), (rs.RS_VERTICAL_SLASH, 48, 160), (rs.RS_BLOCK_SPARSE, 4, 0), (rs.RS_DENSE, 0, 0)]
+    cfg = rs.RouteConfig(budget_frac=0.5, cert_max=0.6)
+    data = []
+    for seed in (301, 302):
+        L = make_layer(tiny_spec(seed, n, Hq, Hkv))
+        data.append((dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])))
+    want = []
+    for Q, K, V in data:
+        layer = rs.RoutedPrefillLayer(p, lib, cfg)
+        layer.forward(Q, K, V)
+        torch.cuda.synchronize()
+        want.append((layer.O.clone(), layer.choice.clone(), layer.lse_sel.clone()))
+    layers = [rs.RoutedPrefillLayer(p, lib, cfg) for _ in range(2)]
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    torch.cuda.synchronize()
+    for rep in range(4):
+        for k in range(2):
+            with torch.cuda.stream(streams[k]):
+                layers[k].forward(*data[k])
+    torch.cuda.synchronize()
+    for k in range(2):
+        rs.check_status(layers[k].status, f"stream {k}")
+        assert torch.equal(layers[k].O, want[k][0]) and torch.equal(layers[k].choice, want[k][1])
+        assert torch.equal(layers[k].lse_sel, want[k][2])
