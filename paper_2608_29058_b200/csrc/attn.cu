@@ -695,6 +695,67 @@ WsPlan plan_ws(const rs_problem* p, int max_kv) {
   return w;
 }
 
+// Scratch of one attention launch: the work list (cost, items, launch order: one entry per 128-row tile) and, for
+// vertical-slash items, the packed K / V rows of the gathered columns.
+struct AttnScratch { int* cost; int2* items; int2* order; __nv_bfloat16 *Kp, *Vp; int kv_pad; int n_work, n_items; };
+
+// Enqueues the work-list kernels, the gather of the vertical columns and the attention launch.  Arguments are checked
+// by the callers; `sc` says where the scratch lives (caller workspace or the library's built-in array).
+int enqueue_attn(const rs_problem* p, const void* Q, const void* K, const void* V, const rs_candidate* lib, int n_cand,
+                 const rs_index_set* idx, const int32_t* choice, bool any_vs, bool vs_eval_layout, void* O, int o_dtype,
+                 float* lse, float* onorm, uint64_t* counters, const AttnScratch& sc, int32_t* status,
+                 cudaStream_t stream) {
+  AttnParams P{};
+  P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = p->n_q_heads / p->n_kv_heads;
+  P.n_seg = p->n_segments; P.n_cand = n_cand;
+  int tiles = 0;
+  for (int s = 0; s <= p->n_segments; ++s) {
+    P.seg_bounds[s] = p->seg_bounds[s];
+    P.tile_base[s] = tiles;
+    if (s < p->n_segments) tiles += (p->seg_bounds[s + 1] - p->seg_bounds[s] + kTileM - 1) / kTileM;
+  }
+  P.tiles_per_head = tiles;
+  for (int c = 0; c < n_cand; ++c) P.lib[c] = lib[c];
+  P.choice = choice;
+  if (idx) P.idx = *idx;
+  P.vs_eval_layout = vs_eval_layout ? 1 : 0;
+  P.kv_pad = sc.kv_pad;
+  P.order = sc.order;
+  P.O = O; P.o_f32 = o_dtype; P.lse = lse; P.onorm = onorm;
+  P.counters = reinterpret_cast<unsigned long long*>(counters);
+  P.status = status;
+  P.scale_log2e = (float)(1.4426950408889634 / sqrt((double)RS_HEAD_DIM));
+
+  CUtensorMap tmQ, tmK, tmV, tmKp, tmVp;
+  if (rs_make_tmap_bf16_2d(&tmQ, Q, (uint64_t)P.Hq * P.n, RS_HEAD_DIM, kTileM, 64) ||
+      rs_make_tmap_bf16_2d(&tmK, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kChunk, 64) ||
+      rs_make_tmap_bf16_2d(&tmV, V, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kChunk, 64))
+    return RS_ERR_CUDA;
+  if (sc.Kp != nullptr) {
+    const uint64_t pack_rows = (uint64_t)sc.n_items * (uint64_t)sc.kv_pad;
+    if (rs_make_tmap_bf16_2d(&tmKp, sc.Kp, pack_rows, RS_HEAD_DIM, kChunk, 64) ||
+        rs_make_tmap_bf16_2d(&tmVp, sc.Vp, pack_rows, RS_HEAD_DIM, kChunk, 64))
+      return RS_ERR_CUDA;
+  } else {          // no gathered columns in this launch: the packed maps are never read and alias K and V
+    tmKp = tmK; tmVp = tmV;
+  }
+
+  const int n_work = sc.n_work;
+  // every entry of cost / items / order is rewritten by the two kernels below, so nothing has to be cleared
+  rs_attn_cost_kernel<<<(n_work + 255) / 256, 256, 0, stream>>>(P, n_work, sc.cost, sc.items);
+  const int n_bins = (P.n >> 6) + 66;
+  rs_attn_order_kernel<<<P.Hkv, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work / P.Hkv, n_bins, sc.cost, sc.items,
+                                                                            sc.order);
+  if (choice != nullptr && any_vs && sc.Kp != nullptr) {
+    dim3 grid((P.kv_pad + 15) / 16, sc.n_items);
+    rs_pack_vertical_kernel<<<grid, 256, 0, stream>>>(P, reinterpret_cast<const __nv_bfloat16*>(K),
+                                                      reinterpret_cast<const __nv_bfloat16*>(V), sc.Kp, sc.Vp);
+  }
+  if (rs_ensure_dynamic_smem(g_attn_smem, rs_attn_kernel, 116 * 1024) != RS_OK) return RS_ERR_CUDA;
+  rs_attn_kernel<<<n_work, kThreads, attn_smem_bytes(P.n), stream>>>(tmQ, tmK, tmV, tmKp, tmVp, P);
+  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+}
+
 int launch_attn(const rs_problem* p, const void* Q, const void* K, const void* V, const rs_candidate* lib,
                 int n_cand, const rs_index_set* idx, const int32_t* choice, void* O, int o_dtype, float* lse,
                 float* onorm, uint64_t* counters, void* ws, size_t ws_bytes, int32_t* status, void* stream_) {
@@ -705,7 +766,6 @@ int launch_attn(const rs_problem* p, const void* Q, const void* K, const void* V
   if (choice != nullptr && (lib == nullptr || idx == nullptr || n_cand == 0)) return RS_ERR_INVALID_ARG;
   rc = rs_check_device();
   if (rc != RS_OK) return rc;
-  cudaStream_t stream = (cudaStream_t)stream_;
 
   int max_kv = 0;
   bool any_vs = false;
@@ -724,56 +784,12 @@ int launch_attn(const rs_problem* p, const void* Q, const void* K, const void* V
   const WsPlan w = plan_ws(p, max_kv);
   if (ws_bytes < w.total) return RS_ERR_WORKSPACE_TOO_SMALL;
   if (((uintptr_t)ws & 255) != 0) return RS_ERR_INVALID_ARG;
-
-  AttnParams P{};
-  P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = p->n_q_heads / p->n_kv_heads;
-  P.n_seg = p->n_segments; P.n_cand = n_cand;
-  int tiles = 0;
-  for (int s = 0; s <= p->n_segments; ++s) {
-    P.seg_bounds[s] = p->seg_bounds[s];
-    P.tile_base[s] = tiles;
-    if (s < p->n_segments) tiles += (p->seg_bounds[s + 1] - p->seg_bounds[s] + kTileM - 1) / kTileM;
-  }
-  P.tiles_per_head = tiles;
-  for (int c = 0; c < n_cand; ++c) P.lib[c] = lib[c];
-  P.choice = choice;
-  if (idx) P.idx = *idx;
-  P.vs_eval_layout = vs_eval_layout ? 1 : 0;
-  P.kv_pad = w.kv_pad > 0 ? w.kv_pad : 64;
   uint8_t* wsb = reinterpret_cast<uint8_t*>(ws);
-  P.order = reinterpret_cast<const int2*>(wsb + w.order);
-  P.O = O; P.o_f32 = o_dtype; P.lse = lse; P.onorm = onorm;
-  P.counters = reinterpret_cast<unsigned long long*>(counters);
-  P.status = status;
-  P.scale_log2e = (float)(1.4426950408889634 / sqrt((double)RS_HEAD_DIM));
-
-  __nv_bfloat16* Kp = reinterpret_cast<__nv_bfloat16*>(wsb + w.kpack);
-  __nv_bfloat16* Vp = reinterpret_cast<__nv_bfloat16*>(wsb + w.vpack);
-  CUtensorMap tmQ, tmK, tmV, tmKp, tmVp;
-  const uint64_t pack_rows = (uint64_t)w.n_items * (uint64_t)P.kv_pad;
-  if (rs_make_tmap_bf16_2d(&tmQ, Q, (uint64_t)P.Hq * P.n, RS_HEAD_DIM, kTileM, 64) ||
-      rs_make_tmap_bf16_2d(&tmK, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kChunk, 64) ||
-      rs_make_tmap_bf16_2d(&tmV, V, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kChunk, 64) ||
-      rs_make_tmap_bf16_2d(&tmKp, Kp, pack_rows, RS_HEAD_DIM, kChunk, 64) ||
-      rs_make_tmap_bf16_2d(&tmVp, Vp, pack_rows, RS_HEAD_DIM, kChunk, 64))
-    return RS_ERR_CUDA;
-
-  const int n_work = w.n_work;
-  int* cost = reinterpret_cast<int*>(wsb + w.cost);
-  int2* items = reinterpret_cast<int2*>(wsb + w.items);
-  int2* order = reinterpret_cast<int2*>(wsb + w.order);
-  rs_attn_cost_kernel<<<(n_work + 255) / 256, 256, 0, stream>>>(P, n_work, cost, items);
-  const int n_bins = (P.n >> 6) + 66;
-  rs_attn_order_kernel<<<P.Hkv, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work / P.Hkv, n_bins, cost, items, order);
-  if (choice != nullptr && any_vs) {
-    dim3 grid((P.kv_pad + 15) / 16, w.n_items);
-    rs_pack_vertical_kernel<<<grid, 256, 0, stream>>>(P, reinterpret_cast<const __nv_bfloat16*>(K),
-                                                      reinterpret_cast<const __nv_bfloat16*>(V), Kp, Vp);
-  }
-  const size_t smem = attn_smem_bytes(P.n);
-  if (rs_ensure_dynamic_smem(g_attn_smem, rs_attn_kernel, 116 * 1024) != RS_OK) return RS_ERR_CUDA;
-  rs_attn_kernel<<<n_work, kThreads, smem, stream>>>(tmQ, tmK, tmV, tmKp, tmVp, P);
-  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+  AttnScratch sc{reinterpret_cast<int*>(wsb + w.cost), reinterpret_cast<int2*>(wsb + w.items),
+                 reinterpret_cast<int2*>(wsb + w.order), reinterpret_cast<__nv_bfloat16*>(wsb + w.kpack),
+                 reinterpret_cast<__nv_bfloat16*>(wsb + w.vpack), w.kv_pad > 0 ? w.kv_pad : 64, w.n_work, w.n_items};
+  return enqueue_attn(p, Q, K, V, lib, n_cand, idx, choice, any_vs, vs_eval_layout, O, o_dtype, lse, onorm, counters, sc,
+                      status, (cudaStream_t)stream_);
 }
 
 }  // namespace
@@ -844,40 +860,11 @@ extern "C" int rs_dense_prefill_attn_noalloc(const rs_problem* p, const void* Q,
   void* scratch = nullptr;
   rc = noalloc_scratch_ptr(&scratch);
   if (rc != RS_OK) return rc;
-  cudaStream_t stream = (cudaStream_t)stream_;
-  const int n_work = (int)n_work_ll;
-
-  AttnParams P{};
-  P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = p->n_q_heads / p->n_kv_heads;
-  P.n_seg = p->n_segments; P.n_cand = 0;
-  int acc = 0;
-  for (int s = 0; s <= p->n_segments; ++s) {
-    P.seg_bounds[s] = p->seg_bounds[s];
-    P.tile_base[s] = acc;
-    if (s < p->n_segments) acc += (p->seg_bounds[s + 1] - p->seg_bounds[s] + kTileM - 1) / kTileM;
-  }
-  P.tiles_per_head = acc;
-  P.choice = nullptr;
-  P.kv_pad = 64;
   unsigned char* sb = reinterpret_cast<unsigned char*>(scratch);
-  int* cost = reinterpret_cast<int*>(sb);
-  int2* items = reinterpret_cast<int2*>(sb + (size_t)kNoAllocMaxTiles * 4);
-  int2* order = reinterpret_cast<int2*>(sb + (size_t)kNoAllocMaxTiles * 12);
-  P.order = order;
-  P.O = O; P.o_f32 = o_dtype; P.lse = lse; P.onorm = onorm; P.counters = nullptr; P.status = status;
-  P.scale_log2e = (float)(1.4426950408889634 / sqrt((double)RS_HEAD_DIM));
-
-  CUtensorMap tmQ, tmK, tmV;
-  if (rs_make_tmap_bf16_2d(&tmQ, Q, (uint64_t)P.Hq * P.n, RS_HEAD_DIM, kTileM, 64) ||
-      rs_make_tmap_bf16_2d(&tmK, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kChunk, 64) ||
-      rs_make_tmap_bf16_2d(&tmV, V, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kChunk, 64))
-    return RS_ERR_CUDA;
-  // every entry of cost / items / order is rewritten by the two kernels below, so nothing has to be cleared
-  rs_attn_cost_kernel<<<(n_work + 255) / 256, 256, 0, stream>>>(P, n_work, cost, items);
-  const int n_bins = (P.n >> 6) + 66;
-  rs_attn_order_kernel<<<P.Hkv, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work / P.Hkv, n_bins, cost, items, order);
-  if (rs_ensure_dynamic_smem(g_attn_smem, rs_attn_kernel, 116 * 1024) != RS_OK) return RS_ERR_CUDA;
-  // the gathered-column maps are never read by dense tiles; they alias K and V
-  rs_attn_kernel<<<n_work, kThreads, attn_smem_bytes(P.n), stream>>>(tmQ, tmK, tmV, tmK, tmV, P);
-  return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+  AttnScratch sc{reinterpret_cast<int*>(sb), reinterpret_cast<int2*>(sb + (size_t)kNoAllocMaxTiles * 4),
+                 reinterpret_cast<int2*>(sb + (size_t)kNoAllocMaxTiles * 12), nullptr, nullptr, 64, (int)n_work_ll,
+                 p->n_segments * p->n_q_heads};
+  // the same enqueue as rs_dense_prefill_attn: same kernels, same work list, only the scratch lives elsewhere
+  return enqueue_attn(p, Q, K, V, nullptr, 0, nullptr, nullptr, false, false, O, o_dtype, lse, onorm, nullptr, sc, status,
+                      (cudaStream_t)stream_);
 }

@@ -54,13 +54,16 @@ def test_dense_bf16_output_and_segments():
     n, Hq, Hkv = 576, 2, 2
     L = make_layer(tiny_spec(5, n, Hq, Hkv))
     p = rs.Problem(Hq, Hkv, n, [0, 192, 576])       # a segment boundary that is not a multiple of 128
-    O, lse, _, _ = _run_dense(L, p, torch.bfloat16)
+    O32, lse, _, _ = _run_dense(L, p, torch.float32)
     Qs, Ks, Vs = f64_heads(L)
     for h in range(Hq):
         Oo, lo = A.dense_attention(Qs[h], Ks[h], Vs[h])
-        err = np.abs(O[h] - Oo)
-        assert err.max() < 2e-2 + 2.0 ** -8 * np.abs(Oo).max() and err.mean() < 5e-3
+        assert_attention_close(O32[h], Oo, f"dense, segments, h={h}")
         assert np.abs(lse[h] - lo).max() < 2e-3
+    # the bf16 output is the same result rounded once (round to nearest even): bit-identical to rounding the fp32 output
+    O16, lse16, _, _ = _run_dense(L, p, torch.bfloat16)
+    assert np.array_equal(O16, torch.from_numpy(O32).to(torch.bfloat16).float().numpy())
+    assert np.array_equal(lse16, lse)
 
 
 CANDS = [C(PT.DENSE), C(PT.A_SHAPE, 8, 96), C(PT.A_SHAPE, 70, 200), C(PT.VERTICAL_SLASH, 24, 40),

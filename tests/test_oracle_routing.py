@@ -235,3 +235,62 @@ def test_global_router_is_the_best_constant_assignment():
     cov, cost = _instance(rng)
     choice, rep = RT.route(LIB, cov, cost, np.ones(4, np.float32), RT.RouteParams(budget=405, t_probe=5, global_pattern=True))
     assert np.all(choice == DENSE_C) and rep.total_risk == 0.0
+
+
+def _greedy_by_cross_multiplication(Rnum, den, cost, dense_c, budget, t_probe):
+    """The greedy substitution with "risk per unit of cost" (Section 3.4: the risk-per-microsecond substitution) compared
+    exactly: risks are the rationals Rnum / den, and dR1 / dT1 < dR2 / dT2 is decided as dR1 * dT2 < dR2 * dT1 in
+    integers (dT > 0).  Ties: larger saving, lower item, lower candidate."""
+    n_items, n_cand = Rnum.shape
+    choice = [dense_c] * n_items
+    total = t_probe + int(cost[:, dense_c].sum())
+    while total > budget:
+        best = None                     # (dR numerator, dT, item, k)
+        for it in range(n_items):
+            cur = choice[it]
+            for k in range(n_cand):
+                dT = int(cost[it, cur]) - int(cost[it, k])
+                if dT <= 0:
+                    continue
+                dR = int(Rnum[it, k]) - int(Rnum[it, cur])
+                if best is None:
+                    best = (dR, dT, it, k)
+                    continue
+                lhs, rhs = dR * best[1], best[0] * dT          # dR / dT  vs  best dR / best dT
+                if lhs < rhs or (lhs == rhs and (-dT, it, k) < (-best[1], best[2], best[3])):
+                    best = (dR, dT, it, k)
+        if best is None:
+            return choice, total, 0
+        choice[best[2]] = best[3]
+        total -= best[1]
+    return choice, total, 1
+
+
+def test_one_division_orders_substitutions_like_exact_cross_multiplication():
+    """The oracle ranks substitutions by the single IEEE division dR / dT inside the tuple (ratio, -dT, item, k).  The
+    sentence it reads (Section 3.4, "greedily apply the risk-per-microsecond substitution") fixes the exact quotient;
+    here the two are shown to agree wherever the quotient is decided exactly: risks that are multiples of 1/64 and
+    integer costs below 2^20 make dR and dT exact, equal rationals divide to the same double and different rationals
+    (which differ by more than 2^-46 relative) to different doubles.  Thousands of random instances with many exact ties
+    between different (dR, dT) pairs -- 1/64 over 1 against 2/64 over 2 -- plus planted duplicates of whole items."""
+    rng = np.random.default_rng(2608)
+    n_cand, dense_c = 6, 5
+    n_ties = 0
+    for trial in range(3000):
+        n_items = int(rng.integers(2, 7))
+        Rnum = rng.integers(0, 40, size=(n_items, n_cand))           # risk = Rnum / 64
+        cost = rng.integers(1, 24, size=(n_items, n_cand)) * int(rng.choice([1, 1000, 65536]))
+        Rnum[:, dense_c] = 0
+        cost[:, dense_c] = cost.max() + int(rng.integers(1, 9))
+        if trial % 3 == 0 and n_items >= 3:                          # planted ties: an item repeated
+            Rnum[2], cost[2] = Rnum[0], cost[0]
+        R = Rnum.astype(np.float64) / 64.0
+        budget = int(cost[:, dense_c].sum() * rng.uniform(0.05, 0.9))
+        want = _greedy_by_cross_multiplication(Rnum, 64, cost, dense_c, budget, 3)
+        got = RT.greedy_solve(R, cost, dense_c, budget, 3)
+        assert (list(got[0]), got[1], got[2]) == (want[0], want[1], want[2]), trial
+        # count instances where the first step already has an exact tie of the quotient between different pairs
+        first = sorted((Rnum[it, k] * 1.0 / (cost[it, dense_c] - cost[it, k]), it, k)
+                       for it in range(n_items) for k in range(n_cand - 1))
+        n_ties += first[0][0] == first[1][0]
+    assert n_ties > 100                                              # the tie-break branch really is exercised
