@@ -73,11 +73,22 @@ def fixed_choice_for(lib, n_q_heads):
     return np.array([index_of[int(x)] for x in pat], dtype=np.int32)
 
 
-# ----------------------------------------------------------------------------------------- clocks
-# DRAM bytes of the attention launch measured with ncu (one-pass metrics, full-size workload, clocks untouched); the
-# algorithmic minimum of the config-3 launch is Q + K + V + O + row outputs = 2.71e9 bytes.
-ATTN_DRAM_BYTES_PER_LAUNCH = {("config3", 131072, "flops", False, False): 3.20e9 + 1.08e9}
+# ----------------------------------------------------------------------------------------- measured DRAM traffic
+def measured_traffic(workload: str, n: int, plain: bool):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture recorded
+    in profiles/dram_traffic.json (null for workloads and router settings that were not captured)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not plain or not os.path.exists(path):
+        return None, None
+    with open(path) as f:
+        table = json.load(f)
+    rec = table.get(f"{workload}:n={n}")
+    if rec is None:
+        return None, None
+    return float(rec["dram_bytes_read"]) + float(rec["dram_bytes_write"]), rec.get("how")
 
+
+# ----------------------------------------------------------------------------------------- clocks
 
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
@@ -147,7 +158,8 @@ def aggregate_over_ranks(ms_local: float, units_local: float, device=None):
 
 
 # ----------------------------------------------------------------------------------------- CPU oracle leg
-def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float = 20.0, n_heads: int = 8, n_blocks: int = 20):
+def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float = 20.0, n_heads: int = 8, n_blocks: int = 20,
+                  routes: str = "under the routes and index lists the GPU pass chose for this layer"):
     """Times the oracle's masked attention on sampled query blocks under the routed masks.
 
     Returns (effective TFLOP/s, description, cores, max abs difference to gpu_O on the sampled rows).
@@ -182,31 +194,19 @@ def oracle_sample(L, spec, cands, choice, sets_fn, gpu_O=None, budget_s: float =
                 worst = max(worst, float(np.abs(gpu_O[h, rows].astype(np.float64) - Om).max()))
     tflops = 512.0 * pairs_done / max(t_used, 1e-9) / 1e12
     desc = (f"oracle masked attention on {rows_done} sampled query rows (heads {heads}, query blocks {blocks}) of the "
-            f"same routed layer, {t_used:.1f} s; effective = 512 FLOP x selected pairs / time")
+            f"same layer {routes}, {t_used:.1f} s; effective = 512 FLOP x selected pairs / time")
     return tflops, desc, os.cpu_count(), worst
 
 
 def download_sets(layer, cands, choice):
     """Device index lists of the routed candidates -> the oracle's IndexSet objects (CPU-baseline leg only)."""
     from oracle import patterns as PT
-    p = layer.p
-    nb = p.n_keys // 64
-    reuse = getattr(layer, "_reuse_eval", False)       # vertical-slash lists may still sit in the evaluation layout
-    vs = layer.idx_eval if reuse else layer.idx
-    cnt = vs.vs_count.cpu().numpy()
-    cols, offs, diag = (t.cpu().numpy() for t in (vs.vs_cols, vs.vs_offs, vs.vs_diag))
-    blk, bcnt = layer.idx.bs_blk.cpu().numpy(), layer.idx.bs_count.cpu().numpy()
     sets = []
-    for item in range(p.n_items):
-        s, h = divmod(item, p.n_q_heads)
-        q0, q1 = p.seg_bounds[s], p.seg_bounds[s + 1]
-        cand = cands[choice[item]]
-        ix = PT.IndexSet(cand=cand, q0=q0, q1=q1)
-        if cand.pattern == PT.VERTICAL_SLASH:
-            sl = item * len(cands) + int(choice[item]) if reuse else item
-            ix.V, ix.S, ix.D = cols[sl, :cnt[sl, 0]], offs[sl, :cnt[sl, 1]], diag[sl, :cnt[sl, 2]]
-        elif cand.pattern == PT.BLOCK_SPARSE:
-            ix.blk = [blk[h * nb + qb, :bcnt[h * nb + qb]] for qb in range(q0 // 64, q1 // 64)]
+    for item, d in enumerate(layer.download_index_lists(choice)):
+        ix = PT.IndexSet(cand=cands[choice[item]], q0=d["q0"], q1=d["q1"])
+        for name in ("V", "S", "D", "blk"):
+            if name in d:
+                setattr(ix, name, d[name])
         sets.append(ix)
     return sets
 
@@ -237,6 +237,10 @@ def main():
                     help="also time the layer replayed from a CUDA graph (whole pass captured once; for launch-bound sizes)")
     ap.add_argument("--sweep", action="store_true", help="config-5 sweep: n x budget x forced-dense cells, JSONL output")
     ap.add_argument("--n", type=int, default=None, help="override the sequence length (smaller profiling case)")
+    ap.add_argument("--out-dir", default="bench_out", help="directory for the JSONL files of --sweep and --ablations")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="config3: skip the two untimed side runs (the literal planted-structure generator at this length, "
+                         "and the certificate read in ABS mode)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
@@ -252,9 +256,14 @@ def main():
     from synth import make_layer
     spec, lib, route_kw, fixed = workload_spec(args.workload, args.n)
     metric = "effective TFLOP/s of routed sparse prefill attention (FLOPs of selected query-key pairs / layer time)"
+    generator = {"config1": "planted-structure generator with the task's literal constants (sinks 4, verticals 3, local 0.5)",
+                 "config2": "planted-structure generator, per-head random sink / vertical / local strengths",
+                 "config3": "archetype generator (local / vertical / topic / diffuse heads), boosts scaled by log(n/4096)"}
     config = {"workload": f"{args.workload}: Hq={spec.n_q_heads} Hkv={spec.n_kv_heads} d=128 n={spec.n}, "
+                          + generator.get(args.workload, "") + ", "
                           + ("routes fixed from seed" if fixed else
-                             f"online routing, budget {route_kw['budget_frac']:.2f} of dense FLOPs, cert_max {route_kw['cert_max']}"),
+                             f"online routing, budget {route_kw['budget_frac']:.2f} of dense FLOPs, cert_max {route_kw['cert_max']} "
+                             f"with cert_mode=REL (Eq. 5 without the V_max factor)"),
               "l2": "inputs (Q,K,V,O > 126 MB) exceed L2; no explicit flush" if spec.n >= 32768 else "small case, L2 resident",
               "replicas": args.gpus}
 
@@ -450,6 +459,12 @@ def main():
     if rank != 0:
         return 0
 
+    plain = args.cost == "flops" and not (args.rescue or args.mixture or args.calibration)
+    # ---- side runs outside the timed region: what the headline would be under the two literal readings of the task
+    extra = None
+    if args.workload == "config3" and not args.no_extra and plain:
+        extra = side_runs(rs, torch, dev, spec, p, Q, K, V, layer, route_kw, dense_ms)
+
     # ---- CPU oracle on a bounded sample of the same workload (also a full-size parity spot check)
     cpu = None
     if not args.no_cpu_baseline:
@@ -463,14 +478,11 @@ def main():
                "max_abs_diff_vs_gpu_on_sample": worst}
 
     peak = peaks["bf16_tflops_sustained"]
+    traffic, traffic_how = measured_traffic(args.workload, spec.n, plain)
     attn_ms = stages["attention"]
     achieved = f_tile / (attn_ms * 1e-3) / 1e12
     overhead_ms = stages["probe"] + stages["evaluate"] + stages["route"] + stages["materialise"] + stages["certificate"]
-    hist = {}
-    for it in range(p.n_items):
-        c = layer.cands[choice[it]]
-        key = {0: "dense", 1: "a_shape", 2: "vertical_slash", 3: "block_sparse"}[c[0]] + (f"({c[1]},{c[2]})" if c[0] else "")
-        hist[key] = hist.get(key, 0) + 1
+    hist = _route_hist(layer, choice)
     any_vs = any(c[0] == 2 for c in layer.cands)
     any_bs = any(c[0] == 3 for c in layer.cands)
     # kernels of this library per layer pass, stage by stage (memsets and torch copies are not counted)
@@ -506,14 +518,63 @@ def main():
                      "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": f"bf16_tflops_sustained, {peaks['source']}",
                      "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
-                     "traffic": ATTN_DRAM_BYTES_PER_LAUNCH.get((args.workload, spec.n, args.cost, bool(args.rescue), bool(args.mixture))),
-                     "traffic_note": "dram__bytes_read.sum + dram__bytes_write.sum of this launch from a one-pass ncu capture of this "
-                                     "workload (profiles/rs_attn_kernel_config3_n16384.md); null for workloads that were not captured",
+                     "traffic": traffic, "traffic_note": traffic_how,
                      "note": "achieved = 512 FLOP x 128 x 64 pairs per issued chunk / attention-call time (CUDA events)"},
+        "stage_ms_targets": {"probe": 0.30, "evaluate": 0.35, "at": "n=131072, config3"},
+        "extra": extra,
         "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
     }
     print(json.dumps(out))
     return 0
+
+
+def _route_hist(layer, choice):
+    hist = {}
+    for it in range(len(choice)):
+        c = layer.cands[choice[it]]
+        key = {0: "dense", 1: "a_shape", 2: "vertical_slash", 3: "block_sparse"}[c[0]] + (f"({c[1]},{c[2]})" if c[0] else "")
+        hist[key] = hist.get(key, 0) + 1
+    return hist
+
+
+def side_runs(rs, torch, dev, spec, p, Q, K, V, layer, route_kw, dense_ms, reps: int = 3):
+    """Two untimed companions of the config-3 headline, so that the JSON line itself shows what the workload choices do:
+    (a) the same layer pass with the certificate read in ABS mode (2 (1 - m_low) V_max against cert_max);
+    (b) the same online routing on a layer from the planted-structure generator of configs 1-2 (per-head random sink /
+        vertical / local strengths, no scaling with n) at this length."""
+    def run(lyr, q, k, v):
+        for _ in range(2):
+            lyr.forward(q, k, v)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            lyr.forward(q, k, v)
+        b.record()
+        torch.cuda.synchronize()
+        rs.check_status(lyr.status, "side run")
+        ms = a.elapsed_time(b) / reps
+        choice = lyr.choice.cpu().numpy()
+        rep = lyr.route_report()
+        return {"ms_per_layer": ms, "speedup_vs_own_dense": (dense_ms / ms) if dense_ms else None,
+                "routes": _route_hist(lyr, choice), "fallback_rate": rep["n_fallback"] / p.n_items,
+                "dense_items": int(sum(1 for c in choice if lyr.cands[c][0] == 0))}
+    out = {}
+    saved = layer.cfg.cert_mode
+    layer.cfg.cert_mode = rs.RS_CERT_ABS
+    out["cert_mode_abs"] = run(layer, Q, K, V)
+    out["cert_mode_abs"]["note"] = "same layer and budget; fallback test 2 (1 - m_low) V_max > cert_max"
+    layer.cfg.cert_mode = saved
+    from synth import config2_spec, make_layer
+    lit = make_layer(config2_spec(n=spec.n, n_q_heads=spec.n_q_heads, n_kv_heads=spec.n_kv_heads))
+    q2, k2, v2 = (_to_dev(lit[k], dev) for k in ("Q", "K", "V"))
+    out["literal_generator"] = run(layer, q2, k2, v2)
+    out["literal_generator"]["note"] = ("planted-structure generator of configs 1-2 at this length (constants not scaled "
+                                        "with n), same budget and REL certificate")
+    del q2, k2, v2
+    layer.forward(Q, K, V)             # leave the layer holding the headline pass again
+    torch.cuda.synchronize()
+    return out
 
 
 def _to_dev(bits, dev):
@@ -616,7 +677,7 @@ def ablations(args):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     n = args.n or 131072
-    out_dir = os.path.join(ROOT, "gpurun_out")
+    out_dir = os.path.abspath(args.out_dir)
     os.makedirs(out_dir, exist_ok=True)
     path = os.path.join(out_dir, f"ablations_config3_n{n}.jsonl")
     spec = config3_spec(n)
@@ -698,7 +759,7 @@ def ablations(args):
             torch.cuda.empty_cache()
     print(json.dumps({"ablations": [{k: r[k] for k in ("variant", "ms_per_layer", "fallback_pct", "dense_heads",
                                                        "retained_mass_mean", "retained_mass_worst_decile")} for r in rows],
-                      "file": os.path.relpath(path, ROOT)}))
+                      "file": path}))
     return 0
 
 
@@ -709,7 +770,7 @@ def sweep(args):
     from synth import config3_spec, make_layer
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
-    out_dir = os.path.join(ROOT, "gpurun_out")
+    out_dir = os.path.abspath(args.out_dir)
     os.makedirs(out_dir, exist_ok=True)
     path = os.path.join(out_dir, "sweep_config5.jsonl")
     done = set()
@@ -779,7 +840,7 @@ def sweep(args):
                 cells.append(cell)
         del layer, Q, K, V
         torch.cuda.empty_cache()
-    print(json.dumps({"metric": "config-5 sweep", "cells_run": len(cells), "cells_file": "gpurun_out/sweep_config5.jsonl",
+    print(json.dumps({"metric": "config-5 sweep", "cells_run": len(cells), "cells_file": path,
                       "peak": peaks["bf16_tflops_sustained"], "data": "synthetic"}))
     return 0
 
@@ -799,11 +860,12 @@ def reference_arm(args, spec, lib, route_kw, fixed, metric, config):
     G = spec.n_q_heads // spec.n_kv_heads
     # routes of the sampled heads: a sparse candidate per head in turn (the oracle's own probe builds the indices)
     sparse = [c for c in cands if c.pattern != PT.DENSE]
-    sets = {}
+    sets, names = {}, []
     for t, h in enumerate(heads):
         Qf, Kf = bf16_bits_to_f64(Lq["Q"][h]), bf16_bits_to_f64(L["K"][h // G])
         pr = OP.probe_rows(Qf, Kf, spec.n)
         cand = sparse[(t * 5 + 1) % len(sparse)]
+        names.append(f"head {h}: pattern {cand.pattern} ({cand.b0},{cand.b1})")
         bs = OP.block_scores(Qf, Kf, 0, spec.n) if cand.pattern == PT.BLOCK_SPARSE else None
         sets[h] = PT.build_indices(cand, 0, spec.n, pr.vert, pr.slash, bs)
     Lfull = {"Q": [Lq["Q"].get(h) for h in range(spec.n_q_heads)], "K": L["K"], "V": L["V"]}
@@ -811,7 +873,9 @@ def reference_arm(args, spec, lib, route_kw, fixed, metric, config):
     for it in range(args.warmup + args.steps):
         t0 = time.perf_counter()
         tf, desc, cores, _ = oracle_sample(Lfull, spec, cands, None, lambda h: sets[h], None,
-                                           budget_s=max(2.0, 60.0 / max(1, args.steps + args.warmup)), n_heads=4)
+                                           budget_s=max(2.0, 60.0 / max(1, args.steps + args.warmup)), n_heads=4,
+                                           routes="with one fixed sparse candidate per sampled head, index lists from the "
+                                                  "oracle's own probe (no GPU routes: " + "; ".join(names) + ")")
         if it >= args.warmup:
             vals.append(tf); times.append((time.perf_counter() - t0) * 1e3)
     v = float(np.mean(vals))

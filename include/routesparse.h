@@ -102,8 +102,8 @@ typedef struct {
   int32_t use_cert;        /* 0: no fallback step */
   int32_t cert_mode;       /* rs_cert_mode: REL 2(1-m_low), ABS 2(1-m_low) * V_max */
   int32_t expand_first;    /* 1: next larger budget of the family before dense */
-  int32_t reserved;        /* rescue_any: 1 = when the family has no larger budget, take the cheapest sparse candidate
-                              of any family whose certificate passes before giving up and going dense */
+  int32_t rescue_any;      /* 1 = when the family has no larger budget, take the cheapest sparse candidate of any
+                              family whose certificate passes before giving up and going dense */
   const int32_t* forced_dense;  /* device int32[n_items], non-zero = force dense last; may be NULL */
   const int32_t* fixed_choice;  /* device int32[n_items]; when set, bypasses solve and fallback; may be NULL */
   const double* e;         /* device double[n_items][n_cand]: calibrated error predictor e of Eq. 4 (rs_regressor_eval);
@@ -121,6 +121,10 @@ typedef struct {
   int32_t mix_rows[4];     /* rows per subset (0 = subset unused) */
 } rs_route_params;
 
+/* total_cost and total_risk are those of the final routes (t_probe included in the cost).  feasible is the outcome of
+ * the budgeted solve of Eq. 6-8 alone (0: even the cheapest candidates exceed the budget); the fallback walk and the
+ * forced-dense set run afterwards and may push total_cost above the budget again (Section 3.4, step 5), which a caller
+ * sees by comparing total_cost with the budget it passed. */
 typedef struct { int64_t total_cost; double total_risk; int32_t n_fallback; int32_t feasible; } rs_route_report;
 
 const char* rs_error_string(int code);
@@ -157,8 +161,9 @@ int rs_probe(const rs_problem* p, const void* Q, const void* K, const void* V,
  * largest single stream of the probe (1 GB at 128K) and only heads routed to block-sparse need it. */
 #define RS_PROBE_QPOOL_LAST_ONLY 1
 
-/* 64-row means of Q (the rows of qpool rs_probe left out) for the heads whose routed candidate is block-sparse.
- * choice: device int32[n_items] (NULL: every head).  qpool as for rs_probe. */
+/* 64-row means of Q (the rows of qpool rs_probe left out) for the heads whose routed candidate is block-sparse:
+ * the pooled queries of Section 3.1 ("pooled queries and keys score coarse blocks"), which the block-sparse family
+ * ranks key blocks with.  choice: device int32[n_items] (NULL: every head).  qpool as for rs_probe. */
 int rs_pool_queries(const rs_problem* p, const void* Q, const rs_candidate* lib, int n_cand, const int32_t* choice,
                     float* qpool, int32_t* status, void* stream);
 
@@ -233,7 +238,9 @@ int rs_dense_prefill_attn_noalloc(const rs_problem* p, const void* Q, const void
  * lse_full: [n_q_heads][n_rows].  vmax: [n_kv_heads], any upper bound of the value norms of that KV head
  * (rs_probe's vmax row of the last segment qualifies).
  * Outputs (each may be NULL) m_row, cert_row, cert_tight: [n_q_heads][n_rows]; m_head [n_q_heads];
- * cert_head [n_q_heads][2]. */
+ * cert_head [n_q_heads][2].
+ * A row id outside [0, n_keys) is not read: its outputs are NaN, it is left out of the head-level values, and
+ * RS_ERR_INVALID_ARG is written to `status` (device, may be NULL). */
 int rs_certificate(int n_q_heads, int n_kv_heads, int n_keys, const float* lse_sel, const float* lse_full,
                    const int32_t* rows, int n_rows, const float* vmax, const float* onorm, float delta_q,
                    float* m_row, float* cert_row, float* cert_tight, float* m_head, float* cert_head,

@@ -41,7 +41,7 @@ class rs_index_set(C.Structure):
 class rs_route_params(C.Structure):
     _fields_ = [("budget", C.c_int64), ("t_probe", C.c_int64), ("alpha", C.c_double), ("delta_q", C.c_double),
                 ("cert_max", C.c_double), ("use_cert", C.c_int32), ("cert_mode", C.c_int32),
-                ("expand_first", C.c_int32), ("reserved", C.c_int32),
+                ("expand_first", C.c_int32), ("rescue_any", C.c_int32),
                 ("forced_dense", C.c_void_p), ("fixed_choice", C.c_void_p), ("e", C.c_void_p), ("beta", C.c_double),
                 ("backfill", C.c_int32), ("global_pattern", C.c_int32), ("cov_mix", C.c_void_p), ("mix_rows", C.c_int32 * 4)]
 

@@ -384,7 +384,7 @@ rs_route_kernel(const __grid_constant__ RouteArgs A) {
           if (!(cert > A.prm.cert_max)) break;
           fired = true;
           int nxt = A.prm.expand_first ? A.next_larger[c] : -1;
-          if (nxt < 0 && A.prm.reserved != 0) {
+          if (nxt < 0 && A.prm.rescue_any != 0) {
             // rescue: the cheapest sparse candidate of any family whose certificate passes (ties: lower index)
             for (int k = 0; k < A.n_cand; ++k) {
               if (A.lib[k].pattern == RS_DENSE) continue;

@@ -153,7 +153,7 @@ class RoutedPrefillLayer:
         prm.use_cert = 0 if c.cert_max is None else 1
         prm.cert_max = 0.0 if c.cert_max is None else c.cert_max
         prm.cert_mode, prm.expand_first = c.cert_mode, int(c.expand_first)
-        prm.reserved = int(c.rescue_any)
+        prm.rescue_any = int(c.rescue_any)
         prm.backfill = int(c.backfill)
         prm.global_pattern = int(c.global_pattern)
         if c.mixture_u and getattr(self, "_pp_key", None) is not None:
@@ -371,6 +371,29 @@ class RoutedPrefillLayer:
         e = self.events
         names = ["probe", "evaluate", "route", "materialise", "attention", "certificate"]
         return {names[i]: e[i].elapsed_time(e[i + 1]) for i in range(6)}
+
+    def download_index_lists(self, choice):
+        """The routed candidates' index lists as host arrays, one dict per item (synchronises): vertical-slash items
+        carry V (columns), S (offsets), D (block diagonals); block-sparse items carry blk, one array of key blocks per
+        query block of the segment.  Knows where the lists sit (the evaluation's slots when they were reused)."""
+        p = self.p
+        nb, n_cand = p.n_keys // 64, len(self.cands)
+        vs = self.idx_eval if self._reuse_eval else self.idx
+        cnt = vs.vs_count.cpu().numpy()
+        cols, offs, diag = (t.cpu().numpy() for t in (vs.vs_cols, vs.vs_offs, vs.vs_diag))
+        blk, bcnt = self.idx.bs_blk.cpu().numpy(), self.idx.bs_count.cpu().numpy()
+        out = []
+        for item in range(p.n_items):
+            s, h = divmod(item, p.n_q_heads)
+            c = int(choice[item])
+            d = dict(pattern=self.cands[c][0], q0=p.seg_bounds[s], q1=p.seg_bounds[s + 1])
+            if d["pattern"] == rs.RS_VERTICAL_SLASH:
+                sl = item * n_cand + c if self._reuse_eval else item
+                d.update(V=cols[sl, :cnt[sl, 0]], S=offs[sl, :cnt[sl, 1]], D=diag[sl, :cnt[sl, 2]])
+            elif d["pattern"] == rs.RS_BLOCK_SPARSE:
+                d["blk"] = [blk[h * nb + qb, :bcnt[h * nb + qb]] for qb in range(d["q0"] // 64, d["q1"] // 64)]
+            out.append(d)
+        return out
 
     def route_report(self):
         import numpy as np

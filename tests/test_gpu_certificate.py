@@ -32,6 +32,33 @@ def test_certificate_matches_oracle():
     assert np.all(m_row <= 1.0) and np.all(cert_row >= 0)
 
 
+def test_row_ids_outside_the_sequence_are_reported_not_read():
+    """A row id outside [0, n_keys) is never dereferenced: NaN outputs for that row, the head-level mean over the valid
+    rows only, and RS_ERR_INVALID_ARG in the status words."""
+    rng = np.random.default_rng(1)
+    Hq, n, R = 2, 256, 40
+    rows = np.sort(rng.choice(n, R, replace=False)).astype(np.int32)
+    lse_full = rng.uniform(2, 8, (Hq, R)).astype(np.float32)
+    lse_sel = np.zeros((Hq, n), np.float32)
+    lse_sel[:, rows] = lse_full - rng.exponential(0.05, (Hq, R)).astype(np.float32)
+    bad = rows.copy()
+    bad[3], bad[17] = n, -1
+    vmax = np.float32([3.0, 4.0])
+    t = lambda a: torch.from_numpy(a).cuda()
+    m_row, m_head = torch.zeros((Hq, R), device="cuda"), torch.zeros(Hq, device="cuda")
+    st = rs.new_status()
+    rs.rs_certificate(Hq, Hq, n, t(lse_sel), t(lse_full), t(bad), t(vmax), None, 0.0, m_row, None, None, m_head, None, st)
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[0] == -1
+    got = m_row.cpu().numpy()
+    assert np.isnan(got[:, [3, 17]]).all()
+    ok = np.ones(R, bool); ok[[3, 17]] = False
+    for h in range(Hq):
+        m = CT.certificate(lse_sel[h, rows[ok]], lse_full[h, ok], vmax[h], None, 0.0)[0]
+        assert np.allclose(got[h, ok], m, rtol=1e-5, atol=1e-6)
+        assert abs(float(m_head[h]) - float(np.mean(m))) < 1e-6
+
+
 def test_bounded_wait_gives_up_and_reports():
     """A device-side wait that nothing satisfies runs out by itself; the status words say so and the context lives on."""
     st = rs.new_status()

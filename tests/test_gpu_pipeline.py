@@ -12,33 +12,11 @@ from oracle import certificate as CT
 from oracle import patterns as PT
 from oracle import probe as OP
 from oracle import routing as RT
+from bench import download_sets
 from synth import config1_spec, make_layer, tiny_spec
 
 pytestmark = pytest.mark.gpu
 C = PT.Candidate
-
-
-def download_sets(layer, cands, choice):
-    p = layer.p
-    nb = p.n_keys // 64
-    reuse = getattr(layer, "_reuse_eval", False)       # vertical-slash lists may still sit in the evaluation layout
-    vs = layer.idx_eval if reuse else layer.idx
-    cnt = vs.vs_count.cpu().numpy()
-    cols, offs, diag = (t.cpu().numpy() for t in (vs.vs_cols, vs.vs_offs, vs.vs_diag))
-    blk, bcnt = layer.idx.bs_blk.cpu().numpy(), layer.idx.bs_count.cpu().numpy()
-    sets = []
-    for item in range(p.n_items):
-        s, h = divmod(item, p.n_q_heads)
-        q0, q1 = p.seg_bounds[s], p.seg_bounds[s + 1]
-        cand = cands[choice[item]]
-        ix = PT.IndexSet(cand=cand, q0=q0, q1=q1)
-        if cand.pattern == PT.VERTICAL_SLASH:
-            sl = item * len(cands) + int(choice[item]) if reuse else item
-            ix.V, ix.S, ix.D = cols[sl, :cnt[sl, 0]], offs[sl, :cnt[sl, 1]], diag[sl, :cnt[sl, 2]]
-        elif cand.pattern == PT.BLOCK_SPARSE:
-            ix.blk = [blk[h * nb + qb, :bcnt[h * nb + qb]] for qb in range(q0 // 64, q1 // 64)]
-        sets.append(ix)
-    return sets
 
 
 def run_and_check(spec, bounds, cands, cfg, seed_name):

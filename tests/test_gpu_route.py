@@ -36,7 +36,7 @@ def gpu_route(p, lib, cov, pairs, cost, vmax, **kw):
     prm.use_cert = 0 if kw.get("cert_max") is None else 1
     prm.cert_max = 0.0 if kw.get("cert_max") is None else kw["cert_max"]
     prm.cert_mode = kw.get("cert_mode", rs.RS_CERT_REL); prm.expand_first = int(kw.get("expand_first", True))
-    prm.reserved = int(kw.get("rescue_any", False))
+    prm.rescue_any = int(kw.get("rescue_any", False))
     prm.backfill = int(kw.get("backfill", False))
     prm.global_pattern = int(kw.get("global_pattern", False))
     keep = []
