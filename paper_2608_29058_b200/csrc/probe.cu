@@ -3,13 +3,21 @@
 //
 // For every (segment, KV head) the 64 probe rows of up to four query heads (256 rows) are scored against all
 // causal keys on the tensor cores, twice:
-//   pass 1 (probe_lse):   S = Qp K^T with probe rows on the TMEM lanes; every thread owns one probe row and keeps
-//                         its running maximum and sum, split over key ranges; partials are merged afterwards.
+//   pass 1 (probe_lse):   S = Qp K^T with probe rows on the TMEM lanes; a thread owns one probe row and half of the
+//                         tile's key columns and keeps a running maximum and sum; the partials of all key ranges are
+//                         merged in the prologue of pass 2.  Two more warps form the 64-row means of K from the very
+//                         tile the tensor cores read (no second stream of K for the pooled keys).
 //   pass 2 (probe_accum): S^T = K Qp^T with keys on the TMEM lanes; every thread owns one key, so the column
-//                         mass of a 16-row probe group is a sum inside the thread; the diagonal (slash) mass is
-//                         a skewed sum over a 16 x 128 tile staged in shared memory.
-// Each key tile is read from HBM once per pass (TMA, 128-byte swizzle); both passes are balanced between the
-// HBM stream and the exponential rate.
+//                         mass of a 16-row probe group is a sum inside the thread; the diagonal (slash) mass is a
+//                         skewed sum over the warp's own 16 x 32 tile of probabilities in shared memory.  The four
+//                         lane quadrants of a tile hold four different stretches of the CTA's key range (four TMA
+//                         boxes of 32 keys), so a warp walks 32 consecutive keys per step through a contiguous
+//                         quarter of the range and the part of a diagonal that runs off its tile is carried, in a
+//                         register, into its own next step.  Every offset is produced by exactly one thread: no
+//                         atomics, no zero-filled output, no barrier between warps.
+// Each key tile is read from HBM once per pass (TMA, 128-byte swizzle).
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace {
@@ -19,8 +27,9 @@ constexpr int kHC = 4;                 // head slots per CTA (4 x 64 = 256 probe
 constexpr int kRows = kHC * RS_PROBE_ROWS;
 constexpr int kKeyTile = 128;
 constexpr int kStages = 3;
-constexpr int kThreads1 = 320;         // pass 1: warp 0 TMA, warp 1 MMA, warps 2..9 compute
+constexpr int kThreads1 = 640;         // pass 1: warp 0 TMA, warp 1 MMA, warps 2..17 compute, warps 18..19 pool K
 constexpr int kThreads2 = 576;         // pass 2: warp 0 TMA, warp 1 MMA, warps 2..17 compute
+constexpr int kComputeThreads = 512;
 constexpr uint32_t kTmemCols = 512;
 
 struct rs_candidate_list { int32_t pattern[RS_MAX_CANDIDATES]; };
@@ -29,12 +38,12 @@ struct ProbeParams {
   int n, Hq, Hkv, group, n_seg, n_hc;  // n_hc = head chunks per KV head = ceil(group / 4)
   int seg_bounds[RS_MAX_SEGMENTS + 1];
   int n_splits, per;
-  float4* partial;    // [n_seg*Hkv*n_hc][n_splits][256] (max, sum, sum of p * score, sum of p inside the local band), exp2 domain
-  float* lse2;        // [n_seg*Hkv*n_hc][256] log-sum-exp * log2(e)
+  float4* partial;    // [n_seg*Hkv*n_hc][2*n_splits][256] (max, sum, sum of p * score, sum of p inside the local band), exp2 domain
   float* lse_probe;   // [Hq][n_seg][64]
   float* descr;       // [n_seg][Hq][2] entropy and local-band mass, means over the 64 probe rows (may be NULL)
   float* vert;        // [n_seg][Hq][4][n]
   float* slash;       // [n_seg][Hq][4][n]
+  float* kpool;       // [Hkv][n/64][128] 64-row means of K, written by pass 1 (may be NULL)
   int32_t* status;
   float scale_log2e;
 };
@@ -45,12 +54,15 @@ struct Smem {
   static constexpr uint32_t x = k + kStages * 32768;      // pass 2: [16 compute warps][16 rows][32 keys] fp32
   static constexpr uint32_t lse = x + 32768;              // 256 floats
   static constexpr uint32_t bars = lse + 1024;            // mbarriers
-  static constexpr uint32_t misc = bars + 128;
+  static constexpr uint32_t misc = bars + 256;
   static constexpr uint32_t total = misc + 64 + 1024;     // + alignment slack
 };
+static_assert(Smem::total <= 227 * 1024, "probe shared memory");
 
-__device__ __forceinline__ void named_bar_sync(int id, int count) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
 template <int PASS>
@@ -76,6 +88,12 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int per = P.per;                      // key tiles per CTA, the same for every unit
   const int t0 = blockIdx.x * per, t1 = min(n_tiles, t0 + per);
   const int i_first = q1 - RS_PROBE_ROWS;   // first probe row
+  // Pass 2: the CTA's keys [128 t0, 128 t1) are cut into four contiguous quarters of 32 (t1 - t0) keys, one per lane
+  // quadrant; step st = -1 .. t1 - t0 - 1 of quadrant q covers keys quarter start + 32 st .. + 31.  Step -1 stores
+  // nothing: it only produces the carries of the diagonals that reach back over the start of the quarter.
+  const int n_mma = (PASS == 2) ? (t1 - t0 + 1) : (t1 - t0);      // tiles through the tensor cores
+  // pass 1: the CTAs of the last segment (it sees every key) and of the first head chunk also pool K
+  const bool do_pool = PASS == 1 && P.kpool != nullptr && s == P.n_seg - 1 && hc == 0;
 
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + Smem::bars);
   volatile int* misc = reinterpret_cast<volatile int*>(sm + Smem::misc);
@@ -90,24 +108,73 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
   if (tid == 0) {
     mbar_init(bar_q, 1);
-    for (int i = 0; i < kStages; ++i) { mbar_init(bar_full[i], 1); mbar_init(bar_empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull[i], 1); mbar_init(bar_tempty[i], kThreads - 64); }
+    for (int i = 0; i < kStages; ++i) { mbar_init(bar_full[i], 1); mbar_init(bar_empty[i], do_pool ? 3 : 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull[i], 1); mbar_init(bar_tempty[i], kComputeThreads); }
     misc[1] = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
   }
   if (warp == 1) { tmem_alloc(smem_u32((const void*)&misc[0]), kTmemCols); tmem_relinquish(); }
   if (PASS == 2) {
-    for (int i = tid; i < kRows; i += kThreads) s_lse[i] = P.lse2[(size_t)unit * kRows + i];
+    // Merge of pass 1's partial (max, sum) pairs into the log-sum-exp of the unit's 256 probe rows; every CTA of the
+    // unit forms the same values in the same order, the first one also stores them (and the two descriptors).
+    if (tid < kRows) {
+      const int row = tid, hh = row >> 6;
+      const int n_part = 2 * P.n_splits;
+      const float4* part = P.partial + (size_t)unit * n_part * kRows + row;
+      float m = -INFINITY;
+      for (int k = 0; k < n_part; ++k) m = fmaxf(m, part[(size_t)k * kRows].x);
+      float l = 0.f, a = 0.f, loc = 0.f;
+      for (int k = 0; k < n_part; ++k) {
+        const float4 pk = part[(size_t)k * kRows];
+        if (pk.x > -INFINITY) {
+          const float sc = exp2f(pk.x - m);
+          l += pk.y * sc; a += pk.z * sc; loc += pk.w * sc;
+        }
+      }
+      const float lse2 = m + log2f(l);
+      s_lse[row] = lse2;
+      const bool live = hh < n_heads;
+      if (blockIdx.x == 0 && live)
+        P.lse_probe[((size_t)(h0 + hh) * P.n_seg + s) * RS_PROBE_ROWS + (row & 63)] = lse2 * 0.6931471805599453f;
+      if (blockIdx.x == 0 && P.descr != nullptr) {
+        // H_i = -sum p ln p = ln 2 * (lse2 - E_p[score2]); local mass = local sum / l; then the mean over the head's
+        // 64 rows (fixed order: a butterfly inside each warp, then the two warps of a head)
+        float e = 0.6931471805599453f * (lse2 - a / l), lc = loc / l;
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) {
+          e += __shfl_xor_sync(0xffffffffu, e, off);
+          lc += __shfl_xor_sync(0xffffffffu, lc, off);
+        }
+        float* red = reinterpret_cast<float*>(sm + Smem::x);      // not yet in use
+        if (lane == 0) { red[2 * warp] = e; red[2 * warp + 1] = lc; }
+      }
+    }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (PASS == 2 && blockIdx.x == 0 && P.descr != nullptr && tid < n_heads) {
+    const float* red = reinterpret_cast<const float*>(sm + Smem::x);
+    const int h = h0 + tid;
+    P.descr[((size_t)s * P.Hq + h) * 2 + 0] = (red[4 * tid] + red[4 * tid + 2]) * (1.0f / 64.0f);
+    P.descr[((size_t)s * P.Hq + h) * 2 + 1] = (red[4 * tid + 1] + red[4 * tid + 3]) * (1.0f / 64.0f);
+  }
+  if (PASS == 2 && blockIdx.x == 0) {
+    // offsets beyond the reach of a group's rows (o > first row of the group + 15) have no key: their mass is zero
+    for (int e = tid; e < n_heads * RS_PROBE_GROUPS * 48; e += kThreads) {
+      const int hh = e / (RS_PROBE_GROUPS * 48), grp = (e / 48) % RS_PROBE_GROUPS, k = e % 48;
+      const int o = i_first + grp * 16 + 16 + k;
+      if (o < q1)
+        P.slash[(((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS + grp) * (size_t)P.n + o] = 0.f;
+    }
+  }
+  __syncthreads();
   const uint32_t tmem = (uint32_t)misc[0];
   if (t0 >= t1) {   // nothing to do for this split (uniform across the CTA)
     if (PASS == 1) {
-      for (int i = tid; i < kRows; i += kThreads)
-        P.partial[((size_t)unit * P.n_splits + blockIdx.x) * kRows + i] = make_float4(-INFINITY, 0.f, 0.f, 0.f);
+      for (int i = tid; i < 2 * kRows; i += kThreads)
+        P.partial[((size_t)unit * 2 * P.n_splits + 2 * blockIdx.x) * kRows + i] = make_float4(-INFINITY, 0.f, 0.f, 0.f);
     }
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
@@ -124,15 +191,26 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         tma_load_2d(base + Smem::qp + 32768u + (uint32_t)hh * 8192u, &tmQ, bar_q, 64, row);
       }
       bool ok = true;
-      for (int t = t0; t < t1; ++t) {
-        const int it = t - t0, st = it % kStages;
+      for (int it = 0; it < n_mma; ++it) {
+        const int st = it % kStages;
         ok = mbar_wait(bar_empty[st], ((uint32_t)(it / kStages) & 1u) ^ 1u, abort_flag);
         if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, 11); break; }
         mbar_arrive_expect_tx(bar_full[st], 32768u);
         const uint32_t dst = base + Smem::k + (uint32_t)st * 32768u;
-        const int row = g * P.n + t * kKeyTile;
-        tma_load_2d(dst, &tmK, bar_full[st], 0, row);
-        tma_load_2d(dst + 16384u, &tmK, bar_full[st], 64, row);
+        if (PASS == 1) {
+          const int row = g * P.n + (t0 + it) * kKeyTile;
+          tma_load_2d(dst, &tmK, bar_full[st], 0, row);
+          tma_load_2d(dst + 16384u, &tmK, bar_full[st], 64, row);
+        } else {
+          // rows 32 q .. 32 q + 31 of the tile = the 32 keys of quadrant q's current step (a step that would start
+          // before key 0 loads keys 0..31 instead; its probabilities are zeroed by the consumer)
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int key0 = max(0, t0 * kKeyTile + (q * (t1 - t0) + it - 1) * 32);
+            tma_load_2d(dst + (uint32_t)q * 4096u, &tmK, bar_full[st], 0, g * P.n + key0);
+            tma_load_2d(dst + 16384u + (uint32_t)q * 4096u, &tmK, bar_full[st], 64, g * P.n + key0);
+          }
+        }
       }
       if (!ok) *abort_flag = 1;
     }
@@ -141,8 +219,8 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // ---------------------------------------------------------------- MMA issuer
       bool ok = mbar_wait(bar_q, 0, abort_flag);
       int site = 12;
-      for (int t = t0; t < t1 && ok; ++t) {
-        const int it = t - t0, st = it % kStages, b = it & 1;
+      for (int it = 0; it < n_mma && ok; ++it) {
+        const int st = it % kStages, b = it & 1;
         ok = mbar_wait(bar_full[st], (uint32_t)(it / kStages) & 1u, abort_flag); site = 13;
         if (!ok) break;
         ok = mbar_wait(bar_tempty[b], ((uint32_t)(it >> 1) & 1u) ^ 1u, abort_flag); site = 14;
@@ -179,196 +257,205 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       }
       if (!ok) { rs_report(P.status, RS_ERR_TIMEOUT, site); *abort_flag = 1; }
     }
+  } else if (PASS == 1 && warp >= 18) {
+    // ------------------------------------------------------------------ 64-row means of K from the staged tiles
+    if (do_pool) {
+      const int w = warp - 18;                  // key block inside the tile
+      const int c = lane & 15, par = lane >> 4; // 16-byte column chunk, row parity
+      const uint32_t col_off = (uint32_t)(c >> 3) * 16384u;
+      const int cc = c & 7;
+      bool ok = true;
+      for (int t = t0; t < t1; ++t) {
+        const int it = t - t0, st = it % kStages;
+        ok = mbar_wait(bar_full[st], (uint32_t)(it / kStages) & 1u, abort_flag);
+        if (!ok) break;
+        const int kb = 2 * t + w;
+        if (kb * 64 < q1) {
+          const uint8_t* tile = sm + Smem::k + (uint32_t)st * 32768u + col_off;
+          float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll 8
+          for (int k = 0; k < 32; ++k) {
+            const int r = 64 * w + 2 * k + par;
+            const uint4 u = *reinterpret_cast<const uint4*>(tile + r * 128 + ((cc ^ (r & 7)) << 4));   // 128-byte swizzle
+            const uint32_t wd[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              acc[2 * e] += __uint_as_float(wd[e] << 16);
+              acc[2 * e + 1] += __uint_as_float(wd[e] & 0xffff0000u);
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 16);
+          if (par == 0) {
+            float4* dst = reinterpret_cast<float4*>(P.kpool + ((size_t)g * (P.n >> 6) + kb) * RS_HEAD_DIM + c * 8);
+            const float sc = 1.0f / 64.0f;
+            dst[0] = make_float4(acc[0] * sc, acc[1] * sc, acc[2] * sc, acc[3] * sc);
+            dst[1] = make_float4(acc[4] * sc, acc[5] * sc, acc[6] * sc, acc[7] * sc);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_empty[st]);
+      }
+      if (!ok && lane == 0) { rs_report(P.status, RS_ERR_TIMEOUT, 16); *abort_flag = 1; }
+    }
   } else {
     // ------------------------------------------------------------------ compute warps
-    const int cw = warp - 2;                 // 0..7
+    const int cw = warp - 2;                 // 0..15
     const int quad = warp & 3;               // TMEM lane quadrant this warp may touch
-    const int part = cw >> 2;                // pass 1: head pair
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const float sl2 = P.scale_log2e;
-    uint32_t v[32];
     bool ok = true;
 
     if (PASS == 1) {
+      const int part = (cw >> 2) & 1;                 // head pair
+      const int colhalf = cw >> 3;                    // which 64 of the tile's 128 key columns
       const int r = quad * 32 + lane;                 // row inside the head pair (0..127)
       const int hh = part * 2 + (r >> 6);             // head slot
       const int i = i_first + (r & 63);               // global query row
       const bool want_descr = P.descr != nullptr;
       float m_run = -INFINITY, l_run = 0.f;
       float a_run = 0.f, loc_run = 0.f;               // sum of p * score and local-band sum of p (descriptors)
+      uint32_t v[32];
       for (int t = t0; t < t1; ++t) {
         const int it = t - t0, b = it & 1;
         ok = mbar_wait(bar_tfull[b], (uint32_t)(it >> 1) & 1u, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const int j0 = t * kKeyTile;
-        const bool need_mask = j0 + kKeyTile - 1 > i_first;
-        const bool near = j0 + kKeyTile - 1 > i_first - RS_LOCAL_BAND;   // tile reaches into some row's local band
+        const int j0 = t * kKeyTile + colhalf * 64;
+        const bool need_mask = j0 + 63 > i_first;
+        const bool near = j0 + 63 > i_first - RS_LOCAL_BAND;   // reaches into some row's local band
 #pragma unroll 1
-        for (int c4 = 0; c4 < 4; ++c4) {
-          tmem_ld32(tmem + lane_addr + (uint32_t)(b * 256 + part * 128 + c4 * 32), v);
+        for (int c2 = 0; c2 < 2; ++c2) {
+          tmem_ld32(tmem + lane_addr + (uint32_t)(b * 256 + part * 128 + colhalf * 64 + c2 * 32), v);
           tc_wait_ld();
-          float mx = -INFINITY;
+          const int jc = j0 + c2 * 32;
+          if (need_mask) {
 #pragma unroll
-          for (int x = 0; x < 32; ++x) {
-            float sv = __uint_as_float(v[x]) * sl2;
-            if (need_mask && (j0 + c4 * 32 + x > i)) sv = -INFINITY;
-            v[x] = __float_as_uint(sv);
-            mx = fmaxf(mx, sv);
+            for (int x = 0; x < 32; ++x)
+              if (jc + x > i) v[x] = 0xff800000u;
           }
-          if (mx > m_run) {
+          float mxa[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            mxa[q] = max3f(__uint_as_float(v[8 * q]), __uint_as_float(v[8 * q + 1]), __uint_as_float(v[8 * q + 2]));
+            mxa[q] = max3f(mxa[q], __uint_as_float(v[8 * q + 3]), __uint_as_float(v[8 * q + 4]));
+            mxa[q] = max3f(mxa[q], __uint_as_float(v[8 * q + 5]), __uint_as_float(v[8 * q + 6]));
+            mxa[q] = fmaxf(mxa[q], __uint_as_float(v[8 * q + 7]));
+          }
+          const float mx = fmaxf(max3f(mxa[0], mxa[1], mxa[2]), mxa[3]) * sl2;
+          // the reference only moves when it is exceeded by more than 2^8 (the sums stay far inside fp32 range)
+          if (mx > m_run + 8.0f) {
             const float sc = fast_exp2(m_run - mx);
             l_run *= sc; a_run *= sc; loc_run *= sc;
             m_run = mx;
           }
           if (m_run > -INFINITY) {
-            float acc = 0.f, acc_a = 0.f, acc_l = 0.f;
+            const float neg_m = -m_run;
             if (want_descr) {
+              float acc = 0.f, acc_a = 0.f, acc_l = 0.f;
 #pragma unroll
               for (int x = 0; x < 32; ++x) {
-                const float sv = __uint_as_float(v[x]);
-                const float pe = fast_exp2(sv - m_run);
+                const float sv = __uint_as_float(v[x]) * sl2;
+                const float pe = fast_exp2(sv + neg_m);
                 acc += pe;
                 acc_a = fmaf(pe, fmaxf(sv, -1e30f), acc_a);          // masked entries: pe = 0, keep the product finite
-                if (near && i - (j0 + c4 * 32 + x) < RS_LOCAL_BAND) acc_l += pe;
+                if (near && i - (jc + x) < RS_LOCAL_BAND) acc_l += pe;
               }
+              l_run += acc; a_run += acc_a; loc_run += acc_l;
             } else {
+              float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-              for (int x = 0; x < 32; ++x) acc += fast_exp2(__uint_as_float(v[x]) - m_run);
+              for (int x = 0; x < 32; x += 4) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) acc[q] += fast_exp2(fmaf(__uint_as_float(v[x + q]), sl2, neg_m));
+              }
+              l_run += (acc[0] + acc[1]) + (acc[2] + acc[3]);
             }
-            l_run += acc; a_run += acc_a; loc_run += acc_l;
           }
         }
         tc_fence_before();
         mbar_arrive(bar_tempty[b]);
       }
       if (ok) {
-        P.partial[((size_t)unit * P.n_splits + blockIdx.x) * kRows + hh * 64 + (r & 63)] = make_float4(m_run, l_run, a_run, loc_run);
+        P.partial[((size_t)unit * 2 * P.n_splits + 2 * blockIdx.x + colhalf) * kRows + hh * 64 + (r & 63)] =
+            make_float4(m_run, l_run, a_run, loc_run);
       }
     } else {
-      // Sixteen warps: warp (quad, hh) owns 32 keys of the tile (its TMEM lanes) and the 64 probe rows of head slot hh.
-      // Per probe group: 16 probabilities per key, their sum is the column mass; the diagonal mass is a skewed sum
-      // over the warp's own 16 x 32 tile in shared memory (bin u = l - r + 15, offset o = obase - u).  Bins fed by
-      // this warp alone are stored, the 15 bins on either side also get an addend from the neighbouring 32 keys
-      // and are accumulated with atomics (two addends onto zero: the order does not change the sum).
+      // Sixteen warps: warp (quad, hh) owns the 32 keys of its quadrant's current step (its TMEM lanes) and the 64
+      // probe rows of head slot hh.  Per probe group: 16 probabilities per key, their sum is the column mass; the
+      // diagonal mass is a skewed sum over the warp's own 16 x 32 tile in shared memory.  Row r of the tile is read
+      // rotated by (lane + r + 17) mod 32: for r >= 15 - lane that is key lane - 15 + r, a term of the diagonal that ends
+      // at this lane's key (offset o = first row of the group + 15 - key); otherwise it is key lane + 17 + r, a term of
+      // the diagonal that ends at lane's key of the NEXT step and is carried there in a register.  One conflict-free
+      // read per row serves both.
       const int hh = cw >> 2;                         // head slot
-      const int l128 = quad * 32 + lane;              // key inside the tile
       float* xw = reinterpret_cast<float*>(sm + Smem::x) + cw * (16 * 32);
       const bool live = hh < n_heads;
-      // Row r of the warp's tile is read rotated by (lane + r + 17) mod 32: for r >= 15 - lane that is key
-      // lane - 15 + r (bin u = lane), otherwise key lane + 17 + r (bin u = lane + 32, lanes 0..14 only), so one
-      // conflict-free read per row serves both bins of a lane.
       int rot[16];
 #pragma unroll
       for (int r = 0; r < 16; ++r) rot[r] = r * 32 + ((lane + r + 17) & 31);
-      const int k_lo = 15 - lane;                     // rows r >= k_lo feed bin u = lane
-      auto group = [&](const uint32_t (&v16)[16], int grp, int j, int j0, bool masked) {
-        const int ig = i_first + grp * 16;            // first row of the group
-        const float4* l4 = reinterpret_cast<const float4*>(s_lse + hh * 64 + grp * 16);
-        float lse16[16];
+      const int k_lo = 15 - lane;                     // rows r >= k_lo belong to this step's diagonal
+      const int key_q = t0 * kKeyTile + quad * (t1 - t0) * 32;     // first key of this quadrant's quarter
+      float carry[RS_PROBE_GROUPS] = {0.f, 0.f, 0.f, 0.f};
+      float* const vert_h = P.vert + ((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS * (size_t)P.n;
+      float* const slash_h = P.slash + ((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS * (size_t)P.n;
+      // One step: the four probe groups of the warp's 32 keys.  MASKED steps (those that reach the probe rows, and the
+      // step before key 0) also zero the probabilities of pairs with j > i or j < 0.
+      auto step = [&](auto masked_tag, int b, int j, bool store) {
+        constexpr bool MASKED = decltype(masked_tag)::value;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float4 t4 = l4[q];
-          lse16[4 * q] = t4.x; lse16[4 * q + 1] = t4.y; lse16[4 * q + 2] = t4.z; lse16[4 * q + 3] = t4.w;
-        }
-        float vsum = 0.f;
-        __syncwarp();                                 // the previous group's rotated reads are done
-#pragma unroll
-        for (int r = 0; r < 16; ++r) {
-          float p = fast_exp2(fmaf(__uint_as_float(v16[r]), sl2, -lse16[r]));
-          if (masked && j > ig + r) p = 0.f;
-          vsum += p;
-          xw[r * 32 + lane] = p;
-        }
-        const size_t out = (((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS + grp) * (size_t)P.n;
-        if (live && j < q1) P.vert[out + j] = vsum;
-        __syncwarp();
-        float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll
-        for (int r = 0; r < 16; ++r) {
-          const float x = xw[rot[r]];
-          if (r >= k_lo) acc0 += x; else acc1 += x;
-        }
-        // bin u <-> offset o = obase - u; bins 15..31 are fed by this warp's keys alone
-        const int obase = ig - (j0 + quad * 32) + 15;
-        if (live) {
-          const int o0 = obase - lane;
-          if (o0 >= 0) {
-            if (lane >= 15) P.slash[out + o0] = acc0;
-            else atomicAdd(&P.slash[out + o0], acc0);
-          }
-          const int o1 = o0 - 32;
-          if (lane < 15 && o1 >= 0) atomicAdd(&P.slash[out + o1], acc1);
-        }
-      };
-      for (int t = t0; t < t1; ++t) {
-        const int it = t - t0, b = it & 1;
-        ok = mbar_wait(bar_tfull[b], (uint32_t)(it >> 1) & 1u, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        const int j0 = t * kKeyTile;
-        const int j = j0 + l128;
-        const bool need_mask = j0 + kKeyTile - 1 > i_first;   // only the tiles that reach the probe rows
-#pragma unroll 1
         for (int grp = 0; grp < RS_PROBE_GROUPS; ++grp) {
           uint32_t v16[16];
           tmem_ld16(tmem + lane_addr + (uint32_t)(b * 256 + hh * 64 + grp * 16), v16);
+          const int ig = i_first + grp * 16;            // first row of the group
+          const float4* l4 = reinterpret_cast<const float4*>(s_lse + hh * 64 + grp * 16);
+          float lse16[16];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float4 t4 = l4[q];
+            lse16[4 * q] = t4.x; lse16[4 * q + 1] = t4.y; lse16[4 * q + 2] = t4.z; lse16[4 * q + 3] = t4.w;
+          }
           tc_wait_ld();
-          if (need_mask) group(v16, grp, j, j0, true);
-          else group(v16, grp, j, j0, false);
+          float vs[4] = {0.f, 0.f, 0.f, 0.f};
+          __syncwarp();                                 // the previous group's rotated reads are done
+#pragma unroll
+          for (int r = 0; r < 16; ++r) {
+            float p = fast_exp2(fmaf(__uint_as_float(v16[r]), sl2, -lse16[r]));
+            if (MASKED && (j > ig + r || j < 0)) p = 0.f;
+            vs[r & 3] += p;
+            xw[r * 32 + lane] = p;
+          }
+          if (store && j < q1) vert_h[(size_t)grp * P.n + j] = (vs[0] + vs[1]) + (vs[2] + vs[3]);
+          __syncwarp();
+          float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+          for (int r = 0; r < 16; ++r) {
+            const float x = xw[rot[r]];
+            if (r >= k_lo) acc0 += x; else acc1 += x;
+          }
+          const int o = ig + 15 - j;                    // the offset whose diagonal ends at this key
+          if (store && o >= 0) slash_h[(size_t)grp * P.n + o] = acc0 + carry[grp];
+          carry[grp] = acc1;                            // lanes 15..31: zero
         }
+      };
+      for (int it = 0; it < n_mma; ++it) {
+        const int b = it & 1;
+        ok = mbar_wait(bar_tfull[b], (uint32_t)(it >> 1) & 1u, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const int jw = key_q + (it - 1) * 32;           // first key of the step
+        if (jw + 31 > i_first || jw < 0) step(std::true_type{}, b, jw + lane, it > 0 && live);
+        else step(std::false_type{}, b, jw + lane, it > 0 && live);
         tc_fence_before();
         mbar_arrive(bar_tempty[b]);
       }
     }
-    if (!ok && lane == 0 && cw == 0) { rs_report(P.status, RS_ERR_TIMEOUT, 15); *abort_flag = 1; }
+    if (!ok && lane == 0) { rs_report(P.status, RS_ERR_TIMEOUT, 15); *abort_flag = 1; }
   }
 
   tc_fence_before();
   __syncthreads();
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, kTmemCols); }
-}
-
-// Merges the per-split (max, sum) partials of pass 1 into the probe log-sum-exp.
-__global__ void rs_probe_merge_kernel(ProbeParams P) {
-  const int unit = blockIdx.x;
-  const int row = threadIdx.x;    // 0..255
-  const int hc = unit % P.n_hc;
-  const int g = (unit / P.n_hc) % P.Hkv;
-  const int s = unit / (P.n_hc * P.Hkv);
-  const int hh = row >> 6;
-  const float4* part = P.partial + (size_t)unit * P.n_splits * kRows + row;
-  float m = -INFINITY;
-  for (int k = 0; k < P.n_splits; ++k) m = fmaxf(m, part[(size_t)k * kRows].x);
-  float l = 0.f, a = 0.f, loc = 0.f;
-  for (int k = 0; k < P.n_splits; ++k) {
-    const float4 pk = part[(size_t)k * kRows];
-    if (pk.x > -INFINITY) {
-      const float sc = exp2f(pk.x - m);
-      l += pk.y * sc; a += pk.z * sc; loc += pk.w * sc;
-    }
-  }
-  const float lse2 = m + log2f(l);
-  P.lse2[(size_t)unit * kRows + row] = lse2;
-  const bool live = hc * kHC + hh < P.group;
-  if (live) {
-    const int h = g * P.group + hc * kHC + hh;
-    P.lse_probe[((size_t)h * P.n_seg + s) * RS_PROBE_ROWS + (row & 63)] = lse2 * 0.6931471805599453f;
-  }
-  if (P.descr != nullptr) {
-    // H_i = -sum p ln p = ln 2 * (lse2 - E_p[score2]); local mass = local sum / l; then the mean over the head's 64 rows
-    __shared__ float sh[kRows][2];
-    sh[row][0] = 0.6931471805599453f * (lse2 - a / l);
-    sh[row][1] = loc / l;
-    __syncthreads();
-    if ((row & 63) == 0 && live) {
-      float e = 0.f, lc = 0.f;
-      for (int r = 0; r < 64; ++r) { e += sh[row + r][0]; lc += sh[row + r][1]; }
-      const int h = g * P.group + hc * kHC + hh;
-      P.descr[((size_t)s * P.Hq + h) * 2 + 0] = e * (1.0f / 64.0f);
-      P.descr[((size_t)s * P.Hq + h) * 2 + 1] = lc * (1.0f / 64.0f);
-    }
-  }
 }
 
 // 64-row means of Q and K (fp32) and per-block maxima of ||v||^2.
@@ -455,7 +542,7 @@ __global__ void rs_vmax_kernel(ProbeParams P, const float* blockmax, float* vmax
   }
 }
 
-struct ProbePlan { size_t partial, lse2, blockmax, total; int n_units, n_splits, n_hc, per; };
+struct ProbePlan { size_t partial, blockmax, total; int n_units, n_splits, n_hc, per; };
 
 ProbePlan plan(const rs_problem* p) {
   ProbePlan w{};
@@ -475,8 +562,7 @@ ProbePlan plan(const rs_problem* p) {
   w.per = per;
   w.n_splits = splits;
   size_t off = 0;
-  w.partial = off;  off += rs_align_up((size_t)w.n_units * splits * kRows * sizeof(float4), 256);
-  w.lse2 = off;     off += rs_align_up((size_t)w.n_units * kRows * sizeof(float), 256);
+  w.partial = off;  off += rs_align_up((size_t)w.n_units * 2 * splits * kRows * sizeof(float4), 256);
   w.blockmax = off; off += rs_align_up((size_t)p->n_kv_heads * (p->n_keys / 64) * sizeof(float), 256);
   w.total = off;
   return w;
@@ -606,32 +692,40 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
   for (int s = 0; s <= p->n_segments; ++s) P.seg_bounds[s] = p->seg_bounds[s];
   P.partial = reinterpret_cast<float4*>(wsb + w.partial);
   P.descr = descr;
-  P.lse2 = reinterpret_cast<float*>(wsb + w.lse2);
-  P.lse_probe = lse_probe; P.vert = vert; P.slash = slash; P.status = status;
+  P.lse_probe = lse_probe; P.vert = vert; P.slash = slash; P.kpool = kpool; P.status = status;
   P.scale_log2e = (float)(1.4426950408889634 / sqrt((double)RS_HEAD_DIM));
 
-  const size_t mass_bytes = (size_t)P.n_seg * P.Hq * RS_PROBE_GROUPS * (size_t)P.n * sizeof(float);
-  if (cudaMemsetAsync(vert, 0, mass_bytes, stream) != cudaSuccess) return RS_ERR_CUDA;
-  if (cudaMemsetAsync(slash, 0, mass_bytes, stream) != cudaSuccess) return RS_ERR_CUDA;
+  // Pass 2 writes every entry below a segment's end exactly once; what lies beyond the end of a segment that stops
+  // before n_keys is zero by definition and is cleared here (nothing to do for a single segment).
+  for (int s = 0; s < P.n_seg; ++s) {
+    const int q1 = P.seg_bounds[s + 1];
+    if (q1 >= P.n) continue;
+    const size_t rows = (size_t)P.Hq * RS_PROBE_GROUPS, first = (size_t)s * rows * (size_t)P.n + (size_t)q1;
+    const size_t pitch = (size_t)P.n * sizeof(float), width = (size_t)(P.n - q1) * sizeof(float);
+    if (cudaMemset2DAsync(vert + first, pitch, 0, width, rows, stream) != cudaSuccess ||
+        cudaMemset2DAsync(slash + first, pitch, 0, width, rows, stream) != cudaSuccess)
+      return RS_ERR_CUDA;
+  }
 
-  CUtensorMap tmQ, tmK;
+  CUtensorMap tmQ, tmK, tmK32;      // K in boxes of 128 keys (pass 1) and of 32 keys (pass 2: one box per lane quadrant)
   if (rs_make_tmap_bf16_2d(&tmQ, Q, (uint64_t)P.Hq * P.n, RS_HEAD_DIM, 64, 64) ||
-      rs_make_tmap_bf16_2d(&tmK, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kKeyTile, 64))
+      rs_make_tmap_bf16_2d(&tmK, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kKeyTile, 64) ||
+      rs_make_tmap_bf16_2d(&tmK32, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, 32, 64))
     return RS_ERR_CUDA;
   static rs_smem_attr attr_pass1, attr_pass2;
   if (rs_ensure_dynamic_smem(attr_pass1, rs_probe_kernel<1>, (int)Smem::total) != RS_OK ||
       rs_ensure_dynamic_smem(attr_pass2, rs_probe_kernel<2>, (int)Smem::total) != RS_OK)
     return RS_ERR_CUDA;
-  // The pooled means and the value norms only read Q, K, V: they run beside the two probe passes, on the side
+  // The value norms and the pooled queries only read V and Q: they run beside the two probe passes, on the side
   // stream.  Pass 1 is enqueued first so that its CTAs (one per SM, most of the shared memory) are resident before
   // the small streaming CTAs fill what is left; the other way round the streaming kernels would run alone.
+  // The pooled keys come out of pass 1 itself.
   cudaStream_t side = nullptr;
   rc = rs_side_fork(stream, &side);
   if (rc != RS_OK) return rc;
   dim3 grid(w.n_splits, w.n_units);
   rs_probe_kernel<1><<<grid, kThreads1, Smem::total, stream>>>(tmQ, tmK, P);
   const long long nb = p->n_keys / 64;
-  if (kpool) rs_pool_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(K), kpool, P.Hkv * nb);
   if (vmax) {
     float* blockmax = reinterpret_cast<float*>(wsb + w.blockmax);
     rs_vnorm_block_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(V), blockmax, P.Hkv * nb);
@@ -644,8 +738,7 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
   } else if (qpool) {
     rs_pool_kernel<<<(unsigned)(P.Hq * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(Q), qpool, P.Hq * nb);
   }
-  rs_probe_merge_kernel<<<w.n_units, kRows, 0, stream>>>(P);
-  rs_probe_kernel<2><<<grid, kThreads2, Smem::total, stream>>>(tmQ, tmK, P);
+  rs_probe_kernel<2><<<grid, kThreads2, Smem::total, stream>>>(tmQ, tmK32, P);
   rc = rs_side_join(stream);
   if (rc != RS_OK) return rc;
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
