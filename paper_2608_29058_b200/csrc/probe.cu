@@ -31,6 +31,7 @@ constexpr int kThreads1 = 640;         // pass 1: warp 0 TMA, warp 1 MMA, warps 
 constexpr int kThreads2 = 576;         // pass 2: warp 0 TMA, warp 1 MMA, warps 2..17 compute
 constexpr int kComputeThreads = 512;
 constexpr uint32_t kTmemCols = 512;
+constexpr int kXS = 62;                // floats per row of a warp's probability tile: 15 zeros, 32 keys, 15 zeros
 
 struct rs_candidate_list { int32_t pattern[RS_MAX_CANDIDATES]; };
 
@@ -51,8 +52,8 @@ struct ProbeParams {
 struct Smem {
   static constexpr uint32_t qp = 0;                       // 2 halves x 256 rows x 128 B
   static constexpr uint32_t k = 65536;                    // kStages x (2 halves x 128 rows x 128 B)
-  static constexpr uint32_t x = k + kStages * 32768;      // pass 2: [16 compute warps][16 rows][32 keys] fp32
-  static constexpr uint32_t lse = x + 32768;              // 256 floats
+  static constexpr uint32_t x = k + kStages * 32768;      // pass 2: [16 compute warps][16 rows][kXS] fp32
+  static constexpr uint32_t lse = x + 16 * 16 * kXS * 4;  // 256 floats
   static constexpr uint32_t bars = lse + 1024;            // mbarriers
   static constexpr uint32_t misc = bars + 256;
   static constexpr uint32_t total = misc + 64 + 1024;     // + alignment slack
@@ -109,7 +110,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (tid == 0) {
     mbar_init(bar_q, 1);
     for (int i = 0; i < kStages; ++i) { mbar_init(bar_full[i], 1); mbar_init(bar_empty[i], do_pool ? 3 : 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull[i], 1); mbar_init(bar_tempty[i], kComputeThreads); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull[i], 1); mbar_init(bar_tempty[i], kComputeThreads / 32); }
     misc[1] = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
@@ -118,20 +119,43 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (PASS == 2) {
     // Merge of pass 1's partial (max, sum) pairs into the log-sum-exp of the unit's 256 probe rows; every CTA of the
     // unit forms the same values in the same order, the first one also stores them (and the two descriptors).
-    if (tid < kRows) {
-      const int row = tid, hh = row >> 6;
-      const int n_part = 2 * P.n_splits;
+    // 512 threads: thread (row, half) folds every second partial of the row, eight loads in flight at a time; the two
+    // halves meet through shared memory.  The order of the additions is fixed, so every CTA gets the same bits.
+    float4* mrg = reinterpret_cast<float4*>(sm + Smem::x);        // [2][256] (max, sum, a, loc); x is not yet in use
+    const int n_part = 2 * P.n_splits;
+    if (tid < 2 * kRows) {
+      const int row = tid & (kRows - 1), half = tid >> 8;
       const float4* part = P.partial + (size_t)unit * n_part * kRows + row;
-      float m = -INFINITY;
-      for (int k = 0; k < n_part; ++k) m = fmaxf(m, part[(size_t)k * kRows].x);
-      float l = 0.f, a = 0.f, loc = 0.f;
-      for (int k = 0; k < n_part; ++k) {
-        const float4 pk = part[(size_t)k * kRows];
-        if (pk.x > -INFINITY) {
-          const float sc = exp2f(pk.x - m);
-          l += pk.y * sc; a += pk.z * sc; loc += pk.w * sc;
+      float m = -INFINITY, l = 0.f, a = 0.f, loc = 0.f;
+      for (int k0 = half; k0 < n_part; k0 += 16) {
+        float4 pk[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int k = k0 + 2 * u;
+          pk[u] = k < n_part ? __ldg(part + (size_t)k * kRows) : make_float4(-INFINITY, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          if (pk[u].x > m) {
+            const float sc = exp2f(m - pk[u].x);
+            l *= sc; a *= sc; loc *= sc;
+            m = pk[u].x;
+          }
+          if (pk[u].x > -INFINITY) {
+            const float sc = exp2f(pk[u].x - m);
+            l = fmaf(pk[u].y, sc, l); a = fmaf(pk[u].z, sc, a); loc = fmaf(pk[u].w, sc, loc);
+          }
         }
       }
+      mrg[half * kRows + row] = make_float4(m, l, a, loc);
+    }
+    __syncthreads();
+    if (tid < kRows) {
+      const int row = tid, hh = row >> 6;
+      const float4 p0 = mrg[row], p1 = mrg[kRows + row];
+      const float m = fmaxf(p0.x, p1.x);
+      const float s0 = p0.x > -INFINITY ? exp2f(p0.x - m) : 0.f, s1 = p1.x > -INFINITY ? exp2f(p1.x - m) : 0.f;
+      const float l = p0.y * s0 + p1.y * s1, a = p0.z * s0 + p1.z * s1, loc = p0.w * s0 + p1.w * s1;
       const float lse2 = m + log2f(l);
       s_lse[row] = lse2;
       const bool live = hh < n_heads;
@@ -146,7 +170,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           e += __shfl_xor_sync(0xffffffffu, e, off);
           lc += __shfl_xor_sync(0xffffffffu, lc, off);
         }
-        float* red = reinterpret_cast<float*>(sm + Smem::x);      // not yet in use
+        float* red = reinterpret_cast<float*>(sm + Smem::x) + 4 * 2 * kRows;      // behind the merge scratch
         if (lane == 0) { red[2 * warp] = e; red[2 * warp + 1] = lc; }
       }
     }
@@ -155,7 +179,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   if (PASS == 2 && blockIdx.x == 0 && P.descr != nullptr && tid < n_heads) {
-    const float* red = reinterpret_cast<const float*>(sm + Smem::x);
+    const float* red = reinterpret_cast<const float*>(sm + Smem::x) + 4 * 2 * kRows;
     const int h = h0 + tid;
     P.descr[((size_t)s * P.Hq + h) * 2 + 0] = (red[4 * tid] + red[4 * tid + 2]) * (1.0f / 64.0f);
     P.descr[((size_t)s * P.Hq + h) * 2 + 1] = (red[4 * tid + 1] + red[4 * tid + 3]) * (1.0f / 64.0f);
@@ -170,6 +194,11 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
   }
   __syncthreads();
+  if (PASS == 2) {          // the zero columns on either side of every warp's probability tile (the scratch use is over)
+    float* xz = reinterpret_cast<float*>(sm + Smem::x);
+    for (int i = tid; i < 16 * 16 * kXS; i += kThreads) xz[i] = 0.f;
+    __syncthreads();
+  }
   const uint32_t tmem = (uint32_t)misc[0];
   if (t0 >= t1) {   // nothing to do for this split (uniform across the CTA)
     if (PASS == 1) {
@@ -374,7 +403,8 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
           }
         }
         tc_fence_before();
-        mbar_arrive(bar_tempty[b]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty[b]);   // one arrival per warp: 512 arrivals per tile queue up on the barrier
       }
       if (ok) {
         P.partial[((size_t)unit * 2 * P.n_splits + 2 * blockIdx.x + colhalf) * kRows + hh * 64 + (r & 63)] =
@@ -383,18 +413,14 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     } else {
       // Sixteen warps: warp (quad, hh) owns the 32 keys of its quadrant's current step (its TMEM lanes) and the 64
       // probe rows of head slot hh.  Per probe group: 16 probabilities per key, their sum is the column mass; the
-      // diagonal mass is a skewed sum over the warp's own 16 x 32 tile in shared memory.  Row r of the tile is read
-      // rotated by (lane + r + 17) mod 32: for r >= 15 - lane that is key lane - 15 + r, a term of the diagonal that ends
-      // at this lane's key (offset o = first row of the group + 15 - key); otherwise it is key lane + 17 + r, a term of
-      // the diagonal that ends at lane's key of the NEXT step and is carried there in a register.  One conflict-free
-      // read per row serves both.
+      // diagonal mass is a skewed sum over the warp's own tile in shared memory, 16 rows of [15 zeros | 32 keys |
+      // 15 zeros].  Lane l sums x[r][l + r] over the 16 rows: the diagonal that ends at its key in row 15 (offset
+      // o = first row of the group + 15 - key); the terms of that diagonal that lie in the previous step's keys arrive
+      // through a register: lanes 0..14 also sum x[r][32 + l + r], the part of the diagonal ending at lane's key of the
+      // NEXT step that lies in this step's keys, and carry it over.  No predicates, no index arrays.
       const int hh = cw >> 2;                         // head slot
-      float* xw = reinterpret_cast<float*>(sm + Smem::x) + cw * (16 * 32);
+      float* xw = reinterpret_cast<float*>(sm + Smem::x) + cw * (16 * kXS);
       const bool live = hh < n_heads;
-      int rot[16];
-#pragma unroll
-      for (int r = 0; r < 16; ++r) rot[r] = r * 32 + ((lane + r + 17) & 31);
-      const int k_lo = 15 - lane;                     // rows r >= k_lo belong to this step's diagonal
       const int key_q = t0 * kKeyTile + quad * (t1 - t0) * 32;     // first key of this quadrant's quarter
       float carry[RS_PROBE_GROUPS] = {0.f, 0.f, 0.f, 0.f};
       float* const vert_h = P.vert + ((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS * (size_t)P.n;
@@ -403,10 +429,11 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // step before key 0) also zero the probabilities of pairs with j > i or j < 0.
       auto step = [&](auto masked_tag, int b, int j, bool store) {
         constexpr bool MASKED = decltype(masked_tag)::value;
+        uint32_t v16[16];
+        const uint32_t t_hh = tmem + lane_addr + (uint32_t)(b * 256 + hh * 64);
+        tmem_ld16(t_hh, v16);
 #pragma unroll
         for (int grp = 0; grp < RS_PROBE_GROUPS; ++grp) {
-          uint32_t v16[16];
-          tmem_ld16(tmem + lane_addr + (uint32_t)(b * 256 + hh * 64 + grp * 16), v16);
           const int ig = i_first + grp * 16;            // first row of the group
           const float4* l4 = reinterpret_cast<const float4*>(s_lse + hh * 64 + grp * 16);
           float lse16[16];
@@ -423,19 +450,23 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             float p = fast_exp2(fmaf(__uint_as_float(v16[r]), sl2, -lse16[r]));
             if (MASKED && (j > ig + r || j < 0)) p = 0.f;
             vs[r & 3] += p;
-            xw[r * 32 + lane] = p;
+            xw[r * kXS + 15 + lane] = p;
           }
+          // the scores of the next group travel from TMEM while this group's diagonals are summed
+          if (grp + 1 < RS_PROBE_GROUPS) tmem_ld16(t_hh + (uint32_t)(grp + 1) * 16u, v16);
           if (store && j < q1) vert_h[(size_t)grp * P.n + j] = (vs[0] + vs[1]) + (vs[2] + vs[3]);
           __syncwarp();
-          float acc0 = 0.f, acc1 = 0.f;
+          float acc0[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int r = 0; r < 16; ++r) {
-            const float x = xw[rot[r]];
-            if (r >= k_lo) acc0 += x; else acc1 += x;
-          }
+          for (int r = 0; r < 16; ++r) acc0[r & 3] += xw[r * (kXS + 1) + lane];
           const int o = ig + 15 - j;                    // the offset whose diagonal ends at this key
-          if (store && o >= 0) slash_h[(size_t)grp * P.n + o] = acc0 + carry[grp];
-          carry[grp] = acc1;                            // lanes 15..31: zero
+          if (store && o >= 0) slash_h[(size_t)grp * P.n + o] = ((acc0[0] + acc0[1]) + (acc0[2] + acc0[3])) + carry[grp];
+          if (lane < 15) {
+            float acc1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int r = 0; r < 15; ++r) acc1[r & 3] += xw[r * (kXS + 1) + 32 + lane];
+            carry[grp] = (acc1[0] + acc1[1]) + (acc1[2] + acc1[3]);
+          }
         }
       };
       for (int it = 0; it < n_mma; ++it) {
@@ -447,7 +478,8 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (jw + 31 > i_first || jw < 0) step(std::true_type{}, b, jw + lane, it > 0 && live);
         else step(std::false_type{}, b, jw + lane, it > 0 && live);
         tc_fence_before();
-        mbar_arrive(bar_tempty[b]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_tempty[b]);   // one arrival per warp: 512 arrivals per tile queue up on the barrier
       }
     }
     if (!ok && lane == 0) { rs_report(P.status, RS_ERR_TIMEOUT, 15); *abort_flag = 1; }
