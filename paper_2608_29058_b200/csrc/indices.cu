@@ -6,7 +6,11 @@
 // compaction, coverage is a sum of the same fixed-point values, and pair counts are closed forms.
 // Block-sparse scores are fp32 (fused pooled dot products accumulated k = 0..127 with fmaf, or an explicit
 // score matrix) compared through an order-preserving integer transform.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -84,37 +88,66 @@ __global__ void rs_vblk_kernel(IdxParams P) {
 }
 
 // ------------------------------------------------------------------------------------------ ranking keys, once per line
+// With fuse_vblk the blocks of list 0 also write the 64-key block sums of fx(vert) (what rs_vblk_kernel computes):
+// they hold the four fixed-point values of every key anyway.
 __global__ void __launch_bounds__(256)
-rs_vs_keys_kernel(IdxParams P) {
+rs_vs_keys_kernel(IdxParams P, int fuse_vblk) {
+  __shared__ u64 half_sum[8][RS_PROBE_GROUPS];
   const int item = blockIdx.y >> 1, list = blockIdx.y & 1;
   const int s = item / P.Hq;
   const int q1 = P.seg_bounds[s + 1];
   const int j = blockIdx.x * 256 + threadIdx.x;
-  if (j >= q1) return;
   const float* mass = (list == 0 ? P.vert : P.slash) + (size_t)item * RS_PROBE_GROUPS * P.n;
-  P.keys[((size_t)item * 2 + list) * P.n + j] = line_key(mass, P.n, j);
+  u64 f[RS_PROBE_GROUPS] = {0, 0, 0, 0};
+  if (j < q1) {
+#pragma unroll
+    for (int g = 0; g < RS_PROBE_GROUPS; ++g) f[g] = fx(mass[(size_t)g * P.n + j]);
+    P.keys[((size_t)item * 2 + list) * P.n + j] = (f[0] + f[1]) + (f[2] + f[3]);
+  }
+  if (!fuse_vblk || list != 0) return;                  // uniform over the block
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int g = 0; g < RS_PROBE_GROUPS; ++g) {
+    u64 v = f[g];
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    if (lane == 0) half_sum[warp][g] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x < 4 * RS_PROBE_GROUPS) {
+    const int blk = threadIdx.x >> 2, g = threadIdx.x & 3;
+    const int kb = blockIdx.x * 4 + blk;
+    if (kb < P.nb) P.vblk[((size_t)item * RS_PROBE_GROUPS + g) * P.nb + kb] = half_sum[2 * blk][g] + half_sum[2 * blk + 1][g];
+  }
 }
 
 // ------------------------------------------------------------------------------------------ exact top-k of a line list
-// grid = (2 lists, items, groups of up to kSelMaxC vertical-slash candidates).  list 0: vertical columns over [0, q1);
-// list 1: slash offsets over [1, q1) plus offset 0.  One block serves every budget of the item in the same passes
-// over the keys: the radix digits are histogrammed once per distinct prefix (the first digit once for all budgets),
-// and one counting sweep plus one writing sweep produce all the ordered lists.
+// grid = (kSelCluster, 2 lists x items, groups of up to kSelMaxC vertical-slash candidates); the kSelCluster blocks of
+// a thread-block cluster share one list: block r owns the r-th contiguous eighth of the domain.  list 0: vertical
+// columns over [0, q1); list 1: slash offsets over [1, q1) plus offset 0.  A cluster serves every budget of its group
+// in the same passes over the keys: per radix digit every block histograms its own eighth into shared memory, the
+// blocks read each other's histograms through distributed shared memory (integer counts: the sum does not depend on the
+// order) and each one locates the k-th entry itself; one counting sweep plus one writing sweep produce the ordered
+// lists, the position of a block's first entry being the number of entries the lower-ranked blocks select.
+constexpr int kSelCluster = 8;
 constexpr int kSelThreads = 1024;
 constexpr int kDigitBits = 13;
 constexpr int kBins = 1 << kDigitBits;
-constexpr int kSelMaxC = 2;       // budgets served by one block: two keeps 2 x items x 2 blocks in flight and halves the key passes
+constexpr int kSelMaxC = 2;       // budgets served by one cluster: the two histograms are 64 KB of shared memory per block
 constexpr int kSelBatch = 8;      // independent key loads in flight per thread
 
-__global__ void __launch_bounds__(kSelThreads)
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
 rs_vs_select_kernel(IdxParams P) {
   extern __shared__ unsigned int sel_hist[];             // [unique prefixes <= kSelMaxC][kBins]
   __shared__ unsigned int wsum[32];
   __shared__ u64 sh_prefix[kSelMaxC];
   __shared__ unsigned int sh_k[kSelMaxC];
   __shared__ unsigned int w_gt[kSelMaxC][32], w_eq[kSelMaxC][32];
-  const int list = blockIdx.x, item = blockIdx.y;
-  // the vertical-slash candidates this block serves
+  __shared__ unsigned int cta_tot[2 * kSelMaxC];         // this block's entries above / equal to each threshold
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = (int)cluster.block_rank();
+  const int list = blockIdx.y & 1, item = blockIdx.y >> 1;
+  // the vertical-slash candidates this cluster serves
   int cand_id[kSelMaxC] = {}, slot_id[kSelMaxC] = {}, kk[kSelMaxC] = {};
   int nC = 0;
   {
@@ -130,7 +163,7 @@ rs_vs_select_kernel(IdxParams P) {
       ++seen;
     }
   }
-  if (nC == 0) return;
+  if (nC == 0) return;                                   // the same for every block of the cluster
   const int s = item / P.Hq;
   const int q1 = P.seg_bounds[s + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -145,6 +178,12 @@ rs_vs_select_kernel(IdxParams P) {
     kk[c] = k;
   }
   const int cap = (list == 0) ? P.out.kv_cap : P.out.ks_cap;
+  // this block's part of the domain: [c_lo, c_hi)
+  const int c_len = (((n_dom + kSelCluster - 1) / kSelCluster) + 31) / 32 * 32;
+  const int c_lo = min(n_dom, rank * c_len), c_hi = min(n_dom, c_lo + c_len);
+  const unsigned int* rhist[kSelCluster];
+#pragma unroll
+  for (int r = 0; r < kSelCluster; ++r) rhist[r] = cluster.map_shared_rank(sel_hist, r);
 
   // ---- thresholds: T[c] = key of the k-th entry in "key descending" order, k_eq[c] = how many of its ties are taken
   if (tid < nC) { sh_prefix[tid] = 0; sh_k[tid] = (unsigned)kk[tid]; }
@@ -166,13 +205,13 @@ rs_vs_select_kernel(IdxParams P) {
     for (int i = tid; i < n_hist * kBins; i += kSelThreads) sel_hist[i] = 0;
     __syncthreads();
     // eight independent loads per thread are in flight before any is used: the sweep is latency-bound otherwise
-    for (int base = 0; base < n_dom; base += kSelThreads * kSelBatch) {
+    for (int base = c_lo; base < c_hi; base += kSelThreads * kSelBatch) {
       u64 keyb[kSelBatch];
       bool inb[kSelBatch];
 #pragma unroll
       for (int u = 0; u < kSelBatch; ++u) {
         const int j = base + u * kSelThreads + tid;
-        inb[u] = j < n_dom;
+        inb[u] = j < c_hi;
         keyb[u] = inb[u] ? keys[first + j] : 0ull;
       }
 #pragma unroll
@@ -191,15 +230,24 @@ rs_vs_select_kernel(IdxParams P) {
         }
       }
     }
-    __syncthreads();
-    // per candidate: locate the bin that holds its k-th entry (each thread owns 8 consecutive bins, highest first)
+    cluster.sync();                                      // every block's histogram of this digit is complete
+    // per candidate: locate the bin that holds its k-th entry (each thread owns 8 consecutive bins, highest first);
+    // the counts of a bin are summed over the blocks of the cluster
     _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
-      if (kk[c] == 0) continue;                          // uniform over the block
-      const unsigned int* hist = sel_hist + hsel[c] * kBins;
+      if (kk[c] == 0) continue;                          // uniform over the cluster
       const int b0 = kBins - 8 * (tid + 1);
       unsigned int loc[8], lsum = 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { loc[i] = hist[b0 + i]; lsum += loc[i]; }
+      for (int i = 0; i < 8; ++i) loc[i] = 0;
+#pragma unroll
+      for (int r = 0; r < kSelCluster; ++r) {
+        const uint4* src = reinterpret_cast<const uint4*>(rhist[r] + hsel[c] * kBins + b0);
+        const uint4 lo4 = src[0], hi4 = src[1];
+        loc[0] += lo4.x; loc[1] += lo4.y; loc[2] += lo4.z; loc[3] += lo4.w;
+        loc[4] += hi4.x; loc[5] += hi4.y; loc[6] += hi4.z; loc[7] += hi4.w;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) lsum += loc[i];
       unsigned int incl = lsum;                          // inclusive scan over threads (thread 0 owns the top bins)
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
@@ -226,6 +274,7 @@ rs_vs_select_kernel(IdxParams P) {
       }
       __syncthreads();
     }
+    cluster.sync();                                      // nobody reads this digit's histograms any more
   }
   u64 T[kSelMaxC];
   unsigned int k_eq[kSelMaxC];
@@ -234,9 +283,9 @@ rs_vs_select_kernel(IdxParams P) {
     k_eq[c] = (kk[c] > 0) ? sh_k[c] : 0u;
   }
 
-  // ---- ordered compaction: warp w walks the contiguous range [w * chunk, (w + 1) * chunk)
-  const int chunk = (((n_dom + 31) / 32) + 31) / 32 * 32;
-  const int lo = warp * chunk, hi = min(n_dom, lo + chunk);
+  // ---- ordered compaction: warp w of block r walks the contiguous range [c_lo + w * chunk, c_lo + (w + 1) * chunk)
+  const int chunk = (((c_hi - c_lo + 31) / 32) + 31) / 32 * 32;
+  const int lo = min(c_hi, c_lo + warp * chunk), hi = min(c_hi, lo + chunk);
   unsigned int gt[kSelMaxC], eq[kSelMaxC];
   _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) { gt[c] = 0; eq[c] = 0; }
   for (int base = lo; base < hi; base += 32 * kSelBatch) {
@@ -259,9 +308,20 @@ rs_vs_select_kernel(IdxParams P) {
   if (lane == 0)
     _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) { w_gt[c][warp] = gt[c]; w_eq[c][warp] = eq[c]; }
   __syncthreads();
+  if (tid < 2 * kSelMaxC) {
+    const int c = tid >> 1;
+    unsigned int tot = 0;
+    if (c < nC) for (int w = 0; w < 32; ++w) tot += (tid & 1) ? w_eq[c][w] : w_gt[c][w];
+    cta_tot[tid] = tot;
+  }
+  cluster.sync();                                        // every block's totals are published
   unsigned int pos[kSelMaxC], eq_run[kSelMaxC];
   _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
     unsigned int gt_before = 0, eq_before = 0;
+    for (int r = 0; r < rank; ++r) {
+      const unsigned int* rt = cluster.map_shared_rank(cta_tot, r);
+      gt_before += rt[2 * c]; eq_before += rt[2 * c + 1];
+    }
     for (int w = 0; w < warp; ++w) { gt_before += w_gt[c][w]; eq_before += w_eq[c][w]; }
     pos[c] = gt_before + min(k_eq[c], eq_before) + (list == 1 ? 1u : 0u);
     eq_run[c] = eq_before;
@@ -295,7 +355,7 @@ rs_vs_select_kernel(IdxParams P) {
       }
     }
   }
-  if (tid == 0) {
+  if (tid == 0 && rank == 0) {
     _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
       if (list == 1) {
         P.out.vs_offs[(size_t)slot_id[c] * P.out.ks_cap] = 0;
@@ -305,6 +365,7 @@ rs_vs_select_kernel(IdxParams P) {
       }
     }
   }
+  cluster.sync();                                        // no block leaves while its totals may still be read
 }
 
 // ------------------------------------------------------------------------------------------ pair counts (closed forms)
@@ -325,7 +386,8 @@ __device__ __forceinline__ u64 pairs_block_sparse(int qb_lo, int qb_hi, int k_b)
 }
 
 // ------------------------------------------------------------------------------------------ vertical-slash: D, coverage, pairs
-__global__ void __launch_bounds__(256)
+constexpr int kFinishThreads = 512;
+__global__ void __launch_bounds__(kFinishThreads)
 rs_vs_finish_kernel(IdxParams P) {
   __shared__ uint32_t dbits[128];
   __shared__ int wpre[129];
@@ -356,10 +418,13 @@ rs_vs_finish_kernel(IdxParams P) {
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      if (ob[u] < 0) continue;
-      const int d0 = ob[u] >> 6, d1 = (ob[u] + 63) >> 6;
-      if (d0 < nbs) atomicOr(&dbits[d0 >> 5], 1u << (d0 & 31));
-      if (d1 < nbs) atomicOr(&dbits[d1 >> 5], 1u << (d1 & 31));
+      // offsets are ascending, so the lanes of a warp see runs of equal block diagonals: only the first lane of a run
+      // touches the bitmap (32 lanes hammering one shared-memory word would serialise)
+      const int d0 = ob[u] < 0 ? -1 : ob[u] >> 6, d1 = ob[u] < 0 ? -1 : (ob[u] + 63) >> 6;
+      const int p0 = __shfl_up_sync(0xffffffffu, d0, 1), p1 = __shfl_up_sync(0xffffffffu, d1, 1);
+      const int lane = tid & 31;
+      if (d0 >= 0 && d0 < nbs && (lane == 0 || p0 != d0)) atomicOr(&dbits[d0 >> 5], 1u << (d0 & 31));
+      if (d1 >= 0 && d1 < nbs && d1 != d0 && (lane == 0 || p1 != d1)) atomicOr(&dbits[d1 >> 5], 1u << (d1 & 31));
     }
   }
   __syncthreads();
@@ -438,23 +503,22 @@ rs_vs_finish_kernel(IdxParams P) {
   }
 #pragma unroll
   for (int g = 0; g < RS_PROBE_GROUPS; ++g) if (part[g]) atomicAdd(&cov[g], part[g]);
+  if (tid < 128) {
+    // block diagonals: delta >= 1 is used by every query block qb >= delta of the segment, delta 0 by all
+    uint32_t bits = dbits[tid];
+    while (bits) {
+      const int d = tid * 32 + __ffs(bits) - 1;
+      bits &= bits - 1;
+      if (d == 0) vp += (u64)(nbs - qb_lo) * 2080ull;
+      else if (nbs > max(qb_lo, d)) vp += (u64)(nbs - max(qb_lo, d)) * 4096ull;
+    }
+  }
   if (vp) atomicAdd(&extra_pairs, vp);
   __syncthreads();
   if (tid == 0) {
-    u64 total = extra_pairs;
-    // block diagonals: delta >= 1 is used by every query block qb >= delta of the segment, delta 0 by all
-    for (int w = 0; w < 128; ++w) {
-      uint32_t bits = dbits[w];
-      while (bits) {
-        const int d = w * 32 + __ffs(bits) - 1;
-        bits &= bits - 1;
-        if (d == 0) total += (u64)(nbs - qb_lo) * 2080ull;
-        else if (nbs > max(qb_lo, d)) total += (u64)(nbs - max(qb_lo, d)) * 4096ull;
-      }
-    }
     rs_cand_stats* st = P.stats + (size_t)item * P.n_cand + c;
     for (int g = 0; g < RS_PROBE_GROUPS; ++g) st->cov_fx[g] = cov[g];
-    st->pairs = total;
+    st->pairs = extra_pairs;
   }
 }
 
@@ -621,10 +685,11 @@ rs_bs_eval_kernel(IdxParams P) {
   __shared__ u64 cov[RS_PROBE_GROUPS];
   const int item = blockIdx.x;
   if (P.stats == nullptr && P.choice != nullptr) return;    // materialise mode without stats: rows are built elsewhere
-  bool any = false;
-  for (int c = 0; c < P.n_cand; ++c)
-    any |= P.lib[c].pattern == RS_BLOCK_SPARSE && (P.choice == nullptr || P.choice[item] == c);
-  if (!any) return;
+  // blockIdx.y-th block-sparse candidate of the library
+  int my_c = -1;
+  for (int c = 0, seen = 0; c < P.n_cand; ++c)
+    if (P.lib[c].pattern == RS_BLOCK_SPARSE && seen++ == (int)blockIdx.y) my_c = c;
+  if (my_c < 0 || (P.choice != nullptr && P.choice[item] != my_c)) return;
   const int s = item / P.Hq;
   const int q0 = P.seg_bounds[s], q1 = P.seg_bounds[s + 1];
   const int qb = (q1 >> 6) - 1;
@@ -637,10 +702,9 @@ rs_bs_eval_kernel(IdxParams P) {
     for (int kb = tid; kb < qb; kb += 256) score[kb] = row[kb];
   }
   __syncthreads();
-  for (int c = 0; c < P.n_cand; ++c) {
+  {
+    const int c = my_c;
     const rs_candidate cand = P.lib[c];
-    if (cand.pattern != RS_BLOCK_SPARSE) continue;
-    if (P.choice != nullptr && P.choice[item] != c) continue;
     const int slot = (P.choice != nullptr) ? item : item * P.n_cand + c;
     if (tid < RS_PROBE_GROUPS) cov[tid] = 0;
     __syncthreads();
@@ -1080,7 +1144,8 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   P.scale = (float)(1.0 / sqrt((double)RS_HEAD_DIM));
 
   const int n_jobs = n_items * n_cand;
-  if (stats != nullptr) {
+  const bool fuse_vblk = stats != nullptr && any_vs;     // the ranking-key kernel then also writes the block sums
+  if (stats != nullptr && !fuse_vblk) {
     const long long warps = (long long)n_items * RS_PROBE_GROUPS * nb;
     rs_vblk_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, stream>>>(P);
   }
@@ -1089,8 +1154,8 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   // statistics run on the side stream.
   // launch shape of the select kernel; its attribute is set before the fork so that no error path sits between the
   // fork and the join below
-  int n_vs = 0;
-  for (int c = 0; c < n_cand; ++c) n_vs += (lib[c].pattern == RS_VERTICAL_SLASH);
+  int n_vs = 0, n_bs = 0;
+  for (int c = 0; c < n_cand; ++c) { n_vs += (lib[c].pattern == RS_VERTICAL_SLASH); n_bs += (lib[c].pattern == RS_BLOCK_SPARSE); }
   const int sel_groups = choice ? 1 : (n_vs + kSelMaxC - 1) / kSelMaxC;
   const size_t sel_smem = (size_t)(choice ? 1 : kSelMaxC) * kBins * sizeof(unsigned int);
   static rs_smem_attr sel_attr;
@@ -1098,21 +1163,22 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
     return RS_ERR_CUDA;
   const bool two_chains = any_vs && !skip_vs && (any_bs || stats != nullptr);
   cudaStream_t side = stream;
+  // the ranking keys (and with them the block sums both chains read) come before the fork
+  if (any_vs && !skip_vs) rs_vs_keys_kernel<<<dim3((P.n + 255) / 256, 2 * n_items), 256, 0, stream>>>(P, fuse_vblk ? 1 : 0);
   if (two_chains) {
     rc = rs_side_fork(stream, &side);
     if (rc != RS_OK) return rc;
   }
   if (any_vs && !skip_vs) {
-    rs_vs_keys_kernel<<<dim3((P.n + 255) / 256, 2 * n_items), 256, 0, stream>>>(P);
-    rs_vs_select_kernel<<<dim3(2, n_items, sel_groups), kSelThreads, sel_smem, stream>>>(P);
-    rs_vs_finish_kernel<<<n_jobs, 256, 0, stream>>>(P);
+    rs_vs_select_kernel<<<dim3(kSelCluster, 2 * n_items, sel_groups), kSelThreads, sel_smem, stream>>>(P);
+    rs_vs_finish_kernel<<<n_jobs, kFinishThreads, 0, stream>>>(P);
   }
   if (stats != nullptr) rs_simple_stats_kernel<<<n_jobs, 256, 0, side>>>(P);
   if (any_bs) {
     if ((choice == nullptr || stats != nullptr) && bscore == nullptr)
       rs_bs_eval_scores_kernel<<<dim3((nb + 255) / 256, n_items), 256, 0, side>>>(P);
     if (choice == nullptr || stats != nullptr)
-      rs_bs_eval_kernel<<<n_items, 256, (size_t)nb * sizeof(float), side>>>(P);
+      rs_bs_eval_kernel<<<dim3(n_items, n_bs), 256, (size_t)nb * sizeof(float), side>>>(P);
     if (choice != nullptr) {
       if (bscore == nullptr) {
         const int nt = (nb + 63) / 64;
