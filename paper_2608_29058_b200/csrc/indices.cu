@@ -130,19 +130,24 @@ rs_vs_keys_kernel(IdxParams P, int fuse_vblk) {
 // order) and each one locates the k-th entry itself; one counting sweep plus one writing sweep produce the ordered
 // lists, the position of a block's first entry being the number of entries the lower-ranked blocks select.
 constexpr int kSelCluster = 8;
-constexpr int kSelThreads = 1024;
-constexpr int kDigitBits = 13;
+constexpr int kSelThreads = 256;  // small blocks: all clusters of a layer (2 lists x 32 items x 8 blocks) are resident at once
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kDigitBits = 11;    // four digits cover 44 bits; ranking keys stay below 2^39
+constexpr int kSelPasses = 4;
 constexpr int kBins = 1 << kDigitBits;
-constexpr int kSelMaxC = 2;       // budgets served by one cluster: the two histograms are 64 KB of shared memory per block
-constexpr int kSelBatch = 8;      // independent key loads in flight per thread
+constexpr int kSlice = kBins / kSelCluster;      // bins of a histogram that one block of the cluster scans
+static_assert(kSlice == kSelThreads, "one bin per thread");
+constexpr int kSelMaxC = 4;       // budgets served by one cluster: four histograms are 32 KB of shared memory per block
+constexpr int kSelBatch = 4;      // independent key loads in flight per thread
 
-__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads)
+__global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads, 4)
 rs_vs_select_kernel(IdxParams P) {
   extern __shared__ unsigned int sel_hist[];             // [unique prefixes <= kSelMaxC][kBins]
-  __shared__ unsigned int wsum[32];
-  __shared__ u64 sh_prefix[kSelMaxC];
-  __shared__ unsigned int sh_k[kSelMaxC];
-  __shared__ unsigned int w_gt[kSelMaxC][32], w_eq[kSelMaxC][32];
+  __shared__ unsigned int wsum[kSelMaxC * kSelWarps];
+  __shared__ u64 sh_prefix[kSelMaxC], nx_prefix[kSelMaxC];
+  __shared__ unsigned int sh_k[kSelMaxC], nx_k[kSelMaxC];
+  __shared__ unsigned int slice_tot[kSelMaxC];           // entries in this block's slice of the bins
+  __shared__ unsigned int w_gt[kSelMaxC][kSelWarps], w_eq[kSelMaxC][kSelWarps];
   __shared__ unsigned int cta_tot[2 * kSelMaxC];         // this block's entries above / equal to each threshold
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = (int)cluster.block_rank();
@@ -188,7 +193,7 @@ rs_vs_select_kernel(IdxParams P) {
   // ---- thresholds: T[c] = key of the k-th entry in "key descending" order, k_eq[c] = how many of its ties are taken
   if (tid < nC) { sh_prefix[tid] = 0; sh_k[tid] = (unsigned)kk[tid]; }
   __syncthreads();
-  for (int pass = 2; pass >= 0; --pass) {
+  for (int pass = kSelPasses - 1; pass >= 0; --pass) {
     const int shift = pass * kDigitBits;
     // candidates with the same prefix share a histogram: hsel[c] = index of the first candidate with that prefix
     u64 pre[kSelMaxC];
@@ -231,50 +236,51 @@ rs_vs_select_kernel(IdxParams P) {
       }
     }
     cluster.sync();                                      // every block's histogram of this digit is complete
-    // per candidate: locate the bin that holds its k-th entry (each thread owns 8 consecutive bins, highest first);
-    // the counts of a bin are summed over the blocks of the cluster
-    _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
-      if (kk[c] == 0) continue;                          // uniform over the cluster
-      const int b0 = kBins - 8 * (tid + 1);
-      unsigned int loc[8], lsum = 0;
+    // Block r owns the bins [1024 r, 1024 r + 1024) of every histogram: thread t sums bin 1024 r + 1023 - t over the
+    // blocks of the cluster (counts: the order does not matter) and the block scans its slice from the top.
+    unsigned int v[kSelMaxC], incl[kSelMaxC];
+    _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) {
+      v[c] = 0; incl[c] = 0;
+      if (c >= nC || kk[c] == 0) continue;               // uniform over the cluster
+      const int bin = kSlice * rank + (kSlice - 1 - tid);
+      unsigned int sum = 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) loc[i] = 0;
-#pragma unroll
-      for (int r = 0; r < kSelCluster; ++r) {
-        const uint4* src = reinterpret_cast<const uint4*>(rhist[r] + hsel[c] * kBins + b0);
-        const uint4 lo4 = src[0], hi4 = src[1];
-        loc[0] += lo4.x; loc[1] += lo4.y; loc[2] += lo4.z; loc[3] += lo4.w;
-        loc[4] += hi4.x; loc[5] += hi4.y; loc[6] += hi4.z; loc[7] += hi4.w;
-      }
-#pragma unroll
-      for (int i = 0; i < 8; ++i) lsum += loc[i];
-      unsigned int incl = lsum;                          // inclusive scan over threads (thread 0 owns the top bins)
+      for (int r = 0; r < kSelCluster; ++r) sum += rhist[r][hsel[c] * kBins + bin];
+      v[c] = sum;
+      unsigned int in = sum;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
-        const unsigned int t = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += t;
+        const unsigned int t = __shfl_up_sync(0xffffffffu, in, off);
+        if (lane >= off) in += t;
       }
-      if (lane == 31) wsum[warp] = incl;
-      __syncthreads();
+      if (lane == 31) wsum[c * kSelWarps + warp] = in;
+      incl[c] = in;
+    }
+    __syncthreads();
+    _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) {
+      if (c >= nC || kk[c] == 0) continue;
       unsigned int before = 0;
-      for (int w = 0; w < warp; ++w) before += wsum[w];
-      const unsigned int above = before + incl - lsum;   // entries in bins above this thread's bins
+      for (int w = 0; w < warp; ++w) before += wsum[c * kSelWarps + w];
+      incl[c] += before;
+      if (tid == kSelThreads - 1) slice_tot[c] = incl[c];
+    }
+    cluster.sync();                                      // every block's slice totals are published
+    _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) {
+      if (c >= nC || kk[c] == 0) continue;
+      unsigned int above = incl[c] - v[c];               // entries in higher bins: of this slice, and of the higher slices
+      for (int r = rank + 1; r < kSelCluster; ++r) above += cluster.map_shared_rank(slice_tot, r)[c];
       const unsigned int kq = sh_k[c];
-      __syncthreads();
-      if (above < kq && kq <= above + lsum) {
-        unsigned int acc = above;
-        for (int i = 7; i >= 0; --i) {
-          if (acc + loc[i] >= kq) {
-            sh_prefix[c] = (pre[c] << kDigitBits) | (u64)(b0 + i);
-            sh_k[c] = kq - acc;
-            break;
-          }
-          acc += loc[i];
+      if (above < kq && kq <= above + v[c]) {            // exactly one thread of the cluster: its bin holds the k-th entry
+        const u64 new_prefix = (pre[c] << kDigitBits) | (u64)(kSlice * rank + (kSlice - 1 - tid));
+        for (int r = 0; r < kSelCluster; ++r) {
+          cluster.map_shared_rank(nx_prefix, r)[c] = new_prefix;
+          cluster.map_shared_rank(nx_k, r)[c] = kq - above;
         }
       }
-      __syncthreads();
     }
-    cluster.sync();                                      // nobody reads this digit's histograms any more
+    cluster.sync();                                      // the result has reached every block; this digit's histograms are done
+    if (tid < nC && kk[tid] > 0) { sh_prefix[tid] = nx_prefix[tid]; sh_k[tid] = nx_k[tid]; }
+    __syncthreads();
   }
   u64 T[kSelMaxC];
   unsigned int k_eq[kSelMaxC];
@@ -284,7 +290,7 @@ rs_vs_select_kernel(IdxParams P) {
   }
 
   // ---- ordered compaction: warp w of block r walks the contiguous range [c_lo + w * chunk, c_lo + (w + 1) * chunk)
-  const int chunk = (((c_hi - c_lo + 31) / 32) + 31) / 32 * 32;
+  const int chunk = (((c_hi - c_lo + kSelWarps - 1) / kSelWarps) + 31) / 32 * 32;
   const int lo = min(c_hi, c_lo + warp * chunk), hi = min(c_hi, lo + chunk);
   unsigned int gt[kSelMaxC], eq[kSelMaxC];
   _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) { gt[c] = 0; eq[c] = 0; }
@@ -311,7 +317,7 @@ rs_vs_select_kernel(IdxParams P) {
   if (tid < 2 * kSelMaxC) {
     const int c = tid >> 1;
     unsigned int tot = 0;
-    if (c < nC) for (int w = 0; w < 32; ++w) tot += (tid & 1) ? w_eq[c][w] : w_gt[c][w];
+    if (c < nC) for (int w = 0; w < kSelWarps; ++w) tot += (tid & 1) ? w_eq[c][w] : w_gt[c][w];
     cta_tot[tid] = tot;
   }
   cluster.sync();                                        // every block's totals are published
