@@ -138,7 +138,7 @@ constexpr int kBins = 1 << kDigitBits;
 constexpr int kSlice = kBins / kSelCluster;      // bins of a histogram that one block of the cluster scans
 static_assert(kSlice == kSelThreads, "one bin per thread");
 constexpr int kSelMaxC = 4;       // budgets served by one cluster: four histograms are 32 KB of shared memory per block
-constexpr int kSelBatch = 4;      // independent key loads in flight per thread
+constexpr int kSelBatch = 8;      // independent key loads in flight per thread
 
 __global__ void __cluster_dims__(kSelCluster, 1, 1) __launch_bounds__(kSelThreads, 4)
 rs_vs_select_kernel(IdxParams P) {
@@ -208,6 +208,13 @@ rs_vs_select_kernel(IdxParams P) {
       if (hsel[c] < 0) hsel[c] = n_hist++;
     }
     for (int i = tid; i < n_hist * kBins; i += kSelThreads) sel_hist[i] = 0;
+    // the distinct prefixes, in histogram order: a key matches at most one of them (what lies above this digit fits
+    // 32 bits: keys stay below 2^39 and every prefix has lost at least 11 bits)
+    uint32_t upre[kSelMaxC];
+    _Pragma("unroll") for (int u = 0; u < kSelMaxC; ++u) {
+      upre[u] = 0xffffffffu;
+      _Pragma("unroll") for (int c = kSelMaxC - 1; c >= 0; --c) if (c < nC && hsel[c] == u) upre[u] = (uint32_t)pre[c];
+    }
     __syncthreads();
     // eight independent loads per thread are in flight before any is used: the sweep is latency-bound otherwise
     for (int base = c_lo; base < c_hi; base += kSelThreads * kSelBatch) {
@@ -221,18 +228,15 @@ rs_vs_select_kernel(IdxParams P) {
       }
 #pragma unroll
       for (int u = 0; u < kSelBatch; ++u) {
-        const u64 hi = keyb[u] >> (shift + kDigitBits);
-        const unsigned int dig = (unsigned)((keyb[u] >> shift) & (kBins - 1));
-        int done_hist = -1;                              // histograms are numbered in candidate order
-        _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
-          if (hsel[c] <= done_hist) continue;            // shared with an earlier candidate (or k = 0: hsel = -1)
-          done_hist = hsel[c];
-          unsigned int digit = (inb[u] && hi == pre[c]) ? dig : 0xffffffffu;
-          if (__ballot_sync(0xffffffffu, digit != 0xffffffffu) == 0u) continue;   // nobody in this warp is in the bin
-          const unsigned int peers = __match_any_sync(0xffffffffu, digit);
-          if (digit != 0xffffffffu && lane == (__ffs(peers) - 1))
-            atomicAdd(&sel_hist[hsel[c] * kBins + digit], (unsigned)__popc(peers));
-        }
+        const uint32_t hi = (uint32_t)(keyb[u] >> (shift + kDigitBits));
+        const uint32_t dig = (uint32_t)(keyb[u] >> shift) & (kBins - 1);
+        unsigned int slot = 0xffffffffu;                 // histogram * kBins + digit, or none
+        _Pragma("unroll") for (int h = 0; h < kSelMaxC; ++h)
+          if (hi == upre[h]) slot = (unsigned)h * kBins + dig;
+        if (!inb[u]) slot = 0xffffffffu;
+        if (__ballot_sync(0xffffffffu, slot != 0xffffffffu) == 0u) continue;   // nobody in this warp matches a prefix
+        const unsigned int peers = __match_any_sync(0xffffffffu, slot);
+        if (slot != 0xffffffffu && lane == (__ffs(peers) - 1)) atomicAdd(&sel_hist[slot], (unsigned)__popc(peers));
       }
     }
     cluster.sync();                                      // every block's histogram of this digit is complete
@@ -305,11 +309,17 @@ rs_vs_select_kernel(IdxParams P) {
     }
 #pragma unroll
     for (int u = 0; u < kSelBatch; ++u) {
-      _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
-        gt[c] += __popc(__ballot_sync(0xffffffffu, inb[u] && keyb[u] > T[c]));
-        eq[c] += __popc(__ballot_sync(0xffffffffu, inb[u] && keyb[u] == T[c]));
+      if (inb[u]) {                                      // per-lane counts; the warp sums them once, after the sweep
+        _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+          gt[c] += (keyb[u] > T[c]) ? 1u : 0u;
+          eq[c] += (keyb[u] == T[c]) ? 1u : 0u;
+        }
       }
     }
+  }
+  _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
+    gt[c] = __reduce_add_sync(0xffffffffu, gt[c]);
+    eq[c] = __reduce_add_sync(0xffffffffu, eq[c]);
   }
   if (lane == 0)
     _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) { w_gt[c][warp] = gt[c]; w_eq[c][warp] = eq[c]; }
@@ -346,9 +356,13 @@ rs_vs_select_kernel(IdxParams P) {
     for (int u = 0; u < kSelBatch; ++u) {
       const int j = base + u * 32 + lane;
       _Pragma("unroll") for (int c = 0; c < kSelMaxC; ++c) if (c < nC) {
-        const bool is_eq = inb[u] && keyb[u] == T[c];
-        const unsigned int beq = __ballot_sync(0xffffffffu, is_eq);
-        const bool take = inb[u] && (keyb[u] > T[c] || (is_eq && eq_run[c] + __popc(beq & lt_mask) < k_eq[c]));
+        bool take = inb[u] && keyb[u] > T[c];
+        if (__any_sync(0xffffffffu, inb[u] && keyb[u] == T[c])) {   // ties with the threshold are rare: taken in index order
+          const bool is_eq = inb[u] && keyb[u] == T[c];
+          const unsigned int beq = __ballot_sync(0xffffffffu, is_eq);
+          take = take || (is_eq && eq_run[c] + __popc(beq & lt_mask) < k_eq[c]);
+          eq_run[c] += __popc(beq);
+        }
         const unsigned int bt = __ballot_sync(0xffffffffu, take);
         if (take) {
           const unsigned int p = pos[c] + __popc(bt & lt_mask);
@@ -357,7 +371,6 @@ rs_vs_select_kernel(IdxParams P) {
           if ((int)p < cap) out[p] = first + j;
         }
         pos[c] += __popc(bt);
-        eq_run[c] += __popc(beq);
       }
     }
   }
