@@ -27,5 +27,8 @@ Parts and what pins them (tests/test_oracle_*.py):
   calibration.*                  Section 3.5, predictor e of Eq. 4. Pinned: isotonic fit == scikit-learn's, quantile by
                                                                   counting, monotonicity.  The feature set is this build's
                                                                   reading: "parity unpinned".
+  projection.qkv_project         the producer of Q, K, V (Section 3.4: routing beside the projection kernels).
+                                                                  Pinned: torch linear + rotate-half, rotation special cases,
+                                                                  distance-only dot products, brute-force side outputs.
 """
-from . import attention, calibration, certificate, patterns, probe, routing  # noqa: F401
+from . import attention, calibration, certificate, patterns, probe, projection, routing  # noqa: F401
