@@ -337,6 +337,31 @@ int rs_routed_prefill_layer(const rs_problem* p, const void* Q, const void* K, c
                             const int64_t* cost, const rs_layer_buffers* b, void* ws, size_t ws_bytes,
                             int32_t* status, void* stream);
 
+/* The producer of Q, K, V with the probe's streaming reductions fused into it (Section 3.4: the routing work "runs on
+ * the CPU concurrently with projection kernels or as a fused GPU reduction").  One layer's QKV projection
+ *   Y = X W^T,   X [n_tokens][d_model] bf16,   W [(n_q_heads + 2 n_kv_heads) * 128][d_model] bf16, rows ordered
+ *   Q head 0.., K head 0.., V head 0..  (each head 128 consecutive rows)
+ * on the tensor cores, the rotary embedding of Q and K in the "rotate half" pairing (dimension i with i + 64):
+ *   out[i] = y[i] cos[t][i] - y[i + 64] sin[t][i],  out[i + 64] = y[i + 64] cos[t][i] + y[i] sin[t][i],
+ * rope_cos / rope_sin device fp32 [n_tokens][64]; V is not rotated.  Q, K, V are written as bf16 [heads][n_tokens][128]
+ * (the layout every other call takes), rounded once to nearest even from the fp32 accumulator.
+ * Side outputs (each may be NULL), formed from the ROUNDED values so that they equal what rs_probe would compute
+ * from the tensors just written (up to the order of fp32 additions):
+ *   qpool [n_q_heads][n_tokens/64][128], kpool [n_kv_heads][n_tokens/64][128]   64-row means (Section 3.1: "pooled
+ *         queries and keys score coarse blocks")
+ *   vbmax [n_kv_heads][n_tokens/64]   max over the block's rows of ||v||_2^2 (Eq. 5 needs V_max = max_j ||v_j||;
+ *         rs_value_norm_max turns it into rs_probe's vmax)
+ * A caller that has them passes NULL for qpool, kpool and vmax to rs_probe, which then skips its own pooling of K and
+ * its pass over V.  n_tokens a multiple of 64, d_model a multiple of 64, n_q_heads and n_kv_heads even.
+ * Errors as for the other calls; nothing is allocated; the kernel's waits are bounded (RS_ERR_TIMEOUT in status). */
+int rs_qkv_rope_project(int n_tokens, int d_model, int n_q_heads, int n_kv_heads, const void* X, const void* W,
+                        const float* rope_cos, const float* rope_sin, void* Q, void* K, void* V,
+                        float* qpool, float* kpool, float* vbmax, int32_t* status, void* stream);
+
+/* vmax [n_seg][n_kv_heads] of rs_probe (V_max of Eq. 5 per segment: sqrt of the largest ||v_j||^2 over the keys below
+ * the segment's end) from the block maxima vbmax [n_kv_heads][n_keys/64] written by rs_qkv_rope_project. */
+int rs_value_norm_max(const rs_problem* p, const float* vbmax, float* vmax, int32_t* status, void* stream);
+
 /* Self test of the bounded device-side wait every kernel of this library uses (no passage of the paper: the waits
  * exist because the kernels synchronise TMA, tensor-core and softmax roles through mbarriers).  Launches one small
  * kernel that waits on a barrier nothing arrives on, with a limit of poll_limit (1 .. 2^20) polls; the wait gives up,

@@ -58,7 +58,8 @@ class rs_layer_buffers(C.Structure):
 EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "rs_build_indices", "rs_route",
            "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate",
            "rs_selftest_wait_timeout", "rs_probe_pooled", "rs_probe_pooled_scratch_floats", "rs_regressor_eval",
-           "rs_output_error", "rs_mixture_coverage", "rs_pool_queries", "rs_routed_prefill_layer"]
+           "rs_output_error", "rs_mixture_coverage", "rs_pool_queries", "rs_routed_prefill_layer",
+           "rs_qkv_rope_project", "rs_value_norm_max"]
 
 
 def lib_path() -> str:
@@ -301,6 +302,18 @@ def rs_output_error(Oa, Ob, err, norm_a, status):
     o_dtype = 1 if Oa.dtype == torch.float32 else 0
     _check(load().rs_output_error(C.c_longlong(n_rows), _ptr(Oa), _ptr(Ob), o_dtype, _ptr(err), _ptr(norm_a),
                                   _ptr(status), _stream()), "rs_output_error")
+
+
+def rs_qkv_rope_project(X, W, rope_cos, rope_sin, n_q_heads: int, n_kv_heads: int, Q, K, V, qpool, kpool, vbmax, status):
+    """QKV projection + rotary embedding with the probe's side outputs (pooled Q / K, block maxima of ||v||^2)."""
+    n, dm = int(X.shape[0]), int(X.shape[1])
+    _check(load().rs_qkv_rope_project(n, dm, n_q_heads, n_kv_heads, _ptr(X), _ptr(W), _ptr(rope_cos), _ptr(rope_sin),
+                                      _ptr(Q), _ptr(K), _ptr(V), _ptr(qpool), _ptr(kpool), _ptr(vbmax), _ptr(status),
+                                      _stream()), "rs_qkv_rope_project")
+
+
+def rs_value_norm_max(p: Problem, vbmax, vmax, status):
+    _check(load().rs_value_norm_max(C.byref(p.c), _ptr(vbmax), _ptr(vmax), _ptr(status), _stream()), "rs_value_norm_max")
 
 
 def rs_selftest_wait_timeout(status, poll_limit: int = 2000):
