@@ -235,6 +235,9 @@ def main():
                     help="u of Eq. 4 = disagreement among the recent / uniform / boundary rows of the query mixture (pooled probe)")
     ap.add_argument("--graph", action="store_true",
                     help="also time the layer replayed from a CUDA graph (whole pass captured once; for launch-bound sizes)")
+    ap.add_argument("--from-hidden", action="store_true",
+                    help="the layer pass with its producer in front: QKV projection + rotary embedding (Llama-3.1-8B "
+                         "geometry, seeded weights) with the probe's side outputs fused into its epilogue; --n sets the length")
     ap.add_argument("--sweep", action="store_true", help="config-5 sweep: n x budget x forced-dense cells, JSONL output")
     ap.add_argument("--n", type=int, default=None, help="override the sequence length (smaller profiling case)")
     ap.add_argument("--out-dir", default="bench_out", help="directory for the JSONL files of --sweep and --ablations")
@@ -246,6 +249,8 @@ def main():
     ap.add_argument("--no-dense", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.from_hidden:
+        return from_hidden(args)
     if args.sweep:
         return sweep(args)
     if args.ablations:
@@ -664,6 +669,56 @@ def stack(args):
                         "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "traffic": None},
            "clocks": clocks, "gpu_launches": 23 * args.layers * args.steps}
     print(json.dumps(out))
+    return 0
+
+
+def from_hidden(args):
+    """Projection-fused layer pass (Section 3.4: the probe as a reduction beside the projection kernels).  X and W are
+    seeded Gaussians (no structure is planted, so the router sends most heads to dense); what is measured is the
+    producer itself and what its fused side outputs take off the probe."""
+    import torch
+    import paper_2608_29058_b200 as rs
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    n = args.n or 16384
+    dm, Hq, Hkv = 4096, 32, 8
+    gen = torch.Generator(device=dev).manual_seed(260829058)
+    X = torch.randn((n, dm), generator=gen, device=dev).to(torch.bfloat16)
+    W = (torch.randn(((Hq + 2 * Hkv) * 128, dm), generator=gen, device=dev) / dm ** 0.5).to(torch.bfloat16)
+    inv = 500000.0 ** (-torch.arange(0, 128, 2, device=dev, dtype=torch.float64) / 128)
+    ang = torch.arange(n, device=dev, dtype=torch.float64)[:, None] * inv[None, :]
+    cos, sin = torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()
+    p = rs.Problem(Hq, Hkv, n)
+    layer = rs.RoutedPrefillLayer(p, None, rs.RouteConfig(budget_frac=0.15, cert_max=0.05), device=dev)
+    for _ in range(max(3, args.warmup)):
+        layer.forward_from_hidden(X, W, cos, sin)
+    torch.cuda.synchronize()
+    rs.check_status(layer.status, "warm-up")
+    evs = []
+    for _ in range(args.steps):
+        layer.forward_from_hidden(X, W, cos, sin, record_events=True)
+        evs.append(layer.events_hidden)
+    torch.cuda.synchronize()
+    rs.check_status(layer.status, "timed region")
+    names = ["projection", "probe", "evaluate", "route", "materialise", "attention", "certificate"]
+    st = {nm: float(np.median([e[i].elapsed_time(e[i + 1]) for e in evs])) for i, nm in enumerate(names)}
+    # the same tensors through the ordinary pass (the probe pools by itself): what the fusion takes off the probe
+    Q, K, V = layer._qkv
+    plain = []
+    for _ in range(args.steps):
+        layer.forward(Q, K, V, record_events=True)
+        plain.append(layer.events)
+    torch.cuda.synchronize()
+    probe_plain = float(np.median([e[0].elapsed_time(e[1]) for e in plain]))
+    flops = 2.0 * n * dm * (Hq + 2 * Hkv) * 128
+    peaks = measured_peaks()
+    tf = flops / (st["projection"] * 1e-3) / 1e12
+    print(json.dumps({"metric": "QKV projection + rotary embedding with fused probe side outputs, then the routed layer pass",
+                      "config": {"workload": f"from hidden states: d_model=4096 Hq=32 Hkv=8 d=128 n={n}, seeded Gaussian X and W"},
+                      "stage_ms_median": st, "projection_tflops": tf,
+                      "projection_frac_of_burst_peak": tf / peaks["bf16_tflops"], "peak_source": peaks["source"],
+                      "probe_ms_when_it_pools_itself": probe_plain, "probe_ms_fed_by_projection": st["probe"],
+                      "steps": args.steps, "data": "synthetic", "dtype": "bf16"}))
     return 0
 
 

@@ -364,6 +364,43 @@ class RoutedPrefillLayer:
         self.events = ev
         return self.O
 
+    def forward_from_hidden(self, X, W, rope_cos, rope_sin, forced_dense: Optional[torch.Tensor] = None,
+                            record_events: bool = False) -> torch.Tensor:
+        """The layer pass with its producer in front (Section 3.4: the probe as a reduction fused with the projection
+        kernels): rs_qkv_rope_project writes Q, K, V into buffers owned by the layer together with the pooled queries
+        and keys and the block maxima of the value norms, so rs_probe runs only its two passes over K (no pooling, no
+        stream over V) and no query pooling follows the routing.  X [n, d_model] bf16, W [(Hq + 2 Hkv) * 128, d_model]
+        bf16, rope tables fp32 [n, 64].  Events (record_events): projection, probe, evaluate, route, materialise,
+        attention, certificate."""
+        p = self.p
+        if getattr(self, "_qkv", None) is None:
+            bf = dict(dtype=torch.bfloat16, device=self.O.device)
+            self._qkv = (torch.empty((p.n_q_heads, p.n_keys, 128), **bf), torch.empty((p.n_kv_heads, p.n_keys, 128), **bf),
+                         torch.empty((p.n_kv_heads, p.n_keys, 128), **bf))
+            self._vbmax = torch.empty((p.n_kv_heads, p.n_keys // 64), dtype=torch.float32, device=self.O.device)
+        Q, K, V = self._qkv
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(8)] if record_events else None
+        mark = (lambda i: ev[i].record()) if record_events else (lambda i: None)
+        mark(0)
+        rs.rs_qkv_rope_project(X, W, rope_cos, rope_sin, p.n_q_heads, p.n_kv_heads, Q, K, V, self.qpool, self.kpool,
+                               self._vbmax, self.status)
+        mark(1)
+        rs.rs_probe(p, Q, K, V, self.vert, self.slash, self.lse_probe, None, None, None, None, self.ws, self.status)
+        rs.rs_value_norm_max(p, self._vbmax, self.vmax, self.status)
+        mark(2)
+        self.evaluate_candidates()
+        mark(3)
+        self.route(forced_dense)
+        mark(4)
+        self.materialise(reuse_evaluation=True)
+        mark(5)
+        self.attention(Q, K, V)
+        mark(6)
+        self.certificate()
+        mark(7)
+        self.events_hidden = ev
+        return self.O
+
     def stage_ms(self):
         """Milliseconds per stage of the last forward(record_events=True): probe, evaluate, route, materialise,
         attention, certificate (synchronises)."""

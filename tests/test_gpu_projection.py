@@ -110,3 +110,24 @@ def test_argument_checks():
         rs.rs_qkv_rope_project(torch.zeros((100, 64), device="cuda", dtype=torch.bfloat16), x, x, x, 2, 2, x, x, x, None, None, None, None)
     with pytest.raises(rs.RouteSparseError):
         rs.rs_qkv_rope_project(torch.zeros((128, 64), device="cuda", dtype=torch.bfloat16), x, x, x, 3, 3, x, x, x, None, None, None, None)
+
+
+def test_layer_pass_from_hidden_states_equals_the_pass_on_the_projected_tensors():
+    """RoutedPrefillLayer.forward_from_hidden (projection with fused side outputs, probe without pooling) against the
+    ordinary forward() on the Q, K, V the projection wrote: same routes, bit-identical output."""
+    n, dm, Hq, Hkv = 1088, 256, 4, 2
+    Xb, Wb, cos, sin = _inputs(n, dm, Hq, Hkv, 21)
+    p = rs.Problem(Hq, Hkv, n)
+    lib = [(rs.RS_A_SHAPE, 8, 128), (rs.RS_VERTICAL_SLASH, 32, 48), (rs.RS_BLOCK_SPARSE, 3, 0), (rs.RS_DENSE, 0, 0)]
+    cfg = dict(budget_frac=0.4, cert_max=0.8)
+    a = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(**cfg), out_dtype=torch.float32)
+    Oa = a.forward_from_hidden(_dev_bf16(Xb), _dev_bf16(Wb), torch.from_numpy(cos).cuda(), torch.from_numpy(sin).cuda()).clone()
+    rs.check_status(a.status, "from hidden")
+    Q, K, V = a._qkv
+    b = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(**cfg), out_dtype=torch.float32)
+    b.one_call = False
+    Ob = b.forward(Q, K, V)
+    rs.check_status(b.status, "staged")
+    assert torch.equal(a.choice, b.choice)
+    assert torch.equal(Oa, Ob) and torch.equal(a.lse_sel, b.lse_sel)
+    assert torch.equal(a.stats, b.stats)
