@@ -156,6 +156,29 @@ int rs_probe(const rs_problem* p, const void* Q, const void* K, const void* V,
              float* vert, float* slash, float* lse_probe, float* qpool, float* kpool, float* vmax,
              float* descr, int flags, void* ws, size_t ws_bytes, int32_t* status, void* stream);
 
+/* The same probe on the query mixture of Eq. 3 at key resolution ("a deterministic mixture of recent, uniformly
+ * spaced, and boundary-adjacent positions", Section 3.2): instead of the last 64 rows, four caller-chosen runs of 16
+ * consecutive rows per segment (a diagonal is only visible on consecutive rows, so the mixture is made of runs).
+ *   run_starts  HOST int32 [n_seg][4]: first row of each run; 0 <= start and start + 16 <= segment end
+ *   vert, slash [n_seg][n_q_heads][4][n_keys]: column mass and diagonal mass of run g (group g), fully overwritten;
+ *               slash[..][g][o] = sum over the run's rows i >= o of P[i][i - o]
+ *   lse_probe   [n_q_heads][n_seg][64]: log-sum-exp of the 64 rows in run order
+ * No pooled means, no value norms (rs_probe provides them).  The paper's "Recent queries only" ablation (Table 3) is
+ * rs_probe; with the masses of this call handed to rs_build_indices_ranked the line lists are chosen from the mixture. */
+int rs_probe_runs(const rs_problem* p, const void* Q, const void* K, const int32_t* run_starts,
+                  float* vert, float* slash, float* lse_probe, void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* The query sets I of Eq. 3 ("a deterministic mixture of recent, uniformly spaced, and boundary-adjacent positions";
+ * the paper fixes neither proportions nor spacing, these are this library's choices).  Host functions.
+ * rs_mixture_rows: rows [r_recent + r_uniform + r_boundary] (host, out) = the last r_recent rows of the segment
+ *   [q0, q1), then r_uniform rows at the midpoints of equal strata of what lies between the other two groups, then
+ *   the r_boundary rows right after q0; RS_ERR_UNSUPPORTED_SHAPE when the segment is too short for the groups to be
+ *   disjoint.  This is the row set rs_probe_pooled and rs_mixture_coverage are meant to be given.
+ * rs_mixture_runs: run_starts [4] (host, out) = first rows of the four 16-row runs rs_probe_runs takes: the run right
+ *   after q0, the runs one third and two thirds into the segment (in units of 16 rows), and the last 16 rows. */
+int rs_mixture_rows(int q0, int q1, int r_recent, int r_uniform, int r_boundary, int32_t* rows);
+int rs_mixture_runs(int q0, int q1, int32_t* run_starts);
+
 /* rs_probe flag: fill only the rows of qpool that candidate evaluation reads (the last query block of every segment)
  * and leave the rest to rs_pool_queries once the routes are known; reading all of Q for the pooled means is the
  * largest single stream of the probe (1 GB at 128K) and only heads routed to block-sparse need it. */
@@ -184,6 +207,16 @@ int rs_build_indices(const rs_problem* p, const rs_candidate* lib, int n_cand,
                      const float* bscore, const int32_t* choice,
                      const rs_index_set* out, rs_cand_stats* stats,
                      void* ws, size_t ws_bytes, int32_t* status, void* stream);
+
+/* rs_build_indices with the vertical columns and slash offsets RANKED by another pair of mass arrays (same shapes):
+ * V and S are the top-k of rank_vert / rank_slash (the query mixture of Eq. 3, rs_probe_runs), while coverage, the
+ * uncertainty groups and everything else are still measured on vert / slash (the last 64 rows, which the certificate
+ * audits).  Section 3.2: the probe's mixture of rows decides which lines are worth keeping. */
+int rs_build_indices_ranked(const rs_problem* p, const rs_candidate* lib, int n_cand,
+                            const float* vert, const float* slash, const float* rank_vert, const float* rank_slash,
+                            const float* qpool, const float* kpool, const float* bscore, const int32_t* choice,
+                            const rs_index_set* out, rs_cand_stats* stats,
+                            void* ws, size_t ws_bytes, int32_t* status, void* stream);
 
 /* Risk (Eq. 4), greedy substitution for the budgeted routing problem (Eq. 6-8), fallback walk and forced
  * dense (Section 3.4), solved by one thread block on the device.

@@ -35,9 +35,23 @@ class ProbeResult:
     local_conc: float       # mean over probe rows of the mass with i - j < 1024
 
 
-def probe_rows(Q: np.ndarray, K: np.ndarray, q1: int) -> ProbeResult:
-    """Probe of one head on the segment ending at q1: exact softmax rows q1-64 .. q1-1 over keys [0, q1)."""
-    rows = np.arange(q1 - R_PROBE, q1)
+def mixture_runs(q0: int, q1: int) -> np.ndarray:
+    """First rows of the four 16-row runs of the query mixture at key resolution (Eq. 3: "a deterministic mixture of
+    recent, uniformly spaced, and boundary-adjacent positions"), ascending: the run right after the segment start, two
+    runs one third and two thirds into the segment, and the last 16 rows.  A diagonal is only visible on consecutive
+    rows, so the mixture is made of runs of 16 consecutive rows; the run starts are the uniformly spaced positions.
+    The paper fixes neither the proportions nor the spacing: this is this build's reading."""
+    units = (q1 - q0) // G_ROWS
+    return np.array([q0, q0 + G_ROWS * (units // 3), q0 + G_ROWS * ((2 * units) // 3), q1 - G_ROWS], dtype=np.int64)
+
+
+def probe_rows(Q: np.ndarray, K: np.ndarray, q1: int, starts=None) -> ProbeResult:
+    """Probe of one head on the segment ending at q1: exact softmax rows over the causal keys, reduced per group of 16
+    consecutive rows.  starts: first row of each of the four groups (default: the last 64 rows, q1 - 64 + 16 g)."""
+    if starts is None:
+        starts = [q1 - R_PROBE + G_ROWS * g for g in range(N_GROUPS)]
+    rows = np.concatenate([np.arange(int(s0), int(s0) + G_ROWS) for s0 in starts])
+    assert rows.min() >= 0 and rows.max() < q1
     l = causal_logits(Q, K, rows, q1)
     mx = l.max(axis=1, keepdims=True)
     lse = mx[:, 0] + np.log(np.exp(l - mx).sum(axis=1))

@@ -59,7 +59,8 @@ EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "r
            "rs_sparse_prefill_attn", "rs_dense_prefill_attn", "rs_dense_prefill_attn_noalloc", "rs_certificate",
            "rs_selftest_wait_timeout", "rs_probe_pooled", "rs_probe_pooled_scratch_floats", "rs_regressor_eval",
            "rs_output_error", "rs_mixture_coverage", "rs_pool_queries", "rs_routed_prefill_layer",
-           "rs_qkv_rope_project", "rs_value_norm_max"]
+           "rs_qkv_rope_project", "rs_value_norm_max", "rs_probe_runs", "rs_build_indices_ranked",
+           "rs_mixture_rows", "rs_mixture_runs"]
 
 
 def lib_path() -> str:
@@ -195,6 +196,14 @@ def rs_probe(p: Problem, Q, K, V, vert, slash, lse_probe, qpool, kpool, vmax, de
                            C.c_size_t(ws.numel()), _ptr(status), _stream()), "rs_probe")
 
 
+def rs_probe_runs(p: Problem, Q, K, run_starts, vert, slash, lse_probe, ws, status):
+    """Probe on four 16-row runs per segment (the query mixture at key resolution); run_starts: [n_seg][4] ints."""
+    flat = [int(x) for row in run_starts for x in row]
+    arr = (C.c_int32 * len(flat))(*flat)
+    _check(load().rs_probe_runs(C.byref(p.c), _ptr(Q), _ptr(K), arr, _ptr(vert), _ptr(slash), _ptr(lse_probe), _ptr(ws),
+                                C.c_size_t(ws.numel()), _ptr(status), _stream()), "rs_probe_runs")
+
+
 def rs_pool_queries(p: Problem, Q, lib, choice, qpool, status):
     """64-row means of Q for the heads routed to block-sparse (choice None: every head)."""
     n = 0 if lib is None else len(lib)
@@ -206,6 +215,15 @@ def rs_build_indices(p: Problem, lib, vert, slash, qpool, kpool, bscore, choice,
     _check(load().rs_build_indices(C.byref(p.c), lib, len(lib), _ptr(vert), _ptr(slash), _ptr(qpool), _ptr(kpool),
                                    _ptr(bscore), _ptr(choice), C.byref(out.c), _ptr(stats), _ptr(ws),
                                    C.c_size_t(ws.numel()), _ptr(status), _stream()), "rs_build_indices")
+
+
+def rs_build_indices_ranked(p: Problem, lib, vert, slash, rank_vert, rank_slash, qpool, kpool, bscore, choice,
+                            out: IndexSet, stats, ws, status):
+    """rs_build_indices with the line lists ranked by rank_vert / rank_slash (masses of the query mixture)."""
+    _check(load().rs_build_indices_ranked(C.byref(p.c), lib, len(lib), _ptr(vert), _ptr(slash), _ptr(rank_vert),
+                                          _ptr(rank_slash), _ptr(qpool), _ptr(kpool), _ptr(bscore), _ptr(choice),
+                                          C.byref(out.c), _ptr(stats), _ptr(ws), C.c_size_t(ws.numel()), _ptr(status),
+                                          _stream()), "rs_build_indices_ranked")
 
 
 def rs_route(p: Problem, lib, stats, cost, vmax, params: rs_route_params, choice, report, status):
@@ -257,16 +275,21 @@ def rs_probe_pooled_scratch_floats(p: Problem, r: int) -> int:
 
 
 def mixture_rows(q0: int, q1: int, r_recent: int = 32, r_uniform: int = 16, r_boundary: int = 16):
-    """Row ids of the probe's query mixture (Section 3.2) for the segment [q0, q1), in the order recent, uniform,
-    boundary: the last r_recent rows, r_uniform rows at the midpoints of equal strata of what lies between the two
-    other groups, and the r_boundary rows right after the segment start.  Plain index arithmetic on the host."""
-    span = (q1 - q0) - r_recent - r_boundary
-    if span < r_uniform:
+    """Row ids of the probe's query mixture (Section 3.2) for the segment [q0, q1): rs_mixture_rows of the library."""
+    r = r_recent + r_uniform + r_boundary
+    out = (C.c_int32 * r)()
+    rc = load().rs_mixture_rows(int(q0), int(q1), int(r_recent), int(r_uniform), int(r_boundary), out)
+    if rc == -2:
         raise ValueError("segment too short for this mixture")
-    rows = list(range(q1 - r_recent, q1))
-    rows += [q0 + r_boundary + ((2 * k + 1) * span) // (2 * r_uniform) for k in range(r_uniform)]
-    rows += list(range(q0, q0 + r_boundary))
-    return rows
+    _check(rc, "rs_mixture_rows")
+    return list(out)
+
+
+def rs_mixture_runs(q0: int, q1: int):
+    """First rows of the four 16-row runs of the query mixture at key resolution (rs_mixture_runs of the library)."""
+    out = (C.c_int32 * 4)()
+    _check(load().rs_mixture_runs(int(q0), int(q1), out), "rs_mixture_runs")
+    return list(out)
 
 
 def rs_probe_pooled(p: Problem, Q, K, rows, g: int, sub_bounds, A, lse, colmass, diagmass, descr, scratch, status):

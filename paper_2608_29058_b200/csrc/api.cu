@@ -179,3 +179,25 @@ extern "C" int rs_selftest_wait_timeout(int32_t* status, unsigned int poll_limit
   rs_selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(status, poll_limit);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }
+
+// ------------------------------------------------------------------------------------------ query mixture of Eq. 3 (host)
+extern "C" int rs_mixture_rows(int q0, int q1, int r_recent, int r_uniform, int r_boundary, int32_t* rows) {
+  if (rows == nullptr || q0 < 0 || q1 <= q0 || r_recent < 0 || r_uniform < 0 || r_boundary < 0) return RS_ERR_INVALID_ARG;
+  const long long span = (long long)(q1 - q0) - r_recent - r_boundary;
+  if (span < r_uniform) return RS_ERR_UNSUPPORTED_SHAPE;       // the three groups would overlap
+  int at = 0;
+  for (int k = 0; k < r_recent; ++k) rows[at++] = q1 - r_recent + k;
+  for (int k = 0; k < r_uniform; ++k) rows[at++] = q0 + r_boundary + (int)(((2ll * k + 1) * span) / (2ll * r_uniform));
+  for (int k = 0; k < r_boundary; ++k) rows[at++] = q0 + k;
+  return RS_OK;
+}
+
+extern "C" int rs_mixture_runs(int q0, int q1, int32_t* run_starts) {
+  if (run_starts == nullptr || q0 < 0 || q1 - q0 < RS_PROBE_ROWS || (q1 - q0) % 16 != 0) return RS_ERR_INVALID_ARG;
+  const int units = (q1 - q0) / 16;
+  run_starts[0] = q0;
+  run_starts[1] = q0 + 16 * (units / 3);
+  run_starts[2] = q0 + 16 * ((2 * units) / 3);
+  run_starts[3] = q1 - 16;
+  return RS_OK;
+}

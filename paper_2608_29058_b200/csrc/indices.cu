@@ -21,6 +21,7 @@ struct IdxParams {
   int seg_bounds[RS_MAX_SEGMENTS + 1];
   rs_candidate lib[RS_MAX_CANDIDATES];
   const float* vert; const float* slash; const float* qpool; const float* kpool; const float* bscore;
+  const float* rank_vert; const float* rank_slash;   // masses the line lists are ranked by (== vert / slash unless given)
   const int32_t* choice;
   rs_index_set out;
   rs_cand_stats* stats;
@@ -97,7 +98,7 @@ rs_vs_keys_kernel(IdxParams P, int fuse_vblk) {
   const int s = item / P.Hq;
   const int q1 = P.seg_bounds[s + 1];
   const int j = blockIdx.x * 256 + threadIdx.x;
-  const float* mass = (list == 0 ? P.vert : P.slash) + (size_t)item * RS_PROBE_GROUPS * P.n;
+  const float* mass = (list == 0 ? P.rank_vert : P.rank_slash) + (size_t)item * RS_PROBE_GROUPS * P.n;
   u64 f[RS_PROBE_GROUPS] = {0, 0, 0, 0};
   if (j < q1) {
 #pragma unroll
@@ -1101,10 +1102,10 @@ size_t rs_indices_workspace_bytes(const rs_problem* p, const rs_candidate* lib, 
   return plan(p, lib, n_cand).total;
 }
 
-extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, int n_cand, const float* vert,
-                                const float* slash, const float* qpool, const float* kpool, const float* bscore,
-                                const int32_t* choice, const rs_index_set* out, rs_cand_stats* stats, void* ws,
-                                size_t ws_bytes, int32_t* status, void* stream_) {
+static int build_indices_impl(const rs_problem* p, const rs_candidate* lib, int n_cand, const float* vert,
+                              const float* slash, const float* rank_vert, const float* rank_slash, const float* qpool,
+                              const float* kpool, const float* bscore, const int32_t* choice, const rs_index_set* out,
+                              rs_cand_stats* stats, void* ws, size_t ws_bytes, int32_t* status, void* stream_) {
   int rc = rs_check_problem(p);
   if (rc != RS_OK) return rc;
   if (!lib || n_cand <= 0 || n_cand > RS_MAX_CANDIDATES || !out || !ws) return RS_ERR_INVALID_ARG;
@@ -1156,6 +1157,7 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   for (int s = 0; s <= p->n_segments; ++s) P.seg_bounds[s] = p->seg_bounds[s];
   for (int c = 0; c < n_cand; ++c) P.lib[c] = lib[c];
   P.vert = vert; P.slash = slash; P.qpool = qpool; P.kpool = kpool; P.bscore = bscore; P.choice = choice;
+  P.rank_vert = rank_vert ? rank_vert : vert; P.rank_slash = rank_slash ? rank_slash : slash;
   P.out = *out; P.stats = stats; P.vblk = reinterpret_cast<u64*>(wsb + w.vblk);
   P.bs_ws = reinterpret_cast<float*>(wsb + w.bs_ws); P.status = status;
   P.keys = reinterpret_cast<u64*>(wsb + w.keys);
@@ -1163,7 +1165,8 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
   P.scale = (float)(1.0 / sqrt((double)RS_HEAD_DIM));
 
   const int n_jobs = n_items * n_cand;
-  const bool fuse_vblk = stats != nullptr && any_vs;     // the ranking-key kernel then also writes the block sums
+  // the ranking-key kernel also writes the block sums of fx(vert) when the lists are ranked by vert itself
+  const bool fuse_vblk = stats != nullptr && any_vs && P.rank_vert == vert;
   if (stats != nullptr && !fuse_vblk) {
     const long long warps = (long long)n_items * RS_PROBE_GROUPS * nb;
     rs_vblk_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, stream>>>(P);
@@ -1217,6 +1220,24 @@ extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, in
     if (rc != RS_OK) return rc;
   }
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+}
+
+extern "C" int rs_build_indices(const rs_problem* p, const rs_candidate* lib, int n_cand, const float* vert,
+                                const float* slash, const float* qpool, const float* kpool, const float* bscore,
+                                const int32_t* choice, const rs_index_set* out, rs_cand_stats* stats, void* ws,
+                                size_t ws_bytes, int32_t* status, void* stream) {
+  return build_indices_impl(p, lib, n_cand, vert, slash, nullptr, nullptr, qpool, kpool, bscore, choice, out, stats, ws,
+                            ws_bytes, status, stream);
+}
+
+extern "C" int rs_build_indices_ranked(const rs_problem* p, const rs_candidate* lib, int n_cand, const float* vert,
+                                       const float* slash, const float* rank_vert, const float* rank_slash,
+                                       const float* qpool, const float* kpool, const float* bscore, const int32_t* choice,
+                                       const rs_index_set* out, rs_cand_stats* stats, void* ws, size_t ws_bytes,
+                                       int32_t* status, void* stream) {
+  if (!rank_vert || !rank_slash) return RS_ERR_INVALID_ARG;
+  return build_indices_impl(p, lib, n_cand, vert, slash, rank_vert, rank_slash, qpool, kpool, bscore, choice, out, stats,
+                            ws, ws_bytes, status, stream);
 }
 
 extern "C" int rs_mixture_coverage(const rs_problem* p, const rs_candidate* lib, int n_cand, const float* A,

@@ -38,6 +38,7 @@ struct rs_candidate_list { int32_t pattern[RS_MAX_CANDIDATES]; };
 struct ProbeParams {
   int n, Hq, Hkv, group, n_seg, n_hc;  // n_hc = head chunks per KV head = ceil(group / 4)
   int seg_bounds[RS_MAX_SEGMENTS + 1];
+  int run_start[RS_MAX_SEGMENTS][RS_PROBE_GROUPS];   // first row of each 16-row group of probe rows, per segment
   int n_splits, per;
   float4* partial;    // [n_seg*Hkv*n_hc][2*n_splits][256] (max, sum, sum of p * score, sum of p inside the local band), exp2 domain
   float* lse_probe;   // [Hq][n_seg][64]
@@ -88,7 +89,10 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const int n_tiles = (q1 + kKeyTile - 1) / kKeyTile;
   const int per = P.per;                      // key tiles per CTA, the same for every unit
   const int t0 = blockIdx.x * per, t1 = min(n_tiles, t0 + per);
-  const int i_first = q1 - RS_PROBE_ROWS;   // first probe row
+  int run0[RS_PROBE_GROUPS];               // first row of each group of probe rows
+#pragma unroll
+  for (int q = 0; q < RS_PROBE_GROUPS; ++q) run0[q] = P.run_start[s][q];
+  const int i_min = min(min(run0[0], run0[1]), min(run0[2], run0[3]));   // lowest probe row
   // Pass 2: the CTA's keys [128 t0, 128 t1) are cut into four contiguous quarters of 32 (t1 - t0) keys, one per lane
   // quadrant; step st = -1 .. t1 - t0 - 1 of quadrant q covers keys quarter start + 32 st .. + 31.  Step -1 stores
   // nothing: it only produces the carries of the diagonals that reach back over the start of the quarter.
@@ -184,15 +188,6 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     P.descr[((size_t)s * P.Hq + h) * 2 + 0] = (red[4 * tid] + red[4 * tid + 2]) * (1.0f / 64.0f);
     P.descr[((size_t)s * P.Hq + h) * 2 + 1] = (red[4 * tid + 1] + red[4 * tid + 3]) * (1.0f / 64.0f);
   }
-  if (PASS == 2 && blockIdx.x == 0) {
-    // offsets beyond the reach of a group's rows (o > first row of the group + 15) have no key: their mass is zero
-    for (int e = tid; e < n_heads * RS_PROBE_GROUPS * 48; e += kThreads) {
-      const int hh = e / (RS_PROBE_GROUPS * 48), grp = (e / 48) % RS_PROBE_GROUPS, k = e % 48;
-      const int o = i_first + grp * 16 + 16 + k;
-      if (o < q1)
-        P.slash[(((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS + grp) * (size_t)P.n + o] = 0.f;
-    }
-  }
   __syncthreads();
   if (PASS == 2) {          // the zero columns on either side of every warp's probability tile (the scratch use is over)
     float* xz = reinterpret_cast<float*>(sm + Smem::x);
@@ -215,9 +210,12 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       // ---------------------------------------------------------------- producer
       mbar_arrive_expect_tx(bar_q, (uint32_t)n_heads * 16384u);
       for (int hh = 0; hh < n_heads; ++hh) {
-        const int row = (h0 + hh) * P.n + i_first;
-        tma_load_2d(base + Smem::qp + (uint32_t)hh * 8192u, &tmQ, bar_q, 0, row);
-        tma_load_2d(base + Smem::qp + 32768u + (uint32_t)hh * 8192u, &tmQ, bar_q, 64, row);
+#pragma unroll
+        for (int q = 0; q < RS_PROBE_GROUPS; ++q) {      // one box of 16 rows per group
+          const int row = (h0 + hh) * P.n + run0[q];
+          tma_load_2d(base + Smem::qp + (uint32_t)hh * 8192u + (uint32_t)q * 2048u, &tmQ, bar_q, 0, row);
+          tma_load_2d(base + Smem::qp + 32768u + (uint32_t)hh * 8192u + (uint32_t)q * 2048u, &tmQ, bar_q, 64, row);
+        }
       }
       bool ok = true;
       for (int it = 0; it < n_mma; ++it) {
@@ -340,7 +338,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const int colhalf = cw >> 3;                    // which 64 of the tile's 128 key columns
       const int r = quad * 32 + lane;                 // row inside the head pair (0..127)
       const int hh = part * 2 + (r >> 6);             // head slot
-      const int i = i_first + (r & 63);               // global query row
+      const int i = run0[(r & 63) >> 4] + (r & 15);   // global query row
       const bool want_descr = P.descr != nullptr;
       float m_run = -INFINITY, l_run = 0.f;
       float a_run = 0.f, loc_run = 0.f;               // sum of p * score and local-band sum of p (descriptors)
@@ -351,8 +349,8 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
         tc_fence_after();
         const int j0 = t * kKeyTile + colhalf * 64;
-        const bool need_mask = j0 + 63 > i_first;
-        const bool near = j0 + 63 > i_first - RS_LOCAL_BAND;   // reaches into some row's local band
+        const bool need_mask = j0 + 63 > i_min;
+        const bool near = j0 + 63 > i_min - RS_LOCAL_BAND;   // may reach into some row's local band
 #pragma unroll 1
         for (int c2 = 0; c2 < 2; ++c2) {
           tmem_ld32(tmem + lane_addr + (uint32_t)(b * 256 + part * 128 + colhalf * 64 + c2 * 32), v);
@@ -425,16 +423,20 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       float carry[RS_PROBE_GROUPS] = {0.f, 0.f, 0.f, 0.f};
       float* const vert_h = P.vert + ((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS * (size_t)P.n;
       float* const slash_h = P.slash + ((size_t)s * P.Hq + (size_t)(h0 + hh)) * RS_PROBE_GROUPS * (size_t)P.n;
-      // One step: the four probe groups of the warp's 32 keys.  MASKED steps (those that reach the probe rows, and the
-      // step before key 0) also zero the probabilities of pairs with j > i or j < 0.
-      auto step = [&](auto masked_tag, int b, int j, bool store) {
+      // One step: the four probe groups of the warp's 32 keys.  MASKED steps (those that reach some probe row, and the
+      // step before key 0) also zero the probabilities of pairs with j > i or j < 0, and skip a group altogether when
+      // all of the step's keys lie behind the group's last row.  Every thread writes one column mass and one diagonal
+      // mass per group: the diagonal that ends at its key, offset o = first row of the group + 15 - key, or, when that
+      // is negative, the zero of the offset equal to its key (offsets beyond the group's reach have no key at all).
+      auto step = [&](auto masked_tag, int b, int jw, bool store) {
         constexpr bool MASKED = decltype(masked_tag)::value;
+        const int j = jw + lane;
         uint32_t v16[16];
         const uint32_t t_hh = tmem + lane_addr + (uint32_t)(b * 256 + hh * 64);
         tmem_ld16(t_hh, v16);
 #pragma unroll
         for (int grp = 0; grp < RS_PROBE_GROUPS; ++grp) {
-          const int ig = i_first + grp * 16;            // first row of the group
+          const int ig = run0[grp];                     // first row of the group
           const float4* l4 = reinterpret_cast<const float4*>(s_lse + hh * 64 + grp * 16);
           float lse16[16];
 #pragma unroll
@@ -443,8 +445,14 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             lse16[4 * q] = t4.x; lse16[4 * q + 1] = t4.y; lse16[4 * q + 2] = t4.z; lse16[4 * q + 3] = t4.w;
           }
           tc_wait_ld();
+          if (MASKED && jw > ig + 15) {                 // uniform over the warp: no key of the step is visible to the group
+            if (grp + 1 < RS_PROBE_GROUPS) tmem_ld16(t_hh + (uint32_t)(grp + 1) * 16u, v16);
+            if (store && j < q1) { vert_h[(size_t)grp * P.n + j] = 0.f; slash_h[(size_t)grp * P.n + j] = 0.f; }
+            carry[grp] = 0.f;
+            continue;
+          }
           float vs[4] = {0.f, 0.f, 0.f, 0.f};
-          __syncwarp();                                 // the previous group's rotated reads are done
+          __syncwarp();                                 // the previous group's diagonal reads are done
 #pragma unroll
           for (int r = 0; r < 16; ++r) {
             float p = fast_exp2(fmaf(__uint_as_float(v16[r]), sl2, -lse16[r]));
@@ -460,7 +468,10 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 #pragma unroll
           for (int r = 0; r < 16; ++r) acc0[r & 3] += xw[r * (kXS + 1) + lane];
           const int o = ig + 15 - j;                    // the offset whose diagonal ends at this key
-          if (store && o >= 0) slash_h[(size_t)grp * P.n + o] = ((acc0[0] + acc0[1]) + (acc0[2] + acc0[3])) + carry[grp];
+          if (store) {
+            if (o >= 0) slash_h[(size_t)grp * P.n + o] = ((acc0[0] + acc0[1]) + (acc0[2] + acc0[3])) + carry[grp];
+            else if (j < q1) slash_h[(size_t)grp * P.n + j] = 0.f;
+          }
           if (lane < 15) {
             float acc1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -475,8 +486,8 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         if (!ok) break;
         tc_fence_after();
         const int jw = key_q + (it - 1) * 32;           // first key of the step
-        if (jw + 31 > i_first || jw < 0) step(std::true_type{}, b, jw + lane, it > 0 && live);
-        else step(std::false_type{}, b, jw + lane, it > 0 && live);
+        if (jw + 31 > i_min || jw < 0) step(std::true_type{}, b, jw, it > 0 && live);
+        else step(std::false_type{}, b, jw, it > 0 && live);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tempty[b]);   // one arrival per warp: 512 arrivals per tile queue up on the barrier
@@ -702,14 +713,21 @@ extern "C" int rs_pool_queries(const rs_problem* p, const void* Q, const rs_cand
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }
 
-extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const void* V, float* vert, float* slash,
-                        float* lse_probe, float* qpool, float* kpool, float* vmax, float* descr, int flags, void* ws,
-                        size_t ws_bytes, int32_t* status, void* stream_) {
+// rs_probe and rs_probe_runs.  run_starts: host int32 [n_seg][4], first row of each 16-row group of probe rows, or
+// NULL for the last 64 rows of every segment.
+static int probe_impl(const rs_problem* p, const void* Q, const void* K, const void* V, const int32_t* run_starts,
+                      float* vert, float* slash, float* lse_probe, float* qpool, float* kpool, float* vmax, float* descr,
+                      int flags, void* ws, size_t ws_bytes, int32_t* status, void* stream_) {
   int rc = rs_check_problem(p);
   if (rc != RS_OK) return rc;
   if (!Q || !K || !V || !vert || !slash || !lse_probe || !ws) return RS_ERR_INVALID_ARG;
-  for (int s = 0; s < p->n_segments; ++s)
+  for (int s = 0; s < p->n_segments; ++s) {
     if (p->seg_bounds[s + 1] < RS_PROBE_ROWS) return RS_ERR_UNSUPPORTED_SHAPE;
+    for (int g = 0; run_starts != nullptr && g < RS_PROBE_GROUPS; ++g) {
+      const int r0 = run_starts[s * RS_PROBE_GROUPS + g];
+      if (r0 < 0 || r0 + 16 > p->seg_bounds[s + 1]) return RS_ERR_INVALID_ARG;
+    }
+  }
   rc = rs_check_device();
   if (rc != RS_OK) return rc;
   const ProbePlan w = plan(p);
@@ -722,6 +740,9 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
   P.n = p->n_keys; P.Hq = p->n_q_heads; P.Hkv = p->n_kv_heads; P.group = P.Hq / P.Hkv;
   P.n_seg = p->n_segments; P.n_hc = w.n_hc; P.n_splits = w.n_splits; P.per = w.per;
   for (int s = 0; s <= p->n_segments; ++s) P.seg_bounds[s] = p->seg_bounds[s];
+  for (int s = 0; s < p->n_segments; ++s)
+    for (int g = 0; g < RS_PROBE_GROUPS; ++g)
+      P.run_start[s][g] = run_starts ? run_starts[s * RS_PROBE_GROUPS + g] : p->seg_bounds[s + 1] - RS_PROBE_ROWS + 16 * g;
   P.partial = reinterpret_cast<float4*>(wsb + w.partial);
   P.descr = descr;
   P.lse_probe = lse_probe; P.vert = vert; P.slash = slash; P.kpool = kpool; P.status = status;
@@ -740,7 +761,7 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
   }
 
   CUtensorMap tmQ, tmK, tmK32;      // K in boxes of 128 keys (pass 1) and of 32 keys (pass 2: one box per lane quadrant)
-  if (rs_make_tmap_bf16_2d(&tmQ, Q, (uint64_t)P.Hq * P.n, RS_HEAD_DIM, 64, 64) ||
+  if (rs_make_tmap_bf16_2d(&tmQ, Q, (uint64_t)P.Hq * P.n, RS_HEAD_DIM, 16, 64) ||      // one box per group of probe rows
       rs_make_tmap_bf16_2d(&tmK, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, kKeyTile, 64) ||
       rs_make_tmap_bf16_2d(&tmK32, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, 32, 64))
     return RS_ERR_CUDA;
@@ -774,4 +795,18 @@ extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const
   rc = rs_side_join(stream);
   if (rc != RS_OK) return rc;
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
+}
+
+extern "C" int rs_probe(const rs_problem* p, const void* Q, const void* K, const void* V, float* vert, float* slash,
+                        float* lse_probe, float* qpool, float* kpool, float* vmax, float* descr, int flags, void* ws,
+                        size_t ws_bytes, int32_t* status, void* stream) {
+  return probe_impl(p, Q, K, V, nullptr, vert, slash, lse_probe, qpool, kpool, vmax, descr, flags, ws, ws_bytes, status, stream);
+}
+
+extern "C" int rs_probe_runs(const rs_problem* p, const void* Q, const void* K, const int32_t* run_starts, float* vert,
+                             float* slash, float* lse_probe, void* ws, size_t ws_bytes, int32_t* status, void* stream) {
+  if (run_starts == nullptr) return RS_ERR_INVALID_ARG;
+  // V is only read by the value-norm kernel, which does not run here; K stands in for the argument check
+  return probe_impl(p, Q, K, K, run_starts, vert, slash, lse_probe, nullptr, nullptr, nullptr, nullptr, 0, ws, ws_bytes,
+                    status, stream);
 }

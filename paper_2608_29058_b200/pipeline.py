@@ -48,6 +48,8 @@ class RouteConfig:
     backfill: bool = False             # spend leftover budget on the best risk decrease per added cost
     mixture_u: bool = False            # u of Eq. 4 from the recent / uniform / boundary rows of the query mixture
     global_pattern: bool = False       # comparison router: one candidate for the whole layer (Section 4, baselines)
+    mixture_lists: bool = False        # vertical / slash lists ranked by the query mixture of Eq. 3 (four 16-row runs:
+                                       # boundary, two uniformly spaced, recent) instead of the last 64 rows alone
 
 
 class _IdxView:
@@ -138,7 +140,24 @@ class RoutedPrefillLayer:
     def pool_routed_queries(self, Q):
         rs.rs_pool_queries(self.p, Q, self.lib, self.choice, self.qpool, self.status)
 
+    def mixture_probe(self, Q, K):
+        """Column and diagonal masses of the query mixture at key resolution (rs_probe_runs) into buffers of their own;
+        the run starts come from the library (rs_mixture_runs)."""
+        if getattr(self, "_mix", None) is None:
+            f32 = dict(dtype=torch.float32, device=self.O.device)
+            p = self.p
+            self._mix = dict(vert=torch.empty_like(self.vert), slash=torch.empty_like(self.slash),
+                             lse=torch.empty((p.n_q_heads, p.n_segments, 64), **f32),
+                             runs=[rs.rs_mixture_runs(p.seg_bounds[s], p.seg_bounds[s + 1]) for s in range(p.n_segments)])
+        m = self._mix
+        rs.rs_probe_runs(self.p, Q, K, m["runs"], m["vert"], m["slash"], m["lse"], self.ws, self.status)
+
     def evaluate_candidates(self):
+        if self.cfg.mixture_lists and getattr(self, "_mix", None) is not None:
+            m = self._mix
+            rs.rs_build_indices_ranked(self.p, self.lib, self.vert, self.slash, m["vert"], m["slash"], self.qpool,
+                                       self.kpool, None, None, self.idx_eval, self.stats, self.ws, self.status)
+            return
         rs.rs_build_indices(self.p, self.lib, self.vert, self.slash, self.qpool, self.kpool, None, None,
                             self.idx_eval, self.stats, self.ws, self.status)
 
@@ -322,8 +341,8 @@ class RoutedPrefillLayer:
     def forward(self, Q, K, V, fixed_choice: Optional[torch.Tensor] = None,
                 forced_dense: Optional[torch.Tensor] = None, record_events: bool = False) -> torch.Tensor:
         """Routed sparse prefill attention of one layer; returns O (device). Nothing synchronises."""
-        staged = (record_events or self.cfg.mixture_u or (self.regressor is not None and self.cfg.beta > 0.0)
-                  or not self.one_call)
+        staged = (record_events or self.cfg.mixture_u or self.cfg.mixture_lists
+                  or (self.regressor is not None and self.cfg.beta > 0.0) or not self.one_call)
         if not staged:
             # the whole pass as one library call; the staged path below issues the same calls one by one (needed for
             # per-stage timing and for the steps the one-call entry point does not cover: mixture coverage, predictor e)
@@ -340,6 +359,8 @@ class RoutedPrefillLayer:
         mark(0)
         lazy = not self.cfg.mixture_u        # the mixture coverage reads pooled queries of blocks all over the segment
         self.probe(Q, K, V, lazy_qpool=lazy)
+        if self.cfg.mixture_lists and fixed_choice is None:
+            self.mixture_probe(Q, K)
         mark(1)
         if fixed_choice is None:
             self.evaluate_candidates()

@@ -156,3 +156,30 @@ def test_pooled_probe_invariants():
     Km[1:, 0] = 0.0                                                       # ... of which only key 0 is left
     a_mixed = P.pooled_probe(Qm, Km, rows, g, n, [0, 32, 48, 64]).agreement
     assert a_local > a_mixed + 0.2
+
+
+def test_probe_on_runs_of_the_query_mixture_against_the_full_attention_matrix():
+    """The probe on four arbitrary 16-row runs (the query mixture at key resolution): column and diagonal masses by
+    brute force from the full matrix A; with the runs of the last 64 rows it is the last-64-query probe."""
+    Q, K, V = _head(seed=8, n=448)
+    Am = A.attention_matrix(Q, K)
+    for q0, q1 in ((0, 448), (128, 320)):
+        starts = P.mixture_runs(q0, q1)
+        assert starts[0] == q0 and starts[3] == q1 - 16 and np.all(np.diff(starts) >= 16) and np.all(starts % 16 == 0)
+        pr = P.probe_rows(Q, K, q1, starts)
+        for g, s0 in enumerate(starts):
+            rg = np.arange(s0, s0 + 16)
+            assert np.allclose(pr.vert[g], Am[rg][:, :q1].sum(axis=0), atol=1e-6)
+            want = np.zeros(q1)
+            for i in rg:
+                for o in range(i + 1):
+                    want[o] += Am[i, i - o]
+            assert np.allclose(pr.slash[g], want, atol=1e-6)
+            assert np.all(pr.slash[g, s0 + 16:] == 0)                # no row of the run reaches that far back
+        _, lse = A.dense_attention(Q, K, V, np.concatenate([np.arange(s0, s0 + 16) for s0 in starts]))
+        assert np.allclose(pr.lse, lse, atol=1e-6)
+    a, b = P.probe_rows(Q, K, 320), P.probe_rows(Q, K, 320, [256, 272, 288, 304])
+    assert np.array_equal(a.vert, b.vert) and np.array_equal(a.slash, b.slash) and np.array_equal(a.lse, b.lse)
+    # thirds of the segment, in units of 16 rows
+    assert P.mixture_runs(0, 64).tolist() == [0, 16, 32, 48]
+    assert P.mixture_runs(64, 64 + 960).tolist() == [64, 64 + 320, 64 + 640, 64 + 944]
