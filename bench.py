@@ -233,6 +233,9 @@ def main():
                     help="router ablations of the paper's Table 3 on the config-3 layer, JSONL output")
     ap.add_argument("--mixture", action="store_true",
                     help="u of Eq. 4 = disagreement among the recent / uniform / boundary rows of the query mixture (pooled probe)")
+    ap.add_argument("--mixture-lists", action="store_true",
+                    help="vertical / slash lists ranked by the query mixture of Eq. 3 at key resolution (four 16-row runs) "
+                         "instead of the last 64 rows alone (the paper's 'Recent queries only' ablation is the default)")
     ap.add_argument("--graph", action="store_true",
                     help="also time the layer replayed from a CUDA graph (whole pass captured once; for launch-bound sizes)")
     ap.add_argument("--from-hidden", action="store_true",
@@ -290,7 +293,8 @@ def main():
     to_dev = lambda bits: torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
     Q, K, V = to_dev(L["Q"]), to_dev(L["K"]), to_dev(L["V"])
     p = rs.Problem(spec.n_q_heads, spec.n_kv_heads, spec.n, [int(x) for x in L["seg_bounds"]])
-    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(rescue_any=args.rescue, mixture_u=args.mixture, **route_kw), device=dev)
+    layer = rs.RoutedPrefillLayer(p, lib, rs.RouteConfig(rescue_any=args.rescue, mixture_u=args.mixture,
+                                                           mixture_lists=args.mixture_lists, **route_kw), device=dev)
     risk_calibration = None
     if args.calibration:
         with open(args.calibration) as f:
@@ -464,7 +468,7 @@ def main():
     if rank != 0:
         return 0
 
-    plain = args.cost == "flops" and not (args.rescue or args.mixture or args.calibration)
+    plain = args.cost == "flops" and not (args.rescue or args.mixture or args.calibration or args.mixture_lists)
     # ---- side runs outside the timed region: what the headline would be under the two literal readings of the task
     extra = None
     if args.workload == "config3" and not args.no_extra and plain:
@@ -519,6 +523,7 @@ def main():
         "cost_model": args.cost, "calibration": calibration, "risk_calibration": risk_calibration, "launch_ablation": launch_ablation,
         "cuda_graph_ms_per_layer": graph_ms,
         "fallback_rescue": bool(args.rescue), "mixture_uncertainty": bool(args.mixture),
+        "mixture_lists": bool(args.mixture_lists),
         "roofline": {"kernel": "rs_attn_kernel (one launch, all heads)", "bound": "tensor", "achieved": achieved,
                      "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": f"bf16_tflops_sustained, {peaks['source']}",
@@ -760,6 +765,8 @@ def ablations(args):
         ("greedy back-fill of leftover budget", None, rs.RouteConfig(backfill=True, **base), {}),
         ("uncertainty from recent / uniform / boundary rows (query mixture)", None, rs.RouteConfig(mixture_u=True, **base), {}),
         ("the same with alpha = 4", None, rs.RouteConfig(mixture_u=True, alpha=4.0, **base), {}),
+        ("lists ranked by the query mixture (four 16-row runs) instead of the recent rows only", None,
+         rs.RouteConfig(mixture_lists=True, **base), {}),
         ("layer-level router: one candidate for all heads", None, rs.RouteConfig(global_pattern=True, **base), {}),
         ("layer-level router without fallback", None, rs.RouteConfig(global_pattern=True, budget_frac=0.15, cert_max=None), {}),
     ]
