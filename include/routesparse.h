@@ -330,6 +330,25 @@ int rs_regressor_eval(const rs_problem* p, const rs_candidate* lib, int n_cand, 
                       const float* descr, const double* w, const double* bp_z, const double* bp_e, int n_bp,
                       double* e_out, int32_t* status, void* stream);
 
+/* Offline calibration of Section 3.5 and the predictor e of Section 3.3 / Eq. 4 from audit records (HOST function, host
+ * arrays; a few hundred records, run once per model / library / length bucket):
+ *   features [n_records][n_features], target [n_records] (audited error, e.g. mean row error / V_max),
+ *   residual [n_records] (m_hat - m_true of the audited (head, candidate)), q in (0, 1]
+ * Outputs: delta_q = the ceil(q n)-th smallest residual floored at 0 ("a one-sided residual quantile", Section 3.3);
+ *   w [n_features] >= 0 minimising ||features w - target||^2 (w = e_0 when the minimiser is 0); the non-decreasing
+ *   least-squares step function of target on z = features . w as breakpoints bp_z (ascending) / bp_e (non-decreasing),
+ *   thinned to at most max_breakpoints (<= 64 for rs_regressor_eval) by dropping the smallest jumps; n_bp their number.
+ *   bp_z, bp_e need room for n_records entries. */
+int rs_calibration_fit(int n_records, int n_features, const double* features, const double* target,
+                       const double* residual, double q, int max_breakpoints, double* delta_q, double* w,
+                       double* bp_z, double* bp_e, int* n_bp);
+
+/* Measured latency table of Section 3.1 ("we profile every (p, b, n) tuple"): cand_ms [n_cand] = measured time of one
+ * attention launch with every item routed to candidate c; it is split over the items in proportion to their exact
+ * pair counts pairs [n_items][n_cand] and written as integer nanoseconds (>= 1) to table [n_items][n_cand], the
+ * `cost` argument of rs_route.  HOST function, host arrays. */
+int rs_cost_table_from_times(int n_items, int n_cand, const double* cand_ms, const uint64_t* pairs, int64_t* table);
+
 /* Dense audit of Section 3.5: row-wise output error between two attention outputs of the same shape,
  *   err[i] = || Oa_i - Ob_i ||_2,  norm_a[i] = || Oa_i ||_2   (fp32 accumulation over the 128 dimensions)
  * Oa, Ob: [n_rows][128] bf16 (o_dtype 0) or fp32 (o_dtype 1); err, norm_a (may be NULL): device fp32[n_rows]. */

@@ -60,7 +60,7 @@ EXPORTS = ["rs_error_string", "rs_version", "rs_workspace_bytes", "rs_probe", "r
            "rs_selftest_wait_timeout", "rs_probe_pooled", "rs_probe_pooled_scratch_floats", "rs_regressor_eval",
            "rs_output_error", "rs_mixture_coverage", "rs_pool_queries", "rs_routed_prefill_layer",
            "rs_qkv_rope_project", "rs_value_norm_max", "rs_probe_runs", "rs_build_indices_ranked",
-           "rs_mixture_rows", "rs_mixture_runs"]
+           "rs_mixture_rows", "rs_mixture_runs", "rs_calibration_fit", "rs_cost_table_from_times"]
 
 
 def lib_path() -> str:
@@ -337,6 +337,34 @@ def rs_qkv_rope_project(X, W, rope_cos, rope_sin, n_q_heads: int, n_kv_heads: in
 
 def rs_value_norm_max(p: Problem, vbmax, vmax, status):
     _check(load().rs_value_norm_max(C.byref(p.c), _ptr(vbmax), _ptr(vmax), _ptr(status), _stream()), "rs_value_norm_max")
+
+
+def rs_calibration_fit(features, target, residual, q: float, max_breakpoints: int = 64):
+    """Host statistics of the offline calibration (library function): returns (delta_q, w, bp_z, bp_e)."""
+    import numpy as np
+    X = np.ascontiguousarray(features, dtype=np.float64)
+    y = np.ascontiguousarray(target, dtype=np.float64)
+    r = np.ascontiguousarray(residual, dtype=np.float64)
+    n, nf = X.shape
+    dq, nbp = C.c_double(0.0), C.c_int(0)
+    w = np.zeros(nf); bz = np.zeros(n); be = np.zeros(n)
+    dp = lambda a: a.ctypes.data_as(C.POINTER(C.c_double))
+    _check(load().rs_calibration_fit(n, nf, dp(X), dp(y), dp(r), C.c_double(q), int(max_breakpoints), C.byref(dq), dp(w),
+                                     dp(bz), dp(be), C.byref(nbp)), "rs_calibration_fit")
+    k = int(nbp.value)
+    return float(dq.value), w.tolist(), bz[:k].tolist(), be[:k].tolist()
+
+
+def rs_cost_table_from_times(cand_ms, pairs):
+    """Measured candidate times split over the items in proportion to their pair counts -> int64 nanosecond table."""
+    import numpy as np
+    ms = np.ascontiguousarray(cand_ms, dtype=np.float64)
+    pr = np.ascontiguousarray(pairs, dtype=np.uint64)
+    table = np.zeros(pr.shape, dtype=np.int64)
+    _check(load().rs_cost_table_from_times(pr.shape[0], pr.shape[1], ms.ctypes.data_as(C.POINTER(C.c_double)),
+                                           pr.ctypes.data_as(C.POINTER(C.c_uint64)),
+                                           table.ctypes.data_as(C.POINTER(C.c_int64))), "rs_cost_table_from_times")
+    return table
 
 
 def rs_selftest_wait_timeout(status, poll_limit: int = 2000):

@@ -1,8 +1,8 @@
 """Offline calibration (Section 3.5): dense audits of calibration layers give the true retained mass and the output
 error of every (head, candidate); from them come the one-sided residual quantile delta_q of the probe's mass estimate,
 the coverage of the resulting empirical certificate (Eq. 5 with m_low = max(0, m_hat - delta_q)), and the monotone
-predictor e of Eq. 4.  Every attention launch, certificate and row error runs in the library's kernels; the host only
-does the statistics over a few hundred (head, candidate) records.
+predictor e of Eq. 4.  Every attention launch, certificate and row error runs in the library's kernels and the statistics over
+the few hundred (head, candidate) records in its host function rs_calibration_fit; this module only gathers records.
 
 Not part of the hot path: run once per model / library / length bucket, then RoutedPrefillLayer.use_calibration().
 
@@ -12,7 +12,6 @@ from __future__ import annotations
 
 import argparse
 import json
-import math
 from typing import Dict, List, Optional, Sequence
 
 import numpy as np
@@ -22,55 +21,6 @@ from . import binding as rs
 from .pipeline import RoutedPrefillLayer, RouteConfig
 
 FEATURES = ("1 - m_hat", "u", "entropy", "1 - local", "1 - agreement", "1 - pairs / dense pairs")
-
-
-# ------------------------------------------------------------------------------------------ host statistics
-def residual_quantile(residuals: Sequence[float], q: float) -> float:
-    """delta_q: the ceil(q N)-th smallest residual m_hat - m_true, floored at 0 (only over-estimates are corrected)."""
-    r = sorted(float(x) for x in residuals)
-    if not r:
-        return 0.0
-    k = min(max(int(math.ceil(q * len(r))), 1), len(r))
-    return max(0.0, r[k - 1])
-
-
-def nonneg_least_squares(X: np.ndarray, y: np.ndarray, iters: int = 4000) -> np.ndarray:
-    """min ||X w - y||^2 subject to w >= 0 by projected gradient (six unknowns: convergence is not an issue)."""
-    XtX, Xty = X.T @ X, X.T @ y
-    L = float(np.linalg.eigvalsh(XtX).max()) or 1.0
-    w = np.zeros(X.shape[1])
-    for _ in range(iters):
-        w = np.maximum(0.0, w - (XtX @ w - Xty) / L)
-    return w
-
-
-def pool_adjacent_violators(z: np.ndarray, y: np.ndarray):
-    """Non-decreasing least-squares step function of y on z; returns breakpoints (z_k ascending, e_k non-decreasing)."""
-    order = np.argsort(z, kind="stable")
-    z, y = z[order], y[order]
-    stack: List[List[float]] = []                     # [first z, sum of y, count]
-    i = 0
-    while i < len(z):
-        j = i
-        while j + 1 < len(z) and z[j + 1] == z[i]:
-            j += 1
-        stack.append([float(z[i]), float(y[i:j + 1].sum()), float(j - i + 1)])
-        while len(stack) > 1 and stack[-2][1] * stack[-1][2] > stack[-1][1] * stack[-2][2]:
-            top = stack.pop()
-            stack[-1][1] += top[1]
-            stack[-1][2] += top[2]
-        i = j + 1
-    return [b[0] for b in stack], [b[1] / b[2] for b in stack]
-
-
-def thin_breakpoints(bp_z: List[float], bp_e: List[float], limit: int = 64):
-    """At most `limit` breakpoints (the device table's size): neighbouring steps with the smallest jump are merged."""
-    bz, be = list(bp_z), list(bp_e)
-    while len(bz) > limit:
-        k = int(np.argmin(np.diff(be)))               # step k+1 is closest to step k: drop its breakpoint
-        del bz[k + 1]
-        del be[k + 1]
-    return bz, be
 
 
 # ------------------------------------------------------------------------------------------ audits
@@ -146,14 +96,10 @@ def calibrate(calibration_records: List[Dict], held_out: Optional[Dict[str, List
               g: int = 64) -> Dict:
     """delta_q, certificate coverage (in-domain and per held-out domain) and the predictor e from audit records."""
     res = [r["m_hat"] - r["m_true"] for r in calibration_records]
-    delta_q = residual_quantile(res, q)
     X = np.array([r["features"] for r in calibration_records], dtype=np.float64)
     y = np.array([r["mean_err"] / max(r["vmax"], 1e-30) for r in calibration_records], dtype=np.float64)
-    w = nonneg_least_squares(X, y)
-    if not np.any(w > 0):
-        w = np.array([1.0, 0, 0, 0, 0, 0])
-    bp_z, bp_e = pool_adjacent_violators(X @ w, y)
-    bp_z, bp_e = thin_breakpoints(bp_z, bp_e)
+    delta_q, w, bp_z, bp_e = rs.rs_calibration_fit(X, y, res, q)          # the statistics run in the library
+    w = np.array(w)
     fit = np.array([max([e for zk, e in zip(bp_z, bp_e) if zk <= z], default=0.0) for z in X @ w])
     out = {"q": q, "delta_q": delta_q, "n_records": len(calibration_records),
            "residual_mean": float(np.mean(res)), "residual_max": float(np.max(res)),

@@ -1,8 +1,8 @@
 """Call sequence of one routed prefill attention layer (the six-step procedure of Section 3.4).
 
 This is the public, user-level entry of the package: it owns the device buffers of one layer and enqueues the
-C-ABI calls in order on the current CUDA stream.  It contains no arithmetic of the method -- every step runs
-in the library's kernels.
+C-ABI calls in order on the current CUDA stream.  It contains no arithmetic of the method: every step runs in the
+library's kernels or host functions (profile_costs only times launches and hands the times to the library).
 """
 from __future__ import annotations
 
@@ -287,7 +287,6 @@ class RoutedPrefillLayer:
         a.record(); self.probe(Q, K, V); self.evaluate_candidates(); b.record()
         torch.cuda.synchronize()
         t_probe_ns = a.elapsed_time(b) * 1e6
-        pairs = self.stats.cpu().numpy()[:, :, 4].astype(np.float64)
         ms, tail = np.zeros(n_cand), np.zeros(n_cand)     # median and tail (maximum of the repetitions)
         saved = self.choice.clone()
         for c in range(n_cand):
@@ -303,7 +302,7 @@ class RoutedPrefillLayer:
             ms[c] = float(np.median(ts))
             tail[c] = float(np.max(ts))
         self.choice.copy_(saved)
-        table = np.maximum(1, np.rint(ms[None, :] * 1e6 * pairs / pairs.sum(axis=0, keepdims=True))).astype(np.int64)
+        table = rs.rs_cost_table_from_times(ms, self.stats.cpu().numpy()[:, :, 4].astype(np.uint64))
         dense_c = [i for i, c in enumerate(self.cands) if c[0] == rs.RS_DENSE][0]
         self.cost_table = torch.from_numpy(table).to(self.O.device)
         self.cost_budget = int(self.cfg.budget_frac * ms[dense_c] * 1e6)
