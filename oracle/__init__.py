@@ -18,9 +18,13 @@ Parts and what pins them (tests/test_oracle_*.py):
                                                                   build's reading: "parity unpinned".
   certificate.certificate        Eq. 5.                           Pinned: equality case, L1 identity, bound on every row.
   probe.pooled_probe             Eq. 3, general form + descriptors. Pinned: width 1 == exact probe, per-key brute force,
-                                                                  identical keys -> uniform rows.  The mixture, the pooling
-                                                                  of a straddling block and the agreement formula are this
-                                                                  build's reading: beyond those "parity unpinned".
+                                                                  identical keys -> uniform rows, agreement and signature
+                                                                  bins in a closed-form case (sink rows against uniform
+                                                                  rows).  The proportions of the mixture and the pooling of
+                                                                  a straddling block are this build's reading.
+  probe.probe_rows(starts=...)   Eq. 3 at key resolution on four 16-row runs of the query mixture.  Pinned: brute force
+                                                                  against the full attention matrix; the last-64-row runs
+                                                                  give the ordinary probe bit for bit.
   patterns.mixture_coverage_fx   coverage on the mixture's rows.   Pinned: closed cases (whole blocks, half blocks, columns).
                                                                   The even split of a block's mass over its visible keys
                                                                   is this build's reading: "parity unpinned".

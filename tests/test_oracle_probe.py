@@ -183,3 +183,30 @@ def test_probe_on_runs_of_the_query_mixture_against_the_full_attention_matrix():
     # thirds of the segment, in units of 16 rows
     assert P.mixture_runs(0, 64).tolist() == [0, 16, 32, 48]
     assert P.mixture_runs(64, 64 + 960).tolist() == [64, 64 + 320, 64 + 640, 64 + 944]
+
+
+def test_agreement_descriptor_in_a_closed_form_case():
+    """Recent rows that put all their mass on key block 0 (a sink 60 logits above everything else) against uniform-group
+    rows whose queries are zero (uniform over the visible blocks): the recent signature is the unit vector of the
+    [block 0] bin, a uniform row with v > 17 visible blocks has 1/v in that bin, so the total-variation distance is
+    1 - mean(1/v) and agreement = mean(1/v).  Entropy: 0 for the recent rows, 1 for the uniform ones."""
+    n, d, g = 64 * 40, 128, 64
+    K = np.zeros((n, d)); Q = np.zeros((n, d))
+    u = np.zeros(d); u[3] = 1.0
+    K[:64] = u                                              # block 0: the sink direction, every other key is zero
+    rows = np.array([n - 4, n - 3, n - 2, n - 1, 64 * 20 + 5, 64 * 25 + 63, 64 * 30])
+    Q[rows[:4]] = 60.0 * np.sqrt(d) * u                     # logit 60 on block 0, 0 elsewhere
+    pp = P.pooled_probe(Q, K, rows, g, n, [0, 4, 7])
+    vis = np.array([21, 26, 31])
+    assert abs(pp.agreement - np.mean(1.0 / vis)) < 1e-12
+    assert abs(pp.entropy - 3.0 / 7.0) < 1e-12
+    # identical groups agree completely; disjoint supports not at all
+    same = P.pooled_probe(Q, K, rows[[0, 1, 2, 3]], g, n, [0, 2, 4])
+    assert abs(same.agreement - 1.0) < 1e-12
+    Q2 = Q.copy(); K2 = K.copy()
+    K2[64 * 39:] = u; K2[:64] = 0.0                         # second pair of rows: all mass on their own block instead
+    sig_a = P.row_signature(np.eye(40)[0], n - 1, g)        # everything on block 0 -> bin 0
+    sig_b = P.row_signature(np.eye(40)[39], n - 1, g)       # everything on the row's own block -> offset 0 -> bin 1
+    assert sig_a.tolist() == [1.0] + [0.0] * 17 and sig_b.tolist() == [0.0, 1.0] + [0.0] * 16
+    assert P.row_signature(np.eye(40)[10], n - 1, g)[17] == 1.0          # far from both ends -> the [rest] bin
+    assert P.row_signature(np.eye(40)[24], n - 1, g)[1 + 15] == 1.0      # relative offset 15 is still local
