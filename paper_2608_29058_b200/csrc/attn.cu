@@ -589,10 +589,8 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 }
 
 // -------------------------------------------------------------------------------------------- work list
-// One thread per (item, tile): estimated number of 64-key chunks, used only to order the launch (heavy first).
-__global__ void rs_attn_cost_kernel(AttnParams P, int n_work, int* cost, int2* items) {
-  const int wid = blockIdx.x * blockDim.x + threadIdx.x;
-  if (wid >= n_work) return;
+// Estimated number of 64-key chunks of work item wid = (head, tile of the head), used only to order the launch.
+__device__ __forceinline__ int rs_tile_cost(const AttnParams& P, int wid, int2* item_tile) {
   const int h = wid / P.tiles_per_head;
   const int tt = wid - h * P.tiles_per_head;
   int s = 0;
@@ -619,30 +617,36 @@ __global__ void rs_attn_cost_kernel(AttnParams P, int n_work, int* cost, int2* i
     const size_t row = (size_t)h * (P.n >> 6) + qb0;
     c = P.idx.bs_count[row] + (qb_last > qb0 ? P.idx.bs_count[row + 1] : 0);
   }
-  cost[wid] = c;
-  items[wid] = make_int2(item, tile);
+  *item_tile = make_int2(item, tile);
+  return c;
 }
 
-// Launch order: KV groups one after the other (the CTAs in flight then stream the same K / V, which keeps them in L2),
-// inside a group heaviest item first.  One block per KV group runs a counting sort by cost over the group's items,
-// which are contiguous in the item enumeration (head-major).
-__global__ void rs_attn_order_kernel(int per_group, int n_bins, const int* cost, const int2* items, int2* order) {
+// Work list of the launch (Section 3.4: heads are grouped into one launch).  KV groups run one after the other (the
+// CTAs in flight then stream the same K / V, which keeps them in L2), inside a group the heaviest item first.  One block
+// per KV group: cost of each of the group's items (they are contiguous in the head-major enumeration), then a
+// counting sort by cost.  cost / items are scratch of the block itself.
+__global__ void __launch_bounds__(1024)
+rs_attn_worklist_kernel(AttnParams P, int per_group, int n_bins, int* cost, int2* items, int2* order) {
   extern __shared__ int hist[];
-  const int n_work = per_group;
-  cost += (size_t)blockIdx.x * per_group;
-  items += (size_t)blockIdx.x * per_group;
-  order += (size_t)blockIdx.x * per_group;
+  const int base = blockIdx.x * per_group;
+  cost += base; items += base; order += base;
   for (int i = threadIdx.x; i <= n_bins; i += blockDim.x) hist[i] = 0;
   __syncthreads();
-  for (int i = threadIdx.x; i < n_work; i += blockDim.x) atomicAdd(&hist[min(cost[i], n_bins - 1)], 1);
+  for (int i = threadIdx.x; i < per_group; i += blockDim.x) {
+    int2 it;
+    const int c = min(rs_tile_cost(P, base + i, &it), n_bins - 1);
+    cost[i] = c;
+    items[i] = it;
+    atomicAdd(&hist[c], 1);
+  }
   __syncthreads();
   if (threadIdx.x == 0) {
     int acc = 0;
     for (int b = n_bins - 1; b >= 0; --b) { int c = hist[b]; hist[b] = acc; acc += c; }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < n_work; i += blockDim.x) {
-    const int pos = atomicAdd(&hist[min(cost[i], n_bins - 1)], 1);
+  for (int i = threadIdx.x; i < per_group; i += blockDim.x) {
+    const int pos = atomicAdd(&hist[cost[i]], 1);
     order[pos] = items[i];
   }
 }
@@ -741,11 +745,10 @@ int enqueue_attn(const rs_problem* p, const void* Q, const void* K, const void* 
   }
 
   const int n_work = sc.n_work;
-  // every entry of cost / items / order is rewritten by the two kernels below, so nothing has to be cleared
-  rs_attn_cost_kernel<<<(n_work + 255) / 256, 256, 0, stream>>>(P, n_work, sc.cost, sc.items);
+  // every entry of cost / items / order is rewritten by the kernel below, so nothing has to be cleared
   const int n_bins = (P.n >> 6) + 66;
-  rs_attn_order_kernel<<<P.Hkv, 1024, (n_bins + 1) * sizeof(int), stream>>>(n_work / P.Hkv, n_bins, sc.cost, sc.items,
-                                                                            sc.order);
+  rs_attn_worklist_kernel<<<P.Hkv, 1024, (n_bins + 1) * sizeof(int), stream>>>(P, n_work / P.Hkv, n_bins, sc.cost, sc.items,
+                                                                               sc.order);
   if (choice != nullptr && any_vs && sc.Kp != nullptr) {
     dim3 grid((P.kv_pad + 15) / 16, sc.n_items);
     rs_pack_vertical_kernel<<<grid, 256, 0, stream>>>(P, reinterpret_cast<const __nv_bfloat16*>(K),
