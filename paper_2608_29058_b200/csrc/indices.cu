@@ -45,6 +45,15 @@ __device__ __forceinline__ u64 fx(float x) {
   return (sh > -24) ? (m >> (-sh)) : 0ull;
 }
 
+// Adds v of every thread of the block to *target (shared memory): the warp sums first, so that one 64-bit atomic per
+// warp reaches the word (hundreds of threads on one shared 64-bit word serialise in a compare-and-swap loop).
+// Integer addition: the result does not depend on the order.  All threads of the warp must call it.
+__device__ __forceinline__ void warp_sum_then_add(u64 v, u64* target) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  if ((threadIdx.x & 31) == 0 && v != 0) atomicAdd(target, v);
+}
+
 __device__ __forceinline__ u64 line_key(const float* mass, int n, int j) {
   return fx(mass[j]) + fx(mass[(size_t)n + j]) + fx(mass[2 * (size_t)n + j]) + fx(mass[3 * (size_t)n + j]);
 }
@@ -522,7 +531,7 @@ rs_vs_finish_kernel(IdxParams P) {
     }
   }
 #pragma unroll
-  for (int g = 0; g < RS_PROBE_GROUPS; ++g) if (part[g]) atomicAdd(&cov[g], part[g]);
+  for (int g = 0; g < RS_PROBE_GROUPS; ++g) warp_sum_then_add(part[g], &cov[g]);
   if (tid < 128) {
     // block diagonals: delta >= 1 is used by every query block qb >= delta of the segment, delta 0 by all
     uint32_t bits = dbits[tid];
@@ -533,7 +542,7 @@ rs_vs_finish_kernel(IdxParams P) {
       else if (nbs > max(qb_lo, d)) vp += (u64)(nbs - max(qb_lo, d)) * 4096ull;
     }
   }
-  if (vp) atomicAdd(&extra_pairs, vp);
+  warp_sum_then_add(vp, &extra_pairs);
   __syncthreads();
   if (tid == 0) {
     rs_cand_stats* st = P.stats + (size_t)item * P.n_cand + c;
@@ -571,6 +580,7 @@ rs_simple_stats_kernel(IdxParams P) {
   const int n_off = window_covers_all ? q1 : win;
   const int n_col = window_covers_all ? 0 : min(n_sink, q1);
   u64 part[RS_PROBE_GROUPS] = {0, 0, 0, 0};
+#pragma unroll 4
   for (int o = tid; o < n_off; o += blockDim.x)
 #pragma unroll
     for (int g = 0; g < RS_PROBE_GROUPS; ++g) part[g] += fx(slash[(size_t)g * P.n + o]);
@@ -578,7 +588,7 @@ rs_simple_stats_kernel(IdxParams P) {
 #pragma unroll
     for (int g = 0; g < RS_PROBE_GROUPS; ++g) part[g] += fx(vert[(size_t)g * P.n + j]);
 #pragma unroll
-  for (int g = 0; g < RS_PROBE_GROUPS; ++g) if (part[g]) atomicAdd(&cov[g], part[g]);
+  for (int g = 0; g < RS_PROBE_GROUPS; ++g) warp_sum_then_add(part[g], &cov[g]);
   __syncthreads();
   if (tid == 0) {
     for (int g = 0; g < RS_PROBE_GROUPS; ++g) st->cov_fx[g] = cov[g];
@@ -742,7 +752,7 @@ rs_bs_eval_kernel(IdxParams P) {
 #pragma unroll
         for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) part[gg] += vblk[(size_t)gg * P.nb + sel[i]];
 #pragma unroll
-      for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) if (part[gg]) atomicAdd(&cov[gg], part[gg]);
+      for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) warp_sum_then_add(part[gg], &cov[gg]);
       __syncthreads();
       if (tid == 0) {
         rs_cand_stats* st = P.stats + (size_t)item * P.n_cand + c;
