@@ -676,7 +676,7 @@ def stack(args):
                         "achieved": f_tile / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                         "frac": f_tile / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                         "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "traffic": None},
-           "clocks": clocks, "gpu_launches": 23 * args.layers * args.steps}
+           "clocks": clocks, "gpu_launches": 20 * args.layers * args.steps}
     print(json.dumps(out))
     return 0
 
