@@ -496,21 +496,20 @@ def main():
     any_bs = any(c[0] == 3 for c in layer.cands)
     # kernels of this library per layer pass, stage by stage (memsets and torch copies are not counted)
     nb = spec.n // 64
-    n_probe = 2 + 2 + 1                                   # two passes (K is pooled inside pass 1); value norms, V_max; Q pooling
+    n_probe = 2 + 1                                       # two passes (K pooled in pass 1; V_max and the last Q block in pass 2); value norms
     n_probe += 2 if (args.mixture_lists and not fixed) else 0          # the probe on the mixture's runs
-    n_bs_rows = 2 if nb > 1025 else 1                     # warp-per-row kernel, block-per-row kernel for long rows
     if fixed:
         n_eval, n_route = 0, 0
-        n_mat = 3 * any_vs + (1 + n_bs_rows) * any_bs     # keys / select / finish; fused scores / rows
+        n_mat = 3 * any_vs + 2 * any_bs                   # keys / select / finish; fused scores / rows
     else:
-        n_eval = 1 + (3 if any_vs else 1) + 2 * any_bs    # closed-form stats; VS chain (keys + block sums, select, finish) or block sums alone; BS evaluation
+        n_eval = 1 + (3 if any_vs else 1) + 1 * any_bs    # closed-form stats + pooled scores; VS chain (keys + block sums, select, finish) or block sums alone; BS evaluation
         n_eval += 1 if (args.mixture_lists and any_vs) else 0          # block sums separate from the ranking keys
         n_eval += 4 if args.mixture else 0                # pooled probe (3) + mixture coverage
         n_eval += (0 if args.mixture else 3) + 1 if (args.calibration and args.beta > 0) else 0   # pooled probe + predictor
         n_route = 1
-        n_mat = (1 + n_bs_rows) * any_bs                  # the evaluation's vertical-slash lists are reused
+        n_mat = 2 * any_bs                                # the evaluation's vertical-slash lists are reused
     n_mat += 0 if (args.mixture and not fixed) else int(any_bs)     # queries of the heads routed to block-sparse
-    launches_per_step = n_probe + n_eval + n_route + n_mat + (2 + any_vs) + 1   # + work list, gather, attention + certificate
+    launches_per_step = n_probe + n_eval + n_route + n_mat + 2 + 1  # + preparation (work list, gather), attention + certificate
     out = {
         "metric": metric, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
@@ -676,7 +675,7 @@ def stack(args):
                         "achieved": f_tile / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                         "frac": f_tile / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                         "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "traffic": None},
-           "clocks": clocks, "gpu_launches": 20 * args.layers * args.steps}
+           "clocks": clocks, "gpu_launches": 15 * args.layers * args.steps}
     print(json.dumps(out))
     return 0
 

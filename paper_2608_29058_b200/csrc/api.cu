@@ -61,7 +61,7 @@ namespace {
 struct SideStream {
   std::mutex mu;
   cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr, mid = nullptr;
 };
 SideStream g_side[64];
 thread_local int t_side_dev = -1;   // device whose side stream this thread holds between fork and join
@@ -76,7 +76,8 @@ int rs_side_fork(cudaStream_t main, cudaStream_t* side) {
   if (S.stream == nullptr) {
     if (cudaStreamCreateWithFlags(&S.stream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&S.fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&S.join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&S.join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&S.mid, cudaEventDisableTiming) != cudaSuccess) {
       S.stream = nullptr;
       S.mu.unlock();
       return RS_ERR_CUDA;
@@ -89,6 +90,13 @@ int rs_side_fork(cudaStream_t main, cudaStream_t* side) {
   t_side_dev = dev;
   *side = S.stream;
   return RS_OK;
+}
+
+int rs_side_sync_here(cudaStream_t main) {
+  if (t_side_dev < 0) return RS_ERR_INVALID_ARG;
+  SideStream& S = g_side[t_side_dev];
+  return cudaEventRecord(S.mid, S.stream) == cudaSuccess && cudaStreamWaitEvent(main, S.mid, 0) == cudaSuccess ? RS_OK
+                                                                                                               : RS_ERR_CUDA;
 }
 
 int rs_side_join(cudaStream_t main) {

@@ -621,13 +621,39 @@ __device__ __forceinline__ int rs_tile_cost(const AttnParams& P, int wid, int2* 
   return c;
 }
 
-// Work list of the launch (Section 3.4: heads are grouped into one launch).  KV groups run one after the other (the
-// CTAs in flight then stream the same K / V, which keeps them in L2), inside a group the heaviest item first.  One block
-// per KV group: cost of each of the group's items (they are contiguous in the head-major enumeration), then a
-// counting sort by cost.  cost / items are scratch of the block itself.
+// Preparation of the launch, one kernel with two kinds of blocks.
+// Blocks 0 .. Hkv-1: the work list (Section 3.4: heads are grouped into one launch).  KV groups run one after the
+// other (the CTAs in flight then stream the same K / V, which keeps them in L2), inside a group the heaviest item first.
+// One block per KV group: cost of each of the group's items (they are contiguous in the head-major enumeration), then
+// a counting sort by cost.  cost / items are scratch of the block itself.
+// Blocks Hkv ..: the vertical key / value rows of every vertical-slash item are gathered into a contiguous,
+// zero-padded buffer; pack_blocks blocks per item, 64 rows each (16 threads move one 256-byte row).
 __global__ void __launch_bounds__(1024)
-rs_attn_worklist_kernel(AttnParams P, int per_group, int n_bins, int* cost, int2* items, int2* order) {
+rs_attn_prepare_kernel(AttnParams P, int per_group, int n_bins, int* cost, int2* items, int2* order, int pack_blocks,
+                       const __nv_bfloat16* K, const __nv_bfloat16* V, __nv_bfloat16* Kp, __nv_bfloat16* Vp) {
   extern __shared__ int hist[];
+  if ((int)blockIdx.x >= P.Hkv) {
+    const int pb = blockIdx.x - P.Hkv;
+    const int item = pb / pack_blocks;
+    if (P.choice == nullptr || P.lib[P.choice[item]].pattern != RS_VERTICAL_SLASH) return;
+    const int h = item % P.Hq, g = h / P.group;
+    const int slot = P.vs_eval_layout ? item * P.n_cand + P.choice[item] : item;
+    const int n_cols = P.idx.vs_count[4 * slot];
+    const int row = (pb - item * pack_blocks) * 64 + (threadIdx.x >> 4);
+    if (row >= P.kv_pad) return;
+    const int l16 = threadIdx.x & 15;
+    uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
+    if (row < n_cols) {
+      const int j = P.idx.vs_cols[(size_t)slot * P.idx.kv_cap + row];
+      const size_t src = ((size_t)g * P.n + (size_t)j) * RS_HEAD_DIM;
+      kv = reinterpret_cast<const uint4*>(K + src)[l16];
+      vv = reinterpret_cast<const uint4*>(V + src)[l16];
+    }
+    const size_t dst = ((size_t)item * P.kv_pad + row) * RS_HEAD_DIM;
+    reinterpret_cast<uint4*>(Kp + dst)[l16] = kv;
+    reinterpret_cast<uint4*>(Vp + dst)[l16] = vv;
+    return;
+  }
   const int base = blockIdx.x * per_group;
   cost += base; items += base; order += base;
   for (int i = threadIdx.x; i <= n_bins; i += blockDim.x) hist[i] = 0;
@@ -649,29 +675,6 @@ rs_attn_worklist_kernel(AttnParams P, int per_group, int n_bins, int* cost, int2
     const int pos = atomicAdd(&hist[cost[i]], 1);
     order[pos] = items[i];
   }
-}
-
-// Gathers the vertical key / value rows of every vertical-slash item into a contiguous, zero-padded buffer.
-__global__ void rs_pack_vertical_kernel(AttnParams P, const __nv_bfloat16* K, const __nv_bfloat16* V,
-                                        __nv_bfloat16* Kp, __nv_bfloat16* Vp) {
-  const int item = blockIdx.y;
-  if (P.choice == nullptr || P.lib[P.choice[item]].pattern != RS_VERTICAL_SLASH) return;
-  const int h = item % P.Hq, g = h / P.group;
-  const int slot = P.vs_eval_layout ? item * P.n_cand + P.choice[item] : item;
-  const int n_cols = P.idx.vs_count[4 * slot];
-  const int row = blockIdx.x * (blockDim.x >> 4) + (threadIdx.x >> 4);   // 16 threads move one 256-byte row
-  if (row >= P.kv_pad) return;
-  const int l16 = threadIdx.x & 15;
-  uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
-  if (row < n_cols) {
-    const int j = P.idx.vs_cols[(size_t)slot * P.idx.kv_cap + row];
-    const size_t src = ((size_t)g * P.n + (size_t)j) * RS_HEAD_DIM;
-    kv = reinterpret_cast<const uint4*>(K + src)[l16];
-    vv = reinterpret_cast<const uint4*>(V + src)[l16];
-  }
-  const size_t dst = ((size_t)item * P.kv_pad + row) * RS_HEAD_DIM;
-  reinterpret_cast<uint4*>(Kp + dst)[l16] = kv;
-  reinterpret_cast<uint4*>(Vp + dst)[l16] = vv;
 }
 
 size_t attn_smem_bytes(int n) {
@@ -703,7 +706,7 @@ WsPlan plan_ws(const rs_problem* p, int max_kv) {
 // vertical-slash items, the packed K / V rows of the gathered columns.
 struct AttnScratch { int* cost; int2* items; int2* order; __nv_bfloat16 *Kp, *Vp; int kv_pad; int n_work, n_items; };
 
-// Enqueues the work-list kernels, the gather of the vertical columns and the attention launch.  Arguments are checked
+// Enqueues the preparation kernel (work list, gather of the vertical columns) and the attention launch.  Arguments are checked
 // by the callers; `sc` says where the scratch lives (caller workspace or the library's built-in array).
 int enqueue_attn(const rs_problem* p, const void* Q, const void* K, const void* V, const rs_candidate* lib, int n_cand,
                  const rs_index_set* idx, const int32_t* choice, bool any_vs, bool vs_eval_layout, void* O, int o_dtype,
@@ -747,13 +750,11 @@ int enqueue_attn(const rs_problem* p, const void* Q, const void* K, const void* 
   const int n_work = sc.n_work;
   // every entry of cost / items / order is rewritten by the kernel below, so nothing has to be cleared
   const int n_bins = (P.n >> 6) + 66;
-  rs_attn_worklist_kernel<<<P.Hkv, 1024, (n_bins + 1) * sizeof(int), stream>>>(P, n_work / P.Hkv, n_bins, sc.cost, sc.items,
-                                                                               sc.order);
-  if (choice != nullptr && any_vs && sc.Kp != nullptr) {
-    dim3 grid((P.kv_pad + 15) / 16, sc.n_items);
-    rs_pack_vertical_kernel<<<grid, 256, 0, stream>>>(P, reinterpret_cast<const __nv_bfloat16*>(K),
-                                                      reinterpret_cast<const __nv_bfloat16*>(V), sc.Kp, sc.Vp);
-  }
+  const bool pack = choice != nullptr && any_vs && sc.Kp != nullptr;
+  const int pack_blocks = pack ? (P.kv_pad + 63) / 64 : 0;
+  rs_attn_prepare_kernel<<<P.Hkv + pack_blocks * sc.n_items, 1024, (n_bins + 1) * sizeof(int), stream>>>(
+      P, n_work / P.Hkv, n_bins, sc.cost, sc.items, sc.order, pack_blocks, reinterpret_cast<const __nv_bfloat16*>(K),
+      reinterpret_cast<const __nv_bfloat16*>(V), sc.Kp, sc.Vp);
   if (rs_ensure_dynamic_smem(g_attn_smem, rs_attn_kernel, 116 * 1024) != RS_OK) return RS_ERR_CUDA;
   rs_attn_kernel<<<n_work, kThreads, attn_smem_bytes(P.n), stream>>>(tmQ, tmK, tmV, tmKp, tmVp, P);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;

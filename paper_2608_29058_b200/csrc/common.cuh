@@ -213,8 +213,10 @@ int rs_make_tmap_f32_2d(CUtensorMap* out, const void* base, uint64_t rows, uint6
 // A second stream per device for kernels of one call that do not depend on each other (fork / join with events,
 // so the caller's stream still sees the call as one ordered piece of work; also valid under stream capture).
 // rs_side_fork locks the device's side stream, makes it wait for everything enqueued so far on `main` and returns
-// it; rs_side_join makes `main` wait for the side stream and unlocks.  Both return an RS_* code.
+// it; rs_side_join makes `main` wait for the side stream and unlocks; rs_side_sync_here, between the two, makes `main`
+// wait for what the side stream holds so far and keeps the lock.  All return an RS_* code.
 int rs_side_fork(cudaStream_t main, cudaStream_t* side);
+int rs_side_sync_here(cudaStream_t main);
 int rs_side_join(cudaStream_t main);
 int rs_check_problem(const rs_problem* p);
 int rs_check_device();

@@ -31,7 +31,6 @@ struct IdxParams {
   float* bs_eval_ws;  // [n_items][nb] pooled scores of each segment's last query block
   int32_t* status;
   float scale;
-  int bs_rows_first;  // first query block served by rs_bs_rows_kernel (the shorter rows go to the warp-per-row kernel)
 };
 
 // floor(x * 2^32) of a non-negative float, exactly, from its bits (no float-to-integer conversion unit involved)
@@ -552,11 +551,10 @@ rs_vs_finish_kernel(IdxParams P) {
 }
 
 // ------------------------------------------------------------------------------------------ A-shape and dense stats
-__global__ void __launch_bounds__(256)
-rs_simple_stats_kernel(IdxParams P) {
+__device__ __forceinline__ void simple_stats_block(const IdxParams& P, int job) {
   __shared__ u64 cov[RS_PROBE_GROUPS];
   int item, c, slot;
-  if (!job_of(P, blockIdx.x, item, c, slot)) return;
+  if (!job_of(P, job, item, c, slot)) return;
   if (P.stats == nullptr) return;
   const rs_candidate cand = P.lib[c];
   if (cand.pattern != RS_A_SHAPE && cand.pattern != RS_DENSE) return;
@@ -622,11 +620,27 @@ __device__ int select_row(const float* score, int m, int take, int qb, int32_t* 
         if (pass == 3 || (key >> (shift + 8)) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
       }
       __syncthreads();
-      if (tid == 0) {
-        uint32_t kk = sh[1], acc = 0;
-        for (int b = 255; b >= 0; --b) {
-          if (acc + hist[b] >= kk) { sh[0] = (prefix << 8) | (uint32_t)b; sh[1] = kk - acc; break; }
-          acc += hist[b];
+      if (warp == 0) {
+        // the bin in which the count from the top reaches kk: eight bins per lane, counts above a lane by a suffix
+        // scan over the lanes, then the one lane that holds the crossing walks its bins from the top
+        const uint32_t kk = sh[1];
+        uint32_t h8[8], local = 0;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) { h8[b] = hist[8 * lane + b]; local += h8[b]; }
+        uint32_t incl = local;                            // sum over lanes >= this one
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const uint32_t o = __shfl_down_sync(0xffffffffu, incl, off);
+          if (lane + off < 32) incl += o;
+        }
+        uint32_t acc = incl - local;
+        __syncwarp();
+        if (acc < kk && incl >= kk) {
+#pragma unroll
+          for (int b = 7; b >= 0; --b) {
+            if (acc + h8[b] >= kk) { sh[0] = (prefix << 8) | (uint32_t)(8 * lane + b); sh[1] = kk - acc; break; }
+            acc += h8[b];
+          }
         }
       }
       __syncthreads();
@@ -688,37 +702,35 @@ __device__ __forceinline__ float pooled_score(const float* q, const float* k, fl
   return acc * scale;
 }
 
-// Pooled scores of the last query block of every item that has a block-sparse candidate to evaluate.
-__global__ void __launch_bounds__(256)
-rs_bs_eval_scores_kernel(IdxParams P) {
+// Pooled scores of the last query block of an item that has a block-sparse candidate to evaluate: 256 key blocks
+// per thread block.
+__device__ __forceinline__ void bs_eval_scores_block(const IdxParams& P, int item, int bx) {
   __shared__ float qrow[RS_HEAD_DIM];
-  const int item = blockIdx.y;
   const int s = item / P.Hq, h = item - s * P.Hq, g = h / P.group;
   const int qb = (P.seg_bounds[s + 1] >> 6) - 1;
-  if (blockIdx.x * 256 >= qb) return;
+  if (bx * 256 >= qb) return;
   if (threadIdx.x < RS_HEAD_DIM) qrow[threadIdx.x] = P.qpool[((size_t)h * P.nb + qb) * RS_HEAD_DIM + threadIdx.x];
   __syncthreads();
-  const int kb = blockIdx.x * 256 + threadIdx.x;
+  const int kb = bx * 256 + threadIdx.x;
   if (kb < qb)
     P.bs_eval_ws[(size_t)item * P.nb + kb] = pooled_score(qrow, P.kpool + ((size_t)g * P.nb + kb) * RS_HEAD_DIM, P.scale);
 }
 
-// Evaluation of the block-sparse candidates of one item: the pooled scores of the segment's last query block are
-// computed once, then every block-sparse candidate selects from them (list, coverage, pairs).
+// Evaluation of one block-sparse candidate of one item: the candidate's selection from the pooled scores of the
+// segment's last query block (list, coverage, pairs).  The blockIdx.y-th block-sparse candidate of the library.
 __global__ void __launch_bounds__(256)
 rs_bs_eval_kernel(IdxParams P) {
   extern __shared__ float score[];      // [nb]
+  const int item = blockIdx.x, bs_index = blockIdx.y;
   __shared__ uint32_t hist[256];
   __shared__ uint32_t sh[8];
   __shared__ unsigned int wcnt[16];
   __shared__ int32_t sel[1024];
   __shared__ u64 cov[RS_PROBE_GROUPS];
-  const int item = blockIdx.x;
   if (P.stats == nullptr && P.choice != nullptr) return;    // materialise mode without stats: rows are built elsewhere
-  // blockIdx.y-th block-sparse candidate of the library
   int my_c = -1;
   for (int c = 0, seen = 0; c < P.n_cand; ++c)
-    if (P.lib[c].pattern == RS_BLOCK_SPARSE && seen++ == (int)blockIdx.y) my_c = c;
+    if (P.lib[c].pattern == RS_BLOCK_SPARSE && seen++ == bs_index) my_c = c;
   if (my_c < 0 || (P.choice != nullptr && P.choice[item] != my_c)) return;
   const int s = item / P.Hq;
   const int q0 = P.seg_bounds[s], q1 = P.seg_bounds[s + 1];
@@ -764,14 +776,24 @@ rs_bs_eval_kernel(IdxParams P) {
   }
 }
 
-// Materialise: one block per (query block, head) of every item routed to block-sparse.
+// What the side chain starts with, one kernel: blocks 0 .. n_simple - 1 the statistics of the closed-form candidates
+// (job = block), the blocks behind them the pooled scores the block-sparse evaluation selects from (score_blocks
+// blocks per item).
 __global__ void __launch_bounds__(256)
-rs_bs_rows_kernel(IdxParams P) {
-  extern __shared__ float score[];
+rs_side_stats_kernel(IdxParams P, int n_simple, int score_blocks) {
+  if ((int)blockIdx.x < n_simple) {
+    simple_stats_block(P, blockIdx.x);
+  } else {
+    const int e = blockIdx.x - n_simple;
+    bs_eval_scores_block(P, e / score_blocks, e % score_blocks);
+  }
+}
+
+// Materialise: one block per (query block, head) of every item routed to block-sparse.
+__device__ __forceinline__ void bs_row_block(const IdxParams& P, int qb, int h, float* score /* [nb] */) {
   __shared__ uint32_t hist[256];
   __shared__ uint32_t sh[8];
   __shared__ unsigned int wcnt[16];
-  const int qb = P.bs_rows_first + blockIdx.x, h = blockIdx.y;
   const int s = seg_of_block(P, qb);
   const int item = s * P.Hq + h;
   const rs_candidate cand = P.lib[P.choice[item]];
@@ -794,11 +816,8 @@ rs_bs_rows_kernel(IdxParams P) {
 // order as select_row (key descending, index ascending), without block-wide barriers.
 constexpr int kWarpRowMax = 1024;
 
-__global__ void __launch_bounds__(256)
-rs_bs_rows_warp_kernel(IdxParams P, int qb_end) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int qb = blockIdx.x * 8 + warp, h = blockIdx.y;
-  if (qb >= qb_end) return;
+__device__ __forceinline__ void bs_row_warp(const IdxParams& P, int qb, int h) {
+  const int lane = threadIdx.x & 31;
   const int s = seg_of_block(P, qb);
   const int item = s * P.Hq + h;
   const rs_candidate cand = P.lib[P.choice[item]];
@@ -856,6 +875,21 @@ rs_bs_rows_warp_kernel(IdxParams P, int qb_end) {
   if (lane == 0) {
     if (take < cap) out[take] = qb;                   // the diagonal block is the largest index: list stays ascending
     P.out.bs_count[orow] = take + 1;
+  }
+}
+
+// Row selection of the materialise call, one kernel: blocks 0 .. ceil(n_short / 8) - 1 serve the query blocks below
+// n_short one warp each, the blocks behind them one longer row each.
+__global__ void __launch_bounds__(256)
+rs_bs_rows_kernel(IdxParams P, int n_short) {
+  extern __shared__ float score[];      // [nb], used by the block-per-row part
+  const int n_warp_blocks = (n_short + 7) / 8;
+  const int h = blockIdx.y;
+  if ((int)blockIdx.x < n_warp_blocks) {
+    const int qb = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (qb < n_short) bs_row_warp(P, qb, h);
+  } else {
+    bs_row_block(P, n_short + ((int)blockIdx.x - n_warp_blocks), h, score);
   }
 }
 
@@ -1205,25 +1239,22 @@ static int build_indices_impl(const rs_problem* p, const rs_candidate* lib, int 
     rs_vs_select_kernel<<<dim3(kSelCluster, 2 * n_items, sel_groups), kSelThreads, sel_smem, stream>>>(P);
     rs_vs_finish_kernel<<<n_jobs, kFinishThreads, 0, stream>>>(P);
   }
-  if (stats != nullptr) rs_simple_stats_kernel<<<n_jobs, 256, 0, side>>>(P);
-  if (any_bs) {
-    if ((choice == nullptr || stats != nullptr) && bscore == nullptr)
-      rs_bs_eval_scores_kernel<<<dim3((nb + 255) / 256, n_items), 256, 0, side>>>(P);
-    if (choice == nullptr || stats != nullptr)
-      rs_bs_eval_kernel<<<dim3(n_items, n_bs), 256, (size_t)nb * sizeof(float), side>>>(P);
-    if (choice != nullptr) {
-      if (bscore == nullptr) {
-        const int nt = (nb + 63) / 64;
-        rs_bs_scores_kernel<<<dim3(nt, nt, P.Hq), 256, 0, side>>>(P);
-      }
-      // short rows one warp each; rows with more than 1024 candidate blocks one thread block each
-      const int n_short = nb < kWarpRowMax + 1 ? nb : kWarpRowMax + 1;       // query blocks 0 .. 1024
-      rs_bs_rows_warp_kernel<<<dim3((n_short + 7) / 8, P.Hq), 256, 0, side>>>(P, n_short);
-      if (nb > n_short) {
-        P.bs_rows_first = n_short;
-        rs_bs_rows_kernel<<<dim3(nb - n_short, P.Hq), 256, (size_t)nb * sizeof(float), side>>>(P);
-      }
+  {
+    const bool eval = any_bs && (choice == nullptr || stats != nullptr);
+    const int n_simple = stats != nullptr ? n_jobs : 0;
+    const int score_blocks = eval && bscore == nullptr ? (nb + 255) / 256 : 0;
+    if (n_simple + score_blocks > 0)
+      rs_side_stats_kernel<<<n_simple + score_blocks * n_items, 256, 0, side>>>(P, n_simple, score_blocks);
+    if (eval) rs_bs_eval_kernel<<<dim3(n_items, n_bs), 256, (size_t)nb * sizeof(float), side>>>(P);
+  }
+  if (any_bs && choice != nullptr) {
+    if (bscore == nullptr) {
+      const int nt = (nb + 63) / 64;
+      rs_bs_scores_kernel<<<dim3(nt, nt, P.Hq), 256, 0, side>>>(P);
     }
+    // short rows one warp each; rows with more than 1024 candidate blocks one thread block each
+    const int n_short = nb < kWarpRowMax + 1 ? nb : kWarpRowMax + 1;       // query blocks 0 .. 1024
+    rs_bs_rows_kernel<<<dim3((n_short + 7) / 8 + (nb - n_short), P.Hq), 256, (size_t)nb * sizeof(float), side>>>(P, n_short);
   }
   if (two_chains) {
     rc = rs_side_join(stream);

@@ -26,7 +26,8 @@ constexpr int RS_LOCAL_BAND = 1024;     // keys with i - j below this count as t
 constexpr int kHC = 4;                 // head slots per CTA (4 x 64 = 256 probe rows)
 constexpr int kRows = kHC * RS_PROBE_ROWS;
 constexpr int kKeyTile = 128;
-constexpr int kStages = 3;
+constexpr int kStages1 = 5;            // K-tile ring of pass 1 (no probability tiles in shared memory)
+constexpr int kStages2 = 3;            // K-tile ring of pass 2
 constexpr int kThreads1 = 640;         // pass 1: warp 0 TMA, warp 1 MMA, warps 2..17 compute, warps 18..19 pool K
 constexpr int kThreads2 = 576;         // pass 2: warp 0 TMA, warp 1 MMA, warps 2..17 compute
 constexpr int kComputeThreads = 512;
@@ -46,20 +47,25 @@ struct ProbeParams {
   float* vert;        // [n_seg][Hq][4][n]
   float* slash;       // [n_seg][Hq][4][n]
   float* kpool;       // [Hkv][n/64][128] 64-row means of K, written by pass 1 (may be NULL)
+  const float* blockmax;  // [Hkv][n/64] block maxima of ||v||^2, complete before pass 2 starts (may be NULL)
+  float* vmax;        // [n_seg][Hkv] written by pass 2 from blockmax (may be NULL)
+  float* qpool_last;  // [Hq][n/64][128]: pass 2 writes the mean of every segment's last 64 query rows (may be NULL)
   int32_t* status;
   float scale_log2e;
 };
 
-struct Smem {
+template <int PASS>
+struct SmemT {
+  static constexpr int stages = PASS == 1 ? kStages1 : kStages2;
   static constexpr uint32_t qp = 0;                       // 2 halves x 256 rows x 128 B
-  static constexpr uint32_t k = 65536;                    // kStages x (2 halves x 128 rows x 128 B)
-  static constexpr uint32_t x = k + kStages * 32768;      // pass 2: [16 compute warps][16 rows][kXS] fp32
-  static constexpr uint32_t lse = x + 16 * 16 * kXS * 4;  // 256 floats
+  static constexpr uint32_t k = 65536;                    // stages x (2 halves x 128 rows x 128 B)
+  static constexpr uint32_t x = k + stages * 32768;       // pass 2: [16 compute warps][16 rows][kXS] fp32
+  static constexpr uint32_t lse = x + (PASS == 2 ? 16 * 16 * kXS * 4 : 0);  // 256 floats
   static constexpr uint32_t bars = lse + 1024;            // mbarriers
   static constexpr uint32_t misc = bars + 256;
   static constexpr uint32_t total = misc + 64 + 1024;     // + alignment slack
 };
-static_assert(Smem::total <= 227 * 1024, "probe shared memory");
+static_assert(SmemT<1>::total <= 227 * 1024 && SmemT<2>::total <= 227 * 1024, "probe shared memory");
 
 __device__ __forceinline__ float max3f(float a, float b, float c) {
   float d;
@@ -77,6 +83,8 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   uint8_t* sm = smem_raw + (base - raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int kThreads = PASS == 1 ? kThreads1 : kThreads2;
+  using Smem = SmemT<PASS>;
+  constexpr int kStages = Smem::stages;
 
   // unit = (segment, kv head, head chunk); blockIdx.x = split of the key range
   const int unit = blockIdx.y;
@@ -107,15 +115,16 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const uint32_t bar_q = smem_u32(&bars[0]);
   uint32_t bar_full[kStages], bar_empty[kStages], bar_tfull[2], bar_tempty[2];
 #pragma unroll
-  for (int i = 0; i < kStages; ++i) { bar_full[i] = smem_u32(&bars[1 + i]); bar_empty[i] = smem_u32(&bars[4 + i]); }
+  for (int i = 0; i < kStages; ++i) { bar_full[i] = smem_u32(&bars[1 + i]); bar_empty[i] = smem_u32(&bars[1 + kStages + i]); }
 #pragma unroll
-  for (int i = 0; i < 2; ++i) { bar_tfull[i] = smem_u32(&bars[7 + i]); bar_tempty[i] = smem_u32(&bars[9 + i]); }
+  for (int i = 0; i < 2; ++i) { bar_tfull[i] = smem_u32(&bars[1 + 2 * kStages + i]); bar_tempty[i] = smem_u32(&bars[3 + 2 * kStages + i]); }
 
   if (tid == 0) {
     mbar_init(bar_q, 1);
     for (int i = 0; i < kStages; ++i) { mbar_init(bar_full[i], 1); mbar_init(bar_empty[i], do_pool ? 3 : 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull[i], 1); mbar_init(bar_tempty[i], kComputeThreads / 32); }
     misc[1] = 0;
+    misc[2] = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK);
   }
@@ -240,6 +249,16 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         }
       }
       if (!ok) *abort_flag = 1;
+    } else if (PASS == 2 && blockIdx.x == 0 && hc == 0 && P.vmax != nullptr) {
+      // vmax[s][g] = sqrt(max over the key blocks below the segment end of the block maxima of ||v||^2), by the 31
+      // lanes of this warp that have nothing else to do (a maximum does not depend on the order)
+      const int nbs = q1 >> 6;
+      const float* bm = P.blockmax + (size_t)g * (P.n >> 6);
+      float m = 0.f;
+      for (int i = lane - 1; i < nbs; i += 31) m = fmaxf(m, __ldg(bm + i));
+      atomicMax(const_cast<int*>(&misc[2]), __float_as_int(m));      // non-negative floats order like their bit patterns
+      __syncwarp(0xfffffffeu);
+      if (lane == 1) P.vmax[s * P.Hkv + g] = sqrtf(__int_as_float(misc[2]));
     }
   } else if (warp == 1) {
     if (lane == 0) {
@@ -332,6 +351,30 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const float sl2 = P.scale_log2e;
     bool ok = true;
+
+    if (PASS == 2 && blockIdx.x == 0 && P.qpool_last != nullptr) {
+      // 64-row mean of the segment's last query block from the staged probe rows (the same rows).  One thread per
+      // (head slot, dimension); the additions run in the order of the streaming pool kernel (rows r, r + 16, r + 32,
+      // r + 48 first, then r = 0 .. 15), so both give the same bits.
+      ok = mbar_wait(bar_q, 0, abort_flag);
+      const int ct = tid - 64, hh = ct >> 7, x = ct & 127;
+      if (ok && hh < n_heads) {
+        const uint8_t* qh = sm + Smem::qp + (uint32_t)(x >> 6) * 32768u + (uint32_t)hh * 8192u + (uint32_t)(x & 7) * 2u;
+        const int chunk = (x & 63) >> 3;
+        float sum = 0.f;
+#pragma unroll
+        for (int r = 0; r < 16; ++r) {
+          float acc = 0.f;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const uint16_t u = *reinterpret_cast<const uint16_t*>(qh + k * 2048 + r * 128 + ((chunk ^ (r & 7)) << 4));
+            acc += __uint_as_float((uint32_t)u << 16);
+          }
+          sum += acc;
+        }
+        P.qpool_last[((size_t)(h0 + hh) * (P.n >> 6) + ((q1 >> 6) - 1)) * RS_HEAD_DIM + x] = sum * (1.0f / 64.0f);
+      }
+    }
 
     if (PASS == 1) {
       const int part = (cw >> 2) & 1;                 // head pair
@@ -501,7 +544,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem, kTmemCols); }
 }
 
-// 64-row means of Q and K (fp32) and per-block maxima of ||v||^2.
+// 64-row means of Q (fp32), every block.
 // One CTA per (tensor row block): 256 threads, thread (rg = tid/16, cc = tid%16) sums rows rg, rg+16, .. of 16-byte
 // column chunk cc; a fixed-order shared-memory reduction over the 16 row groups follows.
 __global__ void __launch_bounds__(256)
@@ -533,6 +576,7 @@ rs_pool_kernel(const __nv_bfloat16* __restrict__ X, float* __restrict__ out, lon
   }
 }
 
+// Block maxima of ||v||^2: one CTA per 64-row block, 16 lanes per row.
 __global__ void __launch_bounds__(256)
 rs_vnorm_block_kernel(const __nv_bfloat16* __restrict__ V, float* __restrict__ blockmax, long long n_blocks) {
   __shared__ float red[8];
@@ -565,23 +609,6 @@ rs_vnorm_block_kernel(const __nv_bfloat16* __restrict__ V, float* __restrict__ b
     float m = red[0];
     for (int i = 1; i < 8; ++i) m = fmaxf(m, red[i]);
     blockmax[blk] = m;
-  }
-}
-
-// vmax[s][g] = sqrt(max over key blocks below the segment end of the block maxima of ||v||^2)
-__global__ void rs_vmax_kernel(ProbeParams P, const float* blockmax, float* vmax) {
-  const int s = blockIdx.x / P.Hkv, g = blockIdx.x % P.Hkv;
-  const int nb = P.n >> 6, nbs = P.seg_bounds[s + 1] >> 6;
-  float m = 0.f;
-  for (int i = threadIdx.x; i < nbs; i += blockDim.x) m = fmaxf(m, blockmax[(size_t)g * nb + i]);
-  __shared__ float red[32];
-#pragma unroll
-  for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int i = 1; i < (int)(blockDim.x >> 5); ++i) m = fmaxf(m, red[i]);
-    vmax[blockIdx.x] = sqrtf(m);
   }
 }
 
@@ -644,29 +671,9 @@ __device__ __forceinline__ void pool_block(const __nv_bfloat16* __restrict__ X, 
   }
 }
 
-// 64-row means of the Q blocks that are asked for: with `choice`, the blocks of heads routed to block-sparse; with
-// last_only, the last block of every segment.  Same arithmetic and summation order as rs_pool_kernel.
-__global__ void __launch_bounds__(256)
-rs_pool_q_select_kernel(ProbeParams P, const __nv_bfloat16* __restrict__ Q, float* __restrict__ out, rs_candidate_list L,
-                        const int32_t* __restrict__ choice, int last_only) {
-  __shared__ float red[16][128 + 4];
-  const int nb = P.n >> 6;
-  int h, qb;
-  if (last_only) {
-    h = blockIdx.x % P.Hq;
-    qb = (P.seg_bounds[blockIdx.x / P.Hq + 1] >> 6) - 1;
-  } else {
-    h = blockIdx.y;
-    qb = blockIdx.x;
-    int s = 0;
-    while (s + 1 < P.n_seg && qb * 64 >= P.seg_bounds[s + 1]) ++s;
-    if (choice != nullptr && L.pattern[choice[s * P.Hq + h]] != RS_BLOCK_SPARSE) return;
-  }
-  pool_block(Q, out, (long long)h * nb + qb, red);
-}
-
-// The same for a run of kPoolRun consecutive query blocks per CTA: with a choice most heads are not routed to
-// block-sparse, and tens of thousands of CTAs that leave at once still cost a tenth of a millisecond to launch.
+// 64-row means of the Q blocks of the heads routed to block-sparse (every head without a choice), a run of kPoolRun
+// consecutive query blocks per CTA: most heads are not routed to block-sparse, and tens of thousands of CTAs that
+// leave at once still cost a tenth of a millisecond to launch.  Same arithmetic and summation order as rs_pool_kernel.
 constexpr int kPoolRun = 32;
 __global__ void __launch_bounds__(256)
 rs_pool_q_routed_kernel(ProbeParams P, const __nv_bfloat16* __restrict__ Q, float* __restrict__ out, rs_candidate_list L,
@@ -766,34 +773,39 @@ static int probe_impl(const rs_problem* p, const void* Q, const void* K, const v
       rs_make_tmap_bf16_2d(&tmK32, K, (uint64_t)P.Hkv * P.n, RS_HEAD_DIM, 32, 64))
     return RS_ERR_CUDA;
   static rs_smem_attr attr_pass1, attr_pass2;
-  if (rs_ensure_dynamic_smem(attr_pass1, rs_probe_kernel<1>, (int)Smem::total) != RS_OK ||
-      rs_ensure_dynamic_smem(attr_pass2, rs_probe_kernel<2>, (int)Smem::total) != RS_OK)
+  if (rs_ensure_dynamic_smem(attr_pass1, rs_probe_kernel<1>, (int)SmemT<1>::total) != RS_OK ||
+      rs_ensure_dynamic_smem(attr_pass2, rs_probe_kernel<2>, (int)SmemT<2>::total) != RS_OK)
     return RS_ERR_CUDA;
-  // The value norms and the pooled queries only read V and Q: they run beside the two probe passes, on the side
-  // stream.  Pass 1 is enqueued first so that its CTAs (one per SM, most of the shared memory) are resident before
-  // the small streaming CTAs fill what is left; the other way round the streaming kernels would run alone.
-  // The pooled keys come out of pass 1 itself.
-  cudaStream_t side = nullptr;
-  rc = rs_side_fork(stream, &side);
-  if (rc != RS_OK) return rc;
-  dim3 grid(w.n_splits, w.n_units);
-  rs_probe_kernel<1><<<grid, kThreads1, Smem::total, stream>>>(tmQ, tmK, P);
+  // Pass 1 also pools K; pass 2 turns the block maxima of ||v||^2 into vmax and pools the last query block of every
+  // segment from the probe rows it stages.  The block maxima only read V, the pooling of every query block (when it
+  // is asked for) only Q: they run beside the passes on the side stream.  Pass 1 is enqueued first so that its CTAs
+  // (one per SM, most of the shared memory) are resident before the small streaming CTAs fill what is left; the
+  // other way round the streaming kernels would run alone.
   const long long nb = p->n_keys / 64;
+  const bool pool_all = qpool != nullptr && !(flags & RS_PROBE_QPOOL_LAST_ONLY);
+  if (qpool && !pool_all) P.qpool_last = qpool;
+  const bool use_side = vmax != nullptr || pool_all;
+  cudaStream_t side = nullptr;
+  if (use_side) {
+    rc = rs_side_fork(stream, &side);
+    if (rc != RS_OK) return rc;
+  }
+  dim3 grid(w.n_splits, w.n_units);
+  rs_probe_kernel<1><<<grid, kThreads1, SmemT<1>::total, stream>>>(tmQ, tmK, P);
   if (vmax) {
     float* blockmax = reinterpret_cast<float*>(wsb + w.blockmax);
     rs_vnorm_block_kernel<<<(unsigned)(P.Hkv * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(V), blockmax, P.Hkv * nb);
-    rs_vmax_kernel<<<P.n_seg * P.Hkv, 256, 0, side>>>(P, blockmax, vmax);
+    P.blockmax = blockmax; P.vmax = vmax;
+    rc = rs_side_sync_here(stream);          // pass 2 reads the block maxima (they are long done when pass 1 ends)
+    if (rc != RS_OK) { rs_side_join(stream); return rc; }
   }
-  if (qpool && (flags & RS_PROBE_QPOOL_LAST_ONLY)) {
-    rs_candidate_list none{};
-    rs_pool_q_select_kernel<<<(unsigned)(P.n_seg * P.Hq), 256, 0, side>>>(P, reinterpret_cast<const __nv_bfloat16*>(Q), qpool,
-                                                                           none, nullptr, 1);
-  } else if (qpool) {
+  if (pool_all)
     rs_pool_kernel<<<(unsigned)(P.Hq * nb), 256, 0, side>>>(reinterpret_cast<const __nv_bfloat16*>(Q), qpool, P.Hq * nb);
+  rs_probe_kernel<2><<<grid, kThreads2, SmemT<2>::total, stream>>>(tmQ, tmK32, P);
+  if (use_side) {
+    rc = rs_side_join(stream);
+    if (rc != RS_OK) return rc;
   }
-  rs_probe_kernel<2><<<grid, kThreads2, Smem::total, stream>>>(tmQ, tmK32, P);
-  rc = rs_side_join(stream);
-  if (rc != RS_OK) return rc;
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }
 
