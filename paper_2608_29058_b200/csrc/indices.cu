@@ -415,14 +415,13 @@ __device__ __forceinline__ u64 pairs_block_sparse(int qb_lo, int qb_hi, int k_b)
 
 // ------------------------------------------------------------------------------------------ vertical-slash: D, coverage, pairs
 constexpr int kFinishThreads = 512;
-__global__ void __launch_bounds__(kFinishThreads)
-rs_vs_finish_kernel(IdxParams P) {
+__device__ __forceinline__ void vs_finish_block(const IdxParams& P, int job) {
   __shared__ uint32_t dbits[128];
   __shared__ int wpre[129];
   __shared__ u64 cov[RS_PROBE_GROUPS];
   __shared__ u64 extra_pairs;
   int item, c, slot;
-  if (!job_of(P, blockIdx.x, item, c, slot)) return;
+  if (!job_of(P, job, item, c, slot)) return;
   const rs_candidate cand = P.lib[c];
   if (cand.pattern != RS_VERTICAL_SLASH) return;
   const int s = item / P.Hq;
@@ -602,20 +601,22 @@ __device__ __forceinline__ uint32_t f32_order_key(float x) {
 }
 
 // Selects the `take` largest of score[0, m) (ties -> lower index) plus the diagonal block `qb`; writes them
-// ascending to out[] and returns the count.  All 256 threads of the block call it; scores live in shared memory.
+// ascending to out[] and returns the count.  All NT threads of the block call it; scores live in shared memory.
+template <int NT>
 __device__ int select_row(const float* score, int m, int take, int qb, int32_t* out, int cap, uint32_t* hist /*256*/,
-                          uint32_t* sh /*8*/, unsigned int* wcnt /*16*/) {
+                          uint32_t* sh /*8*/, unsigned int* wcnt /* 2 * NT / 32 */) {
+  constexpr int NW = NT / 32;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t T = 0xffffffffu, k_eq = 0;
   take = min(take, m);
   if (take > 0) {
     if (tid == 0) { sh[0] = 0; sh[1] = (uint32_t)take; }
     for (int pass = 3; pass >= 0; --pass) {
-      hist[tid] = 0;
+      if (tid < 256) hist[tid] = 0;
       __syncthreads();
       const uint32_t prefix = sh[0];
       const int shift = pass * 8;
-      for (int i = tid; i < m; i += 256) {
+      for (int i = tid; i < m; i += NT) {
         const uint32_t key = f32_order_key(score[i]);
         if (pass == 3 || (key >> (shift + 8)) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
       }
@@ -649,8 +650,8 @@ __device__ int select_row(const float* score, int m, int take, int qb, int32_t* 
     k_eq = sh[1];
   }
   __syncthreads();
-  // ordered compaction over [0, m): 8 warps, contiguous chunks
-  const int chunk = (((m + 7) / 8) + 31) / 32 * 32;
+  // ordered compaction over [0, m): one contiguous chunk per warp
+  const int chunk = (((m + NW - 1) / NW) + 31) / 32 * 32;
   const int lo = warp * chunk, hi = min(m, lo + chunk);
   unsigned int gt = 0, eq = 0;
   for (int base = lo; base < hi; base += 32) {
@@ -660,10 +661,10 @@ __device__ int select_row(const float* score, int m, int take, int qb, int32_t* 
     gt += __popc(__ballot_sync(0xffffffffu, in && take > 0 && key > T));
     eq += __popc(__ballot_sync(0xffffffffu, in && take > 0 && key == T));
   }
-  if (lane == 0) { wcnt[warp] = gt; wcnt[8 + warp] = eq; }
+  if (lane == 0) { wcnt[warp] = gt; wcnt[NW + warp] = eq; }
   __syncthreads();
   unsigned int gt_before = 0, eq_before = 0;
-  for (int w = 0; w < warp; ++w) { gt_before += wcnt[w]; eq_before += wcnt[8 + w]; }
+  for (int w = 0; w < warp; ++w) { gt_before += wcnt[w]; eq_before += wcnt[NW + w]; }
   unsigned int pos = gt_before + min(k_eq, eq_before), eq_run = eq_before;
   const unsigned int lt_mask = (1u << lane) - 1u;
   for (int base = lo; base < hi; base += 32) {
@@ -717,14 +718,13 @@ __device__ __forceinline__ void bs_eval_scores_block(const IdxParams& P, int ite
 }
 
 // Evaluation of one block-sparse candidate of one item: the candidate's selection from the pooled scores of the
-// segment's last query block (list, coverage, pairs).  The blockIdx.y-th block-sparse candidate of the library.
-__global__ void __launch_bounds__(256)
-rs_bs_eval_kernel(IdxParams P) {
-  extern __shared__ float score[];      // [nb]
-  const int item = blockIdx.x, bs_index = blockIdx.y;
+// segment's last query block (list, coverage, pairs).  bs_index counts the library's block-sparse candidates.
+// All kFinishThreads threads of the block call it.
+__device__ __forceinline__ void bs_eval_block(const IdxParams& P, int item, int bs_index, float* score /* [nb] */) {
+  constexpr int NT = kFinishThreads;
   __shared__ uint32_t hist[256];
   __shared__ uint32_t sh[8];
-  __shared__ unsigned int wcnt[16];
+  __shared__ unsigned int wcnt[2 * NT / 32];
   __shared__ int32_t sel[1024];
   __shared__ u64 cov[RS_PROBE_GROUPS];
   if (P.stats == nullptr && P.choice != nullptr) return;    // materialise mode without stats: rows are built elsewhere
@@ -738,10 +738,10 @@ rs_bs_eval_kernel(IdxParams P) {
   const int tid = threadIdx.x;
   if (P.bscore != nullptr) {
     const float* row = P.bscore + ((size_t)item * P.nb + qb) * P.nb;
-    for (int kb = tid; kb < qb; kb += 256) score[kb] = row[kb];
+    for (int kb = tid; kb < qb; kb += NT) score[kb] = row[kb];
   } else {
     const float* row = P.bs_eval_ws + (size_t)item * P.nb;
-    for (int kb = tid; kb < qb; kb += 256) score[kb] = row[kb];
+    for (int kb = tid; kb < qb; kb += NT) score[kb] = row[kb];
   }
   __syncthreads();
   {
@@ -751,16 +751,16 @@ rs_bs_eval_kernel(IdxParams P) {
     if (tid < RS_PROBE_GROUPS) cov[tid] = 0;
     __syncthreads();
     const int k_b = min(cand.b0, 1024);
-    const int cnt = select_row(score, qb, min(k_b, qb + 1) - 1, qb, sel, 1024, hist, sh, wcnt);
+    const int cnt = select_row<NT>(score, qb, min(k_b, qb + 1) - 1, qb, sel, 1024, hist, sh, wcnt);
     if (P.choice == nullptr) {
       int32_t* dst = P.out.bs_blk + (size_t)slot * P.out.kb_cap;
-      for (int i = tid; i < cnt && i < P.out.kb_cap; i += 256) dst[i] = sel[i];
+      for (int i = tid; i < cnt && i < P.out.kb_cap; i += NT) dst[i] = sel[i];
       if (tid == 0) P.out.bs_count[slot] = cnt;
     }
     if (P.stats != nullptr) {
       const u64* vblk = P.vblk + (size_t)item * RS_PROBE_GROUPS * P.nb;
       u64 part[RS_PROBE_GROUPS] = {0, 0, 0, 0};
-      for (int i = tid; i < cnt; i += 256)
+      for (int i = tid; i < cnt; i += NT)
 #pragma unroll
         for (int gg = 0; gg < RS_PROBE_GROUPS; ++gg) part[gg] += vblk[(size_t)gg * P.nb + sel[i]];
 #pragma unroll
@@ -773,6 +773,19 @@ rs_bs_eval_kernel(IdxParams P) {
       }
     }
     __syncthreads();
+  }
+}
+
+// What follows the line selection, one kernel: blocks 0 .. n_finish - 1 turn the selected lines of a vertical-slash
+// job into D, coverage and pairs (job = block); the blocks behind them evaluate one (item, block-sparse candidate) each.
+__global__ void __launch_bounds__(kFinishThreads)
+rs_finish_eval_kernel(IdxParams P, int n_finish, int n_items) {
+  extern __shared__ float score[];      // [nb], used by the block-sparse part
+  if ((int)blockIdx.x < n_finish) {
+    vs_finish_block(P, blockIdx.x);
+  } else {
+    const int e = blockIdx.x - n_finish;
+    bs_eval_block(P, e % n_items, e / n_items, score);
   }
 }
 
@@ -805,8 +818,8 @@ __device__ __forceinline__ void bs_row_block(const IdxParams& P, int qb, int h, 
   __syncthreads();
   const size_t orow = (size_t)h * P.nb + qb;
   const int k_b = min(cand.b0, P.out.kb_cap);
-  const int cnt = select_row(score, qb, min(k_b, qb + 1) - 1, qb, P.out.bs_blk + orow * P.out.kb_cap, P.out.kb_cap,
-                             hist, sh, wcnt);
+  const int cnt = select_row<256>(score, qb, min(k_b, qb + 1) - 1, qb, P.out.bs_blk + orow * P.out.kb_cap, P.out.kb_cap,
+                                  hist, sh, wcnt);
   if (tid == 0) P.out.bs_count[orow] = cnt;
 }
 
@@ -1055,7 +1068,7 @@ rs_mix_cov_kernel(IdxParams P, MixArgs M) {
     for (int b = 0; b < kMixMaxBS; ++b) {
       if (b >= n_bs) continue;
       const int k_b = min(P.lib[bs_of[b]].b0, P.out.kb_cap);
-      const int cnt = select_row(score, qb_i, min(k_b, qb_i + 1) - 1, qb_i, blist, P.out.kb_cap, hist, sh, wcnt);
+      const int cnt = select_row<256>(score, qb_i, min(k_b, qb_i + 1) - 1, qb_i, blist, P.out.kb_cap, hist, sh, wcnt);
       for (int x = tid; x < cnt; x += 256) { const int kb = blist[x]; atomicOr(&member[b * mw + (kb >> 5)], 1u << (kb & 31)); }
       __syncthreads();
     }
@@ -1215,9 +1228,10 @@ static int build_indices_impl(const rs_problem* p, const rs_candidate* lib, int 
     const long long warps = (long long)n_items * RS_PROBE_GROUPS * nb;
     rs_vblk_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, stream>>>(P);
   }
-  // The vertical-slash chain (keys, select, D / coverage / pairs) and the block-sparse chain (pooled scores, row
-  // selection) do not read each other's results; both read the block sums above.  The second chain and the closed-form
-  // statistics run on the side stream.
+  // The line selection of the vertical-slash candidates on one side, the closed-form statistics, the pooled scores and
+  // the materialised block-sparse rows on the other do not read each other's results; the second group runs on the
+  // side stream.  What comes after the selection (D / coverage / pairs, and the block-sparse evaluation, which reads
+  // the pooled scores) is one kernel behind the join.
   // launch shape of the select kernel; its attribute is set before the fork so that no error path sits between the
   // fork and the join below
   int n_vs = 0, n_bs = 0;
@@ -1235,17 +1249,13 @@ static int build_indices_impl(const rs_problem* p, const rs_candidate* lib, int 
     rc = rs_side_fork(stream, &side);
     if (rc != RS_OK) return rc;
   }
-  if (any_vs && !skip_vs) {
-    rs_vs_select_kernel<<<dim3(kSelCluster, 2 * n_items, sel_groups), kSelThreads, sel_smem, stream>>>(P);
-    rs_vs_finish_kernel<<<n_jobs, kFinishThreads, 0, stream>>>(P);
-  }
+  if (any_vs && !skip_vs) rs_vs_select_kernel<<<dim3(kSelCluster, 2 * n_items, sel_groups), kSelThreads, sel_smem, stream>>>(P);
+  const bool eval = any_bs && (choice == nullptr || stats != nullptr);
   {
-    const bool eval = any_bs && (choice == nullptr || stats != nullptr);
     const int n_simple = stats != nullptr ? n_jobs : 0;
     const int score_blocks = eval && bscore == nullptr ? (nb + 255) / 256 : 0;
     if (n_simple + score_blocks > 0)
       rs_side_stats_kernel<<<n_simple + score_blocks * n_items, 256, 0, side>>>(P, n_simple, score_blocks);
-    if (eval) rs_bs_eval_kernel<<<dim3(n_items, n_bs), 256, (size_t)nb * sizeof(float), side>>>(P);
   }
   if (any_bs && choice != nullptr) {
     if (bscore == nullptr) {
@@ -1259,6 +1269,13 @@ static int build_indices_impl(const rs_problem* p, const rs_candidate* lib, int 
   if (two_chains) {
     rc = rs_side_join(stream);
     if (rc != RS_OK) return rc;
+  }
+  // after the line selection (and, for the block-sparse evaluation, the pooled scores of the side chain)
+  {
+    const int n_finish = any_vs && !skip_vs ? n_jobs : 0;
+    const int n_eval = eval ? n_items * n_bs : 0;
+    if (n_finish + n_eval > 0)
+      rs_finish_eval_kernel<<<n_finish + n_eval, kFinishThreads, (size_t)nb * sizeof(float), stream>>>(P, n_finish, n_items);
   }
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
 }
