@@ -396,6 +396,19 @@ def main():
         dense_ms = d0.elapsed_time(d1) / reps
         del O_d, lse_d
 
+    # ---- the same layer pass through the one-call entry point (no stage events, no Python between the stages)
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    o0.record()
+    for _ in range(args.steps):
+        step()
+    o1.record()
+    torch.cuda.synchronize()
+    rs.check_status(layer.status, "one-call passes")
+    one_call_ms = o0.elapsed_time(o1) / args.steps
+
     # ---- the same layer pass replayed from a CUDA graph (no host work between the launches)
     graph_ms = None
     if args.graph:
@@ -524,7 +537,7 @@ def main():
                   "selected_fraction_of_dense": f_mask / f_dense},
         "routes": hist, "route_report": layer.route_report() if not fixed else None,
         "cost_model": args.cost, "calibration": calibration, "risk_calibration": risk_calibration, "launch_ablation": launch_ablation,
-        "cuda_graph_ms_per_layer": graph_ms,
+        "one_call_ms_per_layer": one_call_ms, "cuda_graph_ms_per_layer": graph_ms,
         "fallback_rescue": bool(args.rescue), "mixture_uncertainty": bool(args.mixture),
         "mixture_lists": bool(args.mixture_lists),
         "roofline": {"kernel": "rs_attn_kernel (one launch, all heads)", "bound": "tensor", "achieved": achieved,

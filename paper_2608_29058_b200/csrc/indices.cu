@@ -33,15 +33,10 @@ struct IdxParams {
   float scale;
 };
 
-// floor(x * 2^32) of a non-negative float, exactly, from its bits (no float-to-integer conversion unit involved)
+// floor(x * 2^32) of a non-negative float, exactly: the scaling by a power of two is exact in fp32 (the masses are far
+// below 2^95) and the conversion rounds toward zero.
 __device__ __forceinline__ u64 fx(float x) {
-  const uint32_t b = __float_as_uint(x);
-  const int e = (int)((b >> 23) & 0xffu);
-  if (e == 0) return 0ull;                               // zero and subnormals: far below 2^-32
-  const u64 m = (u64)((b & 0x7fffffu) | 0x800000u);      // x = m * 2^(e - 150)
-  const int sh = e - 118;                                // x * 2^32 = m * 2^(e - 118)
-  if (sh >= 0) return m << min(sh, 40);
-  return (sh > -24) ? (m >> (-sh)) : 0ull;
+  return __float2ull_rz(x * 4294967296.0f);
 }
 
 // Adds v of every thread of the block to *target (shared memory): the warp sums first, so that one 64-bit atomic per
@@ -244,8 +239,14 @@ rs_vs_select_kernel(IdxParams P) {
           if (hi == upre[h]) slot = (unsigned)h * kBins + dig;
         if (!inb[u]) slot = 0xffffffffu;
         if (__ballot_sync(0xffffffffu, slot != 0xffffffffu) == 0u) continue;   // nobody in this warp matches a prefix
-        const unsigned int peers = __match_any_sync(0xffffffffu, slot);
-        if (slot != 0xffffffffu && lane == (__ffs(peers) - 1)) atomicAdd(&sel_hist[slot], (unsigned)__popc(peers));
+        // the upper digits of most keys are equal (small masses): one addition for the warp when all 32 agree,
+        // one per lane otherwise (in the lower digits the lanes rarely meet)
+        const unsigned int slot0 = __shfl_sync(0xffffffffu, slot, 0);
+        if (__all_sync(0xffffffffu, slot == slot0)) {
+          if (lane == 0) atomicAdd(&sel_hist[slot], 32u);
+        } else if (slot != 0xffffffffu) {
+          atomicAdd(&sel_hist[slot], 1u);
+        }
       }
     }
     cluster.sync();                                      // every block's histogram of this digit is complete

@@ -122,3 +122,31 @@ def test_lazy_query_pooling_equals_full_pooling_where_it_is_read():
     assert np.all(got[0, 1:4] == 123.0) and np.all(got[3, 0:4] == 123.0)   # heads not routed to block-sparse stay untouched
     rs.rs_pool_queries(p, Q, None, None, qpool, st)                     # no choice: every head
     assert np.array_equal(qpool.cpu().numpy(), full)
+
+
+@pytest.mark.parametrize("n,Hq,Hkv,bounds", [(1088, 8, 1, [0, 320, 1088]), (640, 6, 2, None), (4096, 8, 2, [0, 64, 4096])])
+def test_last_query_block_from_the_staged_probe_rows(n, Hq, Hkv, bounds):
+    """With RS_PROBE_QPOOL_LAST_ONLY the second pass pools each segment's last query block from the probe rows it has
+    staged (head groups larger than one CTA's four head slots included); V_max comes from the same pass.  Both must
+    hold the bits of the full pooling and of the call without the flag."""
+    L = make_layer(tiny_spec(77 + n, n, Hq, Hkv))
+    p = rs.Problem(Hq, Hkv, n, bounds or [0, n])
+    full = run_probe(L, p)
+    Q, K, V = dev_bf16(L["Q"]), dev_bf16(L["K"]), dev_bf16(L["V"])
+    f32 = dict(dtype=torch.float32, device="cuda")
+    S = p.n_segments
+    vert = torch.zeros((S, Hq, 4, n), **f32); slash = torch.zeros((S, Hq, 4, n), **f32); lse = torch.zeros((Hq, S, 64), **f32)
+    qpool = torch.full((Hq, n // 64, 128), -5.0, **f32)
+    vmax = torch.zeros((S, Hkv), **f32)
+    st = rs.new_status()
+    rs.rs_probe(p, Q, K, V, vert, slash, lse, qpool, None, vmax, None, rs.new_workspace(p, None), st,
+                flags=rs.RS_PROBE_QPOOL_LAST_ONLY)
+    rs.check_status(st, "probe, last block only")
+    got = qpool.cpu().numpy()
+    last = [p.seg_bounds[s + 1] // 64 - 1 for s in range(S)]
+    for qb in last:
+        assert np.array_equal(got[:, qb], full["qpool"][:, qb])
+    others = [qb for qb in range(n // 64) if qb not in last]
+    assert np.all(got[:, others] == -5.0)
+    assert np.array_equal(vmax.cpu().numpy(), full["vmax"])
+    assert np.array_equal(vert.cpu().numpy(), full["vert"]) and np.array_equal(slash.cpu().numpy(), full["slash"])
