@@ -515,7 +515,7 @@ def main():
         n_eval, n_route = 0, 0
         n_mat = 3 * any_vs + 2 * any_bs                   # keys / select / finish; fused scores / rows
     else:
-        n_eval = 1 + (3 if any_vs else 1) + 1 * any_bs    # closed-form stats + pooled scores; VS chain (keys + block sums, select, finish) or block sums alone; BS evaluation
+        n_eval = 1 + (3 if any_vs else 1 + any_bs)        # closed-form stats + pooled scores; keys + block sums, select, finish / BS evaluation (without VS: block sums, BS evaluation)
         n_eval += 1 if (args.mixture_lists and any_vs) else 0          # block sums separate from the ranking keys
         n_eval += 4 if args.mixture else 0                # pooled probe (3) + mixture coverage
         n_eval += (0 if args.mixture else 3) + 1 if (args.calibration and args.beta > 0) else 0   # pooled probe + predictor
@@ -688,7 +688,7 @@ def stack(args):
                         "achieved": f_tile / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                         "frac": f_tile / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
                         "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "traffic": None},
-           "clocks": clocks, "gpu_launches": 15 * args.layers * args.steps}
+           "clocks": clocks, "gpu_launches": 14 * args.layers * args.steps}
     print(json.dumps(out))
     return 0
 
