@@ -26,13 +26,12 @@ constexpr int RS_LOCAL_BAND = 1024;     // keys with i - j below this count as t
 constexpr int kHC = 4;                 // head slots per CTA (4 x 64 = 256 probe rows)
 constexpr int kRows = kHC * RS_PROBE_ROWS;
 constexpr int kKeyTile = 128;
-constexpr int kStages1 = 5;            // K-tile ring of pass 1 (no probability tiles in shared memory)
-constexpr int kStages2 = 3;            // K-tile ring of pass 2
+constexpr int kStages1 = 5;            // K-tile ring of pass 1
+constexpr int kStages2 = 5;            // K-tile ring of pass 2
 constexpr int kThreads1 = 640;         // pass 1: warp 0 TMA, warp 1 MMA, warps 2..17 compute, warps 18..19 pool K
 constexpr int kThreads2 = 576;         // pass 2: warp 0 TMA, warp 1 MMA, warps 2..17 compute
 constexpr int kComputeThreads = 512;
 constexpr uint32_t kTmemCols = 512;
-constexpr int kXS = 62;                // floats per row of a warp's probability tile: 15 zeros, 32 keys, 15 zeros
 
 struct rs_candidate_list { int32_t pattern[RS_MAX_CANDIDATES]; };
 
@@ -59,8 +58,8 @@ struct SmemT {
   static constexpr int stages = PASS == 1 ? kStages1 : kStages2;
   static constexpr uint32_t qp = 0;                       // 2 halves x 256 rows x 128 B
   static constexpr uint32_t k = 65536;                    // stages x (2 halves x 128 rows x 128 B)
-  static constexpr uint32_t x = k + stages * 32768;       // pass 2: [16 compute warps][16 rows][kXS] fp32
-  static constexpr uint32_t lse = x + (PASS == 2 ? 16 * 16 * kXS * 4 : 0);  // 256 floats
+  static constexpr uint32_t x = k;                        // pass 2: scratch of the prologue (the ring is not yet in use)
+  static constexpr uint32_t lse = k + stages * 32768;     // 256 floats
   static constexpr uint32_t bars = lse + 1024;            // mbarriers
   static constexpr uint32_t misc = bars + 256;
   static constexpr uint32_t total = misc + 64 + 1024;     // + alignment slack
@@ -134,7 +133,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     // unit forms the same values in the same order, the first one also stores them (and the two descriptors).
     // 512 threads: thread (row, half) folds every second partial of the row, eight loads in flight at a time; the two
     // halves meet through shared memory.  The order of the additions is fixed, so every CTA gets the same bits.
-    float4* mrg = reinterpret_cast<float4*>(sm + Smem::x);        // [2][256] (max, sum, a, loc); x is not yet in use
+    float4* mrg = reinterpret_cast<float4*>(sm + Smem::x);        // [2][256] (max, sum, a, loc)
     const int n_part = 2 * P.n_splits;
     if (tid < 2 * kRows) {
       const int row = tid & (kRows - 1), half = tid >> 8;
@@ -197,12 +196,9 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     P.descr[((size_t)s * P.Hq + h) * 2 + 0] = (red[4 * tid] + red[4 * tid + 2]) * (1.0f / 64.0f);
     P.descr[((size_t)s * P.Hq + h) * 2 + 1] = (red[4 * tid + 1] + red[4 * tid + 3]) * (1.0f / 64.0f);
   }
+  // pass 2's scratch lies in the first stage of the ring: its generic-proxy accesses are ordered before the TMA writes
+  if (PASS == 2) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   __syncthreads();
-  if (PASS == 2) {          // the zero columns on either side of every warp's probability tile (the scratch use is over)
-    float* xz = reinterpret_cast<float*>(sm + Smem::x);
-    for (int i = tid; i < 16 * 16 * kXS; i += kThreads) xz[i] = 0.f;
-    __syncthreads();
-  }
   const uint32_t tmem = (uint32_t)misc[0];
   if (t0 >= t1) {   // nothing to do for this split (uniform across the CTA)
     if (PASS == 1) {
@@ -454,13 +450,12 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     } else {
       // Sixteen warps: warp (quad, hh) owns the 32 keys of its quadrant's current step (its TMEM lanes) and the 64
       // probe rows of head slot hh.  Per probe group: 16 probabilities per key, their sum is the column mass; the
-      // diagonal mass is a skewed sum over the warp's own tile in shared memory, 16 rows of [15 zeros | 32 keys |
-      // 15 zeros].  Lane l sums x[r][l + r] over the 16 rows: the diagonal that ends at its key in row 15 (offset
-      // o = first row of the group + 15 - key); the terms of that diagonal that lie in the previous step's keys arrive
-      // through a register: lanes 0..14 also sum x[r][32 + l + r], the part of the diagonal ending at lane's key of the
-      // NEXT step that lies in this step's keys, and carry it over.  No predicates, no index arrays.
+      // diagonal mass is a skewed sum over the warp's 16 x 32 probabilities: lane l sums row r's entry of key
+      // l - 15 + r, the diagonal that ends at its key in row 15 (offset o = first row of the group + 15 - key), fetched
+      // by rotating every row over the lanes.  The terms of that diagonal that lie in the previous step's keys arrive
+      // through a register: lanes 0..14 also sum the part of the diagonal ending at the same lane's key of the NEXT
+      // step that lies in this step's keys (the wrapped-around end of the same rotations), and carry it over.
       const int hh = cw >> 2;                         // head slot
-      float* xw = reinterpret_cast<float*>(sm + Smem::x) + cw * (16 * kXS);
       const bool live = hh < n_heads;
       const int key_q = t0 * kKeyTile + quad * (t1 - t0) * 32;     // first key of this quadrant's quarter
       float carry[RS_PROBE_GROUPS] = {0.f, 0.f, 0.f, 0.f};
@@ -495,32 +490,35 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             continue;
           }
           float vs[4] = {0.f, 0.f, 0.f, 0.f};
-          __syncwarp();                                 // the previous group's diagonal reads are done
+          float pr[16];
 #pragma unroll
           for (int r = 0; r < 16; ++r) {
             float p = fast_exp2(fmaf(__uint_as_float(v16[r]), sl2, -lse16[r]));
             if (MASKED && (j > ig + r || j < 0)) p = 0.f;
             vs[r & 3] += p;
-            xw[r * kXS + 15 + lane] = p;
+            pr[r] = p;
           }
           // the scores of the next group travel from TMEM while this group's diagonals are summed
           if (grp + 1 < RS_PROBE_GROUPS) tmem_ld16(t_hh + (uint32_t)(grp + 1) * 16u, v16);
           if (store && j < q1) vert_h[(size_t)grp * P.n + j] = (vs[0] + vs[1]) + (vs[2] + vs[3]);
-          __syncwarp();
-          float acc0[4] = {0.f, 0.f, 0.f, 0.f};
+          // Diagonal sums by lane rotation: the diagonal that ends at this thread's key takes row r from the key
+          // 15 - r to the left.  One rotation per row serves both ends: lanes >= 15 - r receive an entry of their own
+          // diagonal, the lanes below receive (wrapped around) the entry that belongs to the diagonal ending at the
+          // same lane of the NEXT 32 keys, i.e. the carry into the warp's next step.
+          float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int r = 0; r < 16; ++r) acc0[r & 3] += xw[r * (kXS + 1) + lane];
+          for (int r = 0; r < 16; ++r) {
+            const int sh = 15 - r;
+            const float t = sh == 0 ? pr[r] : __shfl_sync(0xffffffffu, pr[r], (lane - sh) & 31);
+            if (lane >= sh) acc0[r & 3] += t;
+            else acc1[r & 3] += t;
+          }
           const int o = ig + 15 - j;                    // the offset whose diagonal ends at this key
           if (store) {
             if (o >= 0) slash_h[(size_t)grp * P.n + o] = ((acc0[0] + acc0[1]) + (acc0[2] + acc0[3])) + carry[grp];
             else if (j < q1) slash_h[(size_t)grp * P.n + j] = 0.f;
           }
-          if (lane < 15) {
-            float acc1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int r = 0; r < 15; ++r) acc1[r & 3] += xw[r * (kXS + 1) + 32 + lane];
-            carry[grp] = (acc1[0] + acc1[1]) + (acc1[2] + acc1[3]);
-          }
+          carry[grp] = (acc1[0] + acc1[1]) + (acc1[2] + acc1[3]);     // zero in lanes 15 and above
         }
       };
       for (int it = 0; it < n_mma; ++it) {
