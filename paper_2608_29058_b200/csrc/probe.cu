@@ -482,7 +482,7 @@ rs_probe_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             const float4 t4 = l4[q];
             lse16[4 * q] = t4.x; lse16[4 * q + 1] = t4.y; lse16[4 * q + 2] = t4.z; lse16[4 * q + 3] = t4.w;
           }
-          tc_wait_ld();
+          tc_wait_ld16(v16);
           if (MASKED && jw > ig + 15) {                 // uniform over the warp: no key of the step is visible to the group
             if (grp + 1 < RS_PROBE_GROUPS) tmem_ld16(t_hh + (uint32_t)(grp + 1) * 16u, v16);
             if (store && j < q1) { vert_h[(size_t)grp * P.n + j] = 0.f; slash_h[(size_t)grp * P.n + j] = 0.f; }
