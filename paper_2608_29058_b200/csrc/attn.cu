@@ -499,6 +499,19 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             mode = 2;
           }
         }
+        if (mode == 0) {
+          // this half of the tile does not take the chunk (uniform over the warp): its probabilities are zeros and
+          // neither the running maximum nor the sum moves, so nothing is loaded or exponentiated
+          uint32_t z[16];
+#pragma unroll
+          for (int q = 0; q < 16; ++q) z[q] = 0u;
+          tmem_st16(t_sc, z);
+          tmem_st16(t_sc + 16u, z);
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar_p + 8u * slot);
+          continue;
+        }
         if (mode >= 0) rs_mask_chunk(t_sc, mode, i, j0, edge, cand.b0, cand.b1, vcols, vbase, n_vcols, d_bits, vk, vd);
       }
       tmem_ld32(t_sc, v);
