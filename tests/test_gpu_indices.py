@@ -52,8 +52,14 @@ def check_slot_vs(idx, slot, ix):
     assert np.array_equal(idx.vs_diag[slot, :len(ix.D)].cpu().numpy(), ix.D)
 
 
-@pytest.mark.parametrize("n,Hq,Hkv,bounds", [(832, 4, 2, None), (1344, 2, 1, [0, 448, 1344])])
-def test_evaluation_mode_is_bit_exact(n, Hq, Hkv, bounds):
+# libraries without one of the families: the kernels that serve two families in one launch then run with one kind of block
+LIB_NO_VS = [C(PT.A_SHAPE, 8, 64), C(PT.BLOCK_SPARSE, 3), C(PT.BLOCK_SPARSE, 7), C(PT.DENSE)]
+LIB_NO_BS = [C(PT.VERTICAL_SLASH, 16, 24), C(PT.A_SHAPE, 8, 128), C(PT.VERTICAL_SLASH, 40, 70), C(PT.DENSE)]
+
+
+@pytest.mark.parametrize("n,Hq,Hkv,bounds,LIB", [(832, 4, 2, None, LIB), (1344, 2, 1, [0, 448, 1344], LIB),
+                                                 (1344, 2, 1, [0, 448, 1344], LIB_NO_VS), (832, 4, 2, None, LIB_NO_BS)])
+def test_evaluation_mode_is_bit_exact(n, Hq, Hkv, bounds, LIB):
     L = make_layer(tiny_spec(41 + n, n, Hq, Hkv))
     p = rs.Problem(Hq, Hkv, n, bounds or [0, n])
     probes, vert, slash, bscore = oracle_scores(L, p)
@@ -129,6 +135,18 @@ def test_fused_block_scores_select_the_same_blocks_up_to_near_ties():
             if len(diff):      # only blocks whose scores are within the fp32 tolerance of each other may swap
                 sc = bs[qb, diff]
                 assert sc.max() - sc.min() <= 1e-3 * max(1.0, np.abs(bs[qb, :qb + 1]).max())
+    # evaluation mode from the pooled arrays (no vertical-slash candidate: the statistics kernel and the evaluation
+    # kernel run with their block-sparse parts only): the list of the last query block is the materialised row
+    idx_e, stats = gpu_build(p, lib_c, vert, slash, None, qpool, kpool, None)
+    for h in range(Hq):
+        row = h * nb + nb - 1
+        got_m = idx.bs_blk[row, :int(idx.bs_count[row])].cpu().numpy()
+        slot = h * len(lib)
+        got_e = idx_e.bs_blk[slot, :int(idx_e.bs_count[slot])].cpu().numpy()
+        assert np.array_equal(got_e, got_m)
+        ix = PT.IndexSet(cand=lib[0], q0=0, q1=n)
+        ix.blk = [None] * (nb - 1) + [got_e]
+        assert stats[h, 0, :4].astype(np.uint64).tolist() == PT.coverage_fx(ix, probes[h][0].vert, probes[h][0].slash).tolist()
 
 
 def test_argument_checks():
