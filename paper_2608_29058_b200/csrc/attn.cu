@@ -635,18 +635,21 @@ __device__ __forceinline__ int rs_tile_cost(const AttnParams& P, int wid, int2* 
 }
 
 // Preparation of the launch, one kernel with two kinds of blocks.
-// Blocks 0 .. Hkv-1: the work list (Section 3.4: heads are grouped into one launch).  KV groups run one after the
-// other (the CTAs in flight then stream the same K / V, which keeps them in L2), inside a group the heaviest item first.
-// One block per KV group: cost of each of the group's items (they are contiguous in the head-major enumeration), then
-// a counting sort by cost.  cost / items are scratch of the block itself.
-// Blocks Hkv ..: the vertical key / value rows of every vertical-slash item are gathered into a contiguous,
+// Blocks 0 .. n_groups-1: the work list (Section 3.4: heads are grouped into one launch).  When K and V of all heads
+// exceed L2, n_groups = Hkv: KV groups run one after the other (the CTAs in flight then stream the same K / V, which
+// keeps them in L2), inside a group the heaviest item first.  When they fit, n_groups = 1: heaviest item first over the
+// whole launch (no long tile of the last group is left to start late).  One block per group: cost of each of the
+// group's items (they are contiguous in the head-major enumeration), then a counting sort by cost.  cost / items are
+// scratch of the block itself.
+// Blocks n_groups ..: the vertical key / value rows of every vertical-slash item are gathered into a contiguous,
 // zero-padded buffer; pack_blocks blocks per item, 64 rows each (16 threads move one 256-byte row).
 __global__ void __launch_bounds__(1024)
-rs_attn_prepare_kernel(AttnParams P, int per_group, int n_bins, int* cost, int2* items, int2* order, int pack_blocks,
-                       const __nv_bfloat16* K, const __nv_bfloat16* V, __nv_bfloat16* Kp, __nv_bfloat16* Vp) {
+rs_attn_prepare_kernel(AttnParams P, int n_groups, int per_group, int n_bins, int* cost, int2* items, int2* order,
+                       int pack_blocks, const __nv_bfloat16* K, const __nv_bfloat16* V, __nv_bfloat16* Kp,
+                       __nv_bfloat16* Vp) {
   extern __shared__ int hist[];
-  if ((int)blockIdx.x >= P.Hkv) {
-    const int pb = blockIdx.x - P.Hkv;
+  if ((int)blockIdx.x >= n_groups) {
+    const int pb = blockIdx.x - n_groups;
     const int item = pb / pack_blocks;
     if (P.choice == nullptr || P.lib[P.choice[item]].pattern != RS_VERTICAL_SLASH) return;
     const int h = item % P.Hq, g = h / P.group;
@@ -715,6 +718,8 @@ WsPlan plan_ws(const rs_problem* p, int max_kv) {
   return w;
 }
 
+constexpr size_t kL2ResidentBytes = 96ull << 20;     // K + V of all heads below this: they stay in the 126 MB L2
+
 // Scratch of one attention launch: the work list (cost, items, launch order: one entry per 128-row tile) and, for
 // vertical-slash items, the packed K / V rows of the gathered columns.
 struct AttnScratch { int* cost; int2* items; int2* order; __nv_bfloat16 *Kp, *Vp; int kv_pad; int n_work, n_items; };
@@ -765,9 +770,11 @@ int enqueue_attn(const rs_problem* p, const void* Q, const void* K, const void* 
   const int n_bins = (P.n >> 6) + 66;
   const bool pack = choice != nullptr && any_vs && sc.Kp != nullptr;
   const int pack_blocks = pack ? (P.kv_pad + 63) / 64 : 0;
-  rs_attn_prepare_kernel<<<P.Hkv + pack_blocks * sc.n_items, 1024, (n_bins + 1) * sizeof(int), stream>>>(
-      P, n_work / P.Hkv, n_bins, sc.cost, sc.items, sc.order, pack_blocks, reinterpret_cast<const __nv_bfloat16*>(K),
-      reinterpret_cast<const __nv_bfloat16*>(V), sc.Kp, sc.Vp);
+  const size_t kv_bytes = 2ull * (size_t)P.Hkv * (size_t)P.n * RS_HEAD_DIM * sizeof(__nv_bfloat16);
+  const int n_groups = (kv_bytes <= kL2ResidentBytes || n_work % P.Hkv != 0) ? 1 : P.Hkv;
+  rs_attn_prepare_kernel<<<n_groups + pack_blocks * sc.n_items, 1024, (n_bins + 1) * sizeof(int), stream>>>(
+      P, n_groups, n_work / n_groups, n_bins, sc.cost, sc.items, sc.order, pack_blocks,
+      reinterpret_cast<const __nv_bfloat16*>(K), reinterpret_cast<const __nv_bfloat16*>(V), sc.Kp, sc.Vp);
   if (rs_ensure_dynamic_smem(g_attn_smem, rs_attn_kernel, 116 * 1024) != RS_OK) return RS_ERR_CUDA;
   rs_attn_kernel<<<n_work, kThreads, attn_smem_bytes(P.n), stream>>>(tmQ, tmK, tmV, tmKp, tmVp, P);
   return cudaGetLastError() == cudaSuccess ? RS_OK : RS_ERR_CUDA;
