@@ -153,7 +153,7 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   uint32_t* d_bits = hi_bits + 128;
   int* wprefix = reinterpret_cast<int*>(d_bits + 128);
   uint64_t* bars = reinterpret_cast<uint64_t*>(wprefix + 132);
-  volatile int* misc = reinterpret_cast<volatile int*>(bars + 14);   // [0] tmem base, [1] abort, [2] n_block, [3] n_vert
+  volatile int* misc = reinterpret_cast<volatile int*>(bars + 14);   // [0] tmem base, [1] abort, [2] n_block, [3] visible gathered columns
   // keep / own-block masks of the gathered-column chunks: [chunk][row half]
   unsigned long long* vkeep = reinterpret_cast<unsigned long long*>(sm + SmemLayout::end_tiles + ((list_cap * 2 + 15) & ~15) +
                                                                       3 * 128 * 4 + 132 * 4 + 14 * 8 + 64);
@@ -241,19 +241,30 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
   }
   __syncthreads();
-  if (tid == 0) {
-    int acc = 0;
-    for (int wd = 0; wd < nb_words; ++wd) { wprefix[wd] = acc; acc += __popc(lo_bits[wd] | hi_bits[wd]); }
-    misc[2] = acc;
-    int nv = 0;
-    if (pattern == RS_VERTICAL_SLASH && n_vcols > 0) {   // verticals with j <= last valid row are a prefix
-      const int* vc = P.idx.vs_cols + (size_t)vs_slot * P.idx.kv_cap;
-      const int i_last = i0 + rows_valid - 1;
-      int lo = 0, hi = n_vcols;
-      while (lo < hi) { int mid = (lo + hi) >> 1; if (vc[mid] <= i_last) lo = mid + 1; else hi = mid; }
-      nv = (lo + kChunk - 1) / kChunk;
+  if (warp == 0) {
+    // exclusive prefix of the words' chunk counts: a warp scan, 32 words at a time
+    int carry = 0;
+    for (int wbase = 0; wbase < nb_words; wbase += 32) {
+      const int wd = wbase + lane;
+      const int c = wd < nb_words ? __popc(lo_bits[wd] | hi_bits[wd]) : 0;
+      int incl = c;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += t;
+      }
+      if (wd < nb_words) wprefix[wd] = carry + incl - c;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
     }
-    misc[3] = nv;
+    if (lane == 0) misc[2] = carry;
+  } else if (pattern == RS_VERTICAL_SLASH && n_vcols > 0) {
+    // verticals with j <= last valid row are a prefix of the ascending list: the other warps count them
+    const int* vc = P.idx.vs_cols + (size_t)vs_slot * P.idx.kv_cap;
+    const int i_last = i0 + rows_valid - 1;
+    int cnt = 0;
+    for (int i = tid - 32; i < n_vcols; i += kThreads - 32) cnt += (vc[i] <= i_last) ? 1 : 0;
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    if (lane == 0 && cnt > 0) atomicAdd(const_cast<int*>(&misc[3]), cnt);
   }
   __syncthreads();
   for (int wd = tid; wd < nb_words; wd += kThreads) {
@@ -276,7 +287,7 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
   }
   __syncthreads();
-  const int n_block = misc[2], n_vert = misc[3];
+  const int n_block = misc[2], n_vert = (misc[3] + kChunk - 1) / kChunk;     // misc[3]: visible gathered columns
   const int n_chunks = n_block + n_vert;
   if (n_vert > 0) {
     // Per gathered-column chunk and row half: which columns survive for every row of the half (valid entry, key
