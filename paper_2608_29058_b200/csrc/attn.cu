@@ -229,12 +229,16 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         lo = sink0 | range_mask(max(0, i0 - win + 1) >> 6, qb0, wd);
         hi = sink1 | range_mask(max(0, i0 + 64 - win + 1) >> 6, qb0 + 1, wd);
       } else {   // vertical-slash: block kb is wanted by query block qb when (qb - kb) is in D
-        for (int b = 0; b < 32; ++b) {
-          const int kb = 32 * wd + b;
-          const int d0 = qb0 - kb, d1 = qb0 + 1 - kb;
-          if (d0 >= 0 && ((d_bits[d0 >> 5] >> (d0 & 31)) & 1u)) lo |= 1u << b;
-          if (d1 >= 0 && ((d_bits[d1 >> 5] >> (d1 & 31)) & 1u)) hi |= 1u << b;
-        }
+        // bit b of the word stands for kb = 32 wd + b, i.e. for the diagonal qb - 32 wd - b: the word is a 32-bit
+        // window of D, read backwards
+        auto d_window = [&](int pos) -> uint32_t {      // D[pos .. pos + 31]; diagonals outside [0, 4096) are not in D
+          const int w0 = pos >> 5;                      // arithmetic shift: floor
+          const uint32_t a = (w0 >= 0 && w0 < 128) ? d_bits[w0] : 0u;
+          const uint32_t b = (w0 + 1 >= 0 && w0 + 1 < 128) ? d_bits[w0 + 1] : 0u;
+          return __funnelshift_r(a, b, (uint32_t)(pos & 31));
+        };
+        lo = __brev(d_window(qb0 - 32 * wd - 31));
+        hi = __brev(d_window(qb0 + 1 - 32 * wd - 31));
       }
       lo_bits[wd] = lo;
       hi_bits[wd] = has_hi ? hi : 0u;
