@@ -262,11 +262,47 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     }
     if (lane == 0) misc[2] = carry;
   } else if (pattern == RS_VERTICAL_SLASH && n_vcols > 0) {
-    // verticals with j <= last valid row are a prefix of the ascending list: the other warps count them
+    // The other five warps walk the ascending list of gathered columns, 32 at a time.  Columns with j <= last valid
+    // row are a prefix: they are counted.  Per 32-column piece and row half: which columns survive for every row of
+    // the half (valid entry, key block not after the half's block, not already covered by a block diagonal of D) and
+    // which of them lie in the half's own key block; a chunk whose 64 columns all survive outside the own block needs
+    // no mask at all.
     const int* vc = P.idx.vs_cols + (size_t)vs_slot * P.idx.kv_cap;
     const int i_last = i0 + rows_valid - 1;
+    const int n_piece = (n_vcols + 31) >> 5;
     int cnt = 0;
-    for (int i = tid - 32; i < n_vcols; i += kThreads - 32) cnt += (vc[i] <= i_last) ? 1 : 0;
+    for (int piece = warp - 1; piece < n_piece; piece += kThreads / 32 - 1) {
+      const int vi = piece * 32 + lane;
+      const bool valid = vi < n_vcols;
+      const int j = valid ? vc[vi] : 0;
+      cnt += (valid && j <= i_last) ? 1 : 0;
+      if (piece < 2 * kMaskChunks) {
+        uint32_t kp[2], dg[2];
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const int dlt = qb0 + hf - (j >> 6);
+          const bool covered = dlt >= 0 && dlt < 4096 && ((d_bits[dlt >> 5] >> (dlt & 31)) & 1u);
+          const bool keep = valid && dlt >= 0 && !covered;
+          kp[hf] = __ballot_sync(0xffffffffu, keep);
+          dg[hf] = __ballot_sync(0xffffffffu, keep && dlt == 0);
+        }
+        if (lane == 0) {
+          uint32_t* k32 = reinterpret_cast<uint32_t*>(vkeep);
+          uint32_t* d32 = reinterpret_cast<uint32_t*>(vdiag);
+          const int chunk = piece >> 1, part = piece & 1;
+          k32[(chunk * 2 + 0) * 2 + part] = kp[0]; k32[(chunk * 2 + 1) * 2 + part] = kp[1];
+          d32[(chunk * 2 + 0) * 2 + part] = dg[0]; d32[(chunk * 2 + 1) * 2 + part] = dg[1];
+        }
+      }
+    }
+    // an odd number of pieces: the second half of the last chunk holds no column
+    if (warp == 1 && lane == 0 && (n_piece & 1) && n_piece < 2 * kMaskChunks) {
+      uint32_t* k32 = reinterpret_cast<uint32_t*>(vkeep);
+      uint32_t* d32 = reinterpret_cast<uint32_t*>(vdiag);
+      const int chunk = n_piece >> 1;
+      k32[(chunk * 2 + 0) * 2 + 1] = 0u; k32[(chunk * 2 + 1) * 2 + 1] = 0u;
+      d32[(chunk * 2 + 0) * 2 + 1] = 0u; d32[(chunk * 2 + 1) * 2 + 1] = 0u;
+    }
     cnt = __reduce_add_sync(0xffffffffu, cnt);
     if (lane == 0 && cnt > 0) atomicAdd(const_cast<int*>(&misc[3]), cnt);
   }
@@ -293,36 +329,6 @@ rs_attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
   __syncthreads();
   const int n_block = misc[2], n_vert = (misc[3] + kChunk - 1) / kChunk;     // misc[3]: visible gathered columns
   const int n_chunks = n_block + n_vert;
-  if (n_vert > 0) {
-    // Per gathered-column chunk and row half: which columns survive for every row of the half (valid entry, key
-    // block not after the half's block, not already covered by a block diagonal of D) and which of them lie in the
-    // half's own key block.  A chunk whose 64 columns all survive outside the own block needs no mask at all.
-    const int* vc = P.idx.vs_cols + (size_t)vs_slot * P.idx.kv_cap;
-    const int n_piece = min(n_vert, kMaskChunks) * 2;          // 32-column pieces, one per warp iteration
-    for (int piece = warp; piece < n_piece; piece += kThreads / 32) {
-      const int vi = piece * 32 + lane;
-      const bool valid = vi < n_vcols;
-      const int j = valid ? vc[vi] : 0;
-      uint32_t kp[2], dg[2];
-#pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        const int dlt = qb0 + hf - (j >> 6);
-        const bool covered = dlt >= 0 && ((d_bits[dlt >> 5] >> (dlt & 31)) & 1u);
-        const bool keep = valid && dlt >= 0 && !covered;
-        kp[hf] = __ballot_sync(0xffffffffu, keep);
-        dg[hf] = __ballot_sync(0xffffffffu, keep && dlt == 0);
-      }
-      if (lane == 0) {
-        uint32_t* k32 = reinterpret_cast<uint32_t*>(vkeep);
-        uint32_t* d32 = reinterpret_cast<uint32_t*>(vdiag);
-        const int chunk = piece >> 1, part = piece & 1;
-        k32[(chunk * 2 + 0) * 2 + part] = kp[0]; k32[(chunk * 2 + 1) * 2 + part] = kp[1];
-        d32[(chunk * 2 + 0) * 2 + part] = dg[0]; d32[(chunk * 2 + 1) * 2 + part] = dg[1];
-      }
-    }
-    __syncthreads();
-  }
-
   // =========================================================================================== roles
   // Everything below is pipelined per 64-key chunk; chunk c uses slot c & 1 of the K / V rings, of the two 64-column
   // score buffers in TMEM and of the barrier pairs, in phase (c >> 1) & 1.  While the softmax warps work on chunk c the
