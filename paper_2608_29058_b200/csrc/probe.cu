@@ -9,12 +9,13 @@
 //                         tile the tensor cores read (no second stream of K for the pooled keys).
 //   pass 2 (probe_accum): S^T = K Qp^T with keys on the TMEM lanes; every thread owns one key, so the column
 //                         mass of a 16-row probe group is a sum inside the thread; the diagonal (slash) mass is a
-//                         skewed sum over the warp's own 16 x 32 tile of probabilities in shared memory.  The four
-//                         lane quadrants of a tile hold four different stretches of the CTA's key range (four TMA
-//                         boxes of 32 keys), so a warp walks 32 consecutive keys per step through a contiguous
-//                         quarter of the range and the part of a diagonal that runs off its tile is carried, in a
-//                         register, into its own next step.  Every offset is produced by exactly one thread: no
-//                         atomics, no zero-filled output, no barrier between warps.
+//                         skewed sum over the warp's own 16 x 32 probabilities, formed by rotating every row over
+//                         the lanes.  The four lane quadrants of a tile hold four different stretches of the CTA's
+//                         key range (four TMA boxes of 32 keys), so a warp walks 32 consecutive keys per step through
+//                         a contiguous quarter of the range and the part of a diagonal that runs off its 32 keys is
+//                         carried, in a register, into its own next step.  Every offset is produced by exactly one
+//                         thread: no atomics, no zero-filled output, no barrier between warps.  The same pass turns
+//                         the block maxima of ||v||^2 into V_max and pools the last query block of every segment.
 // Each key tile is read from HBM once per pass (TMA, 128-byte swizzle).
 #include <type_traits>
 
