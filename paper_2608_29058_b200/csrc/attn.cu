@@ -3,7 +3,7 @@
 //
 // One CTA owns one 128-row query tile of one head.  The keys a tile visits are a list of 64-key chunks:
 // key blocks of K/V selected by the head's pattern (dense, A-shape, the block diagonals of vertical-slash,
-// block-sparse) followed by chunks of gathered vertical columns.  Two chunks form one 128-key MMA tile:
+// block-sparse) followed by chunks of gathered vertical columns.  Per chunk:
 //   S = Q K^T        tcgen05.mma, A and B from shared memory (K-major, 128-byte swizzle), S in TMEM
 //   P = exp2(S - m)  softmax warps: tcgen05.ld, online max / sum in one pass per 64-key chunk (rare chunks are
 //                    masked in place first), bf16 P written back over S in TMEM
